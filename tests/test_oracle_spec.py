@@ -1,0 +1,132 @@
+"""Pins for the oracle's handoff state machine: hand-traced streams and invariants (CPU only)."""
+import os
+
+import numpy as np
+import pytest
+
+from paper_2504_12329_b200 import workloads as W
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+
+def _trace(name):
+    out = {}
+    with open(os.path.join(HERE, "golden", name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            k, v = line.split("=")
+            if k == "handoffs":
+                out[k] = [tuple(int(x) for x in h.split(":")) for h in v.split(",")]
+            elif "," in v:
+                out[k] = [int(x) for x in v.split(",")]
+            else:
+                out[k] = int(v)
+    return out
+
+
+@pytest.fixture(scope="module")
+def tiny(oracle):
+    cfg_s = oracle.Config(**W.TINY_S.as_dict())
+    cfg_l = oracle.Config(**W.TINY_L.as_dict())
+    return oracle.Model(cfg_s, 0, 0), oracle.Model(cfg_l, 0, 1)
+
+
+@pytest.mark.parametrize("name,keep", [("handoff_trace_replace.txt", False), ("handoff_trace_keep.txt", True)])
+def test_hand_traced_streams(oracle, tiny, name, keep):
+    T = _trace(name)
+    r = oracle.generate_spec(tiny[0], tiny[1], [1, 2, 3], delimiter_id=10, keyword_ids=[11, 12, 13], n1=3,
+                             keep_probe=keep, max_new_tokens=12, force=T["force"])
+    assert r.rc == 0
+    assert r.tokens.tolist() == T["tokens"]
+    assert r.source.tolist() == T["source"]
+    assert r.handoffs == T["handoffs"]
+    assert r.emission_source.tolist() == T["emission_source"]
+    assert r.emission_fed.tolist() == T["emission_fed"]
+    assert r.emission_tokens.tolist() == T["force"][: len(r.emission_tokens)]
+    assert (r.kv_len_small, r.kv_len_large) == (T["kv_len_small"], T["kv_len_large"])
+
+
+def _run(oracle, tiny, prompt, force, n1=3, max_new=10, keep=False, eos=-1, large=True):
+    return oracle.generate_spec(tiny[0], tiny[1] if large else None, prompt, delimiter_id=10,
+                                keyword_ids=[11, 12, 13], n1=n1, keep_probe=keep, eos_id=eos,
+                                max_new_tokens=max_new, force=force)
+
+
+def test_scripted_edge_cases(oracle, tiny):
+    # the delimiter is the last prompt token and the first sampled token is a keyword
+    r = _run(oracle, tiny, [4, 10], [12, 30, 31, 32, 33], max_new=4)
+    assert r.handoffs == [(2, 0, 2)] and r.tokens.tolist() == [30, 31, 32, 33] and r.source.tolist() == [1, 1, 1, 0]
+    # a keyword without a delimiter before it does nothing
+    r = _run(oracle, tiny, [4, 5], [11, 12, 13, 9], max_new=4)
+    assert r.handoffs == [] and r.source.tolist() == [0, 0, 0, 0]
+    # the target's own delimiter+keyword does not re-trigger inside its run, but the delimiter that ends
+    # the run followed by a speculative keyword does
+    r = _run(oracle, tiny, [4, 10], [11, 10, 11, 10, 12, 40, 41, 42], max_new=6)
+    assert r.tokens.tolist() == [10, 11, 10, 40, 41, 42]
+    assert r.source.tolist() == [1, 1, 1, 1, 1, 1]
+    assert r.handoffs == [(2, 0, 2), (5, 4, 1)]          # the target only lacks the last token it wrote itself
+    assert r.emission_fed.tolist() == [2, 2, 1, 1, 3, 1, 1, 1]
+    # the token budget ends a run early
+    r = _run(oracle, tiny, [4, 10], [11, 20, 21], max_new=2)
+    assert r.tokens.tolist() == [20, 21] and r.source.tolist() == [1, 1] and r.kv_len_large == 3
+    # EOS inside a run stops at once
+    r = _run(oracle, tiny, [4, 10], [11, 20, 99, 21], max_new=8, eos=99)
+    assert r.tokens.tolist() == [20, 99] and r.source.tolist() == [1, 1]
+    # n1 = 1: control returns after a single target token
+    r = _run(oracle, tiny, [4, 10], [11, 20, 21, 22], n1=1, max_new=3)
+    assert r.source.tolist() == [1, 0, 0] and r.emission_fed.tolist() == [2, 2, 1, 1]
+
+
+def test_no_large_model_or_no_keywords_is_plain_decode(oracle, tiny):
+    prompt = W.prompt_ids(3, 8, 1024)
+    force = W.forcing_schedule(5, 40, mean_interval=4, keyword_rate=0.9)
+    a = _run(oracle, tiny, prompt, force, max_new=20, large=False)
+    b = oracle.generate_spec(tiny[0], tiny[1], prompt, delimiter_id=10, keyword_ids=[], n1=3, max_new_tokens=20,
+                             force=force)
+    assert a.handoffs == [] and b.handoffs == []
+    assert a.tokens.tolist() == b.tokens.tolist() and set(a.source.tolist()) == {0}
+    # and equals feeding the cache by hand with greedy choices
+    kv = oracle.KV(tiny[0], 64)
+    z = kv.forward(prompt)
+    out = []
+    for t in range(20):
+        tok = int(force[t]) if force[t] >= 0 else oracle.argmax(z)[0]
+        out.append(tok)
+        z = kv.forward([tok])
+    assert out == a.tokens.tolist()
+
+
+@pytest.mark.parametrize("keep", [False, True])
+@pytest.mark.parametrize("n1", [1, 4, 20])
+def test_invariants_under_random_schedules(oracle, tiny, keep, n1):
+    prompt = W.prompt_ids(100, 32, 1024)
+    force = W.forcing_schedule(101 + n1, 300, mean_interval=8, keyword_rate=0.5)
+    r = oracle.generate_spec(tiny[0], tiny[1], prompt, delimiter_id=10, keyword_ids=[11, 12, 13], n1=n1,
+                             keep_probe=keep, max_new_tokens=128, force=force)
+    assert r.rc == 0 and len(r.tokens) == 128 and len(r.handoffs) >= 2
+    n_steps = len(r.emission_tokens)
+    assert n_steps == (128 if keep else 128 + len(r.handoffs))
+    seq = np.concatenate([prompt, r.tokens])
+    src = r.source
+    for seg_start, step, catch in r.handoffs:
+        i = seg_start - 32                                   # index into generated tokens
+        if keep:
+            assert seq[seg_start - 2] == 10 and seq[seg_start - 1] in (11, 12, 13) and src[i - 1] == 0
+        else:
+            assert seq[seg_start - 1] == 10
+        run = src[i:i + n1]
+        assert np.all(run == 1)                              # the target writes exactly n1 tokens ...
+        if i + n1 < 128:
+            assert src[i + n1] == 0                          # ... then the speculative model resumes
+        assert r.emission_source[step] == 0 and r.emission_tokens[step] in (11, 12, 13)
+        assert catch >= 0
+    # every target token belongs to some run
+    assert src.sum() == sum(min(n1, 128 - (s - 32)) for s, _, _ in r.handoffs)
+    # each model has ingested everything before the last token it was asked to emit
+    assert r.kv_len_small <= 32 + 128 and r.kv_len_large <= 32 + 128
+    assert sum(r.emission_fed[r.emission_source == 0]) == r.kv_len_small
+    assert sum(r.emission_fed[r.emission_source == 1]) == r.kv_len_large
+    # modify ratio
+    assert 0.0 < src.mean() < 1.0
