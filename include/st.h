@@ -1,0 +1,169 @@
+/*
+ * st.h -- C ABI of the Speculative Thinking decode library (libst.so, CUDA, sm_100a).
+ *
+ * The library runs the hot path of Speculative Thinking (Section 3 of the paper, takeover (1)
+ * "Affirmation/Reflection Takeover", hyper-parameters from the appendix "Hyperparameters of
+ * Speculative Thinking"): key/value-cached greedy decode of a small "speculative" transformer and a
+ * large "target" transformer of the Qwen2 architecture, where the target writes n1 tokens whenever
+ * the speculative model samples a reflection keyword right after a delimiter token, and each model
+ * ingests the tokens it has not seen (catch-up prefill -- the paper's "prefix" pass, Table
+ * "comparison of time") the next time it is asked for a token.
+ *
+ * Conventions
+ *   - Every function returns ST_OK (0) or a negative st_status; nothing throws or aborts.
+ *   - "host" pointers are ordinary CPU memory, "dev" pointers are CUDA device memory on the
+ *     model's device.  The caller owns every buffer it passes; the library owns weights, KV pages
+ *     and scratch, allocated at st_model_create through the allocator in st_config (cudaMalloc when
+ *     the callbacks are NULL) and released by st_model_destroy.
+ *   - All work is enqueued on the CUDA stream given at creation.  st_generate_spec returns after
+ *     the results are in the caller's host buffers; st_prefill / st_decode_step are stream-ordered
+ *     and return once the work is enqueued (their host-pointer arguments are consumed before
+ *     return).
+ *   - Two models used together in st_generate_spec must have been created on the same device and
+ *     stream.
+ *   - There is no CPU fallback: without a CUDA device every entry point except st_strerror fails.
+ */
+#ifndef ST_H
+#define ST_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ST_OK = 0,
+    ST_ERR_ARG = -1,         /* null pointer, size out of range, inconsistent shapes */
+    ST_ERR_OOM = -2,         /* device or host allocation failed */
+    ST_ERR_KV_FULL = -3,     /* not enough free KV pages / sequence slots */
+    ST_ERR_VOCAB = -4,       /* vocab_limit larger than a model's vocabulary, token id out of range */
+    ST_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired */
+    ST_ERR_UNSUPPORTED = -6, /* shape or option the kernels do not cover */
+    ST_ERR_INTERNAL = -7,    /* device status word set, CUDA runtime error */
+    ST_ERR_CAPACITY = -8     /* a caller-provided output buffer is too small */
+} st_status;
+
+typedef struct st_model st_model; /* opaque: weights, paged KV pool, scratch */
+
+/* Device allocator hooks (e.g. backed by a framework's caching allocator). */
+typedef void *(*st_alloc_fn)(uint64_t bytes, void *user);
+typedef void (*st_free_fn)(void *ptr, void *user);
+
+/* Architecture of one decoder-only transformer: RMSNorm -> attention (rotary embedding with
+ * half-split pairing, grouped-query heads: q head i uses kv head i / (n_q_heads / n_kv_heads)) ->
+ * residual -> RMSNorm -> SwiGLU FFN -> residual; final RMSNorm and LM head. */
+typedef struct {
+    int32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
+    float rope_theta, rms_eps;
+    int32_t tie_embeddings; /* LM head shares the embedding matrix */
+    int32_t qkv_bias;       /* q/k/v projections carry a bias */
+    int32_t max_seqs;       /* sequence slots */
+    int32_t max_tokens;     /* total KV capacity in tokens over all slots (rounded up to pages) */
+    int32_t page_size;      /* tokens per KV page: 16, 32 or 64 */
+    st_alloc_fn alloc;      /* NULL -> cudaMalloc */
+    st_free_fn free;        /* NULL -> cudaFree */
+    void *alloc_user;
+} st_config;
+
+/* Handoff rule parameters (Section 3 (1); appendix "Hyperparameters of Speculative Thinking":
+ * n1 = 20).  Keywords and the delimiter are token ids. */
+typedef struct {
+    int32_t delimiter_id;
+    const int32_t *keyword_ids; /* host, n_keywords reflection-keyword ids */
+    int32_t n_keywords;
+    int32_t n1;             /* tokens the target writes per takeover */
+    int32_t keep_probe;     /* 0: the keyword token is dropped and the target writes from its position;
+                               1: the keyword stays and the target continues after it */
+    int32_t eos_id;         /* -1: none */
+    int32_t vocab_limit;    /* tokens are chosen among ids < vocab_limit; 0 = min of the two vocabularies */
+    int32_t max_new_tokens;
+} st_spec_params;
+
+typedef struct {
+    int32_t seg_start;   /* first position the target writes */
+    int32_t step;        /* emission step at which the keyword was sampled */
+    int32_t catchup_len; /* tokens the target has to ingest before its first token */
+} st_handoff;
+
+/* Results of one generation.  All arrays are caller-allocated host memory; a NULL array with
+ * capacity 0 is skipped.  An emission step is one pass of one model that produced one sampled (or
+ * forced) token; a dropped keyword still counts as a step. */
+typedef struct {
+    int32_t *tokens;          /* [cap_tokens] tokens written after the prompt */
+    uint8_t *source;          /* [cap_tokens] 0 = speculative model, 1 = target model */
+    int32_t cap_tokens, n_tokens;
+    st_handoff *handoffs;     /* [cap_handoffs] */
+    int32_t cap_handoffs, n_handoffs;
+    int32_t *emission_tokens; /* [cap_steps] token of every step, dropped ones included */
+    uint8_t *emission_source; /* [cap_steps] */
+    int32_t *emission_fed;    /* [cap_steps] tokens ingested by the emitting model at that step */
+    int32_t *emission_argmax; /* [cap_steps] greedy choice before forcing */
+    int32_t cap_steps, n_steps;
+    int32_t kv_len_small, kv_len_large;
+    float *logits_trace;      /* optional [trace_n_steps][vocab_limit] logits of steps trace_first_step.. */
+    int32_t trace_first_step, trace_n_steps;
+    double seconds;           /* device time of the generation (CUDA events) */
+    int64_t bytes_algorithmic; /* weights + KV bytes the passes had to move (sum over steps) */
+} st_spec_result;
+
+/* Create a model with seeded random-init weights: element idx of tensor tid of model `tag` is
+ * bf16(0.02 * z), z an Irwin-Hall(12) deviate built from SplitMix64 stream outputs (the N(0, 0.02)
+ * initialisation of the workloads; norm gains are 1).  `cuda_stream` is a cudaStream_t (NULL = the
+ * legacy default stream).  Blocks until the weights are initialised. */
+int st_model_create(const st_config *cfg, uint64_t seed, uint32_t model_tag, void *cuda_stream, st_model **out);
+void st_model_destroy(st_model *m);
+
+/* Sequence slots of the paged KV cache.  st_seq_reserve makes sure pages exist for `n_tokens`
+ * positions of the slot (ST_ERR_KV_FULL otherwise); prefill/decode reserve what they need themselves. */
+int st_seq_alloc(st_model *m, int32_t *slot_out);
+int st_seq_free(st_model *m, int32_t slot);
+int st_seq_reserve(st_model *m, int32_t slot, int32_t n_tokens);
+int st_kv_len(st_model *m, int32_t slot, int32_t *len_out);          /* synchronises the stream */
+int st_kv_truncate(st_model *m, int32_t slot, int32_t new_len);      /* drop cached positions >= new_len */
+
+/* Ingest n tokens (host ids) at the slot's next positions -- prompt prefill and catch-up prefill
+ * (the paper's "prefix" pass) are the same call.  last_logits_dev (nullable): fp32 [vocab] logits of
+ * the last ingested position. */
+int st_prefill(st_model *m, int32_t slot, const int32_t *tokens_host, int32_t n, float *last_logits_dev);
+
+/* One KV-cached decode step for `batch` sequences: sequence slots_host[i] ingests tokens_dev[i] at its
+ * next position.  logits_dev (nullable): fp32 [batch][vocab]; argmax_dev (nullable): int32 [batch],
+ * lowest-id argmax over the whole vocabulary. */
+int st_decode_step(st_model *m, const int32_t *slots_host, const int32_t *tokens_dev, int32_t batch,
+                   float *logits_dev, int32_t *argmax_dev);
+
+/* Speculative Thinking generation at batch 1 (Section 3, takeover (1)).  `large` may be NULL (plain
+ * greedy decode of `small`).  prompt: host ids, prompt_len >= 1.  force (nullable): host array,
+ * force[t] >= 0 replaces the token sampled at emission step t.  Routing (which model runs next, how
+ * much it ingests) is decided on the device from the sampled token; the host never reads a token to
+ * choose the next launch. */
+int st_generate_spec(st_model *small, st_model *large, const st_spec_params *params,
+                     const int32_t *prompt, int32_t prompt_len,
+                     const int32_t *force, int32_t n_force, st_spec_result *out);
+
+/* Fill `out_dev` (bf16 bit patterns, device) with elements idx0.. of seeded tensor `tid`: the
+ * generator behind st_model_create, exposed so that it can be compared bit for bit. */
+int st_fill_tensor_bf16(uint64_t seed, uint32_t model_tag, uint32_t tid, uint64_t idx0, uint64_t n,
+                        uint16_t *out_dev, void *cuda_stream);
+
+/* Bytes of weights one decode step streams, and KV bytes per cached token. */
+int64_t st_weight_bytes(const st_model *m);
+int64_t st_kv_bytes_per_token(const st_model *m);
+
+/* Measurement aids.  st_kernel_launches: kernels this library has launched in this process.
+ * st_time_gemv: average device time (CUDA events on the model's stream, after a warm-up round) of
+ * `iters` back-to-back launches of one batch-1 projection kernel, cycling through the layers so that
+ * every launch streams different weights: which = 0 QKV, 1 O, 2 gate/up, 3 down, 4 LM head (the
+ * weight-streaming matrix-vector products of the decode pass).  Scratch activations are overwritten. */
+int64_t st_kernel_launches(void);
+int st_time_gemv(st_model *m, int32_t which, int32_t iters, double *seconds_out);
+
+/* Sticky device status word (0 = clean) and message text. */
+int st_last_device_status(st_model *m);
+const char *st_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ST_H */

@@ -1,0 +1,59 @@
+// Shared device-side definitions of the Speculative Thinking decode library (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace st {
+
+// Which rows a model pass works on.  Written by the host (explicit prefill/decode calls) or by the
+// router kernel (generation), read by every kernel of the pass.
+struct StepDesc {
+    int32_t pos0;     // position of the first ingested token (= cached length before the pass)
+    int32_t m;        // number of tokens ingested by the pass
+    int32_t tok_off;  // tokens of the pass are tok[tok_off .. tok_off + m)
+    int32_t emit;     // 1: the pass ends with LM head + sampling; 0: ingest only
+};
+
+// Device status bits (sticky).
+enum : int32_t {
+    DEV_BAD_TOKEN = 1,     // token id outside the vocabulary
+    DEV_BAD_PAGE = 2,      // block table entry outside the pool
+    DEV_WAIT_EXPIRED = 4,  // a bounded wait ran out
+    DEV_LOG_FULL = 8       // an emission / handoff log overflowed
+};
+
+__device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+
+__device__ __forceinline__ uint4 ldg_nc_v4(const void *p)
+{
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p));
+    return r;
+}
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ uint16_t f32_to_bf16_bits(float f)
+{
+    uint32_t u = __float_as_uint(f);
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+// a = hi + lo with hi = bf16(a), lo = bf16(a - hi): 16 significand bits in two bf16 values.
+__device__ __forceinline__ void split_bf16(float a, uint16_t &hi, uint16_t &lo)
+{
+    hi = f32_to_bf16_bits(a);
+    lo = f32_to_bf16_bits(a - __uint_as_float((uint32_t)hi << 16));
+}
+
+}  // namespace st
