@@ -1,0 +1,320 @@
+"""ctypes binding of libst.so: the same entry points as include/st.h, argument marshalling only.
+
+Device memory handed to the library (and, optionally, the library's own weights and KV pools through
+the allocator hooks) comes from PyTorch; every computation runs in the library's CUDA kernels.  If
+the shared library is missing the import fails -- there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libst.so")
+
+ST_OK, ST_ERR_ARG, ST_ERR_OOM, ST_ERR_KV_FULL, ST_ERR_VOCAB = 0, -1, -2, -3, -4
+ST_ERR_TIMEOUT, ST_ERR_UNSUPPORTED, ST_ERR_INTERNAL, ST_ERR_CAPACITY = -5, -6, -7, -8
+
+ALLOC_FN = C.CFUNCTYPE(C.c_void_p, C.c_uint64, C.c_void_p)
+FREE_FN = C.CFUNCTYPE(None, C.c_void_p, C.c_void_p)
+
+
+class StConfig(C.Structure):
+    _fields_ = [
+        ("n_layers", C.c_int32), ("hidden", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+        ("head_dim", C.c_int32), ("ffn", C.c_int32), ("vocab", C.c_int32),
+        ("rope_theta", C.c_float), ("rms_eps", C.c_float),
+        ("tie_embeddings", C.c_int32), ("qkv_bias", C.c_int32),
+        ("max_seqs", C.c_int32), ("max_tokens", C.c_int32), ("page_size", C.c_int32),
+        ("alloc", ALLOC_FN), ("free", FREE_FN), ("alloc_user", C.c_void_p),
+    ]
+
+
+class StSpecParams(C.Structure):
+    _fields_ = [
+        ("delimiter_id", C.c_int32), ("keyword_ids", C.POINTER(C.c_int32)), ("n_keywords", C.c_int32),
+        ("n1", C.c_int32), ("keep_probe", C.c_int32), ("eos_id", C.c_int32), ("vocab_limit", C.c_int32),
+        ("max_new_tokens", C.c_int32),
+    ]
+
+
+class StHandoff(C.Structure):
+    _fields_ = [("seg_start", C.c_int32), ("step", C.c_int32), ("catchup_len", C.c_int32)]
+
+
+class StSpecResult(C.Structure):
+    _fields_ = [
+        ("tokens", C.POINTER(C.c_int32)), ("source", C.POINTER(C.c_uint8)),
+        ("cap_tokens", C.c_int32), ("n_tokens", C.c_int32),
+        ("handoffs", C.POINTER(StHandoff)), ("cap_handoffs", C.c_int32), ("n_handoffs", C.c_int32),
+        ("emission_tokens", C.POINTER(C.c_int32)), ("emission_source", C.POINTER(C.c_uint8)),
+        ("emission_fed", C.POINTER(C.c_int32)), ("emission_argmax", C.POINTER(C.c_int32)),
+        ("cap_steps", C.c_int32), ("n_steps", C.c_int32),
+        ("kv_len_small", C.c_int32), ("kv_len_large", C.c_int32),
+        ("logits_trace", C.POINTER(C.c_float)), ("trace_first_step", C.c_int32), ("trace_n_steps", C.c_int32),
+        ("seconds", C.c_double), ("bytes_algorithmic", C.c_int64),
+    ]
+
+
+EXPORTS = [
+    "st_model_create", "st_model_destroy", "st_seq_alloc", "st_seq_free", "st_seq_reserve", "st_kv_len",
+    "st_kv_truncate", "st_prefill", "st_decode_step", "st_generate_spec", "st_fill_tensor_bf16",
+    "st_weight_bytes", "st_kv_bytes_per_token", "st_last_device_status", "st_strerror",
+    "st_kernel_launches", "st_time_gemv",
+]
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with paper_2504_12329_b200/build.py "
+                              "(there is no CPU or PyTorch fallback)")
+        L = C.CDLL(LIB_PATH)
+        L.st_model_create.restype = C.c_int
+        L.st_model_create.argtypes = [C.POINTER(StConfig), C.c_uint64, C.c_uint32, C.c_void_p, C.POINTER(C.c_void_p)]
+        L.st_model_destroy.restype = None
+        L.st_model_destroy.argtypes = [C.c_void_p]
+        L.st_seq_alloc.restype = C.c_int
+        L.st_seq_alloc.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
+        L.st_seq_free.restype = C.c_int
+        L.st_seq_free.argtypes = [C.c_void_p, C.c_int32]
+        L.st_seq_reserve.restype = C.c_int
+        L.st_seq_reserve.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
+        L.st_kv_len.restype = C.c_int
+        L.st_kv_len.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32)]
+        L.st_kv_truncate.restype = C.c_int
+        L.st_kv_truncate.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
+        L.st_prefill.restype = C.c_int
+        L.st_prefill.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p]
+        L.st_decode_step.restype = C.c_int
+        L.st_decode_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+        L.st_generate_spec.restype = C.c_int
+        L.st_generate_spec.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(StSpecParams), C.c_void_p, C.c_int32,
+                                       C.c_void_p, C.c_int32, C.POINTER(StSpecResult)]
+        L.st_fill_tensor_bf16.restype = C.c_int
+        L.st_fill_tensor_bf16.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p]
+        L.st_weight_bytes.restype = C.c_int64
+        L.st_weight_bytes.argtypes = [C.c_void_p]
+        L.st_kv_bytes_per_token.restype = C.c_int64
+        L.st_kv_bytes_per_token.argtypes = [C.c_void_p]
+        L.st_last_device_status.restype = C.c_int
+        L.st_last_device_status.argtypes = [C.c_void_p]
+        L.st_kernel_launches.restype = C.c_int64
+        L.st_kernel_launches.argtypes = []
+        L.st_time_gemv.restype = C.c_int
+        L.st_time_gemv.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_double)]
+        L.st_strerror.restype = C.c_char_p
+        L.st_strerror.argtypes = [C.c_int]
+        _lib = L
+    return _lib
+
+
+class StError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {lib().st_strerror(status).decode()} ({status})")
+
+
+def _check(rc: int, where: str):
+    if rc != ST_OK:
+        raise StError(rc, where)
+
+
+def st_kernel_launches() -> int:
+    return lib().st_kernel_launches()
+
+
+def st_strerror(status: int) -> str:
+    return lib().st_strerror(status).decode()
+
+
+def _np_ptr(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _dev_ptr(t):
+    """Device pointer of a torch CUDA tensor (or None)."""
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    return C.c_void_p(t.data_ptr())
+
+
+class _TorchAllocator:
+    """Allocator hooks that serve the library's device memory from PyTorch's caching allocator."""
+
+    def __init__(self, device):
+        import torch
+        self._torch = torch
+        self.device = device
+        self.live = {}
+        self.alloc_cb = ALLOC_FN(self._alloc)
+        self.free_cb = FREE_FN(self._free)
+
+    def _alloc(self, nbytes, _user):
+        try:
+            t = self._torch.empty(int(nbytes), dtype=self._torch.uint8, device=self.device)
+        except Exception:
+            return None
+        self.live[t.data_ptr()] = t
+        return t.data_ptr()
+
+    def _free(self, ptr, _user):
+        self.live.pop(ptr, None)
+
+
+def st_fill_tensor_bf16(seed: int, tag: int, tid: int, idx0: int, n: int, out, stream: int = 0):
+    """out: torch CUDA tensor of n 16-bit elements (bf16 or int16)."""
+    _check(lib().st_fill_tensor_bf16(seed, tag, tid, idx0, n, _dev_ptr(out), C.c_void_p(stream)), "st_fill_tensor_bf16")
+
+
+@dataclass
+class SpecResult:
+    tokens: np.ndarray
+    source: np.ndarray
+    handoffs: list
+    emission_tokens: np.ndarray
+    emission_source: np.ndarray
+    emission_fed: np.ndarray
+    emission_argmax: np.ndarray
+    kv_len_small: int
+    kv_len_large: int
+    logits_trace: np.ndarray | None
+    seconds: float
+    bytes_algorithmic: int
+    n_steps: int
+
+
+class Model:
+    """One transformer on the current CUDA device (st_model_create / st_model_destroy)."""
+
+    def __init__(self, shape: dict, *, seed: int = 0, tag: int = 0, max_seqs: int = 1, max_tokens: int = 4096,
+                 page_size: int = 64, stream: int | None = None, torch_alloc: bool = True):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required: the library has no CPU path")
+        self._torch = torch
+        self.device = torch.device("cuda", torch.cuda.current_device())
+        self.stream = torch.cuda.current_stream().cuda_stream if stream is None else stream
+        self._allocator = _TorchAllocator(self.device) if torch_alloc else None
+        cfg = StConfig()
+        for k in ("n_layers", "hidden", "n_q_heads", "n_kv_heads", "head_dim", "ffn", "vocab", "tie_embeddings", "qkv_bias"):
+            setattr(cfg, k, int(shape[k]))
+        cfg.rope_theta = float(shape["rope_theta"])
+        cfg.rms_eps = float(shape["rms_eps"])
+        cfg.max_seqs, cfg.max_tokens, cfg.page_size = max_seqs, max_tokens, page_size
+        if self._allocator:
+            cfg.alloc, cfg.free = self._allocator.alloc_cb, self._allocator.free_cb
+        self.cfg = cfg
+        self.vocab = cfg.vocab
+        h = C.c_void_p()
+        _check(lib().st_model_create(C.byref(cfg), seed, tag, C.c_void_p(self.stream), C.byref(h)), "st_model_create")
+        self.h = h
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib().st_model_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # --- sequences -------------------------------------------------------------------------
+    def st_seq_alloc(self) -> int:
+        s = C.c_int32()
+        _check(lib().st_seq_alloc(self.h, C.byref(s)), "st_seq_alloc")
+        return s.value
+
+    def st_seq_free(self, slot: int):
+        _check(lib().st_seq_free(self.h, slot), "st_seq_free")
+
+    def st_seq_reserve(self, slot: int, n_tokens: int):
+        _check(lib().st_seq_reserve(self.h, slot, n_tokens), "st_seq_reserve")
+
+    def st_kv_len(self, slot: int) -> int:
+        n = C.c_int32()
+        _check(lib().st_kv_len(self.h, slot, C.byref(n)), "st_kv_len")
+        return n.value
+
+    def st_kv_truncate(self, slot: int, new_len: int):
+        _check(lib().st_kv_truncate(self.h, slot, new_len), "st_kv_truncate")
+
+    # --- passes ----------------------------------------------------------------------------
+    def st_prefill(self, slot: int, tokens, last_logits=None):
+        t = np.ascontiguousarray(tokens, dtype=np.int32)
+        _check(lib().st_prefill(self.h, slot, _np_ptr(t), t.size, _dev_ptr(last_logits)), "st_prefill")
+
+    def st_decode_step(self, slots, tokens_dev, logits=None, argmax=None):
+        s = np.ascontiguousarray(slots, dtype=np.int32)
+        _check(lib().st_decode_step(self.h, _np_ptr(s), _dev_ptr(tokens_dev), s.size, _dev_ptr(logits), _dev_ptr(argmax)),
+               "st_decode_step")
+
+    def st_weight_bytes(self) -> int:
+        return lib().st_weight_bytes(self.h)
+
+    def st_kv_bytes_per_token(self) -> int:
+        return lib().st_kv_bytes_per_token(self.h)
+
+    def st_time_gemv(self, which: int, iters: int) -> float:
+        sec = C.c_double()
+        _check(lib().st_time_gemv(self.h, which, iters, C.byref(sec)), "st_time_gemv")
+        return sec.value
+
+    def st_last_device_status(self) -> int:
+        return lib().st_last_device_status(self.h)
+
+
+def st_generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id: int, keyword_ids, n1: int = 20,
+                     keep_probe: bool = False, eos_id: int = -1, vocab_limit: int = 0, max_new_tokens: int,
+                     force=None, trace_first_step: int = 0, trace_n_steps: int = 0, cap_steps: int | None = None,
+                     cap_handoffs: int | None = None) -> SpecResult:
+    """Host buffers in, host buffers out: marshals the arguments of st_generate_spec."""
+    prompt = np.ascontiguousarray(prompt, dtype=np.int32)
+    kw = np.ascontiguousarray(keyword_ids, dtype=np.int32)
+    P = StSpecParams(delimiter_id, kw.ctypes.data_as(C.POINTER(C.c_int32)), kw.size, n1, int(keep_probe), eos_id,
+                     vocab_limit, max_new_tokens)
+    if vocab_limit <= 0:
+        vocab_limit = small.vocab if large is None else min(small.vocab, large.vocab)
+    cap_steps = 2 * max_new_tokens + 8 if cap_steps is None else cap_steps
+    cap_handoffs = max_new_tokens + 1 if cap_handoffs is None else cap_handoffs
+    tokens = np.zeros(max_new_tokens + 1, dtype=np.int32)
+    source = np.zeros(max_new_tokens + 1, dtype=np.uint8)
+    hand = (StHandoff * max(cap_handoffs, 1))()
+    e_tok = np.zeros(max(cap_steps, 1), dtype=np.int32)
+    e_src = np.zeros(max(cap_steps, 1), dtype=np.uint8)
+    e_fed = np.zeros(max(cap_steps, 1), dtype=np.int32)
+    e_arg = np.zeros(max(cap_steps, 1), dtype=np.int32)
+    trace = np.zeros((trace_n_steps, vocab_limit), dtype=np.float32) if trace_n_steps > 0 else None
+    R = StSpecResult()
+    R.tokens = tokens.ctypes.data_as(C.POINTER(C.c_int32))
+    R.source = source.ctypes.data_as(C.POINTER(C.c_uint8))
+    R.cap_tokens = tokens.size
+    R.handoffs = C.cast(hand, C.POINTER(StHandoff))
+    R.cap_handoffs = cap_handoffs
+    R.emission_tokens = e_tok.ctypes.data_as(C.POINTER(C.c_int32))
+    R.emission_source = e_src.ctypes.data_as(C.POINTER(C.c_uint8))
+    R.emission_fed = e_fed.ctypes.data_as(C.POINTER(C.c_int32))
+    R.emission_argmax = e_arg.ctypes.data_as(C.POINTER(C.c_int32))
+    R.cap_steps = cap_steps
+    R.logits_trace = trace.ctypes.data_as(C.POINTER(C.c_float)) if trace is not None else None
+    R.trace_first_step = trace_first_step
+    R.trace_n_steps = trace_n_steps
+    f = None if force is None else np.ascontiguousarray(force, dtype=np.int32)
+    rc = lib().st_generate_spec(small.h, large.h if large is not None else None, C.byref(P), _np_ptr(prompt), prompt.size,
+                                _np_ptr(f), 0 if f is None else f.size, C.byref(R))
+    _check(rc, "st_generate_spec")
+    n, s = R.n_tokens, min(R.n_steps, cap_steps)
+    return SpecResult(tokens[:n].copy(), source[:n].copy(),
+                      [(hand[i].seg_start, hand[i].step, hand[i].catchup_len) for i in range(min(R.n_handoffs, cap_handoffs))],
+                      e_tok[:s].copy(), e_src[:s].copy(), e_fed[:s].copy(), e_arg[:s].copy(),
+                      R.kv_len_small, R.kv_len_large, trace, R.seconds, R.bytes_algorithmic, R.n_steps)

@@ -1,0 +1,270 @@
+// Rotary embedding + KV append, and grouped-query attention over the paged KV cache.
+//
+// KV pages: pool[layer][page][kv_head][slot_in_page][head_dim] in bf16, so the tokens of one
+// (page, head) are contiguous.  A sequence's block table maps position / page_size -> page.
+//
+// Attention is a flash-decoding style split over the keys: one CTA per (key split, kv head, query
+// row) processes all G = n_q_heads / n_kv_heads query heads of its kv head against its key range,
+// so every K/V byte is read once per kv head.  Lanes are grouped D/8 per key (each lane owns 8
+// consecutive channels: one 16-byte load of K and of V), scores close with log2(D/8) shuffles, and
+// softmax is kept online in fp32.  Partial results of the splits are merged by the CTA that
+// finishes last (a ticket counter; nothing waits on anything).
+#pragma once
+#include "st_common.cuh"
+
+namespace st {
+
+struct KvView {
+    uint16_t *k, *v;          // this layer's pools
+    const int32_t *block_tab; // this sequence's block table
+    int32_t page_size, page_shift, n_pages, n_kv_heads;
+};
+
+__device__ __forceinline__ size_t kv_offset(const KvView &kv, int pos, int head, int D, int32_t *status)
+{
+    int page = kv.block_tab[pos >> kv.page_shift];
+    if ((unsigned)page >= (unsigned)kv.n_pages) {
+        atomicOr(status, DEV_BAD_PAGE);
+        page = 0;
+    }
+    return (((size_t)page * kv.n_kv_heads + head) * kv.page_size + (pos & (kv.page_size - 1))) * D;
+}
+
+// x[i] = E[token_i] (fp32) and the rotary table of row i: cs[i][j] = (cos, sin)(pos_i * inv_freq[j]),
+// evaluated in double so that long positions lose nothing.
+__global__ void embed_rope_kernel(const StepDesc *desc, const int32_t *tok, const uint16_t *E, int hidden, int vocab,
+                                  float *X, const double *inv_freq, int half, float2 *cs, int32_t *status)
+{
+    const int i = blockIdx.x;
+    if (i >= desc->m) return;
+    int t = tok[desc->tok_off + i];
+    if ((unsigned)t >= (unsigned)vocab) {
+        if (threadIdx.x == 0) atomicOr(status, DEV_BAD_TOKEN);
+        t = 0;
+    }
+    const uint32_t *e = reinterpret_cast<const uint32_t *>(E + (size_t)t * hidden);
+    float2 *x2 = reinterpret_cast<float2 *>(X + (size_t)i * hidden);
+    for (int j = threadIdx.x; j < hidden / 2; j += blockDim.x) {
+        const uint32_t v = e[j];
+        x2[j] = make_float2(bf16_lo(v), bf16_hi(v));
+    }
+    const double pos = (double)(desc->pos0 + i);
+    for (int j = threadIdx.x; j < half; j += blockDim.x) {
+        double s, c;
+        sincos(pos * inv_freq[j], &s, &c);
+        cs[(size_t)i * half + j] = make_float2((float)c, (float)s);
+    }
+}
+
+// Rotate q in place (fp32), rotate k and store k, v into the cache (bf16).
+// qkv: [rows][(Hq + 2 Hkv) * D] = q heads, then k heads, then v heads.
+__global__ void rope_append_kernel(const StepDesc *desc, float *qkv, const float2 *cs, int Hq, int Hkv, int D,
+                                   KvView kv, int32_t *status)
+{
+    const int i = blockIdx.x;
+    if (i >= desc->m) return;
+    const int half = D >> 1, pos = desc->pos0 + i;
+    float *row = qkv + (size_t)i * (Hq + 2 * Hkv) * D;
+    const float2 *c = cs + (size_t)i * half;
+    for (int idx = threadIdx.x; idx < (Hq + Hkv) * half; idx += blockDim.x) {
+        const int h = idx / half, j = idx - h * half;
+        float *v = row + h * D;
+        const float a = v[j], b = v[j + half];
+        const float2 t = c[j];
+        const float ra = a * t.x - b * t.y, rb = b * t.x + a * t.y;
+        if (h < Hq) {
+            v[j] = ra;
+            v[j + half] = rb;
+        } else {
+            const size_t o = kv_offset(kv, pos, h - Hq, D, status);
+            kv.k[o + j] = f32_to_bf16_bits(ra);
+            kv.k[o + j + half] = f32_to_bf16_bits(rb);
+        }
+    }
+    const float *vsrc = row + (Hq + Hkv) * D;
+    for (int idx = threadIdx.x; idx < Hkv * D; idx += blockDim.x) {
+        const int h = idx / D, j = idx - h * D;
+        kv.v[kv_offset(kv, pos, h, D, status) + j] = f32_to_bf16_bits(vsrc[idx]);
+    }
+}
+
+struct AttnParams {
+    const StepDesc *desc;
+    const float *qkv;           // [rows][(Hq + 2 Hkv) * D], q already rotated
+    KvView kv;
+    float *out_f32;             // [rows][Hq * D] (decode) or null
+    uint16_t *out_hi, *out_lo;  // [rows][Hq * D] hi/lo bf16 planes (prefill) or null
+    float *part_o;              // [rows][Hq][n_splits][D]     (n_splits > 1)
+    float *part_ml;             // [rows][Hq][n_splits][2]
+    int32_t *tickets;           // [rows][Hkv], zero between launches
+    int32_t *status;
+    int32_t Hq, n_splits;
+    float scale;
+};
+
+__device__ __forceinline__ void attn_store(const AttnParams &p, size_t oi, float r)
+{
+    if (p.out_f32) p.out_f32[oi] = r;
+    if (p.out_hi) split_bf16(r, p.out_hi[oi], p.out_lo[oi]);
+}
+
+template <int D, int G>
+__global__ void __launch_bounds__(128) attn_kernel(const AttnParams p)
+{
+    constexpr int LPK = D / 8;       // lanes per key
+    constexpr int KPW = 32 / LPK;    // keys per warp step
+    constexpr int NWARP = 4;
+    constexpr int UK = 4;            // key steps in flight
+    const int row = blockIdx.z, hk = blockIdx.y, split = blockIdx.x;
+    if (row >= p.desc->m) return;
+    const int n_keys = p.desc->pos0 + row + 1;
+    const int Hkv = p.kv.n_kv_heads;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int sub = lane / LPK, ch = (lane % LPK) * 8;
+
+    const int per = (n_keys + p.n_splits - 1) / p.n_splits;
+    const int k0 = split * per, k1 = min(n_keys, k0 + per);
+
+    float q[G][8];
+    {
+        const float *qrow = p.qkv + (size_t)row * (p.Hq + 2 * Hkv) * D + (size_t)hk * G * D + ch;
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            const float4 a = *reinterpret_cast<const float4 *>(qrow + g * D);
+            const float4 b = *reinterpret_cast<const float4 *>(qrow + g * D + 4);
+            q[g][0] = a.x * p.scale; q[g][1] = a.y * p.scale; q[g][2] = a.z * p.scale; q[g][3] = a.w * p.scale;
+            q[g][4] = b.x * p.scale; q[g][5] = b.y * p.scale; q[g][6] = b.z * p.scale; q[g][7] = b.w * p.scale;
+        }
+    }
+    float mx[G], den[G], o[G][8];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        mx[g] = -INFINITY;
+        den[g] = 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) o[g][e] = 0.f;
+    }
+
+    for (int base = k0 + (warp * UK) * KPW; base < k1; base += NWARP * UK * KPW) {
+        uint4 kf[UK], vf[UK];
+        bool ok[UK];
+#pragma unroll
+        for (int u = 0; u < UK; ++u) {
+            const int key = base + u * KPW + sub;
+            ok[u] = key < k1;
+            if (ok[u]) {
+                const size_t off = kv_offset(p.kv, key, hk, D, p.status) + ch;
+                kf[u] = *reinterpret_cast<const uint4 *>(p.kv.k + off);
+                vf[u] = *reinterpret_cast<const uint4 *>(p.kv.v + off);
+            } else {
+                kf[u] = make_uint4(0, 0, 0, 0);
+                vf[u] = make_uint4(0, 0, 0, 0);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UK; ++u) {
+            float kk[8] = {bf16_lo(kf[u].x), bf16_hi(kf[u].x), bf16_lo(kf[u].y), bf16_hi(kf[u].y),
+                           bf16_lo(kf[u].z), bf16_hi(kf[u].z), bf16_lo(kf[u].w), bf16_hi(kf[u].w)};
+            float vv[8] = {bf16_lo(vf[u].x), bf16_hi(vf[u].x), bf16_lo(vf[u].y), bf16_hi(vf[u].y),
+                           bf16_lo(vf[u].z), bf16_hi(vf[u].z), bf16_lo(vf[u].w), bf16_hi(vf[u].w)};
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                float s = 0.f;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) s = fmaf(q[g][e], kk[e], s);
+#pragma unroll
+                for (int off = LPK / 2; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+                if (ok[u]) {   // uniform within the lane group of a key
+                    const float mnew = fmaxf(mx[g], s);
+                    const float corr = __expf(mx[g] - mnew), pw = __expf(s - mnew);
+                    den[g] = den[g] * corr + pw;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) o[g][e] = fmaf(pw, vv[e], o[g][e] * corr);
+                    mx[g] = mnew;
+                }
+            }
+        }
+    }
+
+    // ---- merge the lane groups of a warp, then the warps of the CTA ----
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+#pragma unroll
+        for (int off = LPK; off < 32; off <<= 1) {
+            const float m2 = __shfl_xor_sync(0xffffffffu, mx[g], off);
+            const float d2 = __shfl_xor_sync(0xffffffffu, den[g], off);
+            const float mnew = fmaxf(mx[g], m2);
+            const float c1 = mx[g] == -INFINITY ? 0.f : __expf(mx[g] - mnew);
+            const float c2 = m2 == -INFINITY ? 0.f : __expf(m2 - mnew);
+            den[g] = den[g] * c1 + d2 * c2;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float o2 = __shfl_xor_sync(0xffffffffu, o[g][e], off);
+                o[g][e] = o[g][e] * c1 + o2 * c2;
+            }
+            mx[g] = mnew;
+        }
+    }
+    __shared__ float s_o[NWARP][G][D];
+    __shared__ float s_m[NWARP][G], s_d[NWARP][G];
+    __shared__ int s_last;
+    if (sub == 0) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) s_o[warp][g][ch + e] = o[g][e];
+            if (lane == 0) { s_m[warp][g] = mx[g]; s_d[warp][g] = den[g]; }
+        }
+    }
+    __syncthreads();
+    const int hq0 = hk * G;
+    for (int idx = tid; idx < G * D; idx += 128) {
+        const int g = idx / D, c = idx - g * D;
+        float mnew = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < NWARP; ++w) mnew = fmaxf(mnew, s_m[w][g]);
+        float dsum = 0.f, osum = 0.f;
+#pragma unroll
+        for (int w = 0; w < NWARP; ++w) {
+            const float cw = s_m[w][g] == -INFINITY ? 0.f : __expf(s_m[w][g] - mnew);
+            dsum += s_d[w][g] * cw;
+            osum += s_o[w][g][c] * cw;
+        }
+        if (p.n_splits == 1) {
+            attn_store(p, ((size_t)row * p.Hq + hq0 + g) * D + c, osum / dsum);
+        } else {
+            const size_t pi = ((size_t)row * p.Hq + hq0 + g) * p.n_splits + split;
+            p.part_o[pi * D + c] = osum;
+            if (c == 0) { p.part_ml[pi * 2] = mnew; p.part_ml[pi * 2 + 1] = dsum; }
+        }
+    }
+    if (p.n_splits == 1) return;
+
+    // ---- the CTA that finishes last for this (row, kv head) merges the splits ----
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int t = atomicAdd(&p.tickets[row * Hkv + hk], 1);
+        s_last = (t == p.n_splits - 1);
+        if (s_last) p.tickets[row * Hkv + hk] = 0;   // ready for the next launch
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    for (int idx = tid; idx < G * D; idx += 128) {
+        const int g = idx / D, c = idx - g * D;
+        const size_t pi = ((size_t)row * p.Hq + hq0 + g) * p.n_splits;
+        float mnew = -INFINITY;
+        for (int s = 0; s < p.n_splits; ++s) mnew = fmaxf(mnew, __ldcg(&p.part_ml[(pi + s) * 2]));
+        float dsum = 0.f, osum = 0.f;
+        for (int s = 0; s < p.n_splits; ++s) {
+            const float ms = __ldcg(&p.part_ml[(pi + s) * 2]);
+            const float cw = ms == -INFINITY ? 0.f : __expf(ms - mnew);
+            dsum += __ldcg(&p.part_ml[(pi + s) * 2 + 1]) * cw;
+            osum += __ldcg(&p.part_o[(pi + s) * D + c]) * cw;
+        }
+        attn_store(p, ((size_t)row * p.Hq + hq0 + g) * D + c, osum / dsum);
+    }
+}
+
+}  // namespace st

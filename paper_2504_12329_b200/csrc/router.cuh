@@ -1,0 +1,206 @@
+// Greedy sampling fused with the Speculative Thinking handoff rule (paper Section 3, takeover (1)).
+//
+// After a model's LM head, one kernel finds the lowest-id argmax of the logits below vocab_limit
+// and -- in its last-arriving CTA -- advances the generation state on the device: which model is
+// active, how many tokens the target still owes, the write position, each model's cached length,
+// the output and the handoff log, and the description of the next pass.  The host only learns the
+// kind and size of the next pass; it never sees a token before deciding what to launch.
+#pragma once
+#include "st_common.cuh"
+
+namespace st {
+
+constexpr int kClsKeyword = 2;  // class-table bit of a reflection keyword
+
+struct GenState {
+    // --- dynamic ---
+    int32_t active;      // 0 = speculative (small), 1 = target (large)
+    int32_t remaining;   // tokens the target still writes in this takeover
+    int32_t pos;         // next position to write (prompt included)
+    int32_t step;        // emission steps so far
+    int32_t generated;   // tokens written after the prompt
+    int32_t kv_len[2];   // cached length of each model
+    int32_t done;
+    int32_t n_handoffs;
+    int32_t next_model;  // the pass to run next ...
+    int32_t next_m;      // ... ingests this many tokens ...
+    int32_t next_emit;   // ... and samples a token (1) or only ingests (0)
+    // --- parameters ---
+    int32_t has_large, delimiter, n1, keep_probe, eos, vlimit, max_new, n_force;
+    int32_t prompt_len, cap_steps, cap_handoffs, max_chunk;
+    int32_t trace_first, trace_n;
+};
+
+struct GenBuffers {
+    int32_t *tokens;           // [prompt_len + max_new + 1] whole sequence
+    uint8_t *source;           // [max_new]
+    int32_t *em_tok, *em_fed, *em_arg;  // [cap_steps]
+    uint8_t *em_src;           // [cap_steps]
+    int32_t *handoffs;         // [cap_handoffs][3]
+    const int32_t *force;      // [n_force]
+    const uint8_t *cls;        // [vlimit] class bits per token id
+    float *trace;              // [trace_n][vlimit] or null
+};
+
+// Describe the pass that has to run next: the active model ingests everything it has not cached,
+// at most max_chunk tokens at a time; only the last chunk samples a token.
+__device__ __forceinline__ void plan_next_pass(GenState *g, StepDesc *desc_small, StepDesc *desc_large)
+{
+    const int a = g->active;
+    const int pending = g->pos - g->kv_len[a];
+    const int m = pending > g->max_chunk ? g->max_chunk : pending;
+    g->next_model = a;
+    g->next_m = m;
+    g->next_emit = (m == pending);
+    StepDesc *d = a ? desc_large : desc_small;
+    d->pos0 = g->kv_len[a];
+    d->m = m;
+    d->tok_off = g->kv_len[a];
+    d->emit = g->next_emit;
+}
+
+// The state transition of one emission step (model `active` sampled `greedy`).
+__device__ void router_step(GenState *g, const GenBuffers &b, int greedy, StepDesc *desc_small, StepDesc *desc_large,
+                            int32_t *status)
+{
+    const int a = g->active;
+    const int t = g->step;
+    const int fed = g->pos - g->kv_len[a];
+    g->kv_len[a] = g->pos;
+    int tok = greedy;
+    if (t < g->n_force && b.force[t] >= 0) tok = b.force[t];
+    if (t < g->cap_steps) {
+        b.em_tok[t] = tok;
+        b.em_src[t] = (uint8_t)a;
+        b.em_fed[t] = fed;
+        b.em_arg[t] = greedy;
+    } else {
+        atomicOr(status, DEV_LOG_FULL);
+    }
+    g->step = t + 1;
+    if ((unsigned)tok >= (unsigned)g->vlimit) { atomicOr(status, DEV_BAD_TOKEN); tok = 0; }
+    const bool trigger = g->has_large && a == 0 && b.tokens[g->pos - 1] == g->delimiter && (b.cls[tok] & kClsKeyword);
+    if (trigger) {
+        if (g->keep_probe) {
+            b.tokens[g->pos] = tok;
+            b.source[g->generated] = 0;
+            g->pos++;
+            g->generated++;
+            if (tok == g->eos) g->done = 1;
+        }
+        if (g->n_handoffs < g->cap_handoffs) {
+            int32_t *h = b.handoffs + 3 * g->n_handoffs;
+            h[0] = g->pos;
+            h[1] = t;
+            h[2] = g->pos - g->kv_len[1];
+        } else {
+            atomicOr(status, DEV_LOG_FULL);
+        }
+        g->n_handoffs++;
+        g->active = 1;
+        g->remaining = g->n1;
+    } else {
+        b.tokens[g->pos] = tok;
+        b.source[g->generated] = (uint8_t)a;
+        g->pos++;
+        g->generated++;
+        if (tok == g->eos) g->done = 1;
+        if (a == 1 && --g->remaining == 0) g->active = 0;
+    }
+    if (g->generated >= g->max_new) g->done = 1;
+    plan_next_pass(g, desc_small, desc_large);
+}
+
+// An ingest-only chunk finished: advance the cached length and plan the next pass.
+__global__ void advance_ingest_kernel(GenState *g, StepDesc *desc_small, StepDesc *desc_large)
+{
+    const int a = g->next_model;
+    g->kv_len[a] += g->next_m;
+    plan_next_pass(g, desc_small, desc_large);
+}
+
+__global__ void plan_first_pass_kernel(GenState *g, StepDesc *desc_small, StepDesc *desc_large)
+{
+    plan_next_pass(g, desc_small, desc_large);
+}
+
+struct ArgmaxParams {
+    const float *logits;   // [vocab]
+    int32_t limit;         // ids < limit compete
+    float *part_val;       // [gridDim.x]
+    int32_t *part_idx;     // [gridDim.x]
+    int32_t *ticket;       // zero between launches
+    int32_t *argmax_out;   // nullable: plain decode result
+    // generation (all null for plain decode)
+    GenState *gen;
+    GenBuffers buf;
+    StepDesc *desc_small, *desc_large;
+    int32_t *status;
+};
+
+__device__ __forceinline__ void argmax_merge(float &v, int &i, float v2, int i2)
+{
+    if (v2 > v || (v2 == v && i2 < i)) { v = v2; i = i2; }
+}
+
+__global__ void __launch_bounds__(256) argmax_router_kernel(const ArgmaxParams p)
+{
+    __shared__ float s_v[8];
+    __shared__ int s_i[8];
+    __shared__ int s_last;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // optional logits trace of this emission step (the step counter only changes after every CTA
+    // has taken its ticket, i.e. after all of them have read it here)
+    float *trace = nullptr;
+    if (p.gen && p.buf.trace) {
+        const int t = p.gen->step - p.gen->trace_first;
+        if (t >= 0 && t < p.gen->trace_n) trace = p.buf.trace + (size_t)t * p.limit;
+    }
+    float v = -INFINITY;
+    int idx = 0x7fffffff;
+    for (int i = blockIdx.x * 256 + tid; i < p.limit; i += gridDim.x * 256) {
+        const float z = p.logits[i];
+        if (trace) trace[i] = z;
+        argmax_merge(v, idx, z, i);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float v2 = __shfl_xor_sync(0xffffffffu, v, o);
+        const int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
+        argmax_merge(v, idx, v2, i2);
+    }
+    if (lane == 0) { s_v[warp] = v; s_i[warp] = idx; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < 8; ++w) argmax_merge(v, idx, s_v[w], s_i[w]);
+        p.part_val[blockIdx.x] = v;
+        p.part_idx[blockIdx.x] = idx;
+        __threadfence();
+        const int t = atomicAdd(p.ticket, 1);
+        s_last = (t == (int)gridDim.x - 1);
+        if (s_last) *p.ticket = 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    v = -INFINITY;
+    idx = 0x7fffffff;
+    for (int i = tid; i < (int)gridDim.x; i += 256) argmax_merge(v, idx, __ldcg(&p.part_val[i]), __ldcg(&p.part_idx[i]));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float v2 = __shfl_xor_sync(0xffffffffu, v, o);
+        const int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
+        argmax_merge(v, idx, v2, i2);
+    }
+    __syncthreads();
+    if (lane == 0) { s_v[warp] = v; s_i[warp] = idx; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < 8; ++w) argmax_merge(v, idx, s_v[w], s_i[w]);
+        if (idx == 0x7fffffff) idx = 0;   // nothing comparable: fall back to id 0
+        if (p.argmax_out) *p.argmax_out = idx;
+        if (p.gen) router_step(p.gen, p.buf, idx, p.desc_small, p.desc_large, p.status);
+    }
+}
+
+}  // namespace st

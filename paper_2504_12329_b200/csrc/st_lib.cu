@@ -1,0 +1,939 @@
+// Host side of libst.so: model construction, paged KV bookkeeping, pass scheduling and the C ABI.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/st.h"
+#include "attention.cuh"
+#include "gemv.cuh"
+#include "prefill_simt.cuh"
+#include "router.cuh"
+#include "weights.cuh"
+
+using namespace st;
+
+#define CK(expr)                                                     \
+    do {                                                             \
+        cudaError_t e_ = (expr);                                     \
+        if (e_ != cudaSuccess) {                                     \
+            set_error_text(#expr, e_);                               \
+            return e_ == cudaErrorMemoryAllocation ? ST_ERR_OOM : ST_ERR_INTERNAL; \
+        }                                                            \
+    } while (0)
+#define TRY(expr)                  \
+    do {                           \
+        int rc_ = (expr);          \
+        if (rc_ != ST_OK) return rc_; \
+    } while (0)
+
+static thread_local char g_err_text[256];
+static int64_t g_launches = 0;  // kernels launched by this library in this process
+static void set_error_text(const char *what, cudaError_t e)
+{
+    snprintf(g_err_text, sizeof g_err_text, "%s: %s", what, cudaGetErrorString(e));
+}
+
+// Layer-local tensor ids of the seeded streams (stream id = 16 * (layer + 1) + id; 0 = embedding,
+// 1 = LM head).
+enum { TID_WQ = 1, TID_WK = 2, TID_WV = 3, TID_BQ = 4, TID_BK = 5, TID_BV = 6, TID_WO = 7, TID_WG = 9, TID_WU = 10, TID_WD = 11 };
+
+struct LayerWeights {
+    uint16_t *wqkv;  // [(Hq + 2 Hkv) D][h]: q rows, k rows, v rows
+    float *bqkv;     // [(Hq + 2 Hkv) D]
+    uint16_t *wo;    // [h][Hq D]
+    uint16_t *wgu;   // [2 f][h]: row 2j = gate j, row 2j + 1 = up j
+    uint16_t *wd;    // [h][f]
+    float *g1, *g2;  // norm gains [h]
+};
+
+struct st_model {
+    st_config cfg{};
+    uint64_t seed = 0;
+    uint32_t tag = 0;
+    cudaStream_t stream = nullptr;
+    int device = 0, sm_count = 148;
+    std::vector<void *> allocations;
+
+    // weights
+    uint16_t *embed = nullptr, *lm_head = nullptr;
+    float *gf = nullptr;
+    std::vector<LayerWeights> layers;
+    double *inv_freq = nullptr;
+    int64_t weight_bytes = 0;
+
+    // paged KV
+    int n_pages = 0, pages_per_seq = 0, page_shift = 0;
+    uint16_t *kpool = nullptr, *vpool = nullptr;
+    size_t pool_layer_stride = 0;  // elements per layer
+    int32_t *block_tab = nullptr;  // device [max_seqs][pages_per_seq]
+    std::vector<int32_t> free_pages;
+    std::vector<std::vector<int32_t>> seq_pages;
+    std::vector<int32_t> seq_len;  // host view (explicit prefill/decode calls)
+    std::vector<uint8_t> seq_used;
+
+    // scratch
+    int max_rows = 0;          // rows per multi-row pass
+    int max_splits = 0;
+    float *X = nullptr;        // [max_rows][h] residual stream
+    uint16_t *XN = nullptr;    // [2][max_rows][h] hi/lo planes
+    float *QKV = nullptr;      // [max_rows][(Hq + 2 Hkv) D]
+    float *ATT = nullptr;      // [Hq D] (decode)
+    uint16_t *ATTb = nullptr;  // [2][max_rows][Hq D]
+    float *ACT = nullptr;      // [f] (decode)
+    uint16_t *ACTb = nullptr;  // [2][max_rows][f]
+    float2 *cs = nullptr;      // [max_rows][D / 2]
+    float *logits = nullptr;   // [vocab]
+    float *part_o = nullptr, *part_ml = nullptr;
+    int32_t *tickets = nullptr;  // [max_rows * Hkv + 1]; last entry serves the argmax kernel
+    float *amax_val = nullptr;
+    int32_t *amax_idx = nullptr;
+    int32_t *tokbuf = nullptr;   // [max_rows] staging for explicit calls
+    StepDesc *desc = nullptr;    // device
+    int32_t *status = nullptr;   // device sticky status word
+
+    void *dalloc(size_t bytes)
+    {
+        void *p = nullptr;
+        if (bytes == 0) bytes = 16;
+        if (cfg.alloc) p = cfg.alloc(bytes, cfg.alloc_user);
+        else if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); p = nullptr; }
+        if (p) allocations.push_back(p);
+        return p;
+    }
+};
+
+static constexpr int kArgmaxBlocks = 64;
+static constexpr int kGemvWarps = 16;
+
+// ------------------------------------------------------------------------------------------------
+// launch helpers
+// ------------------------------------------------------------------------------------------------
+
+template <int S, int PRO, int EPI>
+static cudaError_t launch_gemv_s(const GemvParams &p, cudaStream_t s, int sms)
+{
+    constexpr int NW = kGemvWarps, R = 2, U = 4;
+    auto kern = gemv_kernel<NW, S, R, U, PRO, EPI>;
+    const size_t smem = (size_t)p.K * 4 + 2 * NW * R * 4;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const int G = NW / S;
+    const int n_tasks = (p.N + R - 1) / R;
+    const int ctas_needed = (n_tasks + G - 1) / G;
+    int per_sm = (int)((220 * 1024) / (smem + 1024));
+    per_sm = per_sm > 4 ? 4 : per_sm < 1 ? 1 : per_sm;
+    int grid = sms * per_sm;
+    if (grid > ctas_needed) grid = ctas_needed;
+    kern<<<grid, NW * 32, smem, s>>>(p);
+    ++g_launches;
+    return cudaGetLastError();
+}
+
+template <int PRO, int EPI>
+static cudaError_t launch_gemv(const GemvParams &p, cudaStream_t s, int sms)
+{
+    const int n_chunks = (p.K + 255) / 256;
+    if (n_chunks >= 64) return launch_gemv_s<8, PRO, EPI>(p, s, sms);
+    if (n_chunks >= 16) return launch_gemv_s<4, PRO, EPI>(p, s, sms);
+    if (n_chunks >= 8) return launch_gemv_s<2, PRO, EPI>(p, s, sms);
+    return launch_gemv_s<1, PRO, EPI>(p, s, sms);
+}
+
+template <int D>
+static cudaError_t launch_attn_d(const AttnParams &p, int G, dim3 grid, cudaStream_t s)
+{
+    switch (G) {
+    case 1: attn_kernel<D, 1><<<grid, 128, 0, s>>>(p); break;
+    case 2: attn_kernel<D, 2><<<grid, 128, 0, s>>>(p); break;
+    case 3: attn_kernel<D, 3><<<grid, 128, 0, s>>>(p); break;
+    case 4: attn_kernel<D, 4><<<grid, 128, 0, s>>>(p); break;
+    case 5: attn_kernel<D, 5><<<grid, 128, 0, s>>>(p); break;
+    case 6: attn_kernel<D, 6><<<grid, 128, 0, s>>>(p); break;
+    case 7: attn_kernel<D, 7><<<grid, 128, 0, s>>>(p); break;
+    case 8: attn_kernel<D, 8><<<grid, 128, 0, s>>>(p); break;
+    default: return cudaErrorInvalidValue;
+    }
+    ++g_launches;
+    return cudaGetLastError();
+}
+
+static cudaError_t launch_attn(const AttnParams &p, int D, int G, dim3 grid, cudaStream_t s)
+{
+    if (D == 64) return launch_attn_d<64>(p, G, grid, s);
+    if (D == 128) return launch_attn_d<128>(p, G, grid, s);
+    return cudaErrorInvalidValue;
+}
+
+template <int EPI>
+static cudaError_t launch_gemm(const GemmParams &p, int m_upper, cudaStream_t s)
+{
+    dim3 grid((p.N + 63) / 64, (m_upper + 63) / 64);
+    gemm_simt_kernel<EPI><<<grid, 256, 0, s>>>(p);
+    ++g_launches;
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// model construction
+// ------------------------------------------------------------------------------------------------
+
+static int fill_rows(st_model *m, uint16_t *out, uint32_t tid, uint64_t rows, uint64_t cols, uint32_t row_mul, uint32_t row_add)
+{
+    const uint64_t key = tensor_stream_key(m->seed, m->tag, tid);
+    const uint64_t n = rows * cols;
+    int blocks = (int)((n + 255) / 256 < 148 * 16 ? (n + 255) / 256 : 148 * 16);
+    fill_bf16_kernel<<<blocks, 256, 0, m->stream>>>(out, key, 0, rows, cols, row_mul, row_add);
+    ++g_launches;
+    CK(cudaGetLastError());
+    return ST_OK;
+}
+
+static int fill_f32(st_model *m, float *out, uint32_t tid, uint64_t n)
+{
+    const uint64_t key = tensor_stream_key(m->seed, m->tag, tid);
+    fill_f32_kernel<<<(int)((n + 255) / 256), 256, 0, m->stream>>>(out, key, n);
+    ++g_launches;
+    CK(cudaGetLastError());
+    return ST_OK;
+}
+
+static int fill_const(st_model *m, float *out, float v, uint64_t n)
+{
+    fill_const_f32_kernel<<<(int)((n + 255) / 256), 256, 0, m->stream>>>(out, v, n);
+    ++g_launches;
+    CK(cudaGetLastError());
+    return ST_OK;
+}
+
+static int check_config(const st_config *c)
+{
+    if (!c) return ST_ERR_ARG;
+    if (c->n_layers < 1 || c->n_layers > 128 || c->hidden < 8 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->ffn < 8 ||
+        c->vocab < 2 || c->max_seqs < 1 || c->max_tokens < 1)
+        return ST_ERR_ARG;
+    if (c->n_q_heads % c->n_kv_heads) return ST_ERR_ARG;
+    if (c->head_dim != 64 && c->head_dim != 128) return ST_ERR_UNSUPPORTED;
+    if (c->n_q_heads / c->n_kv_heads > 8) return ST_ERR_UNSUPPORTED;
+    if (c->hidden % 8 || c->ffn % 8) return ST_ERR_UNSUPPORTED;
+    if ((int64_t)c->hidden * 4 > 160 * 1024 || (int64_t)c->ffn * 4 > 160 * 1024) return ST_ERR_UNSUPPORTED;
+    if (c->page_size != 16 && c->page_size != 32 && c->page_size != 64) return ST_ERR_ARG;
+    if (!(c->rope_theta > 0.f) || !(c->rms_eps >= 0.f)) return ST_ERR_ARG;
+    if ((c->alloc == nullptr) != (c->free == nullptr)) return ST_ERR_ARG;
+    return ST_OK;
+}
+
+static int model_build(st_model *m)
+{
+    const st_config &c = m->cfg;
+    const int h = c.hidden, D = c.head_dim, qd = c.n_q_heads * D, kd = c.n_kv_heads * D, f = c.ffn;
+    const int qkvd = qd + 2 * kd;
+    CK(cudaGetDevice(&m->device));
+    CK(cudaDeviceGetAttribute(&m->sm_count, cudaDevAttrMultiProcessorCount, m->device));
+
+#define ALLOC(ptr, type, count)                                      \
+    do {                                                             \
+        ptr = (type *)m->dalloc((size_t)(count) * sizeof(type));     \
+        if (!ptr) return ST_ERR_OOM;                                 \
+    } while (0)
+
+    // ---- weights ----
+    ALLOC(m->embed, uint16_t, (size_t)c.vocab * h);
+    TRY(fill_rows(m, m->embed, 0, c.vocab, h, 1, 0));
+    if (c.tie_embeddings) {
+        m->lm_head = m->embed;
+    } else {
+        ALLOC(m->lm_head, uint16_t, (size_t)c.vocab * h);
+        TRY(fill_rows(m, m->lm_head, 1, c.vocab, h, 1, 0));
+    }
+    ALLOC(m->gf, float, h);
+    TRY(fill_const(m, m->gf, 1.f, h));
+    m->layers.resize(c.n_layers);
+    for (int l = 0; l < c.n_layers; ++l) {
+        LayerWeights &w = m->layers[l];
+        const uint32_t t = 16u * (uint32_t)(l + 1);
+        ALLOC(w.wqkv, uint16_t, (size_t)qkvd * h);
+        TRY(fill_rows(m, w.wqkv, t + TID_WQ, qd, h, 1, 0));
+        TRY(fill_rows(m, w.wqkv + (size_t)qd * h, t + TID_WK, kd, h, 1, 0));
+        TRY(fill_rows(m, w.wqkv + (size_t)(qd + kd) * h, t + TID_WV, kd, h, 1, 0));
+        ALLOC(w.bqkv, float, qkvd);
+        if (c.qkv_bias) {
+            TRY(fill_f32(m, w.bqkv, t + TID_BQ, qd));
+            TRY(fill_f32(m, w.bqkv + qd, t + TID_BK, kd));
+            TRY(fill_f32(m, w.bqkv + qd + kd, t + TID_BV, kd));
+        } else {
+            TRY(fill_const(m, w.bqkv, 0.f, qkvd));
+        }
+        ALLOC(w.wo, uint16_t, (size_t)h * qd);
+        TRY(fill_rows(m, w.wo, t + TID_WO, h, qd, 1, 0));
+        ALLOC(w.wgu, uint16_t, (size_t)2 * f * h);
+        TRY(fill_rows(m, w.wgu, t + TID_WG, f, h, 2, 0));
+        TRY(fill_rows(m, w.wgu, t + TID_WU, f, h, 2, 1));
+        ALLOC(w.wd, uint16_t, (size_t)h * f);
+        TRY(fill_rows(m, w.wd, t + TID_WD, h, f, 1, 0));
+        ALLOC(w.g1, float, h);
+        ALLOC(w.g2, float, h);
+        TRY(fill_const(m, w.g1, 1.f, h));
+        TRY(fill_const(m, w.g2, 1.f, h));
+    }
+    {
+        const int64_t per_layer = 2ll * ((int64_t)qkvd * h + (int64_t)h * qd + 3ll * f * h) + 4ll * qkvd * (c.qkv_bias ? 1 : 0) + 8ll * h;
+        m->weight_bytes = c.n_layers * per_layer + 4ll * h + 2ll * (int64_t)c.vocab * h;
+    }
+    // rotary frequencies theta^(-2j/D), in double
+    {
+        std::vector<double> fr(D / 2);
+        for (int j = 0; j < D / 2; ++j) fr[j] = std::pow((double)c.rope_theta, -2.0 * (double)j / (double)D);
+        ALLOC(m->inv_freq, double, D / 2);
+        CK(cudaMemcpyAsync(m->inv_freq, fr.data(), fr.size() * sizeof(double), cudaMemcpyHostToDevice, m->stream));
+        CK(cudaStreamSynchronize(m->stream));
+    }
+
+    // ---- paged KV ----
+    m->page_shift = c.page_size == 16 ? 4 : c.page_size == 32 ? 5 : 6;
+    m->n_pages = (c.max_tokens + c.page_size - 1) / c.page_size + c.max_seqs;
+    m->pages_per_seq = (c.max_tokens + c.page_size - 1) / c.page_size + 1;
+    m->pool_layer_stride = (size_t)m->n_pages * c.n_kv_heads * c.page_size * D;
+    ALLOC(m->kpool, uint16_t, m->pool_layer_stride * c.n_layers);
+    ALLOC(m->vpool, uint16_t, m->pool_layer_stride * c.n_layers);
+    ALLOC(m->block_tab, int32_t, (size_t)c.max_seqs * m->pages_per_seq);
+    CK(cudaMemsetAsync(m->block_tab, 0, (size_t)c.max_seqs * m->pages_per_seq * sizeof(int32_t), m->stream));
+    m->free_pages.resize(m->n_pages);
+    for (int i = 0; i < m->n_pages; ++i) m->free_pages[i] = m->n_pages - 1 - i;
+    m->seq_pages.assign(c.max_seqs, {});
+    m->seq_len.assign(c.max_seqs, 0);
+    m->seq_used.assign(c.max_seqs, 0);
+
+    // ---- scratch ----
+    m->max_rows = 1024;
+    m->max_splits = (2 * m->sm_count + c.n_kv_heads - 1) / c.n_kv_heads;
+    ALLOC(m->X, float, (size_t)m->max_rows * h);
+    ALLOC(m->XN, uint16_t, 2 * (size_t)m->max_rows * h);
+    ALLOC(m->QKV, float, (size_t)m->max_rows * qkvd);
+    ALLOC(m->ATT, float, qd);
+    ALLOC(m->ATTb, uint16_t, 2 * (size_t)m->max_rows * qd);
+    ALLOC(m->ACT, float, f);
+    ALLOC(m->ACTb, uint16_t, 2 * (size_t)m->max_rows * f);
+    ALLOC(m->cs, float2, (size_t)m->max_rows * (D / 2));
+    ALLOC(m->logits, float, c.vocab);
+    ALLOC(m->part_o, float, (size_t)c.n_q_heads * m->max_splits * D);
+    ALLOC(m->part_ml, float, (size_t)c.n_q_heads * m->max_splits * 2);
+    ALLOC(m->tickets, int32_t, (size_t)m->max_rows * c.n_kv_heads + 1);
+    CK(cudaMemsetAsync(m->tickets, 0, ((size_t)m->max_rows * c.n_kv_heads + 1) * sizeof(int32_t), m->stream));
+    ALLOC(m->amax_val, float, kArgmaxBlocks);
+    ALLOC(m->amax_idx, int32_t, kArgmaxBlocks);
+    ALLOC(m->tokbuf, int32_t, m->max_rows);
+    ALLOC(m->desc, StepDesc, 1);
+    ALLOC(m->status, int32_t, 1);
+    CK(cudaMemsetAsync(m->status, 0, sizeof(int32_t), m->stream));
+#undef ALLOC
+    CK(cudaStreamSynchronize(m->stream));
+    return ST_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// paged KV bookkeeping (host)
+// ------------------------------------------------------------------------------------------------
+
+static int seq_reserve(st_model *m, int slot, int n_tokens)
+{
+    if (slot < 0 || slot >= m->cfg.max_seqs || !m->seq_used[slot] || n_tokens < 0) return ST_ERR_ARG;
+    const int need = (n_tokens + m->cfg.page_size - 1) / m->cfg.page_size;
+    if (need > m->pages_per_seq) return ST_ERR_KV_FULL;
+    std::vector<int32_t> &pg = m->seq_pages[slot];
+    const int have = (int)pg.size();
+    if (need <= have) return ST_OK;
+    if ((int)m->free_pages.size() < need - have) return ST_ERR_KV_FULL;
+    for (int i = have; i < need; ++i) {
+        pg.push_back(m->free_pages.back());
+        m->free_pages.pop_back();
+    }
+    CK(cudaMemcpyAsync(m->block_tab + (size_t)slot * m->pages_per_seq + have, pg.data() + have,
+                       (size_t)(need - have) * sizeof(int32_t), cudaMemcpyHostToDevice, m->stream));
+    return ST_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// one pass of one model
+// ------------------------------------------------------------------------------------------------
+
+struct SampleCtx {          // what follows the LM head of an emitting pass
+    float *logits_out;      // where the logits go (model scratch when null)
+    int32_t *argmax_out;    // plain decode
+    int32_t vlimit;         // 0 = whole vocabulary
+    GenState *gen;          // generation state (device) or null
+    GenBuffers buf;
+    StepDesc *desc_small, *desc_large;
+    bool want_argmax;
+};
+
+static KvView kv_view(st_model *m, int layer, int slot)
+{
+    KvView kv;
+    kv.k = m->kpool + (size_t)layer * m->pool_layer_stride;
+    kv.v = m->vpool + (size_t)layer * m->pool_layer_stride;
+    kv.block_tab = m->block_tab + (size_t)slot * m->pages_per_seq;
+    kv.page_size = m->cfg.page_size;
+    kv.page_shift = m->page_shift;
+    kv.n_pages = m->n_pages;
+    kv.n_kv_heads = m->cfg.n_kv_heads;
+    return kv;
+}
+
+static int sample_tail(st_model *m, const StepDesc *desc, const SampleCtx &sc)
+{
+    const st_config &c = m->cfg;
+    GemvParams g{};
+    g.W = m->lm_head; g.x = m->X; g.gain = m->gf; g.bias = nullptr;
+    g.y = sc.logits_out ? sc.logits_out : m->logits;
+    g.desc = desc; g.N = c.vocab; g.K = c.hidden; g.x_row = -1; g.eps = c.rms_eps;
+    CK((launch_gemv<PRO_NORM, EPI_STORE>(g, m->stream, m->sm_count)));
+    if (sc.want_argmax) {
+        ArgmaxParams a{};
+        a.logits = g.y;
+        a.limit = sc.vlimit > 0 ? sc.vlimit : c.vocab;
+        a.part_val = m->amax_val; a.part_idx = m->amax_idx;
+        a.ticket = m->tickets + (size_t)m->max_rows * c.n_kv_heads;
+        a.argmax_out = sc.argmax_out;
+        a.gen = sc.gen; a.buf = sc.buf; a.desc_small = sc.desc_small; a.desc_large = sc.desc_large;
+        a.status = m->status;
+        argmax_router_kernel<<<kArgmaxBlocks, 256, 0, m->stream>>>(a);
+        ++g_launches;
+        CK(cudaGetLastError());
+    }
+    return ST_OK;
+}
+
+// Decode pass: exactly one row.  ctx_upper bounds the number of keys (chooses the key split).
+static int pass_decode(st_model *m, const StepDesc *desc, const int32_t *tok, int slot, int ctx_upper, const SampleCtx &sc)
+{
+    const st_config &c = m->cfg;
+    const int h = c.hidden, D = c.head_dim, qd = c.n_q_heads * D, kd = c.n_kv_heads * D, f = c.ffn;
+    const int G = c.n_q_heads / c.n_kv_heads;
+    cudaStream_t s = m->stream;
+    embed_rope_kernel<<<1, 256, 0, s>>>(desc, tok, m->embed, h, c.vocab, m->X, m->inv_freq, D / 2, m->cs, m->status);
+    ++g_launches;
+    CK(cudaGetLastError());
+    int n_splits = ctx_upper / 128;
+    n_splits = n_splits < 1 ? 1 : n_splits > m->max_splits ? m->max_splits : n_splits;
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerWeights &w = m->layers[l];
+        GemvParams g{};
+        g.W = w.wqkv; g.x = m->X; g.gain = w.g1; g.bias = w.bqkv; g.y = m->QKV; g.desc = nullptr;
+        g.N = qd + 2 * kd; g.K = h; g.x_row = 0; g.eps = c.rms_eps;
+        CK((launch_gemv<PRO_NORM, EPI_STORE>(g, s, m->sm_count)));
+        const KvView kv = kv_view(m, l, slot);
+        rope_append_kernel<<<1, 256, 0, s>>>(desc, m->QKV, m->cs, c.n_q_heads, c.n_kv_heads, D, kv, m->status);
+        ++g_launches;
+        CK(cudaGetLastError());
+        AttnParams a{};
+        a.desc = desc; a.qkv = m->QKV; a.kv = kv; a.out_f32 = m->ATT; a.out_hi = a.out_lo = nullptr;
+        a.part_o = m->part_o; a.part_ml = m->part_ml; a.tickets = m->tickets; a.status = m->status;
+        a.Hq = c.n_q_heads; a.n_splits = n_splits; a.scale = 1.f / sqrtf((float)D);
+        CK(launch_attn(a, D, G, dim3(n_splits, c.n_kv_heads, 1), s));
+        g = GemvParams{};
+        g.W = w.wo; g.x = m->ATT; g.y = m->X; g.N = h; g.K = qd; g.x_row = 0;
+        CK((launch_gemv<PRO_PLAIN, EPI_RESADD>(g, s, m->sm_count)));
+        g = GemvParams{};
+        g.W = w.wgu; g.x = m->X; g.gain = w.g2; g.y = m->ACT; g.N = 2 * f; g.K = h; g.x_row = 0; g.eps = c.rms_eps;
+        CK((launch_gemv<PRO_NORM, EPI_SILU>(g, s, m->sm_count)));
+        g = GemvParams{};
+        g.W = w.wd; g.x = m->ACT; g.y = m->X; g.N = h; g.K = f; g.x_row = 0;
+        CK((launch_gemv<PRO_PLAIN, EPI_RESADD>(g, s, m->sm_count)));
+    }
+    return sample_tail(m, desc, sc);
+}
+
+// Multi-row pass: up to m_upper rows (the exact count is desc->m on the device).
+static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int slot, int m_upper, bool emit, const SampleCtx &sc)
+{
+    const st_config &c = m->cfg;
+    const int h = c.hidden, D = c.head_dim, qd = c.n_q_heads * D, kd = c.n_kv_heads * D, f = c.ffn;
+    const int G = c.n_q_heads / c.n_kv_heads;
+    cudaStream_t s = m->stream;
+    if (m_upper > m->max_rows) return ST_ERR_INTERNAL;
+    uint16_t *XN_lo = m->XN + (size_t)m->max_rows * h, *ATT_lo = m->ATTb + (size_t)m->max_rows * qd,
+             *ACT_lo = m->ACTb + (size_t)m->max_rows * f;
+    embed_rope_kernel<<<m_upper, 256, 0, s>>>(desc, tok, m->embed, h, c.vocab, m->X, m->inv_freq, D / 2, m->cs, m->status);
+    ++g_launches;
+    CK(cudaGetLastError());
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerWeights &w = m->layers[l];
+        rmsnorm_rows_kernel<<<m_upper, 256, 0, s>>>(desc, m->X, w.g1, c.rms_eps, h, m->XN, XN_lo);
+        ++g_launches;
+        CK(cudaGetLastError());
+        GemmParams g{};
+        g.desc = desc; g.A_hi = m->XN; g.A_lo = XN_lo; g.W = w.wqkv; g.bias = w.bqkv; g.Yf = m->QKV; g.N = qd + 2 * kd; g.K = h;
+        CK(launch_gemm<GEPI_STORE>(g, m_upper, s));
+        const KvView kv = kv_view(m, l, slot);
+        rope_append_kernel<<<m_upper, 256, 0, s>>>(desc, m->QKV, m->cs, c.n_q_heads, c.n_kv_heads, D, kv, m->status);
+        ++g_launches;
+        CK(cudaGetLastError());
+        AttnParams a{};
+        a.desc = desc; a.qkv = m->QKV; a.kv = kv; a.out_f32 = nullptr; a.out_hi = m->ATTb; a.out_lo = ATT_lo;
+        a.tickets = m->tickets; a.status = m->status;
+        a.Hq = c.n_q_heads; a.n_splits = 1; a.scale = 1.f / sqrtf((float)D);
+        CK(launch_attn(a, D, G, dim3(1, c.n_kv_heads, m_upper), s));
+        g = GemmParams{};
+        g.desc = desc; g.A_hi = m->ATTb; g.A_lo = ATT_lo; g.W = w.wo; g.Yf = m->X; g.N = h; g.K = qd;
+        CK(launch_gemm<GEPI_RESADD>(g, m_upper, s));
+        rmsnorm_rows_kernel<<<m_upper, 256, 0, s>>>(desc, m->X, w.g2, c.rms_eps, h, m->XN, XN_lo);
+        ++g_launches;
+        CK(cudaGetLastError());
+        g = GemmParams{};
+        g.desc = desc; g.A_hi = m->XN; g.A_lo = XN_lo; g.W = w.wgu; g.Yb_hi = m->ACTb; g.Yb_lo = ACT_lo; g.N = 2 * f; g.K = h;
+        CK(launch_gemm<GEPI_SILU>(g, m_upper, s));
+        g = GemmParams{};
+        g.desc = desc; g.A_hi = m->ACTb; g.A_lo = ACT_lo; g.W = w.wd; g.Yf = m->X; g.N = h; g.K = f;
+        CK(launch_gemm<GEPI_RESADD>(g, m_upper, s));
+    }
+    if (emit) return sample_tail(m, desc, sc);
+    return ST_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// C ABI
+// ------------------------------------------------------------------------------------------------
+
+extern "C" {
+
+const char *st_strerror(int status)
+{
+    switch (status) {
+    case ST_OK: return "ok";
+    case ST_ERR_ARG: return "invalid argument";
+    case ST_ERR_OOM: return "out of memory";
+    case ST_ERR_KV_FULL: return "KV cache full";
+    case ST_ERR_VOCAB: return "vocabulary mismatch or token id out of range";
+    case ST_ERR_TIMEOUT: return "device-side wait expired";
+    case ST_ERR_UNSUPPORTED: return "unsupported shape or option";
+    case ST_ERR_INTERNAL: return g_err_text[0] ? g_err_text : "internal error";
+    case ST_ERR_CAPACITY: return "output buffer too small";
+    }
+    return "unknown status";
+}
+
+int st_model_create(const st_config *cfg, uint64_t seed, uint32_t model_tag, void *cuda_stream, st_model **out)
+{
+    if (!out) return ST_ERR_ARG;
+    *out = nullptr;
+    TRY(check_config(cfg));
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev < 1) {
+        cudaGetLastError();
+        snprintf(g_err_text, sizeof g_err_text, "no CUDA device: this library has no CPU path");
+        return ST_ERR_INTERNAL;
+    }
+    st_model *m = new (std::nothrow) st_model();
+    if (!m) return ST_ERR_OOM;
+    m->cfg = *cfg;
+    m->seed = seed;
+    m->tag = model_tag;
+    m->stream = (cudaStream_t)cuda_stream;
+    const int rc = model_build(m);
+    if (rc != ST_OK) {
+        st_model_destroy(m);
+        return rc;
+    }
+    *out = m;
+    return ST_OK;
+}
+
+void st_model_destroy(st_model *m)
+{
+    if (!m) return;
+    cudaStreamSynchronize(m->stream);
+    for (void *p : m->allocations) {
+        if (m->cfg.free) m->cfg.free(p, m->cfg.alloc_user);
+        else cudaFree(p);
+    }
+    delete m;
+}
+
+int64_t st_weight_bytes(const st_model *m) { return m ? m->weight_bytes : 0; }
+
+int64_t st_kv_bytes_per_token(const st_model *m)
+{
+    return m ? 4ll * m->cfg.n_layers * m->cfg.n_kv_heads * m->cfg.head_dim : 0;
+}
+
+int64_t st_kernel_launches(void) { return g_launches; }
+
+int st_seq_alloc(st_model *m, int32_t *slot_out)
+{
+    if (!m || !slot_out) return ST_ERR_ARG;
+    for (int i = 0; i < m->cfg.max_seqs; ++i)
+        if (!m->seq_used[i]) {
+            m->seq_used[i] = 1;
+            m->seq_len[i] = 0;
+            *slot_out = i;
+            return ST_OK;
+        }
+    return ST_ERR_KV_FULL;
+}
+
+int st_seq_free(st_model *m, int32_t slot)
+{
+    if (!m || slot < 0 || slot >= m->cfg.max_seqs || !m->seq_used[slot]) return ST_ERR_ARG;
+    for (int32_t p : m->seq_pages[slot]) m->free_pages.push_back(p);
+    m->seq_pages[slot].clear();
+    m->seq_used[slot] = 0;
+    m->seq_len[slot] = 0;
+    return ST_OK;
+}
+
+int st_seq_reserve(st_model *m, int32_t slot, int32_t n_tokens)
+{
+    if (!m) return ST_ERR_ARG;
+    return seq_reserve(m, slot, n_tokens);
+}
+
+int st_kv_len(st_model *m, int32_t slot, int32_t *len_out)
+{
+    if (!m || !len_out || slot < 0 || slot >= m->cfg.max_seqs || !m->seq_used[slot]) return ST_ERR_ARG;
+    CK(cudaStreamSynchronize(m->stream));
+    *len_out = m->seq_len[slot];
+    return ST_OK;
+}
+
+int st_kv_truncate(st_model *m, int32_t slot, int32_t new_len)
+{
+    if (!m || slot < 0 || slot >= m->cfg.max_seqs || !m->seq_used[slot] || new_len < 0) return ST_ERR_ARG;
+    if (new_len < m->seq_len[slot]) m->seq_len[slot] = new_len;
+    return ST_OK;
+}
+
+int st_last_device_status(st_model *m)
+{
+    if (!m) return ST_ERR_ARG;
+    int32_t v = 0;
+    CK(cudaMemcpyAsync(&v, m->status, sizeof v, cudaMemcpyDeviceToHost, m->stream));
+    CK(cudaStreamSynchronize(m->stream));
+    return v;
+}
+
+int st_fill_tensor_bf16(uint64_t seed, uint32_t model_tag, uint32_t tid, uint64_t idx0, uint64_t n, uint16_t *out_dev, void *cuda_stream)
+{
+    if (!out_dev) return ST_ERR_ARG;
+    if (n == 0) return ST_OK;
+    const uint64_t key = tensor_stream_key(seed, model_tag, tid);
+    // n "rows" of one column starting at row idx0: element index = idx0 + r
+    uint64_t blocks = (n + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    fill_bf16_kernel<<<(int)blocks, 256, 0, (cudaStream_t)cuda_stream>>>(out_dev, key, idx0, n, 1, 1, 0);
+    ++g_launches;
+    CK(cudaGetLastError());
+    return ST_OK;
+}
+
+int st_time_gemv(st_model *m, int32_t which, int32_t iters, double *seconds_out)
+{
+    if (!m || !seconds_out || iters < 1 || which < 0 || which > 4) return ST_ERR_ARG;
+    const st_config &c = m->cfg;
+    const int h = c.hidden, D = c.head_dim, qd = c.n_q_heads * D, kd = c.n_kv_heads * D, f = c.ffn;
+    cudaEvent_t e0, e1;
+    CK(cudaEventCreate(&e0));
+    CK(cudaEventCreate(&e1));
+    CK(cudaMemsetAsync(m->X, 0, (size_t)h * sizeof(float), m->stream));
+    CK(cudaMemsetAsync(m->ATT, 0, (size_t)qd * sizeof(float), m->stream));
+    CK(cudaMemsetAsync(m->ACT, 0, (size_t)f * sizeof(float), m->stream));
+    for (int rep = 0; rep < 2; ++rep) {   // the first round warms up
+        if (rep == 1) CK(cudaEventRecord(e0, m->stream));
+        for (int i = 0; i < iters; ++i) {
+            const LayerWeights &w = m->layers[i % c.n_layers];
+            GemvParams g{};
+            g.x_row = 0; g.eps = c.rms_eps;
+            cudaError_t e = cudaSuccess;
+            switch (which) {
+            case 0: g.W = w.wqkv; g.x = m->X; g.gain = w.g1; g.bias = w.bqkv; g.y = m->QKV; g.N = qd + 2 * kd; g.K = h;
+                    e = launch_gemv<PRO_NORM, EPI_STORE>(g, m->stream, m->sm_count); break;
+            case 1: g.W = w.wo; g.x = m->ATT; g.y = m->X; g.N = h; g.K = qd;
+                    e = launch_gemv<PRO_PLAIN, EPI_RESADD>(g, m->stream, m->sm_count); break;
+            case 2: g.W = w.wgu; g.x = m->X; g.gain = w.g2; g.y = m->ACT; g.N = 2 * f; g.K = h;
+                    e = launch_gemv<PRO_NORM, EPI_SILU>(g, m->stream, m->sm_count); break;
+            case 3: g.W = w.wd; g.x = m->ACT; g.y = m->X; g.N = h; g.K = f;
+                    e = launch_gemv<PRO_PLAIN, EPI_RESADD>(g, m->stream, m->sm_count); break;
+            default: g.W = m->lm_head; g.x = m->X; g.gain = m->gf; g.y = m->logits; g.N = c.vocab; g.K = h;
+                    e = launch_gemv<PRO_NORM, EPI_STORE>(g, m->stream, m->sm_count); break;
+            }
+            CK(e);
+        }
+    }
+    CK(cudaEventRecord(e1, m->stream));
+    CK(cudaEventSynchronize(e1));
+    float ms = 0.f;
+    CK(cudaEventElapsedTime(&ms, e0, e1));
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    *seconds_out = (double)ms * 1e-3 / iters;
+    return ST_OK;
+}
+
+int st_prefill(st_model *m, int32_t slot, const int32_t *tokens_host, int32_t n, float *last_logits_dev)
+{
+    if (!m || !tokens_host || n < 1 || slot < 0 || slot >= m->cfg.max_seqs || !m->seq_used[slot]) return ST_ERR_ARG;
+    for (int i = 0; i < n; ++i)
+        if ((unsigned)tokens_host[i] >= (unsigned)m->cfg.vocab) return ST_ERR_VOCAB;
+    TRY(seq_reserve(m, slot, m->seq_len[slot] + n));
+    for (int done = 0; done < n;) {
+        const int rows = n - done < m->max_rows ? n - done : m->max_rows;
+        const bool last = done + rows == n;
+        StepDesc d{m->seq_len[slot], rows, 0, last ? 1 : 0};
+        CK(cudaMemcpyAsync(m->tokbuf, tokens_host + done, (size_t)rows * sizeof(int32_t), cudaMemcpyHostToDevice, m->stream));
+        CK(cudaMemcpyAsync(m->desc, &d, sizeof d, cudaMemcpyHostToDevice, m->stream));
+        SampleCtx sc{};
+        sc.logits_out = last_logits_dev;
+        sc.want_argmax = false;
+        const bool emit = last && last_logits_dev != nullptr;
+        if (rows == 1 && emit) TRY(pass_decode(m, m->desc, m->tokbuf, slot, d.pos0 + 1, sc));
+        else TRY(pass_rows(m, m->desc, m->tokbuf, slot, rows, emit, sc));
+        m->seq_len[slot] += rows;
+        done += rows;
+        // the staging buffer and descriptor are reused by the next chunk
+        if (!last) CK(cudaStreamSynchronize(m->stream));
+    }
+    return ST_OK;
+}
+
+int st_decode_step(st_model *m, const int32_t *slots_host, const int32_t *tokens_dev, int32_t batch, float *logits_dev, int32_t *argmax_dev)
+{
+    if (!m || !slots_host || !tokens_dev || batch < 1) return ST_ERR_ARG;
+    for (int i = 0; i < batch; ++i) {
+        const int slot = slots_host[i];
+        if (slot < 0 || slot >= m->cfg.max_seqs || !m->seq_used[slot]) return ST_ERR_ARG;
+        for (int j = 0; j < i; ++j)
+            if (slots_host[j] == slot) return ST_ERR_ARG;
+    }
+    for (int i = 0; i < batch; ++i) {
+        const int slot = slots_host[i];
+        TRY(seq_reserve(m, slot, m->seq_len[slot] + 1));
+        StepDesc d{m->seq_len[slot], 1, i, 1};
+        CK(cudaMemcpyAsync(m->desc, &d, sizeof d, cudaMemcpyHostToDevice, m->stream));
+        SampleCtx sc{};
+        sc.logits_out = logits_dev ? logits_dev + (size_t)i * m->cfg.vocab : nullptr;
+        sc.argmax_out = argmax_dev ? argmax_dev + i : nullptr;
+        sc.want_argmax = argmax_dev != nullptr;
+        TRY(pass_decode(m, m->desc, tokens_dev, slot, d.pos0 + 1, sc));
+        m->seq_len[slot] += 1;
+        // the descriptor is rewritten for the next sequence
+        if (i + 1 < batch) CK(cudaStreamSynchronize(m->stream));
+    }
+    return ST_OK;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// generation
+// ------------------------------------------------------------------------------------------------
+
+namespace {
+
+struct DevArena {  // raw device allocations of one generation call, released on scope exit
+    std::vector<void *> ptrs;
+    ~DevArena()
+    {
+        for (void *p : ptrs) cudaFree(p);
+    }
+    template <class T>
+    T *get(size_t n)
+    {
+        void *p = nullptr;
+        if (cudaMalloc(&p, (n ? n : 1) * sizeof(T)) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        ptrs.push_back(p);
+        return (T *)p;
+    }
+};
+
+struct SlotGuard {
+    st_model *m;
+    int slot = -1;
+    ~SlotGuard()
+    {
+        if (m && slot >= 0) st_seq_free(m, slot);
+    }
+};
+
+}  // namespace
+
+extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_params *P, const int32_t *prompt,
+                                int32_t prompt_len, const int32_t *force, int32_t n_force, st_spec_result *out)
+{
+    if (!small || !P || !prompt || !out || prompt_len < 1 || P->max_new_tokens < 0 || P->n1 < 1 || n_force < 0) return ST_ERR_ARG;
+    if (P->n_keywords < 0 || (P->n_keywords > 0 && !P->keyword_ids) || (n_force > 0 && !force)) return ST_ERR_ARG;
+    if (large && (large->stream != small->stream || large->device != small->device)) return ST_ERR_ARG;
+    int vshared = small->cfg.vocab;
+    if (large && large->cfg.vocab < vshared) vshared = large->cfg.vocab;
+    const int vlimit = P->vocab_limit > 0 ? P->vocab_limit : vshared;
+    if (vlimit > vshared) return ST_ERR_VOCAB;
+    for (int i = 0; i < prompt_len; ++i)
+        if ((unsigned)prompt[i] >= (unsigned)vlimit) return ST_ERR_VOCAB;
+    for (int i = 0; i < n_force; ++i)
+        if (force[i] >= vlimit) return ST_ERR_VOCAB;
+    for (int i = 0; i < P->n_keywords; ++i)
+        if ((unsigned)P->keyword_ids[i] >= (unsigned)vlimit) return ST_ERR_VOCAB;
+    if ((unsigned)P->delimiter_id >= (unsigned)vlimit) return ST_ERR_VOCAB;
+    const int max_new = P->max_new_tokens;
+    if (out->cap_tokens < max_new || (max_new > 0 && (!out->tokens || !out->source))) return ST_ERR_CAPACITY;
+    const int cap_steps = out->cap_steps, cap_handoffs = out->cap_handoffs;
+    if ((cap_steps > 0 && (!out->emission_tokens || !out->emission_source)) || (cap_handoffs > 0 && !out->handoffs)) return ST_ERR_ARG;
+    if (out->logits_trace && (out->trace_n_steps < 0 || out->trace_first_step < 0)) return ST_ERR_ARG;
+    out->n_tokens = out->n_handoffs = out->n_steps = 0;
+    out->kv_len_small = out->kv_len_large = 0;
+    out->seconds = 0.0;
+    out->bytes_algorithmic = 0;
+
+    cudaStream_t s = small->stream;
+    CK(cudaMemsetAsync(small->status, 0, sizeof(int32_t), s));
+    if (large) CK(cudaMemsetAsync(large->status, 0, sizeof(int32_t), s));
+    const int total = prompt_len + max_new + 1;
+    SlotGuard gs{small}, gl{large};
+    TRY(st_seq_alloc(small, &gs.slot));
+    TRY(seq_reserve(small, gs.slot, total));
+    if (large) {
+        TRY(st_seq_alloc(large, &gl.slot));
+        TRY(seq_reserve(large, gl.slot, total));
+    }
+
+    DevArena A;
+    GenBuffers b{};
+    GenState *gen = A.get<GenState>(1);
+    StepDesc *desc2 = A.get<StepDesc>(2);
+    b.tokens = A.get<int32_t>(total);
+    b.source = A.get<uint8_t>(max_new + 1);
+    const int dev_steps = cap_steps > 0 ? cap_steps : 1;
+    b.em_tok = A.get<int32_t>(dev_steps);
+    b.em_fed = A.get<int32_t>(dev_steps);
+    b.em_arg = A.get<int32_t>(dev_steps);
+    b.em_src = A.get<uint8_t>(dev_steps);
+    const int dev_hand = cap_handoffs > 0 ? cap_handoffs : 1;
+    b.handoffs = A.get<int32_t>(3 * (size_t)dev_hand);
+    int32_t *d_force = A.get<int32_t>(n_force);
+    uint8_t *d_cls = A.get<uint8_t>(vlimit);
+    const int trace_n = out->logits_trace ? out->trace_n_steps : 0;
+    float *d_trace = trace_n > 0 ? A.get<float>((size_t)trace_n * vlimit) : nullptr;
+    if (!gen || !desc2 || !b.tokens || !b.source || !b.em_tok || !b.em_fed || !b.em_arg || !b.em_src || !b.handoffs ||
+        !d_force || !d_cls || (trace_n > 0 && !d_trace))
+        return ST_ERR_OOM;
+    b.force = d_force;
+    b.cls = d_cls;
+    b.trace = d_trace;
+
+    std::vector<uint8_t> cls(vlimit, 0);
+    for (int i = 0; i < P->n_keywords; ++i) cls[P->keyword_ids[i]] |= kClsKeyword;
+    GenState g0{};
+    g0.has_large = large ? 1 : 0;
+    g0.pos = prompt_len;
+    g0.delimiter = P->delimiter_id;
+    g0.n1 = P->n1;
+    g0.keep_probe = P->keep_probe;
+    g0.eos = P->eos_id;
+    g0.vlimit = vlimit;
+    g0.max_new = max_new;
+    g0.n_force = n_force;
+    g0.prompt_len = prompt_len;
+    g0.cap_steps = cap_steps;
+    g0.cap_handoffs = cap_handoffs;
+    g0.max_chunk = small->max_rows;
+    if (large && large->max_rows < g0.max_chunk) g0.max_chunk = large->max_rows;
+    g0.trace_first = out->trace_first_step;
+    g0.trace_n = trace_n;
+    g0.done = max_new == 0 ? 1 : 0;
+    CK(cudaMemcpyAsync(gen, &g0, sizeof g0, cudaMemcpyHostToDevice, s));
+    CK(cudaMemcpyAsync(b.tokens, prompt, (size_t)prompt_len * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+    if (n_force) CK(cudaMemcpyAsync(d_force, force, (size_t)n_force * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+    CK(cudaMemcpyAsync(d_cls, cls.data(), (size_t)vlimit, cudaMemcpyHostToDevice, s));
+    StepDesc *desc_small = desc2, *desc_large = desc2 + 1;
+    plan_first_pass_kernel<<<1, 1, 0, s>>>(gen, desc_small, desc_large);
+    ++g_launches;
+    CK(cudaGetLastError());
+
+    cudaEvent_t ev0, ev1;
+    CK(cudaEventCreate(&ev0));
+    CK(cudaEventCreate(&ev1));
+    CK(cudaEventRecord(ev0, s));
+
+    // Pass loop.  The host reads only the shape of the next pass (which model, how many rows,
+    // whether it samples) -- enough to size the launch; tokens stay on the device.
+    int64_t bytes = 0;
+    GenState gh = g0;
+    int rc = ST_OK;
+    const int64_t pass_cap = 4ll * (max_new + 2) + (prompt_len / g0.max_chunk + 2) * 4ll;
+    for (int64_t pass = 0; pass < pass_cap; ++pass) {
+        if (cudaMemcpyAsync(&gh, gen, sizeof gh, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            cudaStreamSynchronize(s) != cudaSuccess) {
+            set_error_text("generation state readback", cudaGetLastError());
+            rc = ST_ERR_INTERNAL;
+            break;
+        }
+        if (gh.done) break;
+        st_model *m = gh.next_model ? large : small;
+        const int slot = gh.next_model ? gl.slot : gs.slot;
+        StepDesc *d = gh.next_model ? desc_large : desc_small;
+        SampleCtx sc{};
+        sc.vlimit = vlimit;
+        sc.gen = gen;
+        sc.buf = b;
+        sc.desc_small = desc_small;
+        sc.desc_large = desc_large;
+        sc.want_argmax = true;
+        const int ctx_after = gh.kv_len[gh.next_model] + gh.next_m;
+        if (gh.next_m == 1 && gh.next_emit) rc = pass_decode(m, d, b.tokens, slot, ctx_after, sc);
+        else rc = pass_rows(m, d, b.tokens, slot, gh.next_m, gh.next_emit != 0, sc);
+        if (rc != ST_OK) break;
+        if (!gh.next_emit) {
+            advance_ingest_kernel<<<1, 1, 0, s>>>(gen, desc_small, desc_large);
+            ++g_launches;
+            if (cudaGetLastError() != cudaSuccess) { rc = ST_ERR_INTERNAL; break; }
+        }
+        bytes += m->weight_bytes + st_kv_bytes_per_token(m) * (int64_t)ctx_after;
+    }
+    cudaEventRecord(ev1, s);
+    cudaStreamSynchronize(s);
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, ev0, ev1);
+    cudaEventDestroy(ev0);
+    cudaEventDestroy(ev1);
+    if (rc != ST_OK) return rc;
+    if (!gh.done) return ST_ERR_INTERNAL;
+
+    // ---- results ----
+    out->n_tokens = gh.generated;
+    out->n_steps = gh.step;
+    out->n_handoffs = gh.n_handoffs;
+    out->kv_len_small = gh.kv_len[0];
+    out->kv_len_large = gh.kv_len[1];
+    out->seconds = ms * 1e-3;
+    out->bytes_algorithmic = bytes;
+    const int n_steps = gh.step < cap_steps ? gh.step : cap_steps;
+    const int n_hand = gh.n_handoffs < cap_handoffs ? gh.n_handoffs : cap_handoffs;
+    if (gh.generated > 0) {
+        CK(cudaMemcpyAsync(out->tokens, b.tokens + prompt_len, (size_t)gh.generated * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+        CK(cudaMemcpyAsync(out->source, b.source, (size_t)gh.generated, cudaMemcpyDeviceToHost, s));
+    }
+    if (n_steps > 0) {
+        CK(cudaMemcpyAsync(out->emission_tokens, b.em_tok, (size_t)n_steps * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+        CK(cudaMemcpyAsync(out->emission_source, b.em_src, (size_t)n_steps, cudaMemcpyDeviceToHost, s));
+        if (out->emission_fed) CK(cudaMemcpyAsync(out->emission_fed, b.em_fed, (size_t)n_steps * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+        if (out->emission_argmax) CK(cudaMemcpyAsync(out->emission_argmax, b.em_arg, (size_t)n_steps * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    }
+    if (n_hand > 0) CK(cudaMemcpyAsync(out->handoffs, b.handoffs, (size_t)n_hand * 3 * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    if (trace_n > 0) CK(cudaMemcpyAsync(out->logits_trace, d_trace, (size_t)trace_n * vlimit * sizeof(float), cudaMemcpyDeviceToHost, s));
+    CK(cudaStreamSynchronize(s));
+    int32_t dev_status = 0;
+    CK(cudaMemcpy(&dev_status, small->status, sizeof dev_status, cudaMemcpyDeviceToHost));
+    if (large) {
+        int32_t s2 = 0;
+        CK(cudaMemcpy(&s2, large->status, sizeof s2, cudaMemcpyDeviceToHost));
+        dev_status |= s2;
+    }
+    if (dev_status & DEV_LOG_FULL) return ST_ERR_CAPACITY;
+    if (dev_status & DEV_BAD_TOKEN) return ST_ERR_VOCAB;
+    if (dev_status) return ST_ERR_INTERNAL;
+    return ST_OK;
+}
