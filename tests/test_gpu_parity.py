@@ -1,0 +1,231 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element."""
+import numpy as np
+import pytest
+
+from paper_2504_12329_b200 import workloads as W
+from parity_utils import MARGIN, assert_logits_close, shape_dict
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2504_12329_b200 import binding
+    binding.lib()
+    return binding
+
+
+def test_seeded_weights_bit_identical(B, oracle):
+    for seed, tag, tid, idx0, n in [(0, 0, 0, 0, 100_003), (0, 1, 17, 0, 4096), (5, 2, 16 * 64 + 11, 123_456_789_012, 70_001),
+                                    (0, 0, 1, (1 << 33) + 5, 999)]:
+        out = torch.empty(n, dtype=torch.int16, device="cuda")
+        B.st_fill_tensor_bf16(seed, tag, tid, idx0, n, out)
+        torch.cuda.synchronize()
+        got = out.cpu().numpy().view(np.uint16)
+        want = (oracle.fill_tensor(seed, tag, tid, idx0, n).view(np.uint32) >> 16).astype(np.uint16)
+        assert np.array_equal(got, want)
+
+
+def _teacher_forced(B, oracle, shape, seed, tag, chunks, n_decode, page_size=64, tok_seed=3):
+    """Prefill in the given chunks, then n_decode single steps, all tokens given; compare every logits row."""
+    rng = np.random.default_rng(tok_seed)
+    total = sum(chunks) + n_decode
+    tokens = rng.integers(0, shape["vocab"], size=total).astype(np.int32)
+    om = oracle.Model(oracle.Config(**shape), seed, tag)
+    okv = oracle.KV(om, total + 1)
+    gm = B.Model(shape, seed=seed, tag=tag, max_seqs=2, max_tokens=2 * total + 64, page_size=page_size)
+    slot = gm.st_seq_alloc()
+    logits = torch.empty(shape["vocab"], dtype=torch.float32, device="cuda")
+    worst = (0.0, 1.0)
+    i = 0
+    for c in chunks:
+        want = okv.forward(tokens[i:i + c])
+        gm.st_prefill(slot, tokens[i:i + c], logits)
+        torch.cuda.synchronize()
+        e, cs = assert_logits_close(logits.cpu().numpy(), want, f"prefill chunk at {i} (+{c})")
+        worst = (max(worst[0], e), min(worst[1], cs))
+        i += c
+        assert gm.st_kv_len(slot) == i
+    tok_dev = torch.empty(1, dtype=torch.int32, device="cuda")
+    amax = torch.empty(1, dtype=torch.int32, device="cuda")
+    for _ in range(n_decode):
+        want = okv.forward(tokens[i:i + 1])
+        tok_dev.copy_(torch.from_numpy(tokens[i:i + 1]))
+        gm.st_decode_step([slot], tok_dev, logits, amax)
+        torch.cuda.synchronize()
+        got = logits.cpu().numpy()
+        e, cs = assert_logits_close(got, want, f"decode at {i}")
+        worst = (max(worst[0], e), min(worst[1], cs))
+        gi, margin = oracle.argmax(want)
+        if margin >= MARGIN:
+            assert int(amax.item()) == gi
+        assert int(amax.item()) == int(np.argmax(got))       # lowest-id argmax of its own logits
+        i += 1
+    assert gm.st_last_device_status() == 0
+    gm.close()
+    print(f"{shape['hidden']}x{shape['n_layers']}: worst max-abs {worst[0]:.4f}, worst cosine {worst[1]:.7f}")
+    return worst
+
+
+@pytest.mark.parametrize("shape,tag", [(W.TINY_S, 0), (W.TINY_L, 1)])
+@pytest.mark.parametrize("page_size", [16, 64])
+def test_tiny_models_teacher_forced(B, oracle, shape, tag, page_size):
+    # chunk sizes span one row, a ragged tile, several tiles and a page boundary
+    _teacher_forced(B, oracle, shape_dict(shape), 0, tag, chunks=[1, 2, 37, 65, 130], n_decode=20, page_size=page_size)
+
+
+def test_decode_from_empty_cache_and_long_context(B, oracle):
+    # first token through the decode path, then enough context to use several key splits
+    _teacher_forced(B, oracle, shape_dict(W.TINY_S), 1, 0, chunks=[1], n_decode=3)
+    _teacher_forced(B, oracle, shape_dict(W.TINY_S), 1, 0, chunks=[700], n_decode=4)
+
+
+@pytest.mark.parametrize("shape", [W.QWEN_1P5B, W.QWEN_7B, W.QWEN_32B])
+def test_full_width_two_layers(B, oracle, shape):
+    """Full hidden/FFN/vocabulary widths of the large shapes (so every kernel runs in the launch
+    configuration the full model uses), two layers deep so that the oracle finishes in seconds."""
+    _teacher_forced(B, oracle, shape_dict(shape, n_layers=2), 0, 3, chunks=[19], n_decode=3)
+
+
+def test_qwen1p5b_full_depth(B, oracle):
+    """All 28 layers of the 1.5B shape: prompt prefill, a catch-up sized chunk and decode steps."""
+    _teacher_forced(B, oracle, shape_dict(W.QWEN_1P5B), 0, 0, chunks=[24, 20], n_decode=4)
+
+
+def _gen_both(B, oracle, small_shape, large_shape, prompt, force, *, n1, keep, max_new, trace=0, eos=-1, page_size=64):
+    os_ = oracle.Model(oracle.Config(**small_shape), 0, 0)
+    ol = oracle.Model(oracle.Config(**large_shape), 0, 1) if large_shape else None
+    want = oracle.generate_spec(os_, ol, prompt, delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=n1,
+                                keep_probe=keep, eos_id=eos, max_new_tokens=max_new, force=force, trace_n_steps=trace)
+    cap = len(prompt) + max_new + 64
+    gs = B.Model(small_shape, seed=0, tag=0, max_tokens=cap, page_size=page_size)
+    gl = B.Model(large_shape, seed=0, tag=1, max_tokens=cap, page_size=page_size) if large_shape else None
+    got = B.st_generate_spec(gs, gl, prompt, delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=n1,
+                             keep_probe=keep, eos_id=eos, max_new_tokens=max_new, force=force, trace_n_steps=trace)
+    gs.close()
+    if gl:
+        gl.close()
+    return want, got
+
+
+def _assert_routing_equal(want, got):
+    assert got.tokens.tolist() == want.tokens.tolist()
+    assert got.source.tolist() == want.source.tolist()
+    assert got.handoffs == want.handoffs
+    assert got.emission_tokens.tolist() == want.emission_tokens.tolist()
+    assert got.emission_source.tolist() == want.emission_source.tolist()
+    assert got.emission_fed.tolist() == want.emission_fed.tolist()
+    assert (got.kv_len_small, got.kv_len_large) == (want.kv_len_small, want.kv_len_large)
+    assert got.n_steps == len(want.emission_tokens)
+
+
+@pytest.mark.parametrize("keep", [False, True])
+def test_hand_traced_stream_on_device(B, oracle, keep):
+    force = [5, 10, 11, 7, 8, 9, 6, 10, 4, 10, 12, 20, 21, 22]
+    want, got = _gen_both(B, oracle, shape_dict(W.TINY_S), shape_dict(W.TINY_L), [1, 2, 3], force, n1=3, keep=keep, max_new=12)
+    _assert_routing_equal(want, got)
+    if not keep:
+        assert got.tokens.tolist() == [5, 10, 7, 8, 9, 6, 10, 4, 10, 20, 21, 22]
+        assert got.handoffs == [(5, 2, 5), (12, 10, 5)]
+
+
+@pytest.mark.parametrize("keep", [False, True])
+@pytest.mark.parametrize("n1", [4, 20])
+def test_tiny_pair_fully_forced_routing_and_logits(B, oracle, keep, n1):
+    """Tiny pair, 32-token prompt, 128 tokens, every step forced: routing is bit-exact and every
+    step's logits are within tolerance."""
+    prompt = W.prompt_ids(100, 32, 1024)
+    force = W.full_forcing(101, 300, 1024, mean_interval=8, keyword_rate=0.5)
+    want, got = _gen_both(B, oracle, shape_dict(W.TINY_S), shape_dict(W.TINY_L), prompt, force, n1=n1, keep=keep,
+                          max_new=128, trace=300)
+    _assert_routing_equal(want, got)
+    assert len(want.handoffs) >= 2
+    n = len(want.emission_tokens)
+    for t in range(n):
+        assert_logits_close(got.logits_trace[t], want.logits_trace[t], f"step {t}")
+        if want.emission_margin[t] >= MARGIN:
+            assert got.emission_argmax[t] == want.emission_argmax[t]
+
+
+def test_tiny_pair_free_running(B, oracle):
+    """Tiny pair with the sparse schedule (delimiters/keywords forced, everything else greedy): tokens must
+    match the oracle at every step whose top-2 margin is at least 0.05; after the first low-margin
+    disagreement the comparison continues teacher-forced."""
+    prompt = W.prompt_ids(100, 32, 1024)
+    force = W.forcing_schedule(101, 300, mean_interval=8, keyword_rate=0.5)
+    want, got = _gen_both(B, oracle, shape_dict(W.TINY_S), shape_dict(W.TINY_L), prompt, force, n1=4, keep=False, max_new=128)
+    n = min(len(want.emission_tokens), len(got.emission_tokens))
+    diverged = None
+    for t in range(n):
+        if got.emission_tokens[t] != want.emission_tokens[t]:
+            assert want.emission_margin[t] < MARGIN, f"step {t}: tokens differ at margin {want.emission_margin[t]}"
+            diverged = t
+            break
+    if diverged is None:
+        _assert_routing_equal(want, got)
+    else:
+        forced = want.emission_tokens.copy()
+        want2, got2 = _gen_both(B, oracle, shape_dict(W.TINY_S), shape_dict(W.TINY_L), prompt, forced, n1=4, keep=False, max_new=128)
+        _assert_routing_equal(want2, got2)
+
+
+def test_plain_decode_without_large_model(B, oracle):
+    prompt = W.prompt_ids(7, 16, 1024)
+    want, got = _gen_both(B, oracle, shape_dict(W.TINY_S), None, prompt, None, n1=20, keep=False, max_new=48, trace=48)
+    assert got.handoffs == [] and set(got.source.tolist()) == {0}
+    for t in range(len(want.emission_tokens)):
+        assert_logits_close(got.logits_trace[t], want.logits_trace[t], f"step {t}")
+        if got.emission_tokens[t] != want.emission_tokens[t]:
+            assert want.emission_margin[t] < MARGIN
+            break
+
+
+def test_edge_cases_on_device(B, oracle):
+    S, L = shape_dict(W.TINY_S), shape_dict(W.TINY_L)
+    # delimiter ends the prompt; EOS inside a run; budget ends a run; n1 = 1; re-trigger; zero new tokens
+    for prompt, force, kw in [([4, 10], [12, 30, 31, 32, 33], dict(n1=3, max_new=4)),
+                              ([4, 10], [11, 20, 99, 21], dict(n1=3, max_new=8, eos=99)),
+                              ([4, 10], [11, 20, 21], dict(n1=3, max_new=2)),
+                              ([4, 10], [11, 20, 21, 22], dict(n1=1, max_new=3)),
+                              ([4, 10], [11, 10, 11, 10, 12, 40, 41, 42], dict(n1=3, max_new=6)),
+                              ([4], [], dict(n1=3, max_new=0))]:
+        for keep in (False, True):
+            want, got = _gen_both(B, oracle, S, L, prompt, force if force else None, keep=keep, **kw)
+            _assert_routing_equal(want, got)
+
+
+def test_host_side_errors(B):
+    S = shape_dict(W.TINY_S)
+    m = B.Model(S, max_tokens=128)
+    with pytest.raises(B.StError) as e:
+        B.st_generate_spec(m, None, [1, 2000], delimiter_id=10, keyword_ids=[11], max_new_tokens=4)
+    assert e.value.status == B.ST_ERR_VOCAB
+    with pytest.raises(B.StError) as e:
+        B.st_generate_spec(m, None, [1, 2], delimiter_id=10, keyword_ids=[11], max_new_tokens=4000)
+    assert e.value.status == B.ST_ERR_KV_FULL
+    with pytest.raises(B.StError) as e:
+        B.st_generate_spec(m, None, [1, 2], delimiter_id=10, keyword_ids=[11], max_new_tokens=8, cap_steps=3)
+    assert e.value.status == B.ST_ERR_CAPACITY
+    slot = m.st_seq_alloc()
+    with pytest.raises(B.StError) as e:
+        m.st_seq_alloc()
+    assert e.value.status == B.ST_ERR_KV_FULL
+    with pytest.raises(B.StError) as e:
+        m.st_prefill(slot, [5000])
+    assert e.value.status == B.ST_ERR_VOCAB
+    with pytest.raises(B.StError) as e:
+        m.st_prefill(slot, list(range(400)))
+    assert e.value.status == B.ST_ERR_KV_FULL
+    m.st_seq_free(slot)
+    # the model still works after the refused calls
+    r = B.st_generate_spec(m, None, [1, 2], delimiter_id=10, keyword_ids=[11], max_new_tokens=4)
+    assert len(r.tokens) == 4
+    bad = dict(S, head_dim=48)
+    with pytest.raises(B.StError) as e:
+        B.Model(bad)
+    assert e.value.status == B.ST_ERR_UNSUPPORTED
+    m.close()
