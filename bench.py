@@ -1,0 +1,280 @@
+"""Benchmark: batch-1 Speculative Thinking decode of the 1.5B + 32B pair on one B200.
+
+A step is one whole generation of the workload (prompt prefill, small-model decode, handoffs with
+catch-up prefill, target segments).  Prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2504_12329_b200 import workloads as W
+
+METRIC = "tokens/s batch-1 1.5B+32B spec-thinking decode; % of HBM roofline"
+UNIT = "tokens/s"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "200", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                pass
+        rows = [r for r in self.rows if len(r) >= 6]
+        sm = [float(r[0]) for r in rows if r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in rows if r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[2 + i].lower().startswith("active") for r in rows)]
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None, "reasons": reasons}
+
+
+def cpu_oracle_sample(w: W.Workload, stats: dict | None):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload: decode steps of the small
+    model (all layers) and decode steps of the large model cut to two layers plus its LM head, scaled
+    to the full depth; combined with the workload's pass mix into tokens/s."""
+    import ctypes as C
+    from oracle import oracle as O
+    rng = np.random.default_rng(1)
+    cores = os.cpu_count() or 1
+    om = O.Model(O.Config(**w.small.as_dict()), w.weight_seed, 0)
+    kv = O.KV(om, 64)
+    kv.forward(rng.integers(0, w.small.vocab, 4))
+    n_s = 6
+    t0 = time.perf_counter()
+    for _ in range(n_s):
+        kv.forward(rng.integers(0, w.small.vocab, 1))
+    t_small = (time.perf_counter() - t0) / n_s
+    om.close()
+    t_large = None
+    sample = f"{n_s} decode steps of the {w.small.name} oracle"
+    if w.large is not None:
+        sh = w.large.as_dict()
+        sh["n_layers"] = 2
+        ol = O.Model(O.Config(**sh), w.weight_seed, 1)
+        kv = O.KV(ol, 64)
+        kv.forward(rng.integers(0, w.large.vocab, 2))
+        n_l = 3
+        t0 = time.perf_counter()
+        for _ in range(n_l):
+            kv.forward(rng.integers(0, w.large.vocab, 1))
+        t_with_head = (time.perf_counter() - t0) / n_l
+        t0 = time.perf_counter()
+        for _ in range(n_l):   # the same steps without the LM head (no logits requested)
+            tok = np.ascontiguousarray(rng.integers(0, w.large.vocab, 1), dtype=np.int32)
+            O.lib().orc_forward(ol.h, kv.h, tok.ctypes.data_as(C.c_void_p), 1, 0, None)
+        t_layers2 = (time.perf_counter() - t0) / n_l
+        t_large = t_layers2 / 2 * w.large.n_layers + max(t_with_head - t_layers2, 0.0)
+        ol.close()
+        sample += (f" + {2 * n_l} decode steps of the {w.large.name} oracle cut to 2 layers (with and without LM head), "
+                   f"scaled to {w.large.n_layers} layers")
+    if stats:
+        total = stats["steps_small"] * t_small + stats["steps_large"] * (t_large or 0.0)
+        value = stats["n_tokens"] / total
+        sample += (f"; combined with the run's pass mix ({stats['steps_small']} small, {stats['steps_large']} large passes; "
+                   "a catch-up pass counted as one decode pass)")
+    else:
+        value = 1.0 / t_small
+    return {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+            "s_per_small_step": t_small, "s_per_large_step": t_large}
+
+
+def schedule_stats(w: W.Workload):
+    """Pass mix of the workload from its forcing schedule alone: a replay of the handoff rule on the
+    forced tokens, unforced steps counted as ordinary tokens."""
+    _, force = W.workload_inputs(w)
+    active, remaining, gen, t, last = 0, 0, 0, 0, -1
+    steps = [0, 0]
+    while gen < w.max_new_tokens:
+        tok = int(force[t]) if force is not None and t < len(force) and force[t] >= 0 else -2
+        steps[active] += 1
+        t += 1
+        if w.large is not None and active == 0 and last == W.DELIMITER_ID and tok in W.KEYWORD_IDS:
+            active, remaining = 1, W.N1
+            continue
+        last = tok
+        gen += 1
+        if active == 1:
+            remaining -= 1
+            if remaining == 0:
+                active = 0
+    return {"steps_small": steps[0], "steps_large": steps[1], "n_tokens": gen}
+
+
+def run_reference(args, w):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    stats = schedule_stats(w)
+    vals, base = [], None
+    for _ in range(args.warmup + args.steps):
+        base = cpu_oracle_sample(w, stats)
+        vals.append(base["value"])
+    v = float(np.mean(vals[args.warmup:]))
+    base["value"] = v
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * stats["n_tokens"] / v, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "prompt_len": w.prompt_len, "max_new_tokens": w.max_new_tokens},
+            "cpu_baseline": base,
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--workload", default="qwen1p5b_32b", choices=sorted(W.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = W.CONFIGS[args.workload]
+    if args.impl == "reference":
+        return run_reference(args, w)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2504_12329_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    # The generation is one dependent chain of tokens: it does not shard.  With N > 1 every rank runs
+    # an independent replica of the workload (its own input seed); there is no data-path collective.
+    wl = W.Workload(**{**w.__dict__, "input_seed": w.input_seed + 1000 * rank})
+    prompt, force = W.workload_inputs(wl)
+    cap = wl.prompt_len + wl.max_new_tokens + 64
+    small = B.Model(wl.small.as_dict(), seed=wl.weight_seed, tag=0, max_tokens=cap)
+    large = B.Model(wl.large.as_dict(), seed=wl.weight_seed, tag=1, max_tokens=cap) if wl.large else None
+    kw = dict(delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=W.N1, max_new_tokens=wl.max_new_tokens, force=force)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        B.st_generate_spec(small, large, prompt, **kw)
+    sampler = ClockSampler(local)
+    launches0 = B.st_kernel_launches()
+    barrier()
+    sampler.start()
+    dev_s, e2e_s, results = 0.0, 0.0, []
+    t_region = time.perf_counter()
+    for _ in range(args.steps):
+        t0 = time.perf_counter()
+        r = B.st_generate_spec(small, large, prompt, **kw)   # host buffers in, host buffers out
+        e2e_s += time.perf_counter() - t0
+        dev_s += r.seconds
+        results.append(r)
+    barrier()
+    t_region = time.perf_counter() - t_region
+    clocks = sampler.stop()
+    launches = B.st_kernel_launches() - launches0
+
+    r = results[-1]
+    n_tokens = float(sum(len(x.tokens) for x in results))
+    if world > 1:
+        t = torch.tensor([dev_s, e2e_s], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        n = torch.tensor([n_tokens], dtype=torch.float64, device="cuda")
+        dist.all_reduce(n, op=dist.ReduceOp.SUM)
+        dev_s, e2e_s, n_tokens = float(t[0]), float(t[1]), float(n[0])
+    value = n_tokens / dev_s
+    e2e_value = n_tokens / e2e_s
+
+    peak, peak_kind = measured_peaks()
+    # dominant kernel: the batch-1 gate/up projection of the large model (the largest share of streamed bytes)
+    dom = large if large is not None else small
+    shp = wl.large if wl.large else wl.small
+    gemv_s = dom.st_time_gemv(2, 4 * shp.n_layers)
+    gemv_bytes = 2 * (2 * shp.ffn) * shp.hidden + 4 * shp.hidden * 2 + 4 * shp.ffn
+    achieved = gemv_bytes / gemv_s / 1e9
+    path_gbs = sum(x.bytes_algorithmic for x in results) / sum(x.seconds for x in results) / 1e9
+    steps_small = int((r.emission_source == 0).sum())
+    steps_large = int((r.emission_source == 1).sum())
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * dev_s / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "small": wl.small.name, "large": wl.large.name if wl.large else None,
+                       "prompt_len": wl.prompt_len, "max_new_tokens": wl.max_new_tokens, "n1": W.N1,
+                       "handoffs": len(r.handoffs), "target_share": float(r.source.mean()),
+                       "passes_small": steps_small, "passes_large": steps_large,
+                       "arithmetic": "bf16 weights and KV, fp32 activations and accumulation",
+                       "l2": "inputs larger than L2: every pass streams 3.1 GB (small) or 64 GB (large) of weights",
+                       "multi_gpu": "replicas only" if world > 1 else "single GPU"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT,
+                    "h2d_bytes_per_step": int(prompt.nbytes + (force.nbytes if force is not None else 0) + min(wl.small.vocab, shp.vocab)),
+                    "d2h_bytes_per_step": int(5 * len(r.tokens) + 13 * r.n_steps + 12 * len(r.handoffs) + 80 * r.n_steps)},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "kernel": f"gemv gate/up {shp.name} [{2 * shp.ffn}x{shp.hidden}] bf16",
+                         "peak_source": f"{peak_kind} copy bandwidth", "us_per_launch": gemv_s * 1e6},
+            "path_roofline": {"achieved_gbs": path_gbs, "frac_of_measured_hbm": path_gbs / peak,
+                              "frac_of_nominal_8tbs": path_gbs / 8000.0,
+                              "note": "algorithmic bytes of every pass (weights + KV) / device time of the generation"},
+            "wall_s_timed_region": t_region,
+        }
+        if not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_oracle_sample(wl, {"steps_small": steps_small, "steps_large": steps_large,
+                                                          "n_tokens": len(r.tokens)})
+        print(json.dumps(line), flush=True)
+    small.close()
+    if large:
+        large.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
