@@ -10,7 +10,11 @@
 #include "gemv.cuh"
 #include "prefill_simt.cuh"
 #include "router.cuh"
+#include "tc_gemm.cuh"
 #include "weights.cuh"
+
+#include <cstdlib>
+#include <map>
 
 using namespace st;
 
@@ -39,6 +43,10 @@ static void set_error_text(const char *what, cudaError_t e)
 // 1 = LM head).
 enum { TID_WQ = 1, TID_WK = 2, TID_WV = 3, TID_BQ = 4, TID_BK = 5, TID_BV = 6, TID_WO = 7, TID_WG = 9, TID_WU = 10, TID_WD = 11 };
 
+struct LayerMaps {   // TMA descriptors of one layer's weight matrices
+    CUtensorMap wqkv, wo, wgu, wd;
+};
+
 struct LayerWeights {
     uint16_t *wqkv;  // [(Hq + 2 Hkv) D][h]: q rows, k rows, v rows
     float *bqkv;     // [(Hq + 2 Hkv) D]
@@ -60,6 +68,9 @@ struct st_model {
     uint16_t *embed = nullptr, *lm_head = nullptr;
     float *gf = nullptr;
     std::vector<LayerWeights> layers;
+    std::vector<LayerMaps> maps;
+    std::map<int, CUtensorMap> act_maps;   // key: (buffer * 2 + plane) * 1024 + m_pad
+    bool simt_gemm = false;                // debugging aid: multi-row projections on the CUDA cores
     double *inv_freq = nullptr;
     int64_t weight_bytes = 0;
 
@@ -179,6 +190,83 @@ static cudaError_t launch_gemm(const GemmParams &p, int m_upper, cudaStream_t s)
     return cudaGetLastError();
 }
 
+// ---- TMA descriptors and the tensor-core GEMM launcher ----
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor [rows][K] (K contiguous), boxes of 64 x box_rows elements, 128-byte swizzle,
+// out-of-range elements read as zero.
+static int make_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64_t K, uint32_t box_rows)
+{
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) {
+        snprintf(g_err_text, sizeof g_err_text, "cuTensorMapEncodeTiled is not available");
+        return ST_ERR_INTERNAL;
+    }
+    const cuuint64_t gdim[2] = {K, rows};
+    const cuuint64_t gstride[1] = {K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kTcBlockK, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_err_text, sizeof g_err_text, "cuTensorMapEncodeTiled failed (%d)", (int)r);
+        return ST_ERR_INTERNAL;
+    }
+    return ST_OK;
+}
+
+template <int EPI>
+static int launch_tc_gemm(const CUtensorMap &tw, const CUtensorMap &ta_hi, const CUtensorMap &ta_lo, TcGemmParams p, int m_upper,
+                          int sms, cudaStream_t s)
+{
+    auto kern = tc_gemm_kernel<EPI>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+        attr_set = true;
+    }
+    p.m_pad = (m_upper + 31) / 32 * 32;
+    if (p.m_pad > 256) return ST_ERR_INTERNAL;
+    p.tmem_cols = p.m_pad <= 32 ? 32 : p.m_pad <= 64 ? 64 : p.m_pad <= 128 ? 128 : 256;
+    const int stage_bytes = kTcWBytes + 2 * p.m_pad * kTcBlockK * 2;
+    int stages = (220 * 1024) / stage_bytes;
+    p.stages = stages > 8 ? 8 : stages;
+    const int n_tiles = (p.N + kTcTileW - 1) / kTcTileW;
+    const int kb_total = (p.K + kTcBlockK - 1) / kTcBlockK;
+    int ks = 1;
+    if (EPI != TEPI_SILU) {
+        ks = (sms + n_tiles - 1) / n_tiles;
+        const int ks_max = kb_total / 8 > 1 ? kb_total / 8 : 1;
+        ks = ks > ks_max ? ks_max : ks;
+        ks = ks > 16 ? 16 : ks;
+        const int per = (kb_total + ks - 1) / ks;   // no empty split
+        ks = (kb_total + per - 1) / per;
+    }
+    p.k_splits = ks;
+    if (EPI == TEPI_STORE && ks > 1) CK(cudaMemsetAsync(p.Yf, 0, (size_t)m_upper * p.N * sizeof(float), s));
+    const size_t smem = (size_t)p.stages * stage_bytes + 1024;
+    kern<<<dim3(n_tiles, ks), 192, smem, s>>>(tw, ta_hi, ta_lo, p);
+    ++g_launches;
+    CK(cudaGetLastError());
+    return ST_OK;
+}
+
 // ------------------------------------------------------------------------------------------------
 // model construction
 // ------------------------------------------------------------------------------------------------
@@ -281,6 +369,18 @@ static int model_build(st_model *m)
         TRY(fill_const(m, w.g1, 1.f, h));
         TRY(fill_const(m, w.g2, 1.f, h));
     }
+    m->maps.resize(c.n_layers);
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerWeights &w = m->layers[l];
+        TRY(make_map_bf16(&m->maps[l].wqkv, w.wqkv, qkvd, h, kTcTileW));
+        TRY(make_map_bf16(&m->maps[l].wo, w.wo, h, qd, kTcTileW));
+        TRY(make_map_bf16(&m->maps[l].wgu, w.wgu, 2 * f, h, kTcTileW));
+        TRY(make_map_bf16(&m->maps[l].wd, w.wd, h, f, kTcTileW));
+    }
+    {
+        const char *e = getenv("ST_SIMT_GEMM");
+        m->simt_gemm = e && e[0] == '1';
+    }
     {
         const int64_t per_layer = 2ll * ((int64_t)qkvd * h + (int64_t)h * qd + 3ll * f * h) + 4ll * qkvd * (c.qkv_bias ? 1 : 0) + 8ll * h;
         m->weight_bytes = c.n_layers * per_layer + 4ll * h + 2ll * (int64_t)c.vocab * h;
@@ -310,7 +410,7 @@ static int model_build(st_model *m)
     m->seq_used.assign(c.max_seqs, 0);
 
     // ---- scratch ----
-    m->max_rows = 1024;
+    m->max_rows = 256;   // rows of one multi-row pass = the MMA N limit
     m->max_splits = (2 * m->sm_count + c.n_kv_heads - 1) / c.n_kv_heads;
     ALLOC(m->X, float, (size_t)m->max_rows * h);
     ALLOC(m->XN, uint16_t, 2 * (size_t)m->max_rows * h);
@@ -449,6 +549,42 @@ static int pass_decode(st_model *m, const StepDesc *desc, const int32_t *tok, in
     return sample_tail(m, desc, sc);
 }
 
+// TMA descriptor of one activation plane ([max_rows][K] bf16) with a box of m_pad rows; cached per model.
+static int act_map(st_model *m, int buffer, int plane, const uint16_t *base, int K, int m_pad, const CUtensorMap **out)
+{
+    const int key = (buffer * 2 + plane) * 1024 + m_pad;
+    auto it = m->act_maps.find(key);
+    if (it == m->act_maps.end()) {
+        CUtensorMap map;
+        TRY(make_map_bf16(&map, base, (uint64_t)m->max_rows, (uint64_t)K, (uint32_t)m_pad));
+        it = m->act_maps.emplace(key, map).first;
+    }
+    *out = &it->second;
+    return ST_OK;
+}
+
+// One multi-row projection: tensor cores (default) or the CUDA-core tiled GEMM (debugging aid).
+template <int EPI>
+static int rows_gemm(st_model *m, const StepDesc *desc, int m_upper, int buffer, const uint16_t *A_hi, const uint16_t *A_lo,
+                     const CUtensorMap &tw, const uint16_t *W, const float *bias, float *Yf, uint16_t *Yb_hi, uint16_t *Yb_lo,
+                     int N, int K)
+{
+    if (m->simt_gemm) {
+        GemmParams g{};
+        g.desc = desc; g.A_hi = A_hi; g.A_lo = A_lo; g.W = W; g.bias = bias; g.Yf = Yf; g.Yb_hi = Yb_hi; g.Yb_lo = Yb_lo;
+        g.N = N; g.K = K;
+        CK(launch_gemm<EPI>(g, m_upper, m->stream));
+        return ST_OK;
+    }
+    const int m_pad = (m_upper + 31) / 32 * 32;
+    const CUtensorMap *ta_hi, *ta_lo;
+    TRY(act_map(m, buffer, 0, A_hi, K, m_pad, &ta_hi));
+    TRY(act_map(m, buffer, 1, A_lo, K, m_pad, &ta_lo));
+    TcGemmParams p{};
+    p.desc = desc; p.bias = bias; p.Yf = Yf; p.Yb_hi = Yb_hi; p.Yb_lo = Yb_lo; p.status = m->status; p.N = N; p.K = K;
+    return launch_tc_gemm<EPI>(tw, *ta_hi, *ta_lo, p, m_upper, m->sm_count, m->stream);
+}
+
 // Multi-row pass: up to m_upper rows (the exact count is desc->m on the device).
 static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int slot, int m_upper, bool emit, const SampleCtx &sc)
 {
@@ -459,17 +595,17 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
     if (m_upper > m->max_rows) return ST_ERR_INTERNAL;
     uint16_t *XN_lo = m->XN + (size_t)m->max_rows * h, *ATT_lo = m->ATTb + (size_t)m->max_rows * qd,
              *ACT_lo = m->ACTb + (size_t)m->max_rows * f;
+    static_assert((int)GEPI_STORE == (int)TEPI_STORE && (int)GEPI_RESADD == (int)TEPI_RESADD && (int)GEPI_SILU == (int)TEPI_SILU, "epilogue ids");
     embed_rope_kernel<<<m_upper, 256, 0, s>>>(desc, tok, m->embed, h, c.vocab, m->X, m->inv_freq, D / 2, m->cs, m->status);
     ++g_launches;
     CK(cudaGetLastError());
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerWeights &w = m->layers[l];
+        const LayerMaps &tm = m->maps[l];
         rmsnorm_rows_kernel<<<m_upper, 256, 0, s>>>(desc, m->X, w.g1, c.rms_eps, h, m->XN, XN_lo);
         ++g_launches;
         CK(cudaGetLastError());
-        GemmParams g{};
-        g.desc = desc; g.A_hi = m->XN; g.A_lo = XN_lo; g.W = w.wqkv; g.bias = w.bqkv; g.Yf = m->QKV; g.N = qd + 2 * kd; g.K = h;
-        CK(launch_gemm<GEPI_STORE>(g, m_upper, s));
+        TRY((rows_gemm<TEPI_STORE>(m, desc, m_upper, 0, m->XN, XN_lo, tm.wqkv, w.wqkv, w.bqkv, m->QKV, nullptr, nullptr, qd + 2 * kd, h)));
         const KvView kv = kv_view(m, l, slot);
         rope_append_kernel<<<m_upper, 256, 0, s>>>(desc, m->QKV, m->cs, c.n_q_heads, c.n_kv_heads, D, kv, m->status);
         ++g_launches;
@@ -479,18 +615,12 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
         a.tickets = m->tickets; a.status = m->status;
         a.Hq = c.n_q_heads; a.n_splits = 1; a.scale = 1.f / sqrtf((float)D);
         CK(launch_attn(a, D, G, dim3(1, c.n_kv_heads, m_upper), s));
-        g = GemmParams{};
-        g.desc = desc; g.A_hi = m->ATTb; g.A_lo = ATT_lo; g.W = w.wo; g.Yf = m->X; g.N = h; g.K = qd;
-        CK(launch_gemm<GEPI_RESADD>(g, m_upper, s));
+        TRY((rows_gemm<TEPI_RESADD>(m, desc, m_upper, 1, m->ATTb, ATT_lo, tm.wo, w.wo, nullptr, m->X, nullptr, nullptr, h, qd)));
         rmsnorm_rows_kernel<<<m_upper, 256, 0, s>>>(desc, m->X, w.g2, c.rms_eps, h, m->XN, XN_lo);
         ++g_launches;
         CK(cudaGetLastError());
-        g = GemmParams{};
-        g.desc = desc; g.A_hi = m->XN; g.A_lo = XN_lo; g.W = w.wgu; g.Yb_hi = m->ACTb; g.Yb_lo = ACT_lo; g.N = 2 * f; g.K = h;
-        CK(launch_gemm<GEPI_SILU>(g, m_upper, s));
-        g = GemmParams{};
-        g.desc = desc; g.A_hi = m->ACTb; g.A_lo = ACT_lo; g.W = w.wd; g.Yf = m->X; g.N = h; g.K = f;
-        CK(launch_gemm<GEPI_RESADD>(g, m_upper, s));
+        TRY((rows_gemm<TEPI_SILU>(m, desc, m_upper, 0, m->XN, XN_lo, tm.wgu, w.wgu, nullptr, nullptr, m->ACTb, ACT_lo, 2 * f, h)));
+        TRY((rows_gemm<TEPI_RESADD>(m, desc, m_upper, 2, m->ACTb, ACT_lo, tm.wd, w.wd, nullptr, m->X, nullptr, nullptr, h, f)));
     }
     if (emit) return sample_tail(m, desc, sc);
     return ST_OK;

@@ -1,0 +1,260 @@
+// Multi-row (prefill / catch-up) projection on the 5th-generation tensor cores.
+//
+//   Y[i][n] = sum_k (A_hi[i][k] + A_lo[i][k]) * W[n][k]      i < m <= 256 activation rows
+//
+// "Swap-AB": the weight tile takes the M side of the MMA (128 weight rows = 128 TMEM lanes), the
+// activation rows take the N side (m padded to a multiple of 32 = TMEM columns), so that a pass of a
+// few dozen rows still fills the instruction and every weight byte is read from HBM once per pass.
+// Both operands are K-major bf16 tiles of 64 elements (128 bytes) per row, brought in by TMA with the
+// 128-byte swizzle and consumed from shared memory by tcgen05.mma (kind::f16, fp32 accumulate in
+// TMEM).  The hi and lo activation planes are two MMAs on the same weight tile.
+//
+// One CTA = one 128-row weight tile x one K split.  Warp 0 issues TMA, warp 1 owns TMEM and issues
+// the MMAs, warps 2..5 drain the accumulator (tcgen05.ld) into the epilogue.  Stages hand over
+// through mbarriers; every wait is bounded and, when it runs out, raises a status bit, lets the CTA
+// drain what it armed, frees its TMEM and returns.  No multicast, no clusters.
+#pragma once
+#include <cuda.h>
+
+#include "st_common.cuh"
+
+namespace st {
+
+enum { TEPI_STORE = 0, TEPI_RESADD = 1, TEPI_SILU = 2 };
+
+struct TcGemmParams {
+    const StepDesc *desc;
+    const float *bias;        // [N] or null (added by K split 0)
+    float *Yf;                // TEPI_STORE / TEPI_RESADD: [rows][N] fp32 (accumulated with atomics when k_splits > 1)
+    uint16_t *Yb_hi, *Yb_lo;  // TEPI_SILU: [rows][N / 2] hi/lo planes of silu(row 2j) * row 2j+1
+    int32_t *status;
+    int32_t N, K;
+    int32_t m_pad;            // MMA N: activation rows padded to a multiple of 32, <= 256
+    int32_t stages;           // shared-memory pipeline depth
+    int32_t k_splits;
+    int32_t tmem_cols;        // power of two >= max(32, m_pad)
+};
+
+constexpr int kTcTileW = 128;       // weight rows per CTA
+constexpr int kTcBlockK = 64;       // K elements per stage (128 bytes per row)
+constexpr int kTcWBytes = kTcTileW * kTcBlockK * 2;
+constexpr uint32_t kTcWaitLimit = 1u << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false (and a status bit) when the phase does not complete within the limit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status)
+{
+    for (uint32_t it = 0; it < kTcWaitLimit; ++it) {
+        if (mbar_try(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (it > 64) __nanosleep(64);
+    }
+    *abort_flag = 1;
+    atomicOr(status, DEV_WAIT_EXPIRED);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile with 128-byte rows and the 128-byte swizzle:
+// 8-row groups are 1024 bytes apart (stride byte offset), descriptor version 1, layout type 2.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr)
+{
+    const uint32_t lo = (smem_addr >> 4) & 0x3fffu;
+    const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+    return ((uint64_t)hi << 32) | lo;
+}
+
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t umma_idesc_bf16(int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v)
+{
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW,
+                                                      const __grid_constant__ CUtensorMap tmAhi,
+                                                      const __grid_constant__ CUtensorMap tmAlo, const TcGemmParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t s_full[8], s_empty[8], s_acc;
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+
+    const int m = p.desc->m;
+    if (m <= 0) return;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n0 = blockIdx.x * kTcTileW;
+    const int kb_total = (p.K + kTcBlockK - 1) / kTcBlockK;
+    const int kb_per = (kb_total + p.k_splits - 1) / p.k_splits;
+    const int kb0 = blockIdx.y * kb_per;
+    const int kb1 = min(kb_total, kb0 + kb_per);
+    const int n_kb = kb1 - kb0;
+    if (n_kb <= 0) return;   // uniform for the CTA
+
+    const uint32_t a_bytes = (uint32_t)p.m_pad * kTcBlockK * 2;
+    const uint32_t stage_bytes = kTcWBytes + 2 * a_bytes;
+    const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 1024-byte aligned tile area
+
+    if (tid == 0) {
+        s_abort = 0;
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(smem_u32(&s_full[s]), 1);
+            mbar_init(smem_u32(&s_empty[s]), 1);
+        }
+        mbar_init(smem_u32(&s_acc), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)), "r"((uint32_t)p.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = s_tmem_base;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            int armed = 0;
+            for (int i = 0; i < n_kb; ++i) {
+                const int s = i % p.stages, u = i / p.stages;
+                if (u > 0 && !mbar_wait(smem_u32(&s_empty[s]), (u - 1) & 1, &s_abort, p.status)) break;
+                const uint32_t full = smem_u32(&s_full[s]);
+                const uint32_t base = tiles + (uint32_t)s * stage_bytes;
+                mbar_expect_tx(full, stage_bytes);
+                const int kx = (kb0 + i) * kTcBlockK;
+                tma_load_2d(base, &tmW, kx, n0, full);
+                tma_load_2d(base + kTcWBytes, &tmAhi, kx, 0, full);
+                tma_load_2d(base + kTcWBytes + a_bytes, &tmAlo, kx, 0, full);
+                armed = i + 1;
+            }
+            if (s_abort) {
+                // give the copies already issued a bounded time to land before the CTA leaves
+                for (int i = max(0, armed - p.stages); i < armed; ++i) {
+                    const int s = i % p.stages, u = i / p.stages;
+                    for (uint32_t it = 0; it < (1u << 16) && !mbar_try(smem_u32(&s_full[s]), u & 1); ++it) __nanosleep(128);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16(p.m_pad);
+            bool ok = true;
+            for (int i = 0; i < n_kb && ok; ++i) {
+                const int s = i % p.stages, u = i / p.stages;
+                ok = mbar_wait(smem_u32(&s_full[s]), u & 1, &s_abort, p.status);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t base = tiles + (uint32_t)s * stage_bytes;
+                const uint64_t dw = umma_desc_sw128(base);
+                const uint64_t dh = umma_desc_sw128(base + kTcWBytes);
+                const uint64_t dl = umma_desc_sw128(base + kTcWBytes + a_bytes);
+#pragma unroll
+                for (int k4 = 0; k4 < kTcBlockK / 16; ++k4)   // 16 elements = 32 bytes = 2 descriptor units
+                    umma_bf16(tmem, dw + 2 * k4, dh + 2 * k4, idesc, (i > 0 || k4 > 0) ? 1u : 0u);
+#pragma unroll
+                for (int k4 = 0; k4 < kTcBlockK / 16; ++k4)
+                    umma_bf16(tmem, dw + 2 * k4, dl + 2 * k4, idesc, 1u);
+                umma_commit(smem_u32(&s_empty[s]));
+            }
+            if (ok) umma_commit(smem_u32(&s_acc));
+        }
+    } else {
+        // ---------------- epilogue: TMEM -> registers -> global ----------------
+        const int q = warp & 3;                 // TMEM lane quarter this warp may read
+        const int row = n0 + q * 32 + lane;     // weight row = output feature
+        int ok_i = lane == 0 ? (int)mbar_wait(smem_u32(&s_acc), 0, &s_abort, p.status) : 1;
+        const bool ok = __shfl_sync(0xffffffffu, ok_i, 0) != 0;   // one poller per warp, uniform outcome
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok) {
+            const float bias = (EPI != TEPI_SILU && p.bias && blockIdx.y == 0 && row < p.N) ? p.bias[row] : 0.f;
+            for (int c0 = 0; c0 < m; c0 += 16) {
+                float v[16];
+                tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int c = c0 + j;
+                    if (EPI == TEPI_SILU) {
+                        const float other = __shfl_xor_sync(0xffffffffu, v[j], 1);
+                        if (c < m && !(lane & 1) && row + 1 < p.N) {
+                            const size_t o = (size_t)c * (p.N >> 1) + (row >> 1);
+                            split_bf16(v[j] / (1.f + expf(-v[j])) * other, p.Yb_hi[o], p.Yb_lo[o]);
+                        }
+                    } else if (c < m && row < p.N) {
+                        float *dst = p.Yf + (size_t)c * p.N + row;
+                        const float t = v[j] + bias;
+                        if (p.k_splits > 1) atomicAdd(dst, t);
+                        else if (EPI == TEPI_RESADD) *dst += t;
+                        else *dst = t;
+                    }
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)p.tmem_cols) : "memory");
+    }
+}
+
+}  // namespace st
