@@ -88,6 +88,8 @@ __global__ void rope_append_kernel(const StepDesc *desc, float *qkv, const float
     }
 }
 
+constexpr int kMaxAttnSplits = 160;   // upper bound of n_splits (the host never asks for more)
+
 struct AttnParams {
     const StepDesc *desc;
     const float *qkv;           // [rows][(Hq + 2 Hkv) * D], q already rotated
@@ -251,19 +253,40 @@ __global__ void __launch_bounds__(128) attn_kernel(const AttnParams p)
     __syncthreads();
     if (!s_last) return;
     __threadfence();
+    // weights of the splits: w[g][s] = exp(m_s - max_s m) (0 for empty splits), shared by all channels
+    __shared__ float s_w[G][kMaxAttnSplits], s_l[G][kMaxAttnSplits];
+    __shared__ float s_den[G];
+    for (int idx = tid; idx < G * p.n_splits; idx += 128) {
+        const int g = idx / p.n_splits, sp = idx - g * p.n_splits;
+        const float2 ml = __ldcg(reinterpret_cast<const float2 *>(p.part_ml) + ((size_t)row * p.Hq + hq0 + g) * p.n_splits + sp);
+        s_w[g][sp] = ml.x;
+        s_l[g][sp] = ml.y;
+    }
+    __syncthreads();
+    if (tid < G) {
+        float mnew = -INFINITY;
+        for (int sp = 0; sp < p.n_splits; ++sp) mnew = fmaxf(mnew, s_w[tid][sp]);
+        float dsum = 0.f;
+        for (int sp = 0; sp < p.n_splits; ++sp) {
+            const float ms = s_w[tid][sp];
+            const float cw = ms == -INFINITY ? 0.f : __expf(ms - mnew);
+            s_w[tid][sp] = cw;
+            dsum += s_l[tid][sp] * cw;
+        }
+        s_den[tid] = dsum;
+    }
+    __syncthreads();
     for (int idx = tid; idx < G * D; idx += 128) {
         const int g = idx / D, c = idx - g * D;
-        const size_t pi = ((size_t)row * p.Hq + hq0 + g) * p.n_splits;
-        float mnew = -INFINITY;
-        for (int s = 0; s < p.n_splits; ++s) mnew = fmaxf(mnew, __ldcg(&p.part_ml[(pi + s) * 2]));
-        float dsum = 0.f, osum = 0.f;
-        for (int s = 0; s < p.n_splits; ++s) {
-            const float ms = __ldcg(&p.part_ml[(pi + s) * 2]);
-            const float cw = ms == -INFINITY ? 0.f : __expf(ms - mnew);
-            dsum += __ldcg(&p.part_ml[(pi + s) * 2 + 1]) * cw;
-            osum += __ldcg(&p.part_o[(pi + s) * D + c]) * cw;
+        const float *po = p.part_o + ((size_t)row * p.Hq + hq0 + g) * p.n_splits * D + c;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        int sp = 0;
+        for (; sp + 4 <= p.n_splits; sp += 4) {   // four independent loads in flight
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[j] = fmaf(__ldcg(po + (size_t)(sp + j) * D), s_w[g][sp + j], acc[j]);
         }
-        attn_store(p, ((size_t)row * p.Hq + hq0 + g) * D + c, osum / dsum);
+        for (; sp < p.n_splits; ++sp) acc[0] = fmaf(__ldcg(po + (size_t)sp * D), s_w[g][sp], acc[0]);
+        attn_store(p, ((size_t)row * p.Hq + hq0 + g) * D + c, ((acc[0] + acc[1]) + (acc[2] + acc[3])) / s_den[g]);
     }
 }
 

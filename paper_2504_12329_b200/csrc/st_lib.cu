@@ -117,6 +117,7 @@ struct st_model {
 
 static constexpr int kArgmaxBlocks = 64;
 static constexpr int kGemvWarps = 16;
+static constexpr int kRowSplits = 8;   // most key splits a multi-row pass uses
 
 // ------------------------------------------------------------------------------------------------
 // launch helpers
@@ -412,6 +413,7 @@ static int model_build(st_model *m)
     // ---- scratch ----
     m->max_rows = 256;   // rows of one multi-row pass = the MMA N limit
     m->max_splits = (2 * m->sm_count + c.n_kv_heads - 1) / c.n_kv_heads;
+    if (m->max_splits > kMaxAttnSplits) m->max_splits = kMaxAttnSplits;
     ALLOC(m->X, float, (size_t)m->max_rows * h);
     ALLOC(m->XN, uint16_t, 2 * (size_t)m->max_rows * h);
     ALLOC(m->QKV, float, (size_t)m->max_rows * qkvd);
@@ -421,8 +423,11 @@ static int model_build(st_model *m)
     ALLOC(m->ACTb, uint16_t, 2 * (size_t)m->max_rows * f);
     ALLOC(m->cs, float2, (size_t)m->max_rows * (D / 2));
     ALLOC(m->logits, float, c.vocab);
-    ALLOC(m->part_o, float, (size_t)c.n_q_heads * m->max_splits * D);
-    ALLOC(m->part_ml, float, (size_t)c.n_q_heads * m->max_splits * 2);
+    {   // split-KV partials: one decode row with up to max_splits splits, or max_rows rows with up to kRowSplits
+        size_t n = (size_t)m->max_splits > (size_t)m->max_rows * kRowSplits ? (size_t)m->max_splits : (size_t)m->max_rows * kRowSplits;
+        ALLOC(m->part_o, float, (size_t)c.n_q_heads * n * D);
+        ALLOC(m->part_ml, float, (size_t)c.n_q_heads * n * 2);
+    }
     ALLOC(m->tickets, int32_t, (size_t)m->max_rows * c.n_kv_heads + 1);
     CK(cudaMemsetAsync(m->tickets, 0, ((size_t)m->max_rows * c.n_kv_heads + 1) * sizeof(int32_t), m->stream));
     ALLOC(m->amax_val, float, kArgmaxBlocks);
@@ -586,7 +591,7 @@ static int rows_gemm(st_model *m, const StepDesc *desc, int m_upper, int buffer,
 }
 
 // Multi-row pass: up to m_upper rows (the exact count is desc->m on the device).
-static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int slot, int m_upper, bool emit, const SampleCtx &sc)
+static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int slot, int m_upper, int ctx_upper, bool emit, const SampleCtx &sc)
 {
     const st_config &c = m->cfg;
     const int h = c.hidden, D = c.head_dim, qd = c.n_q_heads * D, kd = c.n_kv_heads * D, f = c.ffn;
@@ -595,6 +600,10 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
     if (m_upper > m->max_rows) return ST_ERR_INTERNAL;
     uint16_t *XN_lo = m->XN + (size_t)m->max_rows * h, *ATT_lo = m->ATTb + (size_t)m->max_rows * qd,
              *ACT_lo = m->ACTb + (size_t)m->max_rows * f;
+    // few rows over a long context: split the keys so that the pass still fills the GPU
+    int row_splits = (3 * m->sm_count + c.n_kv_heads * m_upper - 1) / (c.n_kv_heads * m_upper);
+    if (row_splits > ctx_upper / 256) row_splits = ctx_upper / 256;
+    row_splits = row_splits < 1 ? 1 : row_splits > kRowSplits ? kRowSplits : row_splits;
     static_assert((int)GEPI_STORE == (int)TEPI_STORE && (int)GEPI_RESADD == (int)TEPI_RESADD && (int)GEPI_SILU == (int)TEPI_SILU, "epilogue ids");
     embed_rope_kernel<<<m_upper, 256, 0, s>>>(desc, tok, m->embed, h, c.vocab, m->X, m->inv_freq, D / 2, m->cs, m->status);
     ++g_launches;
@@ -612,9 +621,9 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
         CK(cudaGetLastError());
         AttnParams a{};
         a.desc = desc; a.qkv = m->QKV; a.kv = kv; a.out_f32 = nullptr; a.out_hi = m->ATTb; a.out_lo = ATT_lo;
-        a.tickets = m->tickets; a.status = m->status;
-        a.Hq = c.n_q_heads; a.n_splits = 1; a.scale = 1.f / sqrtf((float)D);
-        CK(launch_attn(a, D, G, dim3(1, c.n_kv_heads, m_upper), s));
+        a.part_o = m->part_o; a.part_ml = m->part_ml; a.tickets = m->tickets; a.status = m->status;
+        a.Hq = c.n_q_heads; a.n_splits = row_splits; a.scale = 1.f / sqrtf((float)D);
+        CK(launch_attn(a, D, G, dim3(row_splits, c.n_kv_heads, m_upper), s));
         TRY((rows_gemm<TEPI_RESADD>(m, desc, m_upper, 1, m->ATTb, ATT_lo, tm.wo, w.wo, nullptr, m->X, nullptr, nullptr, h, qd)));
         rmsnorm_rows_kernel<<<m_upper, 256, 0, s>>>(desc, m->X, w.g2, c.rms_eps, h, m->XN, XN_lo);
         ++g_launches;
@@ -821,7 +830,7 @@ int st_prefill(st_model *m, int32_t slot, const int32_t *tokens_host, int32_t n,
         sc.want_argmax = false;
         const bool emit = last && last_logits_dev != nullptr;
         if (rows == 1 && emit) TRY(pass_decode(m, m->desc, m->tokbuf, slot, d.pos0 + 1, sc));
-        else TRY(pass_rows(m, m->desc, m->tokbuf, slot, rows, emit, sc));
+        else TRY(pass_rows(m, m->desc, m->tokbuf, slot, rows, d.pos0 + rows, emit, sc));
         m->seq_len[slot] += rows;
         done += rows;
         // the staging buffer and descriptor are reused by the next chunk
@@ -1014,7 +1023,7 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
         sc.want_argmax = true;
         const int ctx_after = gh.kv_len[gh.next_model] + gh.next_m;
         if (gh.next_m == 1 && gh.next_emit) rc = pass_decode(m, d, b.tokens, slot, ctx_after, sc);
-        else rc = pass_rows(m, d, b.tokens, slot, gh.next_m, gh.next_emit != 0, sc);
+        else rc = pass_rows(m, d, b.tokens, slot, gh.next_m, ctx_after, gh.next_emit != 0, sc);
         if (rc != ST_OK) break;
         if (!gh.next_emit) {
             advance_ingest_kernel<<<1, 1, 0, s>>>(gen, desc_small, desc_large);
