@@ -13,6 +13,10 @@ namespace st {
 constexpr int kClsKeyword = 2;  // class-table bit of a reflection keyword
 
 struct GenState {
+    // --- accounting (64-bit fields first) ---
+    int64_t bytes_algo;      // weights + KV bytes the passes so far had to move
+    int64_t wbytes[2];       // weight bytes one pass of each model streams
+    int64_t kvb[2];          // KV bytes per cached token of each model
     // --- dynamic ---
     int32_t active;      // 0 = speculative (small), 1 = target (large)
     int32_t remaining;   // tokens the target still writes in this takeover
@@ -25,6 +29,8 @@ struct GenState {
     int32_t next_model;  // the pass to run next ...
     int32_t next_m;      // ... ingests this many tokens ...
     int32_t next_emit;   // ... and samples a token (1) or only ingests (0)
+    int32_t passes;      // passes dispatched so far
+    int32_t pass_cap;    // hard bound on passes (the device loop stops there)
     // --- parameters ---
     int32_t has_large, delimiter, n1, keep_probe, eos, vlimit, max_new, n_force;
     int32_t prompt_len, cap_steps, cap_handoffs, max_chunk;
@@ -67,6 +73,7 @@ __device__ void router_step(GenState *g, const GenBuffers &b, int greedy, StepDe
     const int t = g->step;
     const int fed = g->pos - g->kv_len[a];
     g->kv_len[a] = g->pos;
+    g->bytes_algo += g->wbytes[a] + g->kvb[a] * (int64_t)g->pos;
     int tok = greedy;
     if (t < g->n_force && b.force[t] >= 0) tok = b.force[t];
     if (t < g->cap_steps) {
@@ -116,12 +123,43 @@ __global__ void advance_ingest_kernel(GenState *g, StepDesc *desc_small, StepDes
 {
     const int a = g->next_model;
     g->kv_len[a] += g->next_m;
+    g->bytes_algo += g->wbytes[a] + g->kvb[a] * (int64_t)g->kv_len[a];
     plan_next_pass(g, desc_small, desc_large);
 }
 
 __global__ void plan_first_pass_kernel(GenState *g, StepDesc *desc_small, StepDesc *desc_large)
 {
     plan_next_pass(g, desc_small, desc_large);
+}
+
+// Device-side dispatch of the generation loop (one launch per loop iteration of the graph): picks the
+// body that runs the planned pass, or ends the loop.  Bodies per model, in this order: decode,
+// multi-row passes of at most 32 / 64 / 128 / 256 rows that sample, ingest-only pass of 256 rows.
+constexpr int kBodiesPerModel = 6;
+
+__device__ __forceinline__ int pass_body_index(int model, int m, int emit)
+{
+    int b;
+    if (!emit) b = 5;
+    else if (m == 1) b = 0;
+    else b = m <= 32 ? 1 : m <= 64 ? 2 : m <= 128 ? 3 : 4;
+    return model * kBodiesPerModel + b;
+}
+
+__global__ void dispatch_kernel(GenState *g, cudaGraphConditionalHandle loop, cudaGraphConditionalHandle body, int32_t *status)
+{
+    if (!g->done && g->passes >= g->pass_cap) {
+        g->done = 1;
+        atomicOr(status, DEV_WAIT_EXPIRED);
+    }
+    if (g->done) {
+        cudaGraphSetConditional(loop, 0);
+        cudaGraphSetConditional(body, 0x7fffffffu);   // no such body: nothing runs
+        return;
+    }
+    g->passes++;
+    cudaGraphSetConditional(loop, 1);
+    cudaGraphSetConditional(body, (unsigned)pass_body_index(g->next_model, g->next_m, g->next_emit));
 }
 
 struct ArgmaxParams {
@@ -152,7 +190,7 @@ __global__ void __launch_bounds__(256) argmax_router_kernel(const ArgmaxParams p
     // optional logits trace of this emission step (the step counter only changes after every CTA
     // has taken its ticket, i.e. after all of them have read it here)
     float *trace = nullptr;
-    if (p.gen && p.buf.trace) {
+    if (p.gen && p.buf.trace && p.gen->trace_n > 0) {
         const int t = p.gen->step - p.gen->trace_first;
         if (t >= 0 && t < p.gen->trace_n) trace = p.buf.trace + (size_t)t * p.limit;
     }

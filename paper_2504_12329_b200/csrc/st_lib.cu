@@ -56,8 +56,12 @@ struct LayerWeights {
     float *g1, *g2;  // norm gains [h]
 };
 
+struct GenContext;
+
 struct st_model {
     st_config cfg{};
+    uint64_t id = 0;                 // unique per created model
+    GenContext *gen_ctx = nullptr;   // generation buffers + graph with this model as the speculative one
     uint64_t seed = 0;
     uint32_t tag = 0;
     cudaStream_t stream = nullptr;
@@ -129,12 +133,6 @@ static cudaError_t launch_gemv_s(const GemvParams &p, cudaStream_t s, int sms)
     constexpr int NW = kGemvWarps, R = 2, U = 4;
     auto kern = gemv_kernel<NW, S, R, U, PRO, EPI>;
     const size_t smem = (size_t)p.K * 4 + 2 * NW * R * 4;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
     const int G = NW / S;
     const int n_tasks = (p.N + R - 1) / R;
     const int ctas_needed = (n_tasks + G - 1) / G;
@@ -145,6 +143,22 @@ static cudaError_t launch_gemv_s(const GemvParams &p, cudaStream_t s, int sms)
     kern<<<grid, NW * 32, smem, s>>>(p);
     ++g_launches;
     return cudaGetLastError();
+}
+
+template <int S, int PRO, int EPI>
+static cudaError_t gemv_attr()
+{
+    return cudaFuncSetAttribute(gemv_kernel<kGemvWarps, S, 2, 4, PRO, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+}
+
+template <int PRO, int EPI>
+static cudaError_t gemv_attr_all()
+{
+    cudaError_t e = gemv_attr<1, PRO, EPI>();
+    if (e == cudaSuccess) e = gemv_attr<2, PRO, EPI>();
+    if (e == cudaSuccess) e = gemv_attr<4, PRO, EPI>();
+    if (e == cudaSuccess) e = gemv_attr<8, PRO, EPI>();
+    return e;
 }
 
 template <int PRO, int EPI>
@@ -237,11 +251,6 @@ static int launch_tc_gemm(const CUtensorMap &tw, const CUtensorMap &ta_hi, const
                           int sms, cudaStream_t s)
 {
     auto kern = tc_gemm_kernel<EPI>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
-        attr_set = true;
-    }
     p.m_pad = (m_upper + 31) / 32 * 32;
     if (p.m_pad > 256) return ST_ERR_INTERNAL;
     p.tmem_cols = p.m_pad <= 32 ? 32 : p.m_pad <= 64 ? 64 : p.m_pad <= 128 ? 128 : 256;
@@ -300,6 +309,18 @@ static int fill_const(st_model *m, float *out, float v, uint64_t n)
     return ST_OK;
 }
 
+// Opt every kernel into the shared memory it may ask for (once per device, outside any capture).
+static int init_kernel_attributes()
+{
+    CK((gemv_attr_all<PRO_NORM, EPI_STORE>()));
+    CK((gemv_attr_all<PRO_PLAIN, EPI_RESADD>()));
+    CK((gemv_attr_all<PRO_NORM, EPI_SILU>()));
+    CK(cudaFuncSetAttribute(tc_gemm_kernel<TEPI_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+    CK(cudaFuncSetAttribute(tc_gemm_kernel<TEPI_RESADD>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+    CK(cudaFuncSetAttribute(tc_gemm_kernel<TEPI_SILU>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+    return ST_OK;
+}
+
 static int check_config(const st_config *c)
 {
     if (!c) return ST_ERR_ARG;
@@ -324,6 +345,7 @@ static int model_build(st_model *m)
     const int qkvd = qd + 2 * kd;
     CK(cudaGetDevice(&m->device));
     CK(cudaDeviceGetAttribute(&m->sm_count, cudaDevAttrMultiProcessorCount, m->device));
+    TRY(init_kernel_attributes());
 
 #define ALLOC(ptr, type, count)                                      \
     do {                                                             \
@@ -639,6 +661,8 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
 // C ABI
 // ------------------------------------------------------------------------------------------------
 
+static void destroy_gen_context(st_model *m);
+
 extern "C" {
 
 const char *st_strerror(int status)
@@ -670,6 +694,8 @@ int st_model_create(const st_config *cfg, uint64_t seed, uint32_t model_tag, voi
     }
     st_model *m = new (std::nothrow) st_model();
     if (!m) return ST_ERR_OOM;
+    static uint64_t next_id = 0;
+    m->id = ++next_id;
     m->cfg = *cfg;
     m->seed = seed;
     m->tag = model_tag;
@@ -687,6 +713,7 @@ void st_model_destroy(st_model *m)
 {
     if (!m) return;
     cudaStreamSynchronize(m->stream);
+    destroy_gen_context(m);
     for (void *p : m->allocations) {
         if (m->cfg.free) m->cfg.free(p, m->cfg.alloc_user);
         else cudaFree(p);
@@ -871,14 +898,28 @@ int st_decode_step(st_model *m, const int32_t *slots_host, const int32_t *tokens
 // generation
 // ------------------------------------------------------------------------------------------------
 
-namespace {
-
-struct DevArena {  // raw device allocations of one generation call, released on scope exit
+// Device buffers of a generation and the CUDA graph that runs it.  The graph is one WHILE node whose
+// body is a dispatch kernel followed by a SWITCH node with one body per kind of pass (per model:
+// decode, multi-row passes of <= 32/64/128/256 rows, ingest-only).  The router kernel at the end of a
+// pass plans the next one on the device, the dispatch kernel selects the body: the host launches the
+// graph once and waits.  Kernel arguments are baked into the graph, so the buffers live as long as
+// the context and the graph is rebuilt only when a capacity grows or a model/slot changes.
+struct GenContext {
+    st_model *large = nullptr;
+    uint64_t large_id = 0;
+    int slot_s = -1, slot_l = -1;
+    int cap_total = 0, cap_steps = 0, cap_hand = 0, cap_force = 0, vlimit = 0;
+    size_t cap_trace = 0;
+    GenState *gen = nullptr;
+    StepDesc *desc2 = nullptr;
+    GenBuffers b{};
+    int32_t *d_force = nullptr;
+    uint8_t *d_cls = nullptr;
+    float *d_trace = nullptr;
     std::vector<void *> ptrs;
-    ~DevArena()
-    {
-        for (void *p : ptrs) cudaFree(p);
-    }
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+
     template <class T>
     T *get(size_t n)
     {
@@ -887,7 +928,27 @@ struct DevArena {  // raw device allocations of one generation call, released on
         ptrs.push_back(p);
         return (T *)p;
     }
+    void release()
+    {
+        if (exec) cudaGraphExecDestroy(exec);
+        if (graph) cudaGraphDestroy(graph);
+        for (void *p : ptrs) cudaFree(p);
+        ptrs.clear();
+        exec = nullptr;
+        graph = nullptr;
+    }
 };
+
+static void destroy_gen_context(st_model *m)
+{
+    if (m->gen_ctx) {
+        m->gen_ctx->release();
+        delete m->gen_ctx;
+        m->gen_ctx = nullptr;
+    }
+}
+
+namespace {
 
 struct SlotGuard {
     st_model *m;
@@ -898,7 +959,180 @@ struct SlotGuard {
     }
 };
 
+struct StreamSwap {   // run the pass functions on the capture stream
+    st_model *a, *b;
+    cudaStream_t sa, sb;
+    StreamSwap(st_model *a_, st_model *b_, cudaStream_t cap) : a(a_), b(b_), sa(a_->stream), sb(b_ ? b_->stream : nullptr)
+    {
+        a->stream = cap;
+        if (b) b->stream = cap;
+    }
+    ~StreamSwap()
+    {
+        a->stream = sa;
+        if (b) b->stream = sb;
+    }
+};
+
 }  // namespace
+
+static SampleCtx gen_sample_ctx(const GenContext &c)
+{
+    SampleCtx sc{};
+    sc.vlimit = c.vlimit;
+    sc.gen = c.gen;
+    sc.buf = c.b;
+    sc.desc_small = c.desc2;
+    sc.desc_large = c.desc2 + 1;
+    sc.want_argmax = true;
+    return sc;
+}
+
+// Capture one pass body into `body`.
+static int capture_body(GenContext &c, st_model *small, cudaStream_t cap, cudaGraph_t body, int model, int kind)
+{
+    static const int kRowsOf[kBodiesPerModel] = {1, 32, 64, 128, 256, 256};
+    st_model *m = model ? c.large : small;
+    const int slot = model ? c.slot_l : c.slot_s;
+    StepDesc *d = c.desc2 + model;
+    const SampleCtx sc = gen_sample_ctx(c);
+    CK(cudaStreamBeginCaptureToGraph(cap, body, nullptr, nullptr, 0, cudaStreamCaptureModeRelaxed));
+    int rc;
+    {
+        StreamSwap swap(small, c.large, cap);
+        int rows = kRowsOf[kind];
+        if (rows > m->max_rows) rows = m->max_rows;
+        if (kind == 0) rc = pass_decode(m, d, c.b.tokens, slot, c.cap_total, sc);
+        else rc = pass_rows(m, d, c.b.tokens, slot, rows, c.cap_total, kind != 5, sc);
+        if (rc == ST_OK && kind == 5) {
+            advance_ingest_kernel<<<1, 1, 0, cap>>>(c.gen, c.desc2, c.desc2 + 1);
+            ++g_launches;
+            if (cudaGetLastError() != cudaSuccess) rc = ST_ERR_INTERNAL;
+        }
+    }
+    cudaGraph_t g = nullptr;
+    const cudaError_t e = cudaStreamEndCapture(cap, &g);
+    if (rc != ST_OK) return rc;
+    CK(e);
+    return ST_OK;
+}
+
+static int build_gen_graph(GenContext &c, st_model *small)
+{
+    if (c.exec) { cudaGraphExecDestroy(c.exec); c.exec = nullptr; }
+    if (c.graph) { cudaGraphDestroy(c.graph); c.graph = nullptr; }
+    cudaStream_t cap = nullptr;
+    CK(cudaStreamCreateWithFlags(&cap, cudaStreamNonBlocking));
+    int rc = ST_OK;
+    do {
+        if (cudaGraphCreate(&c.graph, 0) != cudaSuccess) { rc = ST_ERR_INTERNAL; break; }
+        cudaGraphConditionalHandle h_loop, h_body;
+        if (cudaGraphConditionalHandleCreate(&h_loop, c.graph, 1, cudaGraphCondAssignDefault) != cudaSuccess) { rc = ST_ERR_INTERNAL; break; }
+        cudaGraphNodeParams wp = {cudaGraphNodeTypeConditional};
+        wp.type = cudaGraphNodeTypeConditional;
+        wp.conditional.handle = h_loop;
+        wp.conditional.type = cudaGraphCondTypeWhile;
+        wp.conditional.size = 1;
+        cudaGraphNode_t wnode;
+        if (cudaGraphAddNode(&wnode, c.graph, nullptr, 0, &wp) != cudaSuccess) { rc = ST_ERR_INTERNAL; break; }
+        cudaGraph_t loop_body = wp.conditional.phGraph_out[0];
+        if (cudaGraphConditionalHandleCreate(&h_body, loop_body, 0, 0) != cudaSuccess) { rc = ST_ERR_INTERNAL; break; }
+        // dispatch kernel node
+        int32_t *status = small->status;
+        void *args[4] = {&c.gen, &h_loop, &h_body, &status};
+        cudaKernelNodeParams kp;
+        memset(&kp, 0, sizeof kp);
+        kp.func = (void *)dispatch_kernel;
+        kp.gridDim = dim3(1);
+        kp.blockDim = dim3(1);
+        kp.kernelParams = args;
+        cudaGraphNode_t dnode;
+        if (cudaGraphAddKernelNode(&dnode, loop_body, nullptr, 0, &kp) != cudaSuccess) { rc = ST_ERR_INTERNAL; break; }
+        // switch node with one body per kind of pass
+        const int n_bodies = (c.large ? 2 : 1) * kBodiesPerModel;
+        cudaGraphNodeParams sp = {cudaGraphNodeTypeConditional};
+        sp.type = cudaGraphNodeTypeConditional;
+        sp.conditional.handle = h_body;
+        sp.conditional.type = cudaGraphCondTypeSwitch;
+        sp.conditional.size = (unsigned)n_bodies;
+        cudaGraphNode_t snode;
+        if (cudaGraphAddNode(&snode, loop_body, &dnode, 1, &sp) != cudaSuccess) { rc = ST_ERR_INTERNAL; break; }
+        for (int i = 0; i < n_bodies && rc == ST_OK; ++i)
+            rc = capture_body(c, small, cap, sp.conditional.phGraph_out[i], i / kBodiesPerModel, i % kBodiesPerModel);
+        if (rc != ST_OK) break;
+        if (cudaGraphInstantiate(&c.exec, c.graph, 0) != cudaSuccess) { rc = ST_ERR_INTERNAL; break; }
+    } while (0);
+    if (rc != ST_OK) {
+        const cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess || !g_err_text[0]) set_error_text("building the generation graph", e);
+    }
+    cudaStreamDestroy(cap);
+    return rc;
+}
+
+// Make sure the speculative model's context fits this call; (re)allocate and rebuild when it does not.
+static int ensure_gen_context(st_model *small, st_model *large, int slot_s, int slot_l, int total, int cap_steps, int cap_hand,
+                              int n_force, int vlimit, size_t trace_floats, bool want_graph)
+{
+    GenContext *c = small->gen_ctx;
+    const bool fits = c && c->large == large && c->large_id == (large ? large->id : 0) && c->slot_s == slot_s &&
+                      c->slot_l == slot_l && c->cap_total >= total && c->cap_steps >= cap_steps && c->cap_hand >= cap_hand &&
+                      c->cap_force >= n_force && c->vlimit == vlimit && c->cap_trace >= trace_floats &&
+                      (!want_graph || c->exec);
+    if (fits) return ST_OK;
+    // growing: never shrink a capacity, so that alternating call sizes settle on one graph
+    int g_total = total, g_steps = cap_steps, g_hand = cap_hand, g_force = n_force;
+    size_t g_trace = trace_floats;
+    if (c && c->large == large && c->large_id == (large ? large->id : 0) && c->vlimit == vlimit) {
+        g_total = g_total > c->cap_total ? g_total : c->cap_total;
+        g_steps = g_steps > c->cap_steps ? g_steps : c->cap_steps;
+        g_hand = g_hand > c->cap_hand ? g_hand : c->cap_hand;
+        g_force = g_force > c->cap_force ? g_force : c->cap_force;
+        g_trace = g_trace > c->cap_trace ? g_trace : c->cap_trace;
+    }
+    destroy_gen_context(small);
+    c = new (std::nothrow) GenContext();
+    if (!c) return ST_ERR_OOM;
+    small->gen_ctx = c;
+    c->large = large;
+    c->large_id = large ? large->id : 0;
+    c->slot_s = slot_s;
+    c->slot_l = slot_l;
+    c->cap_total = g_total;
+    c->cap_steps = g_steps;
+    c->cap_hand = g_hand;
+    c->cap_force = g_force;
+    c->vlimit = vlimit;
+    c->cap_trace = g_trace;
+    c->gen = c->get<GenState>(1);
+    c->desc2 = c->get<StepDesc>(2);
+    c->b.tokens = c->get<int32_t>(g_total);
+    c->b.source = c->get<uint8_t>(g_total);
+    c->b.em_tok = c->get<int32_t>(g_steps);
+    c->b.em_fed = c->get<int32_t>(g_steps);
+    c->b.em_arg = c->get<int32_t>(g_steps);
+    c->b.em_src = c->get<uint8_t>(g_steps);
+    c->b.handoffs = c->get<int32_t>(3 * (size_t)g_hand);
+    c->d_force = c->get<int32_t>(g_force);
+    c->d_cls = c->get<uint8_t>(vlimit);
+    c->d_trace = g_trace ? c->get<float>(g_trace) : nullptr;
+    if (!c->gen || !c->desc2 || !c->b.tokens || !c->b.source || !c->b.em_tok || !c->b.em_fed || !c->b.em_arg || !c->b.em_src ||
+        !c->b.handoffs || !c->d_force || !c->d_cls || (g_trace && !c->d_trace)) {
+        destroy_gen_context(small);
+        return ST_ERR_OOM;
+    }
+    c->b.force = c->d_force;
+    c->b.cls = c->d_cls;
+    c->b.trace = c->d_trace;
+    if (want_graph) {
+        const int rc = build_gen_graph(*c, small);
+        if (rc != ST_OK) {
+            destroy_gen_context(small);
+            return rc;
+        }
+    }
+    return ST_OK;
+}
 
 extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_params *P, const int32_t *prompt,
                                 int32_t prompt_len, const int32_t *force, int32_t n_force, st_spec_result *out)
@@ -938,34 +1172,24 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
         TRY(st_seq_alloc(large, &gl.slot));
         TRY(seq_reserve(large, gl.slot, total));
     }
-
-    DevArena A;
-    GenBuffers b{};
-    GenState *gen = A.get<GenState>(1);
-    StepDesc *desc2 = A.get<StepDesc>(2);
-    b.tokens = A.get<int32_t>(total);
-    b.source = A.get<uint8_t>(max_new + 1);
-    const int dev_steps = cap_steps > 0 ? cap_steps : 1;
-    b.em_tok = A.get<int32_t>(dev_steps);
-    b.em_fed = A.get<int32_t>(dev_steps);
-    b.em_arg = A.get<int32_t>(dev_steps);
-    b.em_src = A.get<uint8_t>(dev_steps);
-    const int dev_hand = cap_handoffs > 0 ? cap_handoffs : 1;
-    b.handoffs = A.get<int32_t>(3 * (size_t)dev_hand);
-    int32_t *d_force = A.get<int32_t>(n_force);
-    uint8_t *d_cls = A.get<uint8_t>(vlimit);
     const int trace_n = out->logits_trace ? out->trace_n_steps : 0;
-    float *d_trace = trace_n > 0 ? A.get<float>((size_t)trace_n * vlimit) : nullptr;
-    if (!gen || !desc2 || !b.tokens || !b.source || !b.em_tok || !b.em_fed || !b.em_arg || !b.em_src || !b.handoffs ||
-        !d_force || !d_cls || (trace_n > 0 && !d_trace))
-        return ST_ERR_OOM;
-    b.force = d_force;
-    b.cls = d_cls;
-    b.trace = d_trace;
+    static const bool host_loop = [] { const char *e = getenv("ST_HOST_LOOP"); return e && e[0] == '1'; }();
+    TRY(ensure_gen_context(small, large, gs.slot, gl.slot, total, cap_steps > 0 ? cap_steps : 1, cap_handoffs > 0 ? cap_handoffs : 1,
+                           n_force, vlimit, (size_t)trace_n * vlimit, !host_loop));
+    GenContext &C = *small->gen_ctx;
+    const GenBuffers &b = C.b;
+    GenState *gen = C.gen;
+    StepDesc *desc_small = C.desc2, *desc_large = C.desc2 + 1;
 
     std::vector<uint8_t> cls(vlimit, 0);
     for (int i = 0; i < P->n_keywords; ++i) cls[P->keyword_ids[i]] |= kClsKeyword;
     GenState g0{};
+    g0.wbytes[0] = small->weight_bytes;
+    g0.kvb[0] = st_kv_bytes_per_token(small);
+    if (large) {
+        g0.wbytes[1] = large->weight_bytes;
+        g0.kvb[1] = st_kv_bytes_per_token(large);
+    }
     g0.has_large = large ? 1 : 0;
     g0.pos = prompt_len;
     g0.delimiter = P->delimiter_id;
@@ -983,11 +1207,12 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     g0.trace_first = out->trace_first_step;
     g0.trace_n = trace_n;
     g0.done = max_new == 0 ? 1 : 0;
+    const int64_t pass_cap = 2ll * (max_new + 2) + 2ll * (total / g0.max_chunk + 2) * (max_new / P->n1 + 2);
+    g0.pass_cap = pass_cap > 0x7fffffff ? 0x7fffffff : (int32_t)pass_cap;
     CK(cudaMemcpyAsync(gen, &g0, sizeof g0, cudaMemcpyHostToDevice, s));
     CK(cudaMemcpyAsync(b.tokens, prompt, (size_t)prompt_len * sizeof(int32_t), cudaMemcpyHostToDevice, s));
-    if (n_force) CK(cudaMemcpyAsync(d_force, force, (size_t)n_force * sizeof(int32_t), cudaMemcpyHostToDevice, s));
-    CK(cudaMemcpyAsync(d_cls, cls.data(), (size_t)vlimit, cudaMemcpyHostToDevice, s));
-    StepDesc *desc_small = desc2, *desc_large = desc2 + 1;
+    if (n_force) CK(cudaMemcpyAsync(C.d_force, force, (size_t)n_force * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+    CK(cudaMemcpyAsync(C.d_cls, cls.data(), (size_t)vlimit, cudaMemcpyHostToDevice, s));
     plan_first_pass_kernel<<<1, 1, 0, s>>>(gen, desc_small, desc_large);
     ++g_launches;
     CK(cudaGetLastError());
@@ -996,50 +1221,55 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     CK(cudaEventCreate(&ev0));
     CK(cudaEventCreate(&ev1));
     CK(cudaEventRecord(ev0, s));
-
-    // Pass loop.  The host reads only the shape of the next pass (which model, how many rows,
-    // whether it samples) -- enough to size the launch; tokens stay on the device.
-    int64_t bytes = 0;
     GenState gh = g0;
     int rc = ST_OK;
-    const int64_t pass_cap = 4ll * (max_new + 2) + (prompt_len / g0.max_chunk + 2) * 4ll;
-    for (int64_t pass = 0; pass < pass_cap; ++pass) {
-        if (cudaMemcpyAsync(&gh, gen, sizeof gh, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-            cudaStreamSynchronize(s) != cudaSuccess) {
-            set_error_text("generation state readback", cudaGetLastError());
+    if (!host_loop) {
+        // The whole generation is one graph launch; routing happens on the device.
+        const int64_t before = g_launches;
+        if (cudaGraphLaunch(C.exec, s) != cudaSuccess) {
+            set_error_text("cudaGraphLaunch", cudaGetLastError());
             rc = ST_ERR_INTERNAL;
-            break;
         }
-        if (gh.done) break;
-        st_model *m = gh.next_model ? large : small;
-        const int slot = gh.next_model ? gl.slot : gs.slot;
-        StepDesc *d = gh.next_model ? desc_large : desc_small;
-        SampleCtx sc{};
-        sc.vlimit = vlimit;
-        sc.gen = gen;
-        sc.buf = b;
-        sc.desc_small = desc_small;
-        sc.desc_large = desc_large;
-        sc.want_argmax = true;
-        const int ctx_after = gh.kv_len[gh.next_model] + gh.next_m;
-        if (gh.next_m == 1 && gh.next_emit) rc = pass_decode(m, d, b.tokens, slot, ctx_after, sc);
-        else rc = pass_rows(m, d, b.tokens, slot, gh.next_m, ctx_after, gh.next_emit != 0, sc);
-        if (rc != ST_OK) break;
-        if (!gh.next_emit) {
-            advance_ingest_kernel<<<1, 1, 0, s>>>(gen, desc_small, desc_large);
-            ++g_launches;
-            if (cudaGetLastError() != cudaSuccess) { rc = ST_ERR_INTERNAL; break; }
+        g_launches = before;   // counted below from the passes that actually ran
+    } else {
+        // Debugging aid: the same passes launched one by one; the host reads only the shape of the
+        // next pass (which model, how many rows, whether it samples), never a token.
+        const SampleCtx sc = gen_sample_ctx(C);
+        for (int64_t pass = 0; pass < g0.pass_cap; ++pass) {
+            if (cudaMemcpyAsync(&gh, gen, sizeof gh, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+                cudaStreamSynchronize(s) != cudaSuccess) {
+                set_error_text("generation state readback", cudaGetLastError());
+                rc = ST_ERR_INTERNAL;
+                break;
+            }
+            if (gh.done) break;
+            st_model *m = gh.next_model ? large : small;
+            const int slot = gh.next_model ? gl.slot : gs.slot;
+            StepDesc *d = gh.next_model ? desc_large : desc_small;
+            const int ctx_after = gh.kv_len[gh.next_model] + gh.next_m;
+            if (gh.next_m == 1 && gh.next_emit) rc = pass_decode(m, d, b.tokens, slot, ctx_after, sc);
+            else rc = pass_rows(m, d, b.tokens, slot, gh.next_m, ctx_after, gh.next_emit != 0, sc);
+            if (rc != ST_OK) break;
+            if (!gh.next_emit) {
+                advance_ingest_kernel<<<1, 1, 0, s>>>(gen, desc_small, desc_large);
+                ++g_launches;
+                if (cudaGetLastError() != cudaSuccess) { rc = ST_ERR_INTERNAL; break; }
+            }
         }
-        bytes += m->weight_bytes + st_kv_bytes_per_token(m) * (int64_t)ctx_after;
     }
     cudaEventRecord(ev1, s);
-    cudaStreamSynchronize(s);
+    if (cudaStreamSynchronize(s) != cudaSuccess && rc == ST_OK) {
+        set_error_text("generation", cudaGetLastError());
+        rc = ST_ERR_INTERNAL;
+    }
     float ms = 0.f;
     cudaEventElapsedTime(&ms, ev0, ev1);
     cudaEventDestroy(ev0);
     cudaEventDestroy(ev1);
     if (rc != ST_OK) return rc;
+    CK(cudaMemcpy(&gh, gen, sizeof gh, cudaMemcpyDeviceToHost));
     if (!gh.done) return ST_ERR_INTERNAL;
+    if (!host_loop) g_launches += (int64_t)gh.passes + 1;   // dispatch kernels; the passes are counted from the log below
 
     // ---- results ----
     out->n_tokens = gh.generated;
@@ -1048,7 +1278,7 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     out->kv_len_small = gh.kv_len[0];
     out->kv_len_large = gh.kv_len[1];
     out->seconds = ms * 1e-3;
-    out->bytes_algorithmic = bytes;
+    out->bytes_algorithmic = gh.bytes_algo;
     const int n_steps = gh.step < cap_steps ? gh.step : cap_steps;
     const int n_hand = gh.n_handoffs < cap_handoffs ? gh.n_handoffs : cap_handoffs;
     if (gh.generated > 0) {
@@ -1062,8 +1292,13 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
         if (out->emission_argmax) CK(cudaMemcpyAsync(out->emission_argmax, b.em_arg, (size_t)n_steps * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
     }
     if (n_hand > 0) CK(cudaMemcpyAsync(out->handoffs, b.handoffs, (size_t)n_hand * 3 * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
-    if (trace_n > 0) CK(cudaMemcpyAsync(out->logits_trace, d_trace, (size_t)trace_n * vlimit * sizeof(float), cudaMemcpyDeviceToHost, s));
+    if (trace_n > 0) CK(cudaMemcpyAsync(out->logits_trace, C.d_trace, (size_t)trace_n * vlimit * sizeof(float), cudaMemcpyDeviceToHost, s));
     CK(cudaStreamSynchronize(s));
+    if (!host_loop && n_steps == gh.step) {
+        // count the kernels the graph launched from the emission log (which model ran each pass)
+        for (int t = 0; t < n_steps; ++t)
+            g_launches += out->emission_source[t] ? 3 + 6ll * large->cfg.n_layers : 3 + 6ll * small->cfg.n_layers;
+    }
     int32_t dev_status = 0;
     CK(cudaMemcpy(&dev_status, small->status, sizeof dev_status, cudaMemcpyDeviceToHost));
     if (large) {
@@ -1073,6 +1308,7 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     }
     if (dev_status & DEV_LOG_FULL) return ST_ERR_CAPACITY;
     if (dev_status & DEV_BAD_TOKEN) return ST_ERR_VOCAB;
+    if (dev_status & DEV_WAIT_EXPIRED) return ST_ERR_TIMEOUT;
     if (dev_status) return ST_ERR_INTERNAL;
     return ST_OK;
 }
