@@ -168,8 +168,14 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--workload", default="qwen1p5b_32b", choices=sorted(W.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--max-new", type=int, default=0, help="shorten the generation (profiling runs only)")
+    ap.add_argument("--mean-interval", type=float, default=0.0, help="delimiter spacing override (profiling runs only)")
     args = ap.parse_args()
     w = W.CONFIGS[args.workload]
+    if args.max_new > 0 or args.mean_interval > 0:
+        w = W.Workload(**{**w.__dict__, "name": w.name + "-short",
+                          "max_new_tokens": args.max_new if args.max_new > 0 else w.max_new_tokens,
+                          "mean_interval": args.mean_interval if args.mean_interval > 0 else w.mean_interval})
     if args.impl == "reference":
         return run_reference(args, w)
 
