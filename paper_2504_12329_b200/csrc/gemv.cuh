@@ -30,6 +30,11 @@ struct GemvParams {
     float eps;
 };
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may
+// start while its predecessor still runs; it must not touch the predecessor's results before wait().
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 template <int NW, int S, int R, int U, int PRO, int EPI>
 __global__ void __launch_bounds__(NW * 32) gemv_kernel(const GemvParams p)
 {
@@ -43,11 +48,42 @@ __global__ void __launch_bounds__(NW * 32) gemv_kernel(const GemvParams p)
     __shared__ float s_part[32];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int grp = warp / S, ks = warp % S;
+    const int n_tasks = (p.N + R - 1) / R;
+    const int stride = gridDim.x * G;
+    const int n_iter = (n_tasks + stride - 1) / stride;
+    const int n_chunks = (K + 255) >> 8;
+    const int n_cg = (n_chunks + S * U - 1) / (S * U);   // chunk groups per task, the same for every warp
+    const int n_items = n_iter * n_cg;
+
+    // The weight stream is software-pipelined: item j = (task iteration j / n_cg, chunk group j % n_cg);
+    // the loads of item j + 1 are in flight while item j is multiplied.
+    auto issue = [&](int j, uint4 (&w)[U][R]) {
+        const int it = j / n_cg, cg = j - it * n_cg;
+        const int task = it * stride + blockIdx.x * G + grp;
+        const bool live = j < n_items && task < n_tasks;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int e = ((ks + (cg * U + u) * S) << 8) + (lane << 3);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                int row = task * R + r;
+                row = row < p.N ? row : p.N - 1;
+                w[u][r] = (live && e < K) ? ldg_nc_v4(p.W + (size_t)row * K + e) : make_uint4(0, 0, 0, 0);
+            }
+        }
+    };
+
+    uint4 wa[U][R], wb[U][R];
+    issue(0, wa);   // weights do not depend on the previous kernel: fetch before waiting for it
+
+    pdl_wait();
+    pdl_launch_dependents();
     if (p.desc && p.desc->m <= 0) return;
     const int xrow = p.x_row >= 0 ? p.x_row : p.desc->m - 1;
     const float4 *xin = reinterpret_cast<const float4 *>(p.x + (size_t)xrow * K);
 
-    // ---- prologue: bring x into shared memory (normalised if asked) ----
+    // ---- bring x into shared memory (normalised if asked) ----
     // The two halves of each 8-element piece go to separate arrays so that lanes reading
     // consecutive pieces hit consecutive 16-byte slots (no bank conflicts).
     float ss = 0.f;
@@ -74,54 +110,34 @@ __global__ void __launch_bounds__(NW * 32) gemv_kernel(const GemvParams p)
     }
     __syncthreads();
 
-    // ---- persistent loop over row tasks ----
-    const int grp = warp / S, ks = warp % S;
-    const int n_tasks = (p.N + R - 1) / R;
-    const int stride = gridDim.x * G;
-    const int n_iter = (n_tasks + stride - 1) / stride;
-    const int n_chunks = (K + 255) >> 8;
-    for (int it = 0; it < n_iter; ++it) {
+    float acc[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) acc[r] = 0.f;
+
+    auto consume = [&](int j, const uint4 (&w)[U][R]) {
+        if (j >= n_items) return;
+        const int it = j / n_cg, cg = j - it * n_cg;
         const int task = it * stride + blockIdx.x * G + grp;
         const bool live = task < n_tasks;
-        float acc[R];
 #pragma unroll
-        for (int r = 0; r < R; ++r) acc[r] = 0.f;
-        if (live) {
-            const uint16_t *wrow[R];
+        for (int u = 0; u < U; ++u) {
+            const int e = ((ks + (cg * U + u) * S) << 8) + (lane << 3);
+            if (e < K) {
+                const float4 a = xa[e >> 3], b = xb[e >> 3];
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                int row = task * R + r;
-                row = row < p.N ? row : p.N - 1;
-                wrow[r] = p.W + (size_t)row * K;
-            }
-            for (int c0 = ks; c0 < n_chunks; c0 += S * U) {
-                uint4 w[U][R];
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const int e = ((c0 + u * S) << 8) + (lane << 3);
-#pragma unroll
-                    for (int r = 0; r < R; ++r)
-                        w[u][r] = e < K ? ldg_nc_v4(wrow[r] + e) : make_uint4(0, 0, 0, 0);
-                }
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const int e = ((c0 + u * S) << 8) + (lane << 3);
-                    if (e < K) {
-                        const float4 a = xa[e >> 3], b = xb[e >> 3];
-#pragma unroll
-                        for (int r = 0; r < R; ++r) {
-                            const uint4 v = w[u][r];
-                            float s = acc[r];
-                            s = fmaf(bf16_lo(v.x), a.x, s); s = fmaf(bf16_hi(v.x), a.y, s);
-                            s = fmaf(bf16_lo(v.y), a.z, s); s = fmaf(bf16_hi(v.y), a.w, s);
-                            s = fmaf(bf16_lo(v.z), b.x, s); s = fmaf(bf16_hi(v.z), b.y, s);
-                            s = fmaf(bf16_lo(v.w), b.z, s); s = fmaf(bf16_hi(v.w), b.w, s);
-                            acc[r] = s;
-                        }
-                    }
+                for (int r = 0; r < R; ++r) {
+                    const uint4 v = w[u][r];
+                    float t = acc[r];
+                    t = fmaf(bf16_lo(v.x), a.x, t); t = fmaf(bf16_hi(v.x), a.y, t);
+                    t = fmaf(bf16_lo(v.y), a.z, t); t = fmaf(bf16_hi(v.y), a.w, t);
+                    t = fmaf(bf16_lo(v.z), b.x, t); t = fmaf(bf16_hi(v.z), b.y, t);
+                    t = fmaf(bf16_lo(v.w), b.z, t); t = fmaf(bf16_hi(v.w), b.w, t);
+                    acc[r] = t;
                 }
             }
         }
+        if (cg != n_cg - 1) return;
+        // ---- the task is complete: close the rows ----
 #pragma unroll
         for (int r = 0; r < R; ++r) acc[r] = warp_sum(acc[r]);
         float *rbuf = red + (size_t)(it & 1) * NW * R;
@@ -141,7 +157,7 @@ __global__ void __launch_bounds__(NW * 32) gemv_kernel(const GemvParams p)
                 if (S > 1) {
                     t = 0.f;
 #pragma unroll
-                    for (int s = 0; s < S; ++s) t += rbuf[(grp * S + s) * R + r];
+                    for (int s2 = 0; s2 < S; ++s2) t += rbuf[(grp * S + s2) * R + r];
                 }
                 v[r] = t;
             }
@@ -166,6 +182,15 @@ __global__ void __launch_bounds__(NW * 32) gemv_kernel(const GemvParams p)
                 }
             }
         }
+#pragma unroll
+        for (int r = 0; r < R; ++r) acc[r] = 0.f;
+    };
+
+    for (int j = 0; j < n_items; j += 2) {
+        issue(j + 1, wb);
+        consume(j, wa);
+        issue(j + 2, wa);
+        consume(j + 1, wb);
     }
 }
 

@@ -120,12 +120,20 @@ struct st_model {
 };
 
 static constexpr int kArgmaxBlocks = 64;
-static constexpr int kGemvWarps = 16;
+static constexpr int kGemvWarps = 8;
 static constexpr int kRowSplits = 8;   // most key splits a multi-row pass uses
 
 // ------------------------------------------------------------------------------------------------
 // launch helpers
 // ------------------------------------------------------------------------------------------------
+
+// Programmatic dependent launch lets a weight-streaming kernel fetch its first weights while its
+// predecessor drains (ST_PDL=0 turns it off for debugging).
+static bool use_pdl()
+{
+    static const bool on = [] { const char *e = getenv("ST_PDL"); return !(e && e[0] == '0'); }();
+    return on;
+}
 
 template <int S, int PRO, int EPI>
 static cudaError_t launch_gemv_s(const GemvParams &p, cudaStream_t s, int sms)
@@ -136,13 +144,30 @@ static cudaError_t launch_gemv_s(const GemvParams &p, cudaStream_t s, int sms)
     const int G = NW / S;
     const int n_tasks = (p.N + R - 1) / R;
     const int ctas_needed = (n_tasks + G - 1) / G;
-    int per_sm = (int)((220 * 1024) / (smem + 1024));
-    per_sm = per_sm > 4 ? 4 : per_sm < 1 ? 1 : per_sm;
-    int grid = sms * per_sm;
+    // persistent CTAs: as many as are resident at once (at most two per SM, leaving room for the
+    // next kernel of the chain to start its prefetch)
+    static int occ_cache[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    const int bucket = smem <= 8 * 1024 ? 0 : smem <= 24 * 1024 ? 1 : smem <= 48 * 1024 ? 2 : smem <= 80 * 1024 ? 3 : 4;
+    if (!occ_cache[bucket]) {
+        int n = 0;
+        const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, NW * 32, smem);
+        if (e != cudaSuccess) return e;
+        occ_cache[bucket] = n < 1 ? 1 : n > 2 ? 2 : n;
+    }
+    int grid = sms * occ_cache[bucket];
     if (grid > ctas_needed) grid = ctas_needed;
-    kern<<<grid, NW * 32, smem, s>>>(p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(NW * 32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = use_pdl() ? 1 : 0;
     ++g_launches;
-    return cudaGetLastError();
+    return cudaLaunchKernelEx(&cfg, kern, p);
 }
 
 template <int S, int PRO, int EPI>
