@@ -7,6 +7,7 @@
 
 #include "../../include/st.h"
 #include "attention.cuh"
+#include "decode_mega.cuh"
 #include "gemv.cuh"
 #include "prefill_simt.cuh"
 #include "router.cuh"
@@ -107,6 +108,14 @@ struct st_model {
     int32_t *tokbuf = nullptr;   // [max_rows] staging for explicit calls
     StepDesc *desc = nullptr;    // device
     int32_t *status = nullptr;   // device sticky status word
+    // single-kernel decode step
+    MegaLayer *mega_layers = nullptr;   // device [n_layers]
+    float *X0 = nullptr, *X1 = nullptr, *D1 = nullptr, *D2 = nullptr;   // [h] each
+    unsigned *mega_sync = nullptr;      // [4]
+    int32_t *mega_tickets = nullptr;    // [Hkv]
+    int mega_stages = 0, mega_xarea = 0, mega_splits = 0;
+    size_t mega_smem = 0;
+    bool multi_kernel_decode = false;   // debugging aid: one kernel per phase instead
 
     void *dalloc(size_t bytes)
     {
@@ -334,6 +343,8 @@ static int fill_const(st_model *m, float *out, float v, uint64_t n)
     return ST_OK;
 }
 
+static int mega_attr_all();
+
 // Opt every kernel into the shared memory it may ask for (once per device, outside any capture).
 static int init_kernel_attributes()
 {
@@ -343,8 +354,16 @@ static int init_kernel_attributes()
     CK(cudaFuncSetAttribute(tc_gemm_kernel<TEPI_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
     CK(cudaFuncSetAttribute(tc_gemm_kernel<TEPI_RESADD>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
     CK(cudaFuncSetAttribute(tc_gemm_kernel<TEPI_SILU>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
-    return ST_OK;
+    return mega_attr_all();
 }
+
+static size_t mega_scratch_bytes(int D, int G)
+{
+    // sizeof(MegaAttnScratch<D, G>)
+    return sizeof(float) * ((size_t)kMegaAttnWarps * G * D + 2 * (size_t)kMegaAttnWarps * G + 2 * (size_t)G * kMaxAttnSplits + G);
+}
+
+static int mega_attr_all();
 
 static int check_config(const st_config *c)
 {
@@ -477,12 +496,47 @@ static int model_build(st_model *m)
     }
     ALLOC(m->tickets, int32_t, (size_t)m->max_rows * c.n_kv_heads + 1);
     CK(cudaMemsetAsync(m->tickets, 0, ((size_t)m->max_rows * c.n_kv_heads + 1) * sizeof(int32_t), m->stream));
-    ALLOC(m->amax_val, float, kArgmaxBlocks);
-    ALLOC(m->amax_idx, int32_t, kArgmaxBlocks);
+    ALLOC(m->amax_val, float, kArgmaxBlocks > m->sm_count ? kArgmaxBlocks : m->sm_count);
+    ALLOC(m->amax_idx, int32_t, kArgmaxBlocks > m->sm_count ? kArgmaxBlocks : m->sm_count);
     ALLOC(m->tokbuf, int32_t, m->max_rows);
     ALLOC(m->desc, StepDesc, 1);
     ALLOC(m->status, int32_t, 1);
     CK(cudaMemsetAsync(m->status, 0, sizeof(int32_t), m->stream));
+    // ---- single-kernel decode step ----
+    {
+        std::vector<MegaLayer> ml(c.n_layers);
+        for (int l = 0; l < c.n_layers; ++l) {
+            const LayerWeights &w = m->layers[l];
+            ml[l] = MegaLayer{w.wqkv, w.wo, w.wgu, w.wd, w.bqkv, w.g1, w.g2,
+                              m->kpool + (size_t)l * m->pool_layer_stride, m->vpool + (size_t)l * m->pool_layer_stride};
+        }
+        ALLOC(m->mega_layers, MegaLayer, c.n_layers);
+        CK(cudaMemcpyAsync(m->mega_layers, ml.data(), ml.size() * sizeof(MegaLayer), cudaMemcpyHostToDevice, m->stream));
+        CK(cudaStreamSynchronize(m->stream));
+        ALLOC(m->X0, float, h);
+        ALLOC(m->X1, float, h);
+        ALLOC(m->D1, float, h);
+        ALLOC(m->D2, float, h);
+        ALLOC(m->mega_sync, unsigned, 4);
+        ALLOC(m->mega_tickets, int32_t, c.n_kv_heads);
+        CK(cudaMemsetAsync(m->mega_sync, 0, 4 * sizeof(unsigned), m->stream));
+        CK(cudaMemsetAsync(m->mega_tickets, 0, c.n_kv_heads * sizeof(int32_t), m->stream));
+        int widest = h > qd ? h : qd;
+        widest = widest > f ? widest : f;
+        size_t xarea = (size_t)widest * 4;
+        const size_t scratch = 2 * mega_scratch_bytes(D, c.n_q_heads / c.n_kv_heads);
+        if (scratch > xarea) xarea = scratch;
+        xarea = (xarea + 1023) / 1024 * 1024;
+        int stages = (int)((226 * 1024 - 1024 - (long long)xarea) / kMegaTileBytes);
+        if (stages < 2) return ST_ERR_UNSUPPORTED;
+        m->mega_stages = stages > kMegaMaxStages ? kMegaMaxStages : stages;
+        m->mega_xarea = (int)xarea;
+        m->mega_smem = 1024 + xarea + (size_t)m->mega_stages * kMegaTileBytes;
+        m->mega_splits = (2 * m->sm_count + c.n_kv_heads - 1) / c.n_kv_heads;
+        if (m->mega_splits > kMaxAttnSplits) m->mega_splits = kMaxAttnSplits;
+        const char *e = getenv("ST_MULTI_KERNEL");
+        m->multi_kernel_decode = e && e[0] == '1';
+    }
 #undef ALLOC
     CK(cudaStreamSynchronize(m->stream));
     return ST_OK;
@@ -561,8 +615,75 @@ static int sample_tail(st_model *m, const StepDesc *desc, const SampleCtx &sc)
     return ST_OK;
 }
 
-// Decode pass: exactly one row.  ctx_upper bounds the number of keys (chooses the key split).
+template <int D, int G>
+static cudaError_t mega_launch_dg(const MegaParams &p, int grid, size_t smem, cudaStream_t s, bool attr_only)
+{
+    auto kern = decode_mega_kernel<D, G>;
+    if (attr_only) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
+    kern<<<grid, kMegaThreads, smem, s>>>(p);
+    return cudaGetLastError();
+}
+
+template <int D>
+static cudaError_t mega_launch_d(const MegaParams &p, int G, int grid, size_t smem, cudaStream_t s, bool attr_only)
+{
+    switch (G) {
+    case 1: return mega_launch_dg<D, 1>(p, grid, smem, s, attr_only);
+    case 2: return mega_launch_dg<D, 2>(p, grid, smem, s, attr_only);
+    case 3: return mega_launch_dg<D, 3>(p, grid, smem, s, attr_only);
+    case 4: return mega_launch_dg<D, 4>(p, grid, smem, s, attr_only);
+    case 5: return mega_launch_dg<D, 5>(p, grid, smem, s, attr_only);
+    case 6: return mega_launch_dg<D, 6>(p, grid, smem, s, attr_only);
+    case 7: return mega_launch_dg<D, 7>(p, grid, smem, s, attr_only);
+    case 8: return mega_launch_dg<D, 8>(p, grid, smem, s, attr_only);
+    }
+    return cudaErrorInvalidValue;
+}
+
+static cudaError_t mega_launch(const MegaParams &p, int D, int G, int grid, size_t smem, cudaStream_t s, bool attr_only)
+{
+    if (D == 64) return mega_launch_d<64>(p, G, grid, smem, s, attr_only);
+    if (D == 128) return mega_launch_d<128>(p, G, grid, smem, s, attr_only);
+    return cudaErrorInvalidValue;
+}
+
+static int mega_attr_all()
+{
+    for (int D = 64; D <= 128; D += 64)
+        for (int G = 1; G <= 8; ++G) CK(mega_launch(MegaParams{}, D, G, 0, 0, nullptr, true));
+    return ST_OK;
+}
+
+static int pass_decode_multi(st_model *m, const StepDesc *desc, const int32_t *tok, int slot, int ctx_upper, const SampleCtx &sc);
+
+// Decode pass as one persistent kernel.
 static int pass_decode(st_model *m, const StepDesc *desc, const int32_t *tok, int slot, int ctx_upper, const SampleCtx &sc)
+{
+    if (m->multi_kernel_decode) return pass_decode_multi(m, desc, tok, slot, ctx_upper, sc);
+    const st_config &c = m->cfg;
+    MegaParams p{};
+    p.layers = m->mega_layers;
+    p.embed = m->embed; p.lm_head = m->lm_head; p.gf = m->gf; p.inv_freq = m->inv_freq;
+    p.desc = desc; p.tok = tok;
+    p.kv = kv_view(m, 0, slot);
+    p.X0 = m->X0; p.X1 = m->X1; p.QKV = m->QKV; p.ATT = m->ATT; p.D1 = m->D1; p.D2 = m->D2; p.ACT = m->ACT;
+    p.logits = sc.logits_out ? sc.logits_out : m->logits;
+    p.part_o = m->part_o; p.part_ml = m->part_ml; p.tickets = m->mega_tickets; p.sync = m->mega_sync; p.status = m->status;
+    p.n_layers = c.n_layers; p.h = c.hidden; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.f = c.ffn; p.vocab = c.vocab;
+    p.n_splits = m->mega_splits; p.stages = m->mega_stages; p.xarea_bytes = m->mega_xarea;
+    p.eps = c.rms_eps; p.scale = 1.f / sqrtf((float)c.head_dim);
+    p.want_argmax = sc.want_argmax ? 1 : 0;
+    p.limit = sc.vlimit > 0 ? sc.vlimit : c.vocab;
+    p.part_val = m->amax_val; p.part_idx = m->amax_idx; p.argmax_out = sc.argmax_out;
+    p.gen = sc.gen; p.buf = sc.buf; p.desc_small = sc.desc_small; p.desc_large = sc.desc_large;
+    (void)ctx_upper;
+    CK(mega_launch(p, c.head_dim, c.n_q_heads / c.n_kv_heads, m->sm_count, m->mega_smem, m->stream, false));
+    ++g_launches;
+    return ST_OK;
+}
+
+// Decode pass, one kernel per phase (debugging aid).  ctx_upper bounds the number of keys (chooses the key split).  ctx_upper bounds the number of keys (chooses the key split).
+static int pass_decode_multi(st_model *m, const StepDesc *desc, const int32_t *tok, int slot, int ctx_upper, const SampleCtx &sc)
 {
     const st_config &c = m->cfg;
     const int h = c.hidden, D = c.head_dim, qd = c.n_q_heads * D, kd = c.n_kv_heads * D, f = c.ffn;
@@ -871,6 +992,7 @@ int st_prefill(st_model *m, int32_t slot, const int32_t *tokens_host, int32_t n,
     for (int i = 0; i < n; ++i)
         if ((unsigned)tokens_host[i] >= (unsigned)m->cfg.vocab) return ST_ERR_VOCAB;
     TRY(seq_reserve(m, slot, m->seq_len[slot] + n));
+    CK(cudaMemsetAsync(m->mega_sync, 0, 4 * sizeof(unsigned), m->stream));
     for (int done = 0; done < n;) {
         const int rows = n - done < m->max_rows ? n - done : m->max_rows;
         const bool last = done + rows == n;
@@ -900,6 +1022,7 @@ int st_decode_step(st_model *m, const int32_t *slots_host, const int32_t *tokens
         for (int j = 0; j < i; ++j)
             if (slots_host[j] == slot) return ST_ERR_ARG;
     }
+    CK(cudaMemsetAsync(m->mega_sync, 0, 4 * sizeof(unsigned), m->stream));
     for (int i = 0; i < batch; ++i) {
         const int slot = slots_host[i];
         TRY(seq_reserve(m, slot, m->seq_len[slot] + 1));
@@ -1188,7 +1311,13 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
 
     cudaStream_t s = small->stream;
     CK(cudaMemsetAsync(small->status, 0, sizeof(int32_t), s));
-    if (large) CK(cudaMemsetAsync(large->status, 0, sizeof(int32_t), s));
+    CK(cudaMemsetAsync(small->mega_sync, 0, 4 * sizeof(unsigned), s));
+    CK(cudaMemsetAsync(small->mega_tickets, 0, small->cfg.n_kv_heads * sizeof(int32_t), s));
+    if (large) {
+        CK(cudaMemsetAsync(large->status, 0, sizeof(int32_t), s));
+        CK(cudaMemsetAsync(large->mega_sync, 0, 4 * sizeof(unsigned), s));
+        CK(cudaMemsetAsync(large->mega_tickets, 0, large->cfg.n_kv_heads * sizeof(int32_t), s));
+    }
     const int total = prompt_len + max_new + 1;
     SlotGuard gs{small}, gl{large};
     TRY(st_seq_alloc(small, &gs.slot));
