@@ -170,12 +170,17 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--max-new", type=int, default=0, help="shorten the generation (profiling runs only)")
     ap.add_argument("--mean-interval", type=float, default=0.0, help="delimiter spacing override (profiling runs only)")
+    ap.add_argument("--layers", type=int, default=0, help="cut both models to this many layers (profiling runs only)")
     args = ap.parse_args()
     w = W.CONFIGS[args.workload]
     if args.max_new > 0 or args.mean_interval > 0:
         w = W.Workload(**{**w.__dict__, "name": w.name + "-short",
                           "max_new_tokens": args.max_new if args.max_new > 0 else w.max_new_tokens,
                           "mean_interval": args.mean_interval if args.mean_interval > 0 else w.mean_interval})
+    if args.layers > 0:
+        import dataclasses
+        cut = lambda sh: None if sh is None else dataclasses.replace(sh, name=f"{sh.name}-{args.layers}L", n_layers=args.layers)
+        w = W.Workload(**{**w.__dict__, "name": w.name + f"-{args.layers}L", "small": cut(w.small), "large": cut(w.large)})
     if args.impl == "reference":
         return run_reference(args, w)
 
