@@ -29,8 +29,8 @@ constexpr int kMegaCT = 32 * kMegaConsumers;                      // consumer th
 constexpr int kMegaRowsPerWarp = 4;
 constexpr int kMegaTileRows = kMegaConsumers * kMegaRowsPerWarp;  // 32
 constexpr int kMegaSeg = 512;                                     // K elements per tile
-constexpr int kMegaRowPitch = kMegaSeg * 2;                       // bytes per tile row
-constexpr int kMegaTileBytes = kMegaTileRows * kMegaRowPitch;     // 32 KB
+constexpr int kMegaBoxBytes = kMegaTileRows * 256 * 2;            // one TMA box: 32 rows x 256 elements = 16 KB
+constexpr int kMegaTileBytes = 2 * kMegaBoxBytes;                 // 32 KB: two boxes side by side in K
 constexpr int kMegaMaxStages = 6;
 constexpr uint32_t kMegaSpinLimit = 1u << 22;
 constexpr int kMegaAttnWarps = 4;                                 // warps per attention unit (two units per CTA)
@@ -41,8 +41,14 @@ struct MegaLayer {
     uint16_t *kpool, *vpool;
 };
 
+// TMA descriptors of the weight matrices for the decode ring: boxes of 256 elements x 32 rows, no
+// swizzle (a tile row is 512 contiguous bytes in shared memory), zero fill outside the matrix.
+// Device array: 4 per layer (QKV, O, gate/up, down), then the LM head.
+constexpr int kMegaBoxK = 256;
+
 struct MegaParams {
     const MegaLayer *layers;
+    const CUtensorMap *maps;   // [4 * n_layers + 1], global memory
     const uint16_t *embed, *lm_head;
     const float *gf;
     const double *inv_freq;
@@ -184,21 +190,34 @@ __device__ __forceinline__ void mega_load_x(MegaShared &sh, float4 *xa, float4 *
 {
     const int K8 = K >> 3;
     float ss = 0.f;
-    for (int q = ctid; q < 2 * K8; q += kMegaCT) {
-        float4 v;
-        if (src_embed) {
-            const uint2 e = reinterpret_cast<const uint2 *>(src_embed)[q];
-            v = make_float4(bf16_lo(e.x), bf16_hi(e.x), bf16_lo(e.y), bf16_hi(e.y));
-        } else {
-            v = __ldcg(reinterpret_cast<const float4 *>(x) + q);
+    constexpr int XU = 4;   // loads in flight per thread
+    for (int q0 = ctid; q0 < 2 * K8; q0 += XU * kMegaCT) {
+        float4 v[XU], a[XU];
+#pragma unroll
+        for (int u = 0; u < XU; ++u) {
+            const int q = q0 + u * kMegaCT;
+            v[u] = a[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (q < 2 * K8) {
+                if (src_embed) {
+                    const uint2 e = reinterpret_cast<const uint2 *>(src_embed)[q];
+                    v[u] = make_float4(bf16_lo(e.x), bf16_hi(e.x), bf16_lo(e.y), bf16_hi(e.y));
+                } else {
+                    v[u] = __ldcg(reinterpret_cast<const float4 *>(x) + q);
+                }
+                if (add) a[u] = __ldcg(reinterpret_cast<const float4 *>(add) + q);
+            }
         }
-        if (add) {
-            const float4 a = __ldcg(reinterpret_cast<const float4 *>(add) + q);
-            v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
+#pragma unroll
+        for (int u = 0; u < XU; ++u) {
+            const int q = q0 + u * kMegaCT;
+            if (q < 2 * K8) {
+                float4 t = v[u];
+                t.x += a[u].x; t.y += a[u].y; t.z += a[u].z; t.w += a[u].w;
+                if (x_out && blockIdx.x == 0) reinterpret_cast<float4 *>(x_out)[q] = t;
+                ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
+                ((q & 1) ? xb : xa)[q >> 1] = t;
+            }
         }
-        if (x_out && blockIdx.x == 0) reinterpret_cast<float4 *>(x_out)[q] = v;
-        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-        ((q & 1) ? xb : xa)[q >> 1] = v;
     }
     if (norm) {
         ss = warp_sum(ss);
@@ -231,37 +250,44 @@ __device__ __forceinline__ bool mega_run_tiles(const MegaParams &p, MegaShared &
 {
     int t0, t1, nseg;
     mega_range(ph, blockIdx.x, gridDim.x, t0, t1, nseg);
-    float acc[kMegaRowsPerWarp];
+    float acc[kMegaRowsPerWarp], acc2[kMegaRowsPerWarp];
 #pragma unroll
-    for (int r = 0; r < kMegaRowsPerWarp; ++r) acc[r] = 0.f;
+    for (int r = 0; r < kMegaRowsPerWarp; ++r) acc[r] = acc2[r] = 0.f;
     bool first_seg_seen = false;
     for (int t = t0; t < t1; ++t, ++it) {
         const int slot = it % p.stages, u = it / p.stages;
         const int rb = t / nseg, seg = t - rb * nseg;
         if (seg == 0 || t == t0) first_seg_seen = (seg == 0);
         const int k0 = seg * kMegaSeg;
-        const int kl = min(kMegaSeg, ph.K - k0);
         // after an expired wait every later wait returns at once: the step runs to its end (with a
         // status bit set) instead of leaving warps behind at a barrier
         mbar_wait(smem_u32(&sh.full[slot]), u & 1, &sh.abort, p.status);
-        const uint32_t tile = ring + (uint32_t)slot * kMegaTileBytes + (uint32_t)(cw * kMegaRowsPerWarp) * kMegaRowPitch;
+        const uint32_t tile = ring + (uint32_t)slot * kMegaTileBytes + (uint32_t)(cw * kMegaRowsPerWarp) * (kMegaBoxK * 2);
+        // all weight loads of the tile first (8 x 16 bytes per lane), then the multiplies: two
+        // independent accumulation chains per row
+        uint4 w[kMegaSeg / kMegaBoxK][kMegaRowsPerWarp];
 #pragma unroll
-        for (int c = 0; c < kMegaSeg / 256; ++c) {
-            const int e = c * 256 + lane * 8;
-            if (e < kl) {
+        for (int c = 0; c < kMegaSeg / kMegaBoxK; ++c)
+#pragma unroll
+            for (int r = 0; r < kMegaRowsPerWarp; ++r)
+                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                             : "=r"(w[c][r].x), "=r"(w[c][r].y), "=r"(w[c][r].z), "=r"(w[c][r].w)
+                             : "r"(tile + (uint32_t)c * kMegaBoxBytes + (uint32_t)r * (kMegaBoxK * 2) + (uint32_t)lane * 16));
+#pragma unroll
+        for (int c = 0; c < kMegaSeg / kMegaBoxK; ++c) {
+            const int e = c * kMegaBoxK + lane * 8;
+            if (k0 + e < ph.K) {
                 const float4 a = xa[(k0 + e) >> 3], b = xb[(k0 + e) >> 3];
 #pragma unroll
                 for (int r = 0; r < kMegaRowsPerWarp; ++r) {
-                    uint4 v;
-                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                                 : "r"(tile + (uint32_t)r * kMegaRowPitch + (uint32_t)e * 2));
-                    float s = acc[r];
-                    s = fmaf(bf16_lo(v.x), a.x, s); s = fmaf(bf16_hi(v.x), a.y, s);
-                    s = fmaf(bf16_lo(v.y), a.z, s); s = fmaf(bf16_hi(v.y), a.w, s);
-                    s = fmaf(bf16_lo(v.z), b.x, s); s = fmaf(bf16_hi(v.z), b.y, s);
-                    s = fmaf(bf16_lo(v.w), b.z, s); s = fmaf(bf16_hi(v.w), b.w, s);
-                    acc[r] = s;
+                    const uint4 v = w[c][r];
+                    float s0 = acc[r], s1 = acc2[r];
+                    s0 = fmaf(bf16_lo(v.x), a.x, s0); s1 = fmaf(bf16_hi(v.x), a.y, s1);
+                    s0 = fmaf(bf16_lo(v.y), a.z, s0); s1 = fmaf(bf16_hi(v.y), a.w, s1);
+                    s0 = fmaf(bf16_lo(v.z), b.x, s0); s1 = fmaf(bf16_hi(v.z), b.y, s1);
+                    s0 = fmaf(bf16_lo(v.w), b.z, s0); s1 = fmaf(bf16_hi(v.w), b.w, s1);
+                    acc[r] = s0;
+                    acc2[r] = s1;
                 }
             }
         }
@@ -270,7 +296,7 @@ __device__ __forceinline__ bool mega_run_tiles(const MegaParams &p, MegaShared &
         if (seg == nseg - 1 || t == t1 - 1) {
             // close this CTA's share of the row block
 #pragma unroll
-            for (int r = 0; r < kMegaRowsPerWarp; ++r) acc[r] = warp_sum(acc[r]);
+            for (int r = 0; r < kMegaRowsPerWarp; ++r) acc[r] = warp_sum(acc[r] + acc2[r]);
             const int row0 = rb * kMegaTileRows + cw * kMegaRowsPerWarp;
             if (EPI == MEPI_SILU) {
                 if (lane < kMegaRowsPerWarp / 2) {
@@ -289,7 +315,7 @@ __device__ __forceinline__ bool mega_run_tiles(const MegaParams &p, MegaShared &
                 }
             }
 #pragma unroll
-            for (int r = 0; r < kMegaRowsPerWarp; ++r) acc[r] = 0.f;
+            for (int r = 0; r < kMegaRowsPerWarp; ++r) acc[r] = acc2[r] = 0.f;
             first_seg_seen = false;
         }
     }
@@ -549,14 +575,15 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
                 }
                 const int rb = t / nseg, seg = t - rb * nseg;
                 const int r0 = rb * kMegaTileRows, k0 = seg * kMegaSeg;
-                const int kl = min(kMegaSeg, ph.K - k0);
-                const int rows = min(kMegaTileRows, ph.N - r0);
-                const uint32_t full = smem_u32(&sh.full[slot]);
-                if (lane == 0) mbar_expect_tx(full, (uint32_t)rows * (uint32_t)kl * 2u);
+                if (lane == 0) {
+                    const uint32_t full = smem_u32(&sh.full[slot]);
+                    const uint32_t dst = ring + (uint32_t)slot * kMegaTileBytes;
+                    const bool two = k0 + kMegaBoxK < ph.K;     // the second box lies inside the matrix
+                    mbar_expect_tx(full, two ? kMegaTileBytes : kMegaBoxBytes);
+                    tma_load_2d(dst, p.maps + idx, k0, r0, full);
+                    if (two) tma_load_2d(dst + kMegaBoxBytes, p.maps + idx, k0 + kMegaBoxK, r0, full);
+                }
                 __syncwarp();
-                if (lane < rows)
-                    bulk_copy_g2s(ring + (uint32_t)slot * kMegaTileBytes + (uint32_t)lane * kMegaRowPitch,
-                                  ph.W + (size_t)(r0 + lane) * ph.K + k0, (uint32_t)kl * 2u, full);
             }
         }
         if (!ok && lane == 0) {

@@ -110,6 +110,7 @@ struct st_model {
     int32_t *status = nullptr;   // device sticky status word
     // single-kernel decode step
     MegaLayer *mega_layers = nullptr;   // device [n_layers]
+    CUtensorMap *mega_maps = nullptr;   // device [4 * n_layers + 1]
     float *X0 = nullptr, *X1 = nullptr, *D1 = nullptr, *D2 = nullptr;   // [h] each
     unsigned *mega_sync = nullptr;      // [4]
     int32_t *mega_tickets = nullptr;    // [Hkv]
@@ -257,9 +258,10 @@ static EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
-// 2-D bf16 tensor [rows][K] (K contiguous), boxes of 64 x box_rows elements, 128-byte swizzle,
-// out-of-range elements read as zero.
-static int make_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64_t K, uint32_t box_rows)
+// 2-D bf16 tensor [rows][K] (K contiguous), boxes of box_k x box_rows elements (64 wide with the
+// 128-byte swizzle by default), out-of-range elements read as zero.
+static int make_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64_t K, uint32_t box_rows,
+                         uint32_t box_k = kTcBlockK, bool swizzle128 = true)
 {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) {
@@ -268,10 +270,11 @@ static int make_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint
     }
     const cuuint64_t gdim[2] = {K, rows};
     const cuuint64_t gstride[1] = {K * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kTcBlockK, box_rows};
+    const cuuint32_t box[2] = {box_k, box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estr,
-                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         snprintf(g_err_text, sizeof g_err_text, "cuTensorMapEncodeTiled failed (%d)", (int)r);
@@ -513,6 +516,20 @@ static int model_build(st_model *m)
         ALLOC(m->mega_layers, MegaLayer, c.n_layers);
         CK(cudaMemcpyAsync(m->mega_layers, ml.data(), ml.size() * sizeof(MegaLayer), cudaMemcpyHostToDevice, m->stream));
         CK(cudaStreamSynchronize(m->stream));
+        {   // decode-ring TMA descriptors: 256 x 32 boxes without swizzle
+            std::vector<CUtensorMap> maps(4 * c.n_layers + 1);
+            for (int l = 0; l < c.n_layers; ++l) {
+                const LayerWeights &w = m->layers[l];
+                TRY(make_map_bf16(&maps[4 * l + 0], w.wqkv, qkvd, h, kMegaTileRows, kMegaBoxK, false));
+                TRY(make_map_bf16(&maps[4 * l + 1], w.wo, h, qd, kMegaTileRows, kMegaBoxK, false));
+                TRY(make_map_bf16(&maps[4 * l + 2], w.wgu, 2 * f, h, kMegaTileRows, kMegaBoxK, false));
+                TRY(make_map_bf16(&maps[4 * l + 3], w.wd, h, f, kMegaTileRows, kMegaBoxK, false));
+            }
+            TRY(make_map_bf16(&maps[4 * c.n_layers], m->lm_head, c.vocab, h, kMegaTileRows, kMegaBoxK, false));
+            ALLOC(m->mega_maps, CUtensorMap, maps.size());
+            CK(cudaMemcpyAsync(m->mega_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, m->stream));
+            CK(cudaStreamSynchronize(m->stream));
+        }
         ALLOC(m->X0, float, h);
         ALLOC(m->X1, float, h);
         ALLOC(m->D1, float, h);
@@ -663,6 +680,7 @@ static int pass_decode(st_model *m, const StepDesc *desc, const int32_t *tok, in
     const st_config &c = m->cfg;
     MegaParams p{};
     p.layers = m->mega_layers;
+    p.maps = m->mega_maps;
     p.embed = m->embed; p.lm_head = m->lm_head; p.gf = m->gf; p.inv_freq = m->inv_freq;
     p.desc = desc; p.tok = tok;
     p.kv = kv_view(m, 0, slot);
