@@ -33,7 +33,7 @@ constexpr int kMegaBoxBytes = kMegaTileRows * 256 * 2;            // one TMA box
 constexpr int kMegaTileBytes = 2 * kMegaBoxBytes;                 // 32 KB: two boxes side by side in K
 constexpr int kMegaMaxStages = 6;
 constexpr uint32_t kMegaSpinLimit = 1u << 22;
-constexpr int kMegaAttnWarps = 4;                                 // warps per attention unit (two units per CTA)
+constexpr int kMegaAttnWarps = kMegaConsumers;                    // all consumer warps work on one attention unit
 
 struct MegaLayer {
     const uint16_t *wqkv, *wo, *wgu, *wd;
@@ -91,10 +91,14 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
     return v;
 }
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kMegaCT) : "memory"); }
-__device__ __forceinline__ void attn_group_sync(int grp)
-{
-    asm volatile("bar.sync %0, %1;" ::"r"(2 + grp), "n"(32 * kMegaAttnWarps) : "memory");
-}
+constexpr int kMegaAttnUK = 4;   // key steps in flight per lane
+
+// First batch of cached keys/values of an attention unit, fetched before the grid barrier that
+// precedes the attention phase (cached K/V do not depend on this layer's QKV).
+struct MegaKvPrefetch {
+    uint4 kf[kMegaAttnUK], vf[kMegaAttnUK];
+    bool ok[kMegaAttnUK];
+};
 
 // The weight matrix of weight phase idx: 4 per layer (QKV, O, gate/up, down), then the LM head.
 struct MegaPhase {
@@ -166,8 +170,8 @@ __device__ __forceinline__ bool mega_grid_barrier(const MegaParams &p, MegaShare
         bool ok = false;
         for (uint32_t it = 0; it < kMegaSpinLimit; ++it) {
             if (ld_acquire_u32(&p.sync[0]) >= target) { ok = true; break; }
-            if (ld_acquire_u32(&p.sync[2])) break;
-            if (it > 32) __nanosleep(40);
+            if ((it & 63) == 63 && ld_acquire_u32(&p.sync[2])) break;
+            if (it > 256) __nanosleep(32);
         }
         if (!ok) {
             atomicExch(&p.sync[2], 1u);
@@ -322,33 +326,68 @@ __device__ __forceinline__ bool mega_run_tiles(const MegaParams &p, MegaShared &
     return true;
 }
 
-// Attention of one (kv head, key split) unit by 4 warps: rotary embedding of q on the fly, cached keys
-// [k0, k1), and the step's own key/value (position pos) taken from the QKV vector by the last split,
-// which also appends them to the cache.  Partials go to part_o / part_ml; the unit that finishes last
-// for its kv head merges the splits into ATT.
-template <int D, int G>
-__device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaShared &sh, MegaAttnScratch<D, G> &sc,
-                                                    const KvView &kv, int hk, int split, int n_splits, int pos, int grp, int gw,
-                                                    int lane)
+// Key range of split `split` of `n_splits` over keys 0..pos.
+__device__ __forceinline__ void mega_split_range(int pos, int split, int n_splits, int &k0, int &k1)
 {
-    constexpr int LPK = D / 8, KPW = 32 / LPK, UK = 4, half = D / 2;
-    const int gt = gw * 32 + lane;                  // thread within the unit
-    const int sub = lane / LPK, ch = (lane % LPK) * 8;
     const int n_keys = pos + 1;
     const int per = (n_keys + n_splits - 1) / n_splits;
-    const int k0 = split * per, k1 = min(n_keys, k0 + per);
+    k0 = split * per;
+    k1 = min(n_keys, k0 + per);
+}
+
+template <int D>
+__device__ __forceinline__ void mega_attention_prefetch(const MegaParams &p, const KvView &kv, int hk, int split, int n_splits,
+                                                        int pos, int cw, int lane, MegaKvPrefetch &pf)
+{
+    constexpr int LPK = D / 8, KPW = 32 / LPK;
+    const int sub = lane / LPK, ch = (lane % LPK) * 8;
+    int k0, k1;
+    mega_split_range(pos, split, n_splits, k0, k1);
+    const int k1c = min(k1, pos);
+    const int base = k0 + (cw * kMegaAttnUK) * KPW;
+#pragma unroll
+    for (int u = 0; u < kMegaAttnUK; ++u) {
+        const int key = base + u * KPW + sub;
+        pf.ok[u] = key < k1c;
+        if (pf.ok[u]) {
+            const size_t off = kv_offset(kv, key, hk, D, p.status) + ch;
+            pf.kf[u] = __ldcg(reinterpret_cast<const uint4 *>(kv.k + off));
+            pf.vf[u] = __ldcg(reinterpret_cast<const uint4 *>(kv.v + off));
+        } else {
+            pf.kf[u] = make_uint4(0, 0, 0, 0);
+            pf.vf[u] = make_uint4(0, 0, 0, 0);
+        }
+    }
+}
+
+// Attention of one (kv head, key split) unit by the CTA's consumer warps: rotary embedding of q on the
+// fly, cached keys [k0, k1) (the first batch already in registers), and the step's own key/value
+// (position pos) taken from the QKV vector by the split that owns it, which also appends them to the
+// cache.  Partials go to part_o / part_ml; the unit that finishes last for its kv head merges the
+// splits into ATT.
+template <int D, int G>
+__device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaShared &sh, MegaAttnScratch<D, G> &sc,
+                                                    const KvView &kv, int hk, int split, int n_splits, int pos, int cw, int lane,
+                                                    MegaKvPrefetch &pf)
+{
+    constexpr int LPK = D / 8, KPW = 32 / LPK, UK = kMegaAttnUK, half = D / 2;
+    const int gt = cw * 32 + lane;                  // thread within the unit
+    const int sub = lane / LPK, ch = (lane % LPK) * 8;
+    int k0, k1;
+    mega_split_range(pos, split, n_splits, k0, k1);
     const int k1c = min(k1, pos);                   // cached keys only
-    const int qkvd = (p.Hq + 2 * p.Hkv) * D;
-    (void)qkvd;
     // rotate 8 channels starting at ch of a head vector v (fp32, unrotated) at this step's position
     auto rotated8 = [&](const float *v, float *out8) {
         const int other = ch < half ? ch + half : ch - half;
         const int j0 = ch < half ? ch : ch - half;
+        const float4 m0 = __ldcg(reinterpret_cast<const float4 *>(v + ch)), m1 = __ldcg(reinterpret_cast<const float4 *>(v + ch + 4));
+        const float4 o0 = __ldcg(reinterpret_cast<const float4 *>(v + other)), o1 = __ldcg(reinterpret_cast<const float4 *>(v + other + 4));
+        const float mine[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+        const float oth[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
             const float2 t = sh.cs[j0 + e];
-            const float mine = __ldcg(v + ch + e), oth = __ldcg(v + other + e);
-            out8[e] = ch < half ? mine * t.x - oth * t.y : mine * t.x + oth * t.y;
+            out8[e] = ch < half ? mine[e] * t.x - oth[e] * t.y : mine[e] * t.x + oth[e] * t.y;
         }
     };
     float q[G][8];
@@ -384,43 +423,43 @@ __device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaSha
             }
         }
     };
-    for (int base = k0 + (gw * UK) * KPW; base < k1c; base += kMegaAttnWarps * UK * KPW) {
-        uint4 kf[UK], vf[UK];
-        bool ok[UK];
+    for (int base = k0 + (cw * UK) * KPW; base < k1c; base += kMegaAttnWarps * UK * KPW) {
+        if (base != k0 + (cw * UK) * KPW) {   // later batches; the first one was fetched ahead of the barrier
 #pragma unroll
-        for (int u = 0; u < UK; ++u) {
-            const int key = base + u * KPW + sub;
-            ok[u] = key < k1c;
-            if (ok[u]) {
-                const size_t off = kv_offset(kv, key, hk, D, p.status) + ch;
-                kf[u] = __ldcg(reinterpret_cast<const uint4 *>(kv.k + off));
-                vf[u] = __ldcg(reinterpret_cast<const uint4 *>(kv.v + off));
-            } else {
-                kf[u] = make_uint4(0, 0, 0, 0);
-                vf[u] = make_uint4(0, 0, 0, 0);
+            for (int u = 0; u < UK; ++u) {
+                const int key = base + u * KPW + sub;
+                pf.ok[u] = key < k1c;
+                if (pf.ok[u]) {
+                    const size_t off = kv_offset(kv, key, hk, D, p.status) + ch;
+                    pf.kf[u] = __ldcg(reinterpret_cast<const uint4 *>(kv.k + off));
+                    pf.vf[u] = __ldcg(reinterpret_cast<const uint4 *>(kv.v + off));
+                } else {
+                    pf.kf[u] = make_uint4(0, 0, 0, 0);
+                    pf.vf[u] = make_uint4(0, 0, 0, 0);
+                }
             }
         }
 #pragma unroll
         for (int u = 0; u < UK; ++u) {
-            const float kk[8] = {bf16_lo(kf[u].x), bf16_hi(kf[u].x), bf16_lo(kf[u].y), bf16_hi(kf[u].y),
-                                 bf16_lo(kf[u].z), bf16_hi(kf[u].z), bf16_lo(kf[u].w), bf16_hi(kf[u].w)};
-            const float vv[8] = {bf16_lo(vf[u].x), bf16_hi(vf[u].x), bf16_lo(vf[u].y), bf16_hi(vf[u].y),
-                                 bf16_lo(vf[u].z), bf16_hi(vf[u].z), bf16_lo(vf[u].w), bf16_hi(vf[u].w)};
-            update(kk, vv, ok[u]);
+            const float kk[8] = {bf16_lo(pf.kf[u].x), bf16_hi(pf.kf[u].x), bf16_lo(pf.kf[u].y), bf16_hi(pf.kf[u].y),
+                                 bf16_lo(pf.kf[u].z), bf16_hi(pf.kf[u].z), bf16_lo(pf.kf[u].w), bf16_hi(pf.kf[u].w)};
+            const float vv[8] = {bf16_lo(pf.vf[u].x), bf16_hi(pf.vf[u].x), bf16_lo(pf.vf[u].y), bf16_hi(pf.vf[u].y),
+                                 bf16_lo(pf.vf[u].z), bf16_hi(pf.vf[u].z), bf16_lo(pf.vf[u].w), bf16_hi(pf.vf[u].w)};
+            update(kk, vv, pf.ok[u]);
         }
     }
-    if (k0 <= pos && pos < k1 && gw == 0) {
+    if (k0 <= pos && pos < k1 && cw == 0) {
         // this step's own key/value: rotate k, round both to bf16 (what the cache holds), append, attend
         float kk[8], vv[8];
         rotated8(p.QKV + (size_t)(p.Hq + hk) * D, kk);
         const float *vsrc = p.QKV + (size_t)(p.Hq + p.Hkv + hk) * D + ch;
+        const float4 v0 = __ldcg(reinterpret_cast<const float4 *>(vsrc)), v1 = __ldcg(reinterpret_cast<const float4 *>(vsrc + 4));
+        const float vraw[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
         uint32_t kb[4], vb[4];
 #pragma unroll
         for (int e = 0; e < 8; e += 2) {
-            const uint16_t k0b = f32_to_bf16_bits(kk[e]), k1b = f32_to_bf16_bits(kk[e + 1]);
-            const uint16_t v0b = f32_to_bf16_bits(__ldcg(vsrc + e)), v1b = f32_to_bf16_bits(__ldcg(vsrc + e + 1));
-            kb[e >> 1] = (uint32_t)k0b | ((uint32_t)k1b << 16);
-            vb[e >> 1] = (uint32_t)v0b | ((uint32_t)v1b << 16);
+            kb[e >> 1] = (uint32_t)f32_to_bf16_bits(kk[e]) | ((uint32_t)f32_to_bf16_bits(kk[e + 1]) << 16);
+            vb[e >> 1] = (uint32_t)f32_to_bf16_bits(vraw[e]) | ((uint32_t)f32_to_bf16_bits(vraw[e + 1]) << 16);
             kk[e] = bf16_lo(kb[e >> 1]); kk[e + 1] = bf16_hi(kb[e >> 1]);
             vv[e] = bf16_lo(vb[e >> 1]); vv[e + 1] = bf16_hi(vb[e >> 1]);
         }
@@ -431,7 +470,7 @@ __device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaSha
         }
         update(kk, vv, sub == 0);
     }
-    // ---- merge lane groups, then the unit's warps ----
+    // ---- merge lane groups, then the warps ----
 #pragma unroll
     for (int g = 0; g < G; ++g) {
 #pragma unroll
@@ -454,13 +493,13 @@ __device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaSha
 #pragma unroll
         for (int g = 0; g < G; ++g) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) sc.o[gw][g][ch + e] = o[g][e];
-            if (lane == 0) { sc.m[gw][g] = mx[g]; sc.d[gw][g] = den[g]; }
+            for (int e = 0; e < 8; ++e) sc.o[cw][g][ch + e] = o[g][e];
+            if (lane == 0) { sc.m[cw][g] = mx[g]; sc.d[cw][g] = den[g]; }
         }
     }
-    attn_group_sync(grp);
+    consumer_sync();
     const int hq0 = hk * G;
-    for (int idx = gt; idx < G * D; idx += 32 * kMegaAttnWarps) {
+    for (int idx = gt; idx < G * D; idx += kMegaCT) {
         const int g = idx / D, c = idx - g * D;
         float mnew = -INFINITY;
 #pragma unroll
@@ -473,26 +512,31 @@ __device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaSha
             osum += sc.o[w][g][c] * cw2;
         }
         const size_t pi = (size_t)(hq0 + g) * n_splits + split;
-        p.part_o[pi * D + c] = osum;
-        if (c == 0) { p.part_ml[pi * 2] = mnew; p.part_ml[pi * 2 + 1] = dsum; }
+        if (n_splits == 1) {
+            p.ATT[(size_t)(hq0 + g) * D + c] = osum / dsum;   // a single split is the final result
+        } else {
+            p.part_o[pi * D + c] = osum;
+            if (c == 0) { p.part_ml[pi * 2] = mnew; p.part_ml[pi * 2 + 1] = dsum; }
+        }
     }
+    if (n_splits == 1) return;
     __threadfence();
-    attn_group_sync(grp);
+    consumer_sync();
     if (gt == 0) {
         const int t = atomicAdd(&p.tickets[hk], 1);
-        sh.last[grp] = (t == n_splits - 1);
-        if (sh.last[grp]) p.tickets[hk] = 0;
+        sh.last[0] = (t == n_splits - 1);
+        if (sh.last[0]) p.tickets[hk] = 0;
     }
-    attn_group_sync(grp);
-    if (sh.last[grp]) {
+    consumer_sync();
+    if (sh.last[0]) {
         __threadfence();
-        for (int idx = gt; idx < G * n_splits; idx += 32 * kMegaAttnWarps) {
+        for (int idx = gt; idx < G * n_splits; idx += kMegaCT) {
             const int g = idx / n_splits, sp = idx - g * n_splits;
             const float2 ml = __ldcg(reinterpret_cast<const float2 *>(p.part_ml) + (size_t)(hq0 + g) * n_splits + sp);
             sc.w[g][sp] = ml.x;
             sc.l[g][sp] = ml.y;
         }
-        attn_group_sync(grp);
+        consumer_sync();
         if (gt < G) {
             float mnew = -INFINITY;
             for (int sp = 0; sp < n_splits; ++sp) mnew = fmaxf(mnew, sc.w[gt][sp]);
@@ -505,8 +549,8 @@ __device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaSha
             }
             sc.den[gt] = dsum;
         }
-        attn_group_sync(grp);
-        for (int idx = gt; idx < G * D; idx += 32 * kMegaAttnWarps) {
+        consumer_sync();
+        for (int idx = gt; idx < G * D; idx += kMegaCT) {
             const int g = idx / D, c = idx - g * D;
             const float *po = p.part_o + (size_t)(hq0 + g) * n_splits * D + c;
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -519,7 +563,6 @@ __device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaSha
             p.ATT[(size_t)(hq0 + g) * D + c] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) / sc.den[g];
         }
     }
-    attn_group_sync(grp);   // the scratch is reused by the unit's next turn
 }
 
 __device__ __forceinline__ void mega_zero(float *buf, int n, int ctid)
@@ -630,19 +673,19 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
         mega_load_x(sh, xa, xb_of(p.h), p.h, p.X1, l > 0 ? p.D2 : nullptr, l == 0 ? p.embed + (size_t)tokid * p.h : nullptr, p.X0,
                     L.g1, p.eps, true, ctid, cw, lane);
         mega_run_tiles<MEPI_ADD>(p, sh, mega_phase<D>(p, 4 * l), ring, xa, xb_of(p.h), p.QKV, L.bqkv, it, cw, lane);
-        mega_grid_barrier(p, sh, epoch, ctid);
-        // ---- attention (two units per CTA at a time) ----
-        mega_zero(p.D2, p.h, ctid);
+        // ---- attention: one (kv head, key split) unit per CTA; its first keys are fetched before the barrier ----
         kv.k = L.kpool;
         kv.v = L.vpool;
-        {
-            const int grp = cw / kMegaAttnWarps, gw = cw % kMegaAttnWarps;
-            // short contexts use fewer key splits (every CTA derives the same number from the position)
-            const int ns = max(1, min(p.n_splits, (pos + 64) / 64));
-            const int n_units = p.Hkv * ns;
-            for (int unit = blockIdx.x * 2 + grp; unit < n_units; unit += gridDim.x * 2)
-                mega_attention_unit<D, G>(p, sh, scratch[grp], kv, unit / ns, unit % ns, ns, pos, grp, gw, lane);
-        }
+        // 64 keys per unit while there are CTAs to spare (every CTA derives the same split count)
+        int ns = (pos + 64) / 64;
+        ns = min(ns, min(p.n_splits, max(1, (int)gridDim.x / p.Hkv)));
+        const bool attn_active = (int)blockIdx.x < p.Hkv * ns;
+        const int a_hk = blockIdx.x / ns, a_split = blockIdx.x - a_hk * ns;
+        MegaKvPrefetch pf;
+        if (attn_active) mega_attention_prefetch<D>(p, kv, a_hk, a_split, ns, pos, cw, lane, pf);
+        mega_grid_barrier(p, sh, epoch, ctid);
+        mega_zero(p.D2, p.h, ctid);
+        if (attn_active) mega_attention_unit<D, G>(p, sh, scratch[0], kv, a_hk, a_split, ns, pos, cw, lane, pf);
         mega_grid_barrier(p, sh, epoch, ctid);
         // ---- O projection into D1 ----
         mega_load_x(sh, xa, xb_of(qd), qd, p.ATT, nullptr, nullptr, nullptr, nullptr, 0.f, false, ctid, cw, lane);

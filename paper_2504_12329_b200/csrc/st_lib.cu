@@ -290,11 +290,19 @@ static int launch_tc_gemm(const CUtensorMap &tw, const CUtensorMap &ta_hi, const
     auto kern = tc_gemm_kernel<EPI>;
     p.m_pad = (m_upper + 31) / 32 * 32;
     if (p.m_pad > 256) return ST_ERR_INTERNAL;
-    p.tmem_cols = p.m_pad <= 32 ? 32 : p.m_pad <= 64 ? 64 : p.m_pad <= 128 ? 128 : 256;
-    const int stage_bytes = kTcWBytes + 2 * p.m_pad * kTcBlockK * 2;
+    // as many 128-row weight tiles per CTA as TMEM (512 columns) and shared memory (two stages) allow,
+    // but no more than leaves every SM a tile
+    int wt = 512 / p.m_pad;
+    wt = wt > 4 ? 4 : wt;
+    while (wt > 1 && 2 * (wt * kTcWBytes + 2 * p.m_pad * kTcBlockK * 2) > 220 * 1024) --wt;
+    while (wt > 1 && (p.N + kTcTileW * wt - 1) / (kTcTileW * wt) * (EPI == TEPI_SILU ? 1 : 4) < sms) --wt;
+    p.w_tiles = wt;
+    int cols = wt * p.m_pad;
+    p.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
+    const int stage_bytes = wt * kTcWBytes + 2 * p.m_pad * kTcBlockK * 2;
     int stages = (220 * 1024) / stage_bytes;
     p.stages = stages > 8 ? 8 : stages;
-    const int n_tiles = (p.N + kTcTileW - 1) / kTcTileW;
+    const int n_tiles = (p.N + kTcTileW * wt - 1) / (kTcTileW * wt);
     const int kb_total = (p.K + kTcBlockK - 1) / kTcBlockK;
     int ks = 1;
     if (EPI != TEPI_SILU) {
@@ -541,7 +549,7 @@ static int model_build(st_model *m)
         int widest = h > qd ? h : qd;
         widest = widest > f ? widest : f;
         size_t xarea = (size_t)widest * 4;
-        const size_t scratch = 2 * mega_scratch_bytes(D, c.n_q_heads / c.n_kv_heads);
+        const size_t scratch = mega_scratch_bytes(D, c.n_q_heads / c.n_kv_heads);
         if (scratch > xarea) xarea = scratch;
         xarea = (xarea + 1023) / 1024 * 1024;
         int stages = (int)((226 * 1024 - 1024 - (long long)xarea) / kMegaTileBytes);
@@ -549,7 +557,7 @@ static int model_build(st_model *m)
         m->mega_stages = stages > kMegaMaxStages ? kMegaMaxStages : stages;
         m->mega_xarea = (int)xarea;
         m->mega_smem = 1024 + xarea + (size_t)m->mega_stages * kMegaTileBytes;
-        m->mega_splits = (2 * m->sm_count + c.n_kv_heads - 1) / c.n_kv_heads;
+        m->mega_splits = m->sm_count / c.n_kv_heads > 0 ? m->sm_count / c.n_kv_heads : 1;
         if (m->mega_splits > kMaxAttnSplits) m->mega_splits = kMaxAttnSplits;
         const char *e = getenv("ST_MULTI_KERNEL");
         m->multi_kernel_decode = e && e[0] == '1';

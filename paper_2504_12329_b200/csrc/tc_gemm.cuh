@@ -9,7 +9,7 @@
 // 128-byte swizzle and consumed from shared memory by tcgen05.mma (kind::f16, fp32 accumulate in
 // TMEM).  The hi and lo activation planes are two MMAs on the same weight tile.
 //
-// One CTA = one 128-row weight tile x one K split.  Warp 0 issues TMA, warp 1 owns TMEM and issues
+// One CTA = w_tiles adjacent 128-row weight tiles x one K split.  Warp 0 issues TMA, warp 1 owns TMEM and issues
 // the MMAs, warps 2..5 drain the accumulator (tcgen05.ld) into the epilogue.  Stages hand over
 // through mbarriers; every wait is bounded and, when it runs out, raises a status bit, lets the CTA
 // drain what it armed, frees its TMEM and returns.  No multicast, no clusters.
@@ -32,7 +32,9 @@ struct TcGemmParams {
     int32_t m_pad;            // MMA N: activation rows padded to a multiple of 32, <= 256
     int32_t stages;           // shared-memory pipeline depth
     int32_t k_splits;
-    int32_t tmem_cols;        // power of two >= max(32, m_pad)
+    int32_t tmem_cols;        // power of two >= max(32, w_tiles * m_pad)
+    int32_t w_tiles;          // 128-row weight tiles per CTA (each with its own accumulator); they share the
+                              // activation tiles of a stage, which cuts the activation re-reads per weight byte
 };
 
 constexpr int kTcTileW = 128;       // weight rows per CTA
@@ -139,7 +141,7 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
     const int m = p.desc->m;
     if (m <= 0) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n0 = blockIdx.x * kTcTileW;
+    const int n0 = blockIdx.x * kTcTileW * p.w_tiles;
     const int kb_total = (p.K + kTcBlockK - 1) / kTcBlockK;
     const int kb_per = (kb_total + p.k_splits - 1) / p.k_splits;
     const int kb0 = blockIdx.y * kb_per;
@@ -148,7 +150,8 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
     if (n_kb <= 0) return;   // uniform for the CTA
 
     const uint32_t a_bytes = (uint32_t)p.m_pad * kTcBlockK * 2;
-    const uint32_t stage_bytes = kTcWBytes + 2 * a_bytes;
+    const uint32_t w_bytes = (uint32_t)p.w_tiles * kTcWBytes;
+    const uint32_t stage_bytes = w_bytes + 2 * a_bytes;
     const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 1024-byte aligned tile area
 
     if (tid == 0) {
@@ -180,9 +183,9 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
                 const uint32_t base = tiles + (uint32_t)s * stage_bytes;
                 mbar_expect_tx(full, stage_bytes);
                 const int kx = (kb0 + i) * kTcBlockK;
-                tma_load_2d(base, &tmW, kx, n0, full);
-                tma_load_2d(base + kTcWBytes, &tmAhi, kx, 0, full);
-                tma_load_2d(base + kTcWBytes + a_bytes, &tmAlo, kx, 0, full);
+                for (int t = 0; t < p.w_tiles; ++t) tma_load_2d(base + (uint32_t)t * kTcWBytes, &tmW, kx, n0 + t * kTcTileW, full);
+                tma_load_2d(base + w_bytes, &tmAhi, kx, 0, full);
+                tma_load_2d(base + w_bytes + a_bytes, &tmAlo, kx, 0, full);
                 armed = i + 1;
             }
             if (s_abort) {
@@ -204,15 +207,18 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t base = tiles + (uint32_t)s * stage_bytes;
-                const uint64_t dw = umma_desc_sw128(base);
-                const uint64_t dh = umma_desc_sw128(base + kTcWBytes);
-                const uint64_t dl = umma_desc_sw128(base + kTcWBytes + a_bytes);
+                const uint64_t dh = umma_desc_sw128(base + w_bytes);
+                const uint64_t dl = umma_desc_sw128(base + w_bytes + a_bytes);
+                for (int t = 0; t < p.w_tiles; ++t) {
+                    const uint64_t dw = umma_desc_sw128(base + (uint32_t)t * kTcWBytes);
+                    const uint32_t acc = tmem + (uint32_t)(t * p.m_pad);   // this tile's accumulator columns
 #pragma unroll
-                for (int k4 = 0; k4 < kTcBlockK / 16; ++k4)   // 16 elements = 32 bytes = 2 descriptor units
-                    umma_bf16(tmem, dw + 2 * k4, dh + 2 * k4, idesc, (i > 0 || k4 > 0) ? 1u : 0u);
+                    for (int k4 = 0; k4 < kTcBlockK / 16; ++k4)   // 16 elements = 32 bytes = 2 descriptor units
+                        umma_bf16(acc, dw + 2 * k4, dh + 2 * k4, idesc, (i > 0 || k4 > 0) ? 1u : 0u);
 #pragma unroll
-                for (int k4 = 0; k4 < kTcBlockK / 16; ++k4)
-                    umma_bf16(tmem, dw + 2 * k4, dl + 2 * k4, idesc, 1u);
+                    for (int k4 = 0; k4 < kTcBlockK / 16; ++k4)
+                        umma_bf16(acc, dw + 2 * k4, dl + 2 * k4, idesc, 1u);
+                }
                 umma_commit(smem_u32(&s_empty[s]));
             }
             if (ok) umma_commit(smem_u32(&s_acc));
@@ -220,30 +226,32 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
     } else {
         // ---------------- epilogue: TMEM -> registers -> global ----------------
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
-        const int row = n0 + q * 32 + lane;     // weight row = output feature
         int ok_i = lane == 0 ? (int)mbar_wait(smem_u32(&s_acc), 0, &s_abort, p.status) : 1;
         const bool ok = __shfl_sync(0xffffffffu, ok_i, 0) != 0;   // one poller per warp, uniform outcome
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (ok) {
-            const float bias = (EPI != TEPI_SILU && p.bias && blockIdx.y == 0 && row < p.N) ? p.bias[row] : 0.f;
-            for (int c0 = 0; c0 < m; c0 += 16) {
-                float v[16];
-                tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+            for (int t = 0; t < p.w_tiles; ++t) {
+                const int row = n0 + t * kTcTileW + q * 32 + lane;     // weight row = output feature
+                const float bias = (EPI != TEPI_SILU && p.bias && blockIdx.y == 0 && row < p.N) ? p.bias[row] : 0.f;
+                for (int c0 = 0; c0 < m; c0 += 16) {
+                    float v[16];
+                    tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(t * p.m_pad + c0), v);
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int c = c0 + j;
-                    if (EPI == TEPI_SILU) {
-                        const float other = __shfl_xor_sync(0xffffffffu, v[j], 1);
-                        if (c < m && !(lane & 1) && row + 1 < p.N) {
-                            const size_t o = (size_t)c * (p.N >> 1) + (row >> 1);
-                            split_bf16(v[j] / (1.f + expf(-v[j])) * other, p.Yb_hi[o], p.Yb_lo[o]);
+                    for (int j = 0; j < 16; ++j) {
+                        const int c = c0 + j;
+                        if (EPI == TEPI_SILU) {
+                            const float other = __shfl_xor_sync(0xffffffffu, v[j], 1);
+                            if (c < m && !(lane & 1) && row + 1 < p.N) {
+                                const size_t o = (size_t)c * (p.N >> 1) + (row >> 1);
+                                split_bf16(v[j] / (1.f + expf(-v[j])) * other, p.Yb_hi[o], p.Yb_lo[o]);
+                            }
+                        } else if (c < m && row < p.N) {
+                            float *dst = p.Yf + (size_t)c * p.N + row;
+                            const float tt = v[j] + bias;
+                            if (p.k_splits > 1) atomicAdd(dst, tt);
+                            else if (EPI == TEPI_RESADD) *dst += tt;
+                            else *dst = tt;
                         }
-                    } else if (c < m && row < p.N) {
-                        float *dst = p.Yf + (size_t)c * p.N + row;
-                        const float t = v[j] + bias;
-                        if (p.k_splits > 1) atomicAdd(dst, t);
-                        else if (EPI == TEPI_RESADD) *dst += t;
-                        else *dst = t;
                     }
                 }
             }
