@@ -290,4 +290,181 @@ __global__ void __launch_bounds__(128) attn_kernel(const AttnParams p)
     }
 }
 
+// Multi-row (prefill / catch-up) attention: the 8 warps of a CTA take 8 consecutive query rows of one kv
+// head and walk the keys together, tile by tile through shared memory, so that every K/V byte is read
+// from L2 once per 8 rows instead of once per row.  Each warp keeps its row's online softmax for all G
+// query heads exactly as the decode kernel does; rows are causal (row i sees keys 0 .. pos0 + i).
+template <int D, int G>
+__global__ void __launch_bounds__(256) attn_rows_kernel(const AttnParams p)
+{
+    constexpr int LPK = D / 8, KPW = 32 / LPK, TK = 64, ROWS = 8;
+    __shared__ uint4 s_k[TK * D / 8], s_v[TK * D / 8];
+    __shared__ float s_w[G][kMaxAttnSplits], s_l[G][kMaxAttnSplits];   // split merge (per warp use, one row at a time)
+    __shared__ float s_den[ROWS][G];
+    __shared__ int s_last[ROWS];
+    const int m = p.desc->m;
+    const int row0 = blockIdx.z * ROWS;
+    if (row0 >= m) return;
+    const int hk = blockIdx.y, split = blockIdx.x;
+    const int Hkv = p.kv.n_kv_heads;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int sub = lane / LPK, ch = (lane % LPK) * 8;
+    const int row = row0 + warp;
+    const bool row_live = row < m;
+    const int n_keys = p.desc->pos0 + (row_live ? row : m - 1) + 1;            // keys of this warp's row
+    const int n_keys_cta = p.desc->pos0 + min(m, row0 + ROWS);                 // keys of the CTA's last row
+    // split the CTA's key range; every row uses the same boundaries (rows with fewer keys stop early)
+    const int per = ((n_keys_cta + p.n_splits - 1) / p.n_splits + TK - 1) / TK * TK;
+    const int k0 = split * per, k1_cta = min(n_keys_cta, k0 + per);
+    const int k1 = min(n_keys, k1_cta);
+
+    float q[G][8];
+    {
+        const float *qrow = p.qkv + (size_t)(row_live ? row : 0) * (p.Hq + 2 * Hkv) * D + (size_t)hk * G * D + ch;
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            const float4 a = *reinterpret_cast<const float4 *>(qrow + g * D);
+            const float4 b = *reinterpret_cast<const float4 *>(qrow + g * D + 4);
+            q[g][0] = a.x * p.scale; q[g][1] = a.y * p.scale; q[g][2] = a.z * p.scale; q[g][3] = a.w * p.scale;
+            q[g][4] = b.x * p.scale; q[g][5] = b.y * p.scale; q[g][6] = b.z * p.scale; q[g][7] = b.w * p.scale;
+        }
+    }
+    float mx[G], den[G], o[G][8];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        mx[g] = -INFINITY;
+        den[g] = 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) o[g][e] = 0.f;
+    }
+    for (int t0 = k0; t0 < k1_cta; t0 += TK) {
+        // ---- stage the key tile: TK keys x D channels of K and of V ----
+        for (int i = tid; i < TK * LPK; i += 256) {
+            const int key = t0 + i / LPK, c8 = (i % LPK) * 8;
+            uint4 kq = make_uint4(0, 0, 0, 0), vq = make_uint4(0, 0, 0, 0);
+            if (key < k1_cta) {
+                const size_t off = kv_offset(p.kv, key, hk, D, p.status) + c8;
+                kq = *reinterpret_cast<const uint4 *>(p.kv.k + off);
+                vq = *reinterpret_cast<const uint4 *>(p.kv.v + off);
+            }
+            s_k[i] = kq;
+            s_v[i] = vq;
+        }
+        __syncthreads();
+        if (row_live) {
+            const int tile_keys = min(TK, k1 - t0);   // may be <= 0 for rows that ended earlier
+            for (int j = 0; j < tile_keys; j += KPW) {
+                const int kj = j + sub;
+                const bool ok = kj < tile_keys;
+                const uint4 kf = s_k[min(kj, TK - 1) * LPK + (lane % LPK)], vf = s_v[min(kj, TK - 1) * LPK + (lane % LPK)];
+                const float kk[8] = {bf16_lo(kf.x), bf16_hi(kf.x), bf16_lo(kf.y), bf16_hi(kf.y),
+                                     bf16_lo(kf.z), bf16_hi(kf.z), bf16_lo(kf.w), bf16_hi(kf.w)};
+                const float vv[8] = {bf16_lo(vf.x), bf16_hi(vf.x), bf16_lo(vf.y), bf16_hi(vf.y),
+                                     bf16_lo(vf.z), bf16_hi(vf.z), bf16_lo(vf.w), bf16_hi(vf.w)};
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    float s = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) s = fmaf(q[g][e], kk[e], s);
+#pragma unroll
+                    for (int off = LPK / 2; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+                    if (ok) {
+                        const float mnew = fmaxf(mx[g], s);
+                        const float corr = __expf(mx[g] - mnew), pw = __expf(s - mnew);
+                        den[g] = den[g] * corr + pw;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) o[g][e] = fmaf(pw, vv[e], o[g][e] * corr);
+                        mx[g] = mnew;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+    }
+    // ---- merge the lane groups of the warp: the row's result for this split ----
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+#pragma unroll
+        for (int off = LPK; off < 32; off <<= 1) {
+            const float m2 = __shfl_xor_sync(0xffffffffu, mx[g], off);
+            const float d2 = __shfl_xor_sync(0xffffffffu, den[g], off);
+            const float mnew = fmaxf(mx[g], m2);
+            const float c1 = mx[g] == -INFINITY ? 0.f : __expf(mx[g] - mnew);
+            const float c2 = m2 == -INFINITY ? 0.f : __expf(m2 - mnew);
+            den[g] = den[g] * c1 + d2 * c2;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float o2 = __shfl_xor_sync(0xffffffffu, o[g][e], off);
+                o[g][e] = o[g][e] * c1 + o2 * c2;
+            }
+            mx[g] = mnew;
+        }
+    }
+    const int hq0 = hk * G;
+    if (p.n_splits == 1) {
+        if (row_live && sub == 0) {
+#pragma unroll
+            for (int g = 0; g < G; ++g)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) attn_store(p, ((size_t)row * p.Hq + hq0 + g) * D + ch + e, o[g][e] / den[g]);
+        }
+        return;
+    }
+    if (row_live && sub == 0) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            const size_t pi = ((size_t)row * p.Hq + hq0 + g) * p.n_splits + split;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) p.part_o[pi * D + ch + e] = o[g][e];
+            if (lane == 0) { p.part_ml[pi * 2] = mx[g]; p.part_ml[pi * 2 + 1] = den[g]; }
+        }
+    }
+    // ---- the CTA that finishes a row last (over the splits) merges that row ----
+    __threadfence();
+    __syncwarp();
+    if (lane == 0) {
+        int last = 0;
+        if (row_live) {
+            const int t = atomicAdd(&p.tickets[row * Hkv + hk], 1);
+            last = (t == p.n_splits - 1);
+            if (last) p.tickets[row * Hkv + hk] = 0;
+        }
+        s_last[warp] = last;
+    }
+    __syncthreads();
+    for (int r = 0; r < ROWS; ++r) {       // the whole CTA merges each finished row in turn
+        if (!s_last[r]) continue;          // uniform: shared flag
+        const int rrow = row0 + r;
+        __threadfence();
+        for (int idx = tid; idx < G * p.n_splits; idx += 256) {
+            const int g = idx / p.n_splits, sp = idx - g * p.n_splits;
+            const float2 ml = __ldcg(reinterpret_cast<const float2 *>(p.part_ml) + ((size_t)rrow * p.Hq + hq0 + g) * p.n_splits + sp);
+            s_w[g][sp] = ml.x;
+            s_l[g][sp] = ml.y;
+        }
+        __syncthreads();
+        if (tid < G) {
+            float mnew = -INFINITY;
+            for (int sp = 0; sp < p.n_splits; ++sp) mnew = fmaxf(mnew, s_w[tid][sp]);
+            float dsum = 0.f;
+            for (int sp = 0; sp < p.n_splits; ++sp) {
+                const float ms = s_w[tid][sp];
+                const float cw = ms == -INFINITY ? 0.f : __expf(ms - mnew);
+                s_w[tid][sp] = cw;
+                dsum += s_l[tid][sp] * cw;
+            }
+            s_den[r][tid] = dsum;
+        }
+        __syncthreads();
+        for (int idx = tid; idx < G * D; idx += 256) {
+            const int g = idx / D, c = idx - g * D;
+            const float *po = p.part_o + ((size_t)rrow * p.Hq + hq0 + g) * p.n_splits * D + c;
+            float acc = 0.f;
+            for (int sp = 0; sp < p.n_splits; ++sp) acc = fmaf(__ldcg(po + (size_t)sp * D), s_w[g][sp], acc);
+            attn_store(p, ((size_t)rrow * p.Hq + hq0 + g) * D + c, acc / s_den[r][g]);
+        }
+        __syncthreads();
+    }
+}
+
 }  // namespace st

@@ -224,6 +224,32 @@ static cudaError_t launch_attn_d(const AttnParams &p, int G, dim3 grid, cudaStre
     return cudaGetLastError();
 }
 
+template <int D>
+static cudaError_t launch_attn_rows_d(const AttnParams &p, int G, dim3 grid, cudaStream_t s)
+{
+    switch (G) {
+    case 1: attn_rows_kernel<D, 1><<<grid, 256, 0, s>>>(p); break;
+    case 2: attn_rows_kernel<D, 2><<<grid, 256, 0, s>>>(p); break;
+    case 3: attn_rows_kernel<D, 3><<<grid, 256, 0, s>>>(p); break;
+    case 4: attn_rows_kernel<D, 4><<<grid, 256, 0, s>>>(p); break;
+    case 5: attn_rows_kernel<D, 5><<<grid, 256, 0, s>>>(p); break;
+    case 6: attn_rows_kernel<D, 6><<<grid, 256, 0, s>>>(p); break;
+    case 7: attn_rows_kernel<D, 7><<<grid, 256, 0, s>>>(p); break;
+    case 8: attn_rows_kernel<D, 8><<<grid, 256, 0, s>>>(p); break;
+    default: return cudaErrorInvalidValue;
+    }
+    ++g_launches;
+    return cudaGetLastError();
+}
+
+// grid = (key splits, kv heads, ceil(rows / 8))
+static cudaError_t launch_attn_rows(const AttnParams &p, int D, int G, dim3 grid, cudaStream_t s)
+{
+    if (D == 64) return launch_attn_rows_d<64>(p, G, grid, s);
+    if (D == 128) return launch_attn_rows_d<128>(p, G, grid, s);
+    return cudaErrorInvalidValue;
+}
+
 static cudaError_t launch_attn(const AttnParams &p, int D, int G, dim3 grid, cudaStream_t s)
 {
     if (D == 64) return launch_attn_d<64>(p, G, grid, s);
@@ -795,7 +821,8 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
     uint16_t *XN_lo = m->XN + (size_t)m->max_rows * h, *ATT_lo = m->ATTb + (size_t)m->max_rows * qd,
              *ACT_lo = m->ACTb + (size_t)m->max_rows * f;
     // few rows over a long context: split the keys so that the pass still fills the GPU
-    int row_splits = (3 * m->sm_count + c.n_kv_heads * m_upper - 1) / (c.n_kv_heads * m_upper);
+    const int row_ctas = c.n_kv_heads * ((m_upper + 7) / 8);
+    int row_splits = (2 * m->sm_count + row_ctas - 1) / row_ctas;
     if (row_splits > ctx_upper / 256) row_splits = ctx_upper / 256;
     row_splits = row_splits < 1 ? 1 : row_splits > kRowSplits ? kRowSplits : row_splits;
     static_assert((int)GEPI_STORE == (int)TEPI_STORE && (int)GEPI_RESADD == (int)TEPI_RESADD && (int)GEPI_SILU == (int)TEPI_SILU, "epilogue ids");
@@ -817,7 +844,7 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
         a.desc = desc; a.qkv = m->QKV; a.kv = kv; a.out_f32 = nullptr; a.out_hi = m->ATTb; a.out_lo = ATT_lo;
         a.part_o = m->part_o; a.part_ml = m->part_ml; a.tickets = m->tickets; a.status = m->status;
         a.Hq = c.n_q_heads; a.n_splits = row_splits; a.scale = 1.f / sqrtf((float)D);
-        CK(launch_attn(a, D, G, dim3(row_splits, c.n_kv_heads, m_upper), s));
+        CK(launch_attn_rows(a, D, G, dim3(row_splits, c.n_kv_heads, (m_upper + 7) / 8), s));
         TRY((rows_gemm<TEPI_RESADD>(m, desc, m_upper, 1, m->ATTb, ATT_lo, tm.wo, w.wo, nullptr, m->X, nullptr, nullptr, h, qd)));
         rmsnorm_rows_kernel<<<m_upper, 256, 0, s>>>(desc, m->X, w.g2, c.rms_eps, h, m->XN, XN_lo);
         ++g_launches;
