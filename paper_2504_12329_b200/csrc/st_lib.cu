@@ -99,6 +99,7 @@ struct st_model {
     uint16_t *ATTb = nullptr;  // [2][max_rows][Hq D]
     float *ACT = nullptr;      // [f] (decode)
     uint16_t *ACTb = nullptr;  // [2][max_rows][f]
+    float *splitk_ws = nullptr;  // [kMaxKSplits][max_rows][max(qkv width, h)] partial sums of K-split projections
     float2 *cs = nullptr;      // [max_rows][D / 2]
     float *logits = nullptr;   // [vocab]
     float *part_o = nullptr, *part_ml = nullptr;
@@ -131,6 +132,7 @@ struct st_model {
 
 static constexpr int kArgmaxBlocks = 64;
 static constexpr int kGemvWarps = 8;
+static constexpr int kMaxKSplits = 8;  // most K splits of a multi-row projection
 static constexpr int kRowSplits = 8;   // most key splits a multi-row pass uses
 
 // ------------------------------------------------------------------------------------------------
@@ -335,16 +337,22 @@ static int launch_tc_gemm(const CUtensorMap &tw, const CUtensorMap &ta_hi, const
         ks = (sms + n_tiles - 1) / n_tiles;
         const int ks_max = kb_total / 8 > 1 ? kb_total / 8 : 1;
         ks = ks > ks_max ? ks_max : ks;
-        ks = ks > 16 ? 16 : ks;
+        ks = ks > kMaxKSplits ? kMaxKSplits : ks;
         const int per = (kb_total + ks - 1) / ks;   // no empty split
         ks = (kb_total + per - 1) / per;
     }
+    if ((p.N & 3) || !p.Ws) ks = 1;
     p.k_splits = ks;
-    if (EPI == TEPI_STORE && ks > 1) CK(cudaMemsetAsync(p.Yf, 0, (size_t)m_upper * p.N * sizeof(float), s));
     const size_t smem = (size_t)p.stages * stage_bytes + 1024;
     kern<<<dim3(n_tiles, ks), 192, smem, s>>>(tw, ta_hi, ta_lo, p);
     ++g_launches;
     CK(cudaGetLastError());
+    if (ks > 1) {
+        int gx = (p.N / 4 + 255) / 256;
+        splitk_reduce_kernel<<<dim3(gx, m_upper), 256, 0, s>>>(p.desc, p.Ws, ks, p.ws_rows, p.N, p.bias, p.Yf, EPI == TEPI_RESADD ? 1 : 0);
+        ++g_launches;
+        CK(cudaGetLastError());
+    }
     return ST_OK;
 }
 
@@ -524,6 +532,7 @@ static int model_build(st_model *m)
     ALLOC(m->ATTb, uint16_t, 2 * (size_t)m->max_rows * qd);
     ALLOC(m->ACT, float, f);
     ALLOC(m->ACTb, uint16_t, 2 * (size_t)m->max_rows * f);
+    ALLOC(m->splitk_ws, float, (size_t)kMaxKSplits * m->max_rows * (qkvd > h ? qkvd : h));
     ALLOC(m->cs, float2, (size_t)m->max_rows * (D / 2));
     ALLOC(m->logits, float, c.vocab);
     {   // split-KV partials: one decode row with up to max_splits splits, or max_rows rows with up to kRowSplits
@@ -807,6 +816,7 @@ static int rows_gemm(st_model *m, const StepDesc *desc, int m_upper, int buffer,
     TRY(act_map(m, buffer, 1, A_lo, K, m_pad, &ta_lo));
     TcGemmParams p{};
     p.desc = desc; p.bias = bias; p.Yf = Yf; p.Yb_hi = Yb_hi; p.Yb_lo = Yb_lo; p.status = m->status; p.N = N; p.K = K;
+    p.Ws = m->splitk_ws; p.ws_rows = m->max_rows;
     return launch_tc_gemm<EPI>(tw, *ta_hi, *ta_lo, p, m_upper, m->sm_count, m->stream);
 }
 

@@ -25,7 +25,9 @@ enum { TEPI_STORE = 0, TEPI_RESADD = 1, TEPI_SILU = 2 };
 struct TcGemmParams {
     const StepDesc *desc;
     const float *bias;        // [N] or null (added by K split 0)
-    float *Yf;                // TEPI_STORE / TEPI_RESADD: [rows][N] fp32 (accumulated with atomics when k_splits > 1)
+    float *Yf;                // TEPI_STORE / TEPI_RESADD: [rows][N] fp32 when k_splits == 1
+    float *Ws;                // k_splits > 1: partial sums [k_splits][ws_rows][N], reduced by splitk_reduce_kernel
+    int32_t ws_rows;
     uint16_t *Yb_hi, *Yb_lo;  // TEPI_SILU: [rows][N / 2] hi/lo planes of silu(row 2j) * row 2j+1
     int32_t *status;
     int32_t N, K;
@@ -126,6 +128,28 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v)
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Sum the K-split partials of a projection in a fixed order: Y[i][n] (+)= sum_s Ws[s][i][n] (+ bias[n]).
+__global__ void splitk_reduce_kernel(const StepDesc *desc, const float *Ws, int k_splits, int ws_rows, int N, const float *bias,
+                                     float *Y, int accumulate)
+{
+    const int i = blockIdx.y;
+    if (i >= desc->m) return;
+    const int n4 = N >> 2;
+    for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < n4; j += gridDim.x * blockDim.x) {
+        float4 acc = bias ? reinterpret_cast<const float4 *>(bias)[j] : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s = 0; s < k_splits; ++s) {
+            const float4 v = __ldcg(reinterpret_cast<const float4 *>(Ws + ((size_t)s * ws_rows + i) * N) + j);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        float4 *dst = reinterpret_cast<float4 *>(Y + (size_t)i * N) + j;
+        if (accumulate) {
+            const float4 o = *dst;
+            acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w;
+        }
+        *dst = acc;
+    }
 }
 
 template <int EPI>
@@ -246,11 +270,14 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
                                 split_bf16(v[j] / (1.f + expf(-v[j])) * other, p.Yb_hi[o], p.Yb_lo[o]);
                             }
                         } else if (c < m && row < p.N) {
-                            float *dst = p.Yf + (size_t)c * p.N + row;
-                            const float tt = v[j] + bias;
-                            if (p.k_splits > 1) atomicAdd(dst, tt);
-                            else if (EPI == TEPI_RESADD) *dst += tt;
-                            else *dst = tt;
+                            if (p.k_splits > 1) {
+                                p.Ws[((size_t)blockIdx.y * p.ws_rows + c) * p.N + row] = v[j];
+                            } else {
+                                float *dst = p.Yf + (size_t)c * p.N + row;
+                                const float tt = v[j] + bias;
+                                if (EPI == TEPI_RESADD) *dst += tt;
+                                else *dst = tt;
+                            }
                         }
                     }
                 }
