@@ -140,6 +140,22 @@ __device__ __forceinline__ void mega_range(const MegaPhase &ph, int cta, int n_c
     }
 }
 
+// Optional phase timeline (compiled in with -DST_MEGA_TRACE): CTA 0 stamps the global timer at every
+// phase boundary of the step.
+#ifdef ST_MEGA_TRACE
+__device__ unsigned long long g_mega_trace[8192];
+#define MEGA_MARK()                                                         \
+    do {                                                                    \
+        if (blockIdx.x == 0 && ctid == 0 && trace_i < 8192) {               \
+            unsigned long long t_;                                          \
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));          \
+            g_mega_trace[trace_i++] = t_;                                   \
+        }                                                                   \
+    } while (0)
+#else
+#define MEGA_MARK() do { } while (0)
+#endif
+
 struct MegaShared {
     uint64_t full[kMegaMaxStages], empty[kMegaMaxStages];
     float red[kMegaConsumers];
@@ -164,8 +180,8 @@ __device__ __forceinline__ bool mega_grid_barrier(const MegaParams &p, MegaShare
 {
     consumer_sync();
     if (ctid == 0) {
-        __threadfence();
-        atomicAdd(&p.sync[0], 1u);
+        // release-add (no return value to wait for), then poll with acquire loads
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.sync) : "memory");
         const unsigned target = (++epoch) * gridDim.x;
         bool ok = false;
         for (uint32_t it = 0; it < kMegaSpinLimit; ++it) {
@@ -178,7 +194,6 @@ __device__ __forceinline__ bool mega_grid_barrier(const MegaParams &p, MegaShare
             atomicOr(p.status, DEV_WAIT_EXPIRED);
             sh.abort = 1;
         }
-        __threadfence();
     } else {
         ++epoch;
     }
@@ -519,49 +534,58 @@ __device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaSha
             if (c == 0) { p.part_ml[pi * 2] = mnew; p.part_ml[pi * 2 + 1] = dsum; }
         }
     }
-    if (n_splits == 1) return;
-    __threadfence();
-    consumer_sync();
-    if (gt == 0) {
-        const int t = atomicAdd(&p.tickets[hk], 1);
-        sh.last[0] = (t == n_splits - 1);
-        if (sh.last[0]) p.tickets[hk] = 0;
-    }
-    consumer_sync();
-    if (sh.last[0]) {
-        __threadfence();
-        for (int idx = gt; idx < G * n_splits; idx += kMegaCT) {
-            const int g = idx / n_splits, sp = idx - g * n_splits;
-            const float2 ml = __ldcg(reinterpret_cast<const float2 *>(p.part_ml) + (size_t)(hq0 + g) * n_splits + sp);
-            sc.w[g][sp] = ml.x;
-            sc.l[g][sp] = ml.y;
+}
+
+// Merge of the key splits, spread over all CTAs (runs between two grid barriers): CTA c owns a
+// contiguous range of the Hq * D output channels; 16 threads share one channel and stride the splits.
+template <int D, int G>
+__device__ __forceinline__ void mega_attention_merge(const MegaParams &p, MegaAttnScratch<D, G> &sc, int n_splits, int ctid)
+{
+    constexpr int TPO = 16;
+    const int n_out = p.Hq * D;
+    const int per = (n_out + gridDim.x - 1) / gridDim.x;
+    const int o0 = blockIdx.x * per, o1 = min(n_out, o0 + per);
+    if (o0 >= o1) return;   // uniform for the CTA
+    float *w = &sc.w[0][0], *l = &sc.l[0][0];
+    for (int hq = o0 / D; hq <= (o1 - 1) / D; ++hq) {
+        for (int sp = ctid; sp < n_splits; sp += kMegaCT) {
+            const float2 ml = __ldcg(reinterpret_cast<const float2 *>(p.part_ml) + (size_t)hq * n_splits + sp);
+            w[sp] = ml.x;
+            l[sp] = ml.y;
         }
         consumer_sync();
-        if (gt < G) {
+        if (ctid < 32) {
             float mnew = -INFINITY;
-            for (int sp = 0; sp < n_splits; ++sp) mnew = fmaxf(mnew, sc.w[gt][sp]);
+            for (int sp = ctid; sp < n_splits; sp += 32) mnew = fmaxf(mnew, w[sp]);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) mnew = fmaxf(mnew, __shfl_xor_sync(0xffffffffu, mnew, o));
             float dsum = 0.f;
-            for (int sp = 0; sp < n_splits; ++sp) {
-                const float ms = sc.w[gt][sp];
+            for (int sp = ctid; sp < n_splits; sp += 32) {
+                const float ms = w[sp];
                 const float cw2 = ms == -INFINITY ? 0.f : __expf(ms - mnew);
-                sc.w[gt][sp] = cw2;
-                dsum += sc.l[gt][sp] * cw2;
+                w[sp] = cw2;
+                dsum += l[sp] * cw2;
             }
-            sc.den[gt] = dsum;
+            dsum = warp_sum(dsum);
+            if (ctid == 0) sc.den[0] = dsum;
         }
         consumer_sync();
-        for (int idx = gt; idx < G * D; idx += kMegaCT) {
-            const int g = idx / D, c = idx - g * D;
-            const float *po = p.part_o + (size_t)(hq0 + g) * n_splits * D + c;
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            int sp = 0;
-            for (; sp + 4 <= n_splits; sp += 4) {
+        const int lo = max(o0, hq * D), hi = min(o1, (hq + 1) * D);
+        const int j = ctid % TPO;
+        const int n_pass = (hi - lo + kMegaCT / TPO - 1) / (kMegaCT / TPO);   // the same for every thread
+        for (int pass = 0; pass < n_pass; ++pass) {
+            const int oi = lo + pass * (kMegaCT / TPO) + ctid / TPO;
+            const bool live = oi < hi;
+            const int c = (live ? oi : lo) - hq * D;
+            const float *po = p.part_o + (size_t)hq * n_splits * D + c;
+            float acc = 0.f;
+            if (live)
+                for (int sp = j; sp < n_splits; sp += TPO) acc = fmaf(__ldcg(po + (size_t)sp * D), w[sp], acc);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) acc[j] = fmaf(__ldcg(po + (size_t)(sp + j) * D), sc.w[g][sp + j], acc[j]);
-            }
-            for (; sp < n_splits; ++sp) acc[0] = fmaf(__ldcg(po + (size_t)sp * D), sc.w[g][sp], acc[0]);
-            p.ATT[(size_t)(hq0 + g) * D + c] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) / sc.den[g];
+            for (int o = TPO / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            if (live && j == 0) p.ATT[(size_t)hq * D + c] = acc / sc.den[0];
         }
+        consumer_sync();
     }
 }
 
@@ -644,6 +668,9 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
     const int pos = p.desc->pos0;
     const int qd = p.Hq * D, kd = p.Hkv * D, qkvd = qd + 2 * kd;
     unsigned epoch = 0, it = 0;
+    int trace_i = 0;
+    (void)trace_i;
+    MEGA_MARK();
     auto xb_of = [&](int K) { return xa + (K >> 3); };
 
     // step set-up: rotary table, zeroed accumulation vectors
@@ -657,6 +684,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
     mega_zero(p.D2, p.h, ctid);
     mega_zero(p.logits, p.vocab, ctid);
     mega_grid_barrier(p, sh, epoch, ctid);
+    MEGA_MARK();
 
     int tokid = p.tok[p.desc->tok_off];
     if ((unsigned)tokid >= (unsigned)p.vocab) {
@@ -670,9 +698,12 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
         const MegaLayer &L = p.layers[l];
         // ---- QKV: x = (layer 0 ? embedding : x1 + down), normalised ----
         if (l > 0) mega_grid_barrier(p, sh, epoch, ctid);
+        MEGA_MARK();
         mega_load_x(sh, xa, xb_of(p.h), p.h, p.X1, l > 0 ? p.D2 : nullptr, l == 0 ? p.embed + (size_t)tokid * p.h : nullptr, p.X0,
                     L.g1, p.eps, true, ctid, cw, lane);
+    MEGA_MARK();
         mega_run_tiles<MEPI_ADD>(p, sh, mega_phase<D>(p, 4 * l), ring, xa, xb_of(p.h), p.QKV, L.bqkv, it, cw, lane);
+    MEGA_MARK();
         // ---- attention: one (kv head, key split) unit per CTA; its first keys are fetched before the barrier ----
         kv.k = L.kpool;
         kv.v = L.vpool;
@@ -684,28 +715,49 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
         MegaKvPrefetch pf;
         if (attn_active) mega_attention_prefetch<D>(p, kv, a_hk, a_split, ns, pos, cw, lane, pf);
         mega_grid_barrier(p, sh, epoch, ctid);
+    MEGA_MARK();
         mega_zero(p.D2, p.h, ctid);
         if (attn_active) mega_attention_unit<D, G>(p, sh, scratch[0], kv, a_hk, a_split, ns, pos, cw, lane, pf);
+        MEGA_MARK();
+        if (ns > 1) {   // uniform over the grid: ns depends on the position only
+            mega_grid_barrier(p, sh, epoch, ctid);
+            MEGA_MARK();
+            mega_attention_merge<D, G>(p, scratch[0], ns, ctid);
+            MEGA_MARK();
+        }
         mega_grid_barrier(p, sh, epoch, ctid);
+    MEGA_MARK();
         // ---- O projection into D1 ----
         mega_load_x(sh, xa, xb_of(qd), qd, p.ATT, nullptr, nullptr, nullptr, nullptr, 0.f, false, ctid, cw, lane);
+    MEGA_MARK();
         mega_run_tiles<MEPI_ADD>(p, sh, mega_phase<D>(p, 4 * l + 1), ring, xa, xb_of(qd), p.D1, nullptr, it, cw, lane);
+    MEGA_MARK();
         mega_grid_barrier(p, sh, epoch, ctid);
+    MEGA_MARK();
         // ---- gate/up: x1 = x0 + D1, normalised ----
         mega_load_x(sh, xa, xb_of(p.h), p.h, p.X0, p.D1, nullptr, p.X1, L.g2, p.eps, true, ctid, cw, lane);
+    MEGA_MARK();
         mega_zero(p.QKV, qkvd, ctid);
         mega_run_tiles<MEPI_SILU>(p, sh, mega_phase<D>(p, 4 * l + 2), ring, xa, xb_of(p.h), p.ACT, nullptr, it, cw, lane);
+    MEGA_MARK();
         mega_grid_barrier(p, sh, epoch, ctid);
+    MEGA_MARK();
         // ---- down projection into D2 ----
         mega_load_x(sh, xa, xb_of(p.f), p.f, p.ACT, nullptr, nullptr, nullptr, nullptr, 0.f, false, ctid, cw, lane);
+    MEGA_MARK();
         mega_zero(p.D1, p.h, ctid);
         mega_run_tiles<MEPI_ADD>(p, sh, mega_phase<D>(p, 4 * l + 3), ring, xa, xb_of(p.f), p.D2, nullptr, it, cw, lane);
+    MEGA_MARK();
     }
     // ---- LM head ----
     mega_grid_barrier(p, sh, epoch, ctid);
+    MEGA_MARK();
     mega_load_x(sh, xa, xb_of(p.h), p.h, p.X1, p.D2, nullptr, nullptr, p.gf, p.eps, true, ctid, cw, lane);
+    MEGA_MARK();
     mega_run_tiles<MEPI_ADD>(p, sh, mega_phase<D>(p, 4 * p.n_layers), ring, xa, xb_of(p.h), p.logits, nullptr, it, cw, lane);
+    MEGA_MARK();
     mega_grid_barrier(p, sh, epoch, ctid);
+    MEGA_MARK();
 
     // ---- sampling + router ----
     if (p.want_argmax) {

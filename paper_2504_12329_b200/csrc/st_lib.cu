@@ -939,6 +939,10 @@ int64_t st_kv_bytes_per_token(const st_model *m)
 
 int64_t st_kernel_launches(void) { return g_launches; }
 
+#ifdef ST_MEGA_TRACE
+int st_debug_trace(unsigned long long *out, int n) { return (int)cudaMemcpyFromSymbol(out, g_mega_trace, (size_t)n * 8); }
+#endif
+
 int st_seq_alloc(st_model *m, int32_t *slot_out)
 {
     if (!m || !slot_out) return ST_ERR_ARG;
