@@ -30,6 +30,7 @@ struct GenState {
     int32_t next_m;      // ... ingests this many tokens ...
     int32_t next_emit;   // ... and samples a token (1) or only ingests (0)
     int32_t passes;      // passes dispatched so far
+    int32_t body_runs[12];  // how often each graph body ran (per model: decode, 4 row buckets, ingest)
     int32_t pass_cap;    // hard bound on passes (the device loop stops there)
     // --- parameters ---
     int32_t has_large, delimiter, n1, keep_probe, eos, vlimit, max_new, n_force;
@@ -158,8 +159,10 @@ __global__ void dispatch_kernel(GenState *g, cudaGraphConditionalHandle loop, cu
         return;
     }
     g->passes++;
+    const int b = pass_body_index(g->next_model, g->next_m, g->next_emit);
+    g->body_runs[b]++;
     cudaGraphSetConditional(loop, 1);
-    cudaGraphSetConditional(body, (unsigned)pass_body_index(g->next_model, g->next_m, g->next_emit));
+    cudaGraphSetConditional(body, (unsigned)b);
 }
 
 struct ArgmaxParams {

@@ -1134,6 +1134,7 @@ struct GenContext {
     std::vector<void *> ptrs;
     cudaGraph_t graph = nullptr;
     cudaGraphExec_t exec = nullptr;
+    int64_t body_launches[2 * kBodiesPerModel] = {};   // kernels in each captured body
 
     template <class T>
     T *get(size_t n)
@@ -1272,8 +1273,12 @@ static int build_gen_graph(GenContext &c, st_model *small)
         sp.conditional.size = (unsigned)n_bodies;
         cudaGraphNode_t snode;
         if (cudaGraphAddNode(&snode, loop_body, &dnode, 1, &sp) != cudaSuccess) { rc = ST_ERR_INTERNAL; break; }
-        for (int i = 0; i < n_bodies && rc == ST_OK; ++i)
+        for (int i = 0; i < n_bodies && rc == ST_OK; ++i) {
+            const int64_t before = g_launches;
             rc = capture_body(c, small, cap, sp.conditional.phGraph_out[i], i / kBodiesPerModel, i % kBodiesPerModel);
+            c.body_launches[i] = g_launches - before;   // captured, not run
+            g_launches = before;
+        }
         if (rc != ST_OK) break;
         if (cudaGraphInstantiate(&c.exec, c.graph, 0) != cudaSuccess) { rc = ST_ERR_INTERNAL; break; }
     } while (0);
@@ -1490,7 +1495,10 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     if (rc != ST_OK) return rc;
     CK(cudaMemcpy(&gh, gen, sizeof gh, cudaMemcpyDeviceToHost));
     if (!gh.done) return ST_ERR_INTERNAL;
-    if (!host_loop) g_launches += (int64_t)gh.passes + 1;   // dispatch kernels; the passes are counted from the log below
+    if (!host_loop) {   // kernels the graph ran: one dispatch per loop turn plus the kernels of every body that ran
+        g_launches += (int64_t)gh.passes + 1;
+        for (int i = 0; i < 2 * kBodiesPerModel; ++i) g_launches += C.body_launches[i] * gh.body_runs[i];
+    }
 
     // ---- results ----
     out->n_tokens = gh.generated;
@@ -1515,11 +1523,6 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     if (n_hand > 0) CK(cudaMemcpyAsync(out->handoffs, b.handoffs, (size_t)n_hand * 3 * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
     if (trace_n > 0) CK(cudaMemcpyAsync(out->logits_trace, C.d_trace, (size_t)trace_n * vlimit * sizeof(float), cudaMemcpyDeviceToHost, s));
     CK(cudaStreamSynchronize(s));
-    if (!host_loop && n_steps == gh.step) {
-        // count the kernels the graph launched from the emission log (which model ran each pass)
-        for (int t = 0; t < n_steps; ++t)
-            g_launches += out->emission_source[t] ? 3 + 6ll * large->cfg.n_layers : 3 + 6ll * small->cfg.n_layers;
-    }
     int32_t dev_status = 0;
     CK(cudaMemcpy(&dev_status, small->status, sizeof dev_status, cudaMemcpyDeviceToHost));
     if (large) {
