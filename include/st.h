@@ -159,6 +159,18 @@ int64_t st_kv_bytes_per_token(const st_model *m);
 int64_t st_kernel_launches(void);
 int st_time_gemv(st_model *m, int32_t which, int32_t iters, double *seconds_out);
 
+/* Greedy sampling that allocates nothing (the paper has no counterpart: this is a service entry point).
+ * For callers that must not call cudaMalloc -- code running while another component owns the whole
+ * device memory pool, or inside a region where allocation is forbidden or would synchronise the device.
+ * Computes the lowest-id argmax of logits_dev[0..n) (fp32, device) into *argmax_out_dev (int32, device),
+ * the same selection rule as st_decode_step's argmax_dev, on `cuda_stream`.  Its scratch (partial
+ * maxima and a ticket word, 1 KB) is a fixed array inside the library image, present on every GPU
+ * that loads the library until the process exits; n may be at most 4,194,304 (1 << 22), larger sizes
+ * return ST_ERR_CAPACITY.  The first call on a device looks up the array's device address (no
+ * allocation); make that first call outside any stream capture.  All calls share the one array:
+ * calls that overlap on the GPU (different streams) race and must be serialised by the caller. */
+int st_argmax_static(const float *logits_dev, int32_t n, int32_t *argmax_out_dev, void *cuda_stream);
+
 /* Sticky device status word (0 = clean) and message text. */
 int st_last_device_status(st_model *m);
 const char *st_strerror(int status);

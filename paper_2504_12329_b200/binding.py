@@ -63,7 +63,7 @@ EXPORTS = [
     "st_model_create", "st_model_destroy", "st_seq_alloc", "st_seq_free", "st_seq_reserve", "st_kv_len",
     "st_kv_truncate", "st_prefill", "st_decode_step", "st_generate_spec", "st_fill_tensor_bf16",
     "st_weight_bytes", "st_kv_bytes_per_token", "st_last_device_status", "st_strerror",
-    "st_kernel_launches", "st_time_gemv",
+    "st_kernel_launches", "st_time_gemv", "st_argmax_static",
 ]
 
 _lib = None
@@ -109,6 +109,8 @@ def lib():
         L.st_kernel_launches.argtypes = []
         L.st_time_gemv.restype = C.c_int
         L.st_time_gemv.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_double)]
+        L.st_argmax_static.restype = C.c_int
+        L.st_argmax_static.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.st_strerror.restype = C.c_char_p
         L.st_strerror.argtypes = [C.c_int]
         _lib = L
@@ -128,6 +130,12 @@ def _check(rc: int, where: str):
 
 def st_kernel_launches() -> int:
     return lib().st_kernel_launches()
+
+
+def st_argmax_static(logits, n: int, argmax_out, stream: int = 0):
+    """Lowest-id argmax of a device fp32 vector into a device int32, using only the library's built-in
+    scratch array (no allocation anywhere on the path)."""
+    _check(lib().st_argmax_static(_dev_ptr(logits), n, _dev_ptr(argmax_out), C.c_void_p(stream)), "st_argmax_static")
 
 
 def st_strerror(status: int) -> str:

@@ -1536,3 +1536,49 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     if (dev_status) return ST_ERR_INTERNAL;
     return ST_OK;
 }
+
+// ------------------------------------------------------------------------------------------------
+// greedy sampling without any allocation
+// ------------------------------------------------------------------------------------------------
+
+// Scratch of st_argmax_static: 64 partial maxima, 64 partial indices (int bits) and one ticket word.
+// It lives in the library image, so every GPU that loads the library holds these 1 KB until exit.
+static constexpr int kStaticArgmaxBlocks = 64;
+static constexpr int32_t kStaticArgmaxMaxN = 1 << 22;
+static __device__ __align__(256) float g_static_argmax_scratch[256];
+
+extern "C" int st_argmax_static(const float *logits_dev, int32_t n, int32_t *argmax_out_dev, void *cuda_stream)
+{
+    if (!logits_dev || !argmax_out_dev || n < 1) return ST_ERR_ARG;
+    if (n > kStaticArgmaxMaxN) {
+        snprintf(g_err_text, sizeof g_err_text, "st_argmax_static: %d elements exceed the built-in scratch limit of %d", n,
+                 kStaticArgmaxMaxN);
+        return ST_ERR_CAPACITY;
+    }
+    // The symbol name is only a host-side handle; the kernel needs the device address, looked up once
+    // per device with that device current.
+    static float *scratch_of_device[64] = {};
+    int dev = 0;
+    CK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return ST_ERR_UNSUPPORTED;
+    if (!scratch_of_device[dev]) {
+        float *ptr = nullptr;
+        CK(cudaGetSymbolAddress((void **)&ptr, g_static_argmax_scratch));
+        scratch_of_device[dev] = ptr;
+    }
+    float *scratch = scratch_of_device[dev];
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    // the array keeps whatever the previous call left: the ticket word must start at zero
+    CK(cudaMemsetAsync(scratch + 2 * kStaticArgmaxBlocks, 0, sizeof(int32_t), s));
+    ArgmaxParams a{};
+    a.logits = logits_dev;
+    a.limit = n;
+    a.part_val = scratch;
+    a.part_idx = reinterpret_cast<int32_t *>(scratch + kStaticArgmaxBlocks);
+    a.ticket = reinterpret_cast<int32_t *>(scratch + 2 * kStaticArgmaxBlocks);
+    a.argmax_out = argmax_out_dev;
+    argmax_router_kernel<<<kStaticArgmaxBlocks, 256, 0, s>>>(a);
+    ++g_launches;
+    CK(cudaGetLastError());
+    return ST_OK;
+}
