@@ -141,6 +141,23 @@ def schedule_stats(w: W.Workload):
     return {"steps_small": steps[0], "steps_large": steps[1], "n_tokens": gen}
 
 
+def aggregate_over_ranks(dev_s: float, e2e_s: float, n_tokens: float, dist_mod=None, device="cpu"):
+    """Whole-job figures of a replicas-only run: time = the slowest rank, tokens = the sum over ranks."""
+    if dist_mod is None or not dist_mod.is_initialized() or dist_mod.get_world_size() == 1:
+        return dev_s, e2e_s, n_tokens
+    import torch
+    t = torch.tensor([dev_s, e2e_s], dtype=torch.float64, device=device)
+    dist_mod.all_reduce(t, op=dist_mod.ReduceOp.MAX)
+    n = torch.tensor([n_tokens], dtype=torch.float64, device=device)
+    dist_mod.all_reduce(n, op=dist_mod.ReduceOp.SUM)
+    return float(t[0]), float(t[1]), float(n[0])
+
+
+def rank_workload(w: W.Workload, rank: int) -> W.Workload:
+    """Each rank runs an independent replica of the workload with its own input seed."""
+    return W.Workload(**{**w.__dict__, "input_seed": w.input_seed + 1000 * rank})
+
+
 def run_reference(args, w):
     if int(os.environ.get("RANK", "0")) != 0:
         return
@@ -197,7 +214,7 @@ def main():
 
     # The generation is one dependent chain of tokens: it does not shard.  With N > 1 every rank runs
     # an independent replica of the workload (its own input seed); there is no data-path collective.
-    wl = W.Workload(**{**w.__dict__, "input_seed": w.input_seed + 1000 * rank})
+    wl = rank_workload(w, rank)
     prompt, force = W.workload_inputs(wl)
     cap = wl.prompt_len + wl.max_new_tokens + 64
     small = B.Model(wl.small.as_dict(), seed=wl.weight_seed, tag=0, max_tokens=cap)
@@ -231,12 +248,7 @@ def main():
 
     r = results[-1]
     n_tokens = float(sum(len(x.tokens) for x in results))
-    if world > 1:
-        t = torch.tensor([dev_s, e2e_s], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        n = torch.tensor([n_tokens], dtype=torch.float64, device="cuda")
-        dist.all_reduce(n, op=dist.ReduceOp.SUM)
-        dev_s, e2e_s, n_tokens = float(t[0]), float(t[1]), float(n[0])
+    dev_s, e2e_s, n_tokens = aggregate_over_ranks(dev_s, e2e_s, n_tokens, dist if world > 1 else None, "cuda")
     value = n_tokens / dev_s
     e2e_value = n_tokens / e2e_s
 
