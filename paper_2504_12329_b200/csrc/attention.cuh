@@ -1,6 +1,6 @@
 // Rotary embedding + KV append, and grouped-query attention over the paged KV cache.
 //
-// KV pages: pool[layer][page][kv_head][slot_in_page][head_dim] in bf16, so the tokens of one
+// KV pages: pool[layer][page][kv_head][slot_in_page][head_dim] in fp16, so the tokens of one
 // (page, head) are contiguous.  A sequence's block table maps position / page_size -> page.
 //
 // Attention is a flash-decoding style split over the keys: one CTA per (key split, kv head, query
@@ -56,7 +56,7 @@ __global__ void embed_rope_kernel(const StepDesc *desc, const int32_t *tok, cons
     }
 }
 
-// Rotate q in place (fp32), rotate k and store k, v into the cache (bf16).
+// Rotate q in place (fp32), rotate k and store k, v into the cache (fp16).
 // qkv: [rows][(Hq + 2 Hkv) * D] = q heads, then k heads, then v heads.
 __global__ void rope_append_kernel(const StepDesc *desc, float *qkv, const float2 *cs, int Hq, int Hkv, int D,
                                    KvView kv, int32_t *status)
@@ -77,14 +77,14 @@ __global__ void rope_append_kernel(const StepDesc *desc, float *qkv, const float
             v[j + half] = rb;
         } else {
             const size_t o = kv_offset(kv, pos, h - Hq, D, status);
-            kv.k[o + j] = f32_to_bf16_bits(ra);
-            kv.k[o + j + half] = f32_to_bf16_bits(rb);
+            kv.k[o + j] = kv_bits(ra);
+            kv.k[o + j + half] = kv_bits(rb);
         }
     }
     const float *vsrc = row + (Hq + Hkv) * D;
     for (int idx = threadIdx.x; idx < Hkv * D; idx += blockDim.x) {
         const int h = idx / D, j = idx - h * D;
-        kv.v[kv_offset(kv, pos, h, D, status) + j] = f32_to_bf16_bits(vsrc[idx]);
+        kv.v[kv_offset(kv, pos, h, D, status) + j] = kv_bits(vsrc[idx]);
     }
 }
 
@@ -165,10 +165,10 @@ __global__ void __launch_bounds__(128) attn_kernel(const AttnParams p)
         }
 #pragma unroll
         for (int u = 0; u < UK; ++u) {
-            float kk[8] = {bf16_lo(kf[u].x), bf16_hi(kf[u].x), bf16_lo(kf[u].y), bf16_hi(kf[u].y),
-                           bf16_lo(kf[u].z), bf16_hi(kf[u].z), bf16_lo(kf[u].w), bf16_hi(kf[u].w)};
-            float vv[8] = {bf16_lo(vf[u].x), bf16_hi(vf[u].x), bf16_lo(vf[u].y), bf16_hi(vf[u].y),
-                           bf16_lo(vf[u].z), bf16_hi(vf[u].z), bf16_lo(vf[u].w), bf16_hi(vf[u].w)};
+            float kk[8] = {kv_lo(kf[u].x), kv_hi(kf[u].x), kv_lo(kf[u].y), kv_hi(kf[u].y),
+                           kv_lo(kf[u].z), kv_hi(kf[u].z), kv_lo(kf[u].w), kv_hi(kf[u].w)};
+            float vv[8] = {kv_lo(vf[u].x), kv_hi(vf[u].x), kv_lo(vf[u].y), kv_hi(vf[u].y),
+                           kv_lo(vf[u].z), kv_hi(vf[u].z), kv_lo(vf[u].w), kv_hi(vf[u].w)};
 #pragma unroll
             for (int g = 0; g < G; ++g) {
                 float s = 0.f;
@@ -357,10 +357,10 @@ __global__ void __launch_bounds__(256) attn_rows_kernel(const AttnParams p)
                 const int kj = j + sub;
                 const bool ok = kj < tile_keys;
                 const uint4 kf = s_k[min(kj, TK - 1) * LPK + (lane % LPK)], vf = s_v[min(kj, TK - 1) * LPK + (lane % LPK)];
-                const float kk[8] = {bf16_lo(kf.x), bf16_hi(kf.x), bf16_lo(kf.y), bf16_hi(kf.y),
-                                     bf16_lo(kf.z), bf16_hi(kf.z), bf16_lo(kf.w), bf16_hi(kf.w)};
-                const float vv[8] = {bf16_lo(vf.x), bf16_hi(vf.x), bf16_lo(vf.y), bf16_hi(vf.y),
-                                     bf16_lo(vf.z), bf16_hi(vf.z), bf16_lo(vf.w), bf16_hi(vf.w)};
+                const float kk[8] = {kv_lo(kf.x), kv_hi(kf.x), kv_lo(kf.y), kv_hi(kf.y),
+                                     kv_lo(kf.z), kv_hi(kf.z), kv_lo(kf.w), kv_hi(kf.w)};
+                const float vv[8] = {kv_lo(vf.x), kv_hi(vf.x), kv_lo(vf.y), kv_hi(vf.y),
+                                     kv_lo(vf.z), kv_hi(vf.z), kv_lo(vf.w), kv_hi(vf.w)};
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
                     float s = 0.f;

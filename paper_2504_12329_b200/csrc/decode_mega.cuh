@@ -456,15 +456,15 @@ __device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaSha
         }
 #pragma unroll
         for (int u = 0; u < UK; ++u) {
-            const float kk[8] = {bf16_lo(pf.kf[u].x), bf16_hi(pf.kf[u].x), bf16_lo(pf.kf[u].y), bf16_hi(pf.kf[u].y),
-                                 bf16_lo(pf.kf[u].z), bf16_hi(pf.kf[u].z), bf16_lo(pf.kf[u].w), bf16_hi(pf.kf[u].w)};
-            const float vv[8] = {bf16_lo(pf.vf[u].x), bf16_hi(pf.vf[u].x), bf16_lo(pf.vf[u].y), bf16_hi(pf.vf[u].y),
-                                 bf16_lo(pf.vf[u].z), bf16_hi(pf.vf[u].z), bf16_lo(pf.vf[u].w), bf16_hi(pf.vf[u].w)};
+            const float kk[8] = {kv_lo(pf.kf[u].x), kv_hi(pf.kf[u].x), kv_lo(pf.kf[u].y), kv_hi(pf.kf[u].y),
+                                 kv_lo(pf.kf[u].z), kv_hi(pf.kf[u].z), kv_lo(pf.kf[u].w), kv_hi(pf.kf[u].w)};
+            const float vv[8] = {kv_lo(pf.vf[u].x), kv_hi(pf.vf[u].x), kv_lo(pf.vf[u].y), kv_hi(pf.vf[u].y),
+                                 kv_lo(pf.vf[u].z), kv_hi(pf.vf[u].z), kv_lo(pf.vf[u].w), kv_hi(pf.vf[u].w)};
             update(kk, vv, pf.ok[u]);
         }
     }
     if (k0 <= pos && pos < k1 && cw == 0) {
-        // this step's own key/value: rotate k, round both to bf16 (what the cache holds), append, attend
+        // this step's own key/value: rotate k, round both to fp16 (what the cache holds), append, attend
         float kk[8], vv[8];
         rotated8(p.QKV + (size_t)(p.Hq + hk) * D, kk);
         const float *vsrc = p.QKV + (size_t)(p.Hq + p.Hkv + hk) * D + ch;
@@ -473,10 +473,10 @@ __device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaSha
         uint32_t kb[4], vb[4];
 #pragma unroll
         for (int e = 0; e < 8; e += 2) {
-            kb[e >> 1] = (uint32_t)f32_to_bf16_bits(kk[e]) | ((uint32_t)f32_to_bf16_bits(kk[e + 1]) << 16);
-            vb[e >> 1] = (uint32_t)f32_to_bf16_bits(vraw[e]) | ((uint32_t)f32_to_bf16_bits(vraw[e + 1]) << 16);
-            kk[e] = bf16_lo(kb[e >> 1]); kk[e + 1] = bf16_hi(kb[e >> 1]);
-            vv[e] = bf16_lo(vb[e >> 1]); vv[e + 1] = bf16_hi(vb[e >> 1]);
+            kb[e >> 1] = (uint32_t)kv_bits(kk[e]) | ((uint32_t)kv_bits(kk[e + 1]) << 16);
+            vb[e >> 1] = (uint32_t)kv_bits(vraw[e]) | ((uint32_t)kv_bits(vraw[e + 1]) << 16);
+            kk[e] = kv_lo(kb[e >> 1]); kk[e + 1] = kv_hi(kb[e >> 1]);
+            vv[e] = kv_lo(vb[e >> 1]); vv[e + 1] = kv_hi(vb[e >> 1]);
         }
         if (sub == 0) {
             const size_t off = kv_offset(kv, pos, hk, D, p.status) + ch;

@@ -29,6 +29,7 @@ struct GenState {
     int32_t next_model;  // the pass to run next ...
     int32_t next_m;      // ... ingests this many tokens ...
     int32_t next_emit;   // ... and samples a token (1) or only ingests (0)
+    int32_t ingested;    // tokens already ingested by ingest-only chunks of the catch-up in progress
     int32_t passes;      // passes dispatched so far
     int32_t body_runs[12];  // how often each graph body ran (per model: decode, 4 row buckets, ingest)
     int32_t pass_cap;    // hard bound on passes (the device loop stops there)
@@ -72,7 +73,8 @@ __device__ void router_step(GenState *g, const GenBuffers &b, int greedy, StepDe
 {
     const int a = g->active;
     const int t = g->step;
-    const int fed = g->pos - g->kv_len[a];
+    const int fed = g->pos - g->kv_len[a] + g->ingested;   // the whole catch-up, however it was chunked
+    g->ingested = 0;
     g->kv_len[a] = g->pos;
     g->bytes_algo += g->wbytes[a] + g->kvb[a] * (int64_t)g->pos;
     int tok = greedy;
@@ -124,6 +126,7 @@ __global__ void advance_ingest_kernel(GenState *g, StepDesc *desc_small, StepDes
 {
     const int a = g->next_model;
     g->kv_len[a] += g->next_m;
+    g->ingested += g->next_m;
     g->bytes_algo += g->wbytes[a] + g->kvb[a] * (int64_t)g->kv_len[a];
     plan_next_pass(g, desc_small, desc_large);
 }

@@ -1,6 +1,7 @@
 // Shared device-side definitions of the Speculative Thinking decode library (sm_100a).
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -48,6 +49,12 @@ __device__ __forceinline__ uint16_t f32_to_bf16_bits(float f)
     u += 0x7fffu + ((u >> 16) & 1u);
     return (uint16_t)(u >> 16);
 }
+
+// The KV cache holds IEEE half precision (11 significand bits): with bf16 (8 bits) the rounding of K and V
+// alone costs more than the logit tolerance once it has accumulated over 64 layers.
+__device__ __forceinline__ uint16_t kv_bits(float f) { return __half_as_ushort(__float2half_rn(f)); }
+__device__ __forceinline__ float kv_lo(uint32_t v) { return __half2float(__ushort_as_half((unsigned short)(v & 0xffffu))); }
+__device__ __forceinline__ float kv_hi(uint32_t v) { return __half2float(__ushort_as_half((unsigned short)(v >> 16))); }
 
 // a = hi + lo with hi = bf16(a), lo = bf16(a - hi): 16 significand bits in two bf16 values.
 __device__ __forceinline__ void split_bf16(float a, uint16_t &hi, uint16_t &lo)

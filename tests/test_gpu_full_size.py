@@ -1,0 +1,134 @@
+"""GPU parity at the workloads' full sizes, in the launch configuration the benchmark times (one graph
+launch per generation).  The oracle cannot run a 32B model for thousands of tokens, so:
+  * routing is checked against the oracle's state machine on a fully forced token stream (under full
+    forcing the routing does not depend on any logit, so the oracle may run it with the tiny pair);
+  * logits are checked on sampled rows the oracle can compute one by one (all 64 layers, weights
+    generated row by row on the CPU)."""
+import numpy as np
+import pytest
+
+from paper_2504_12329_b200 import workloads as W
+from parity_utils import MARGIN, assert_logits_close, shape_dict
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2504_12329_b200 import binding
+    binding.lib()
+    return binding
+
+
+def _routing_reference(oracle, prompt, force, n1, max_new):
+    """Routing of a fully forced stream from the oracle's state machine (tiny models: logits are irrelevant)."""
+    ts = oracle.Model(oracle.Config(**W.TINY_S.as_dict()), 0, 0)
+    tl = oracle.Model(oracle.Config(**W.TINY_L.as_dict()), 0, 1)
+    return oracle.generate_spec(ts, tl, prompt % 1024, delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=n1,
+                                max_new_tokens=max_new, force=force % 1024, vocab_limit=1024)
+
+
+def test_qwen1p5b_32b_routing_at_full_size(B, oracle):
+    """The benchmark's pair and prompt, 1200 tokens, every step forced (ids below 1024 so that the tiny pair can
+    replay them): sources, handoffs, catch-up lengths, per-step ingested counts and KV lengths are bit-exact."""
+    w = W.CONFIGS["qwen1p5b_32b"]
+    max_new = 1200
+    prompt = W.prompt_ids(w.input_seed, w.prompt_len, 1024)
+    force = W.full_forcing(w.input_seed + 1, 2 * max_new, 1024, mean_interval=w.mean_interval, keyword_rate=w.keyword_rate)
+    want = _routing_reference(oracle, prompt, force, W.N1, max_new)
+    cap = w.prompt_len + max_new + 64
+    small = B.Model(w.small.as_dict(), seed=0, tag=0, max_tokens=cap)
+    large = B.Model(w.large.as_dict(), seed=0, tag=1, max_tokens=cap)
+    got = B.st_generate_spec(small, large, prompt, delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=W.N1,
+                             max_new_tokens=max_new, force=force)
+    assert len(want.handoffs) >= 4
+    assert got.tokens.tolist() == want.tokens.tolist()
+    assert got.source.tolist() == want.source.tolist()
+    assert got.handoffs == want.handoffs
+    assert got.emission_fed.tolist() == want.emission_fed.tolist()
+    assert got.emission_source.tolist() == want.emission_source.tolist()
+    assert (got.kv_len_small, got.kv_len_large) == (want.kv_len_small, want.kv_len_large)
+    assert got.bytes_algorithmic > 0 and got.seconds > 0
+    # the first catch-up of the target includes the prompt and spans two 256-row passes
+    assert want.handoffs[0][2] > 256
+    small.close()
+    large.close()
+
+
+def test_qwen32b_full_depth_sampled_logits(B, oracle):
+    """All 64 layers of the 32B shape: the logits after a 12-token prefill and after two decode steps against the
+    oracle (which generates every weight row on the fly: one pass over the model for all 14 positions)."""
+    shape = shape_dict(W.QWEN_32B)
+    rng = np.random.default_rng(11)
+    tokens = rng.integers(0, shape["vocab"], size=14).astype(np.int32)
+    om = oracle.Model(oracle.Config(**shape), 0, 1, materialize=False)
+    want = oracle.KV(om, 16).forward(tokens, all_rows=True)
+    gm = B.Model(shape, seed=0, tag=1, max_tokens=128)
+    slot = gm.st_seq_alloc()
+    logits = torch.empty(shape["vocab"], dtype=torch.float32, device="cuda")
+    amax = torch.empty(1, dtype=torch.int32, device="cuda")
+    tok = torch.empty(1, dtype=torch.int32, device="cuda")
+    gm.st_prefill(slot, tokens[:12], logits)
+    torch.cuda.synchronize()
+    assert_logits_close(logits.cpu().numpy(), want[11], "row 11 (prefill)")
+    for i in (12, 13):
+        tok.fill_(int(tokens[i]))
+        gm.st_decode_step([slot], tok, logits, amax)
+        torch.cuda.synchronize()
+        assert_logits_close(logits.cpu().numpy(), want[i], f"row {i} (decode)")
+        gi, margin = oracle.argmax(want[i])
+        if margin >= MARGIN:
+            assert int(amax.item()) == gi
+    gm.close()
+
+
+def test_qwen1p5b_alone_free_running(B, oracle):
+    """The 1.5B alone, 256-token prompt, greedy: tokens equal the oracle's wherever its top-2 margin is at least
+    0.05; at the first low-margin disagreement the run continues teacher-forced and the logits are compared."""
+    shape = shape_dict(W.QWEN_1P5B)
+    n_new = 96
+    prompt = W.prompt_ids(100, 256, shape["vocab"])
+    om = oracle.Model(oracle.Config(**shape), 0, 0)
+    want = oracle.generate_spec(om, None, prompt, delimiter_id=W.DELIMITER_ID, keyword_ids=[], max_new_tokens=n_new,
+                                trace_n_steps=n_new)
+    gm = B.Model(shape, seed=0, tag=0, max_tokens=512)
+    got = B.st_generate_spec(gm, None, prompt, delimiter_id=W.DELIMITER_ID, keyword_ids=[], max_new_tokens=n_new)
+    for t in range(n_new):
+        if got.emission_tokens[t] != want.emission_tokens[t]:
+            assert want.emission_margin[t] < MARGIN, f"step {t}: tokens differ at margin {want.emission_margin[t]:.3f}"
+            break
+    forced = B.st_generate_spec(gm, None, prompt, delimiter_id=W.DELIMITER_ID, keyword_ids=[], max_new_tokens=n_new,
+                                force=want.emission_tokens, trace_n_steps=n_new)
+    assert forced.tokens.tolist() == want.tokens.tolist()
+    for t in range(0, n_new, 5):
+        assert_logits_close(forced.logits_trace[t], want.logits_trace[t], f"step {t}")
+        if want.emission_margin[t] >= MARGIN:
+            assert forced.emission_argmax[t] == want.emission_argmax[t]
+    gm.close()
+
+
+def test_qwen7b_32b_long_context_routing(B, oracle):
+    """The long-context pair (7B + 32B shapes, 4096-token prompt): 300 fully forced tokens; the prompt goes through
+    16 chunks of 256 rows on the small model and the target's first catch-up through 17; routing is bit-exact."""
+    w = W.CONFIGS["qwen7b_32b_long"]
+    max_new = 300
+    prompt = W.prompt_ids(w.input_seed, w.prompt_len, 1024)
+    force = W.full_forcing(w.input_seed + 1, 2 * max_new, 1024, mean_interval=w.mean_interval, keyword_rate=w.keyword_rate)
+    want = _routing_reference(oracle, prompt, force, W.N1, max_new)
+    cap = w.prompt_len + max_new + 64
+    small = B.Model(w.small.as_dict(), seed=0, tag=0, max_tokens=cap)
+    large = B.Model(w.large.as_dict(), seed=0, tag=1, max_tokens=cap)
+    got = B.st_generate_spec(small, large, prompt, delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=W.N1,
+                             max_new_tokens=max_new, force=force)
+    assert len(want.handoffs) >= 2 and want.handoffs[0][2] > 4096
+    assert got.tokens.tolist() == want.tokens.tolist()
+    assert got.source.tolist() == want.source.tolist()
+    assert got.handoffs == want.handoffs
+    assert got.emission_fed.tolist() == want.emission_fed.tolist()
+    assert (got.kv_len_small, got.kv_len_large) == (want.kv_len_small, want.kv_len_large)
+    small.close()
+    large.close()
