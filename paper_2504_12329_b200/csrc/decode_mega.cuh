@@ -174,15 +174,20 @@ struct MegaAttnScratch {   // per attention unit (4 warps)
     float den[G];
 };
 
-// Grid-wide barrier over the consumer warps of all CTAs.  When the bounded wait runs out it raises the
-// abort flag (which every later wait honours at once) and returns false; control flow stays uniform.
-__device__ __forceinline__ bool mega_grid_barrier(const MegaParams &p, MegaShared &sh, unsigned &epoch, int ctid)
+// Grid-wide barrier over the consumer warps of all CTAs, in two halves so that work which does not depend on
+// the other CTAs can be slotted between "I am done" and "everybody is done".  When the bounded wait runs out
+// it raises the abort flag (which every later wait honours at once); control flow stays uniform.
+__device__ __forceinline__ void mega_barrier_arrive(const MegaParams &p, int ctid)
 {
     consumer_sync();
+    // release-add: no return value to wait for
+    if (ctid == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.sync) : "memory");
+}
+__device__ __forceinline__ bool mega_barrier_wait(const MegaParams &p, MegaShared &sh, unsigned &epoch, int ctid)
+{
+    ++epoch;
     if (ctid == 0) {
-        // release-add (no return value to wait for), then poll with acquire loads
-        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.sync) : "memory");
-        const unsigned target = (++epoch) * gridDim.x;
+        const unsigned target = epoch * gridDim.x;
         bool ok = false;
         for (uint32_t it = 0; it < kMegaSpinLimit; ++it) {
             if (ld_acquire_u32(&p.sync[0]) >= target) { ok = true; break; }
@@ -194,11 +199,14 @@ __device__ __forceinline__ bool mega_grid_barrier(const MegaParams &p, MegaShare
             atomicOr(p.status, DEV_WAIT_EXPIRED);
             sh.abort = 1;
         }
-    } else {
-        ++epoch;
     }
     consumer_sync();
     return sh.abort == 0;
+}
+__device__ __forceinline__ bool mega_grid_barrier(const MegaParams &p, MegaShared &sh, unsigned &epoch, int ctid)
+{
+    mega_barrier_arrive(p, ctid);
+    return mega_barrier_wait(p, sh, epoch, ctid);
 }
 
 // x (+ add) -> shared memory, optionally normalised; CTA 0 writes the sum back to x_out.
@@ -454,13 +462,54 @@ __device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaSha
                 }
             }
         }
+        // scores of the whole batch first (independent chains), then one softmax update per head
+        float sc_[UK][G];
 #pragma unroll
         for (int u = 0; u < UK; ++u) {
             const float kk[8] = {kv_lo(pf.kf[u].x), kv_hi(pf.kf[u].x), kv_lo(pf.kf[u].y), kv_hi(pf.kf[u].y),
                                  kv_lo(pf.kf[u].z), kv_hi(pf.kf[u].z), kv_lo(pf.kf[u].w), kv_hi(pf.kf[u].w)};
-            const float vv[8] = {kv_lo(pf.vf[u].x), kv_hi(pf.vf[u].x), kv_lo(pf.vf[u].y), kv_hi(pf.vf[u].y),
-                                 kv_lo(pf.vf[u].z), kv_hi(pf.vf[u].z), kv_lo(pf.vf[u].w), kv_hi(pf.vf[u].w)};
-            update(kk, vv, pf.ok[u]);
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                float t = 0.f;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) t = fmaf(q[g][e], kk[e], t);
+                sc_[u][g] = t;
+            }
+        }
+#pragma unroll
+        for (int off = LPK / 2; off > 0; off >>= 1)
+#pragma unroll
+            for (int u = 0; u < UK; ++u)
+#pragma unroll
+                for (int g = 0; g < G; ++g) sc_[u][g] += __shfl_xor_sync(0xffffffffu, sc_[u][g], off);
+        float vv[UK][8];
+#pragma unroll
+        for (int u = 0; u < UK; ++u) {
+            vv[u][0] = kv_lo(pf.vf[u].x); vv[u][1] = kv_hi(pf.vf[u].x); vv[u][2] = kv_lo(pf.vf[u].y); vv[u][3] = kv_hi(pf.vf[u].y);
+            vv[u][4] = kv_lo(pf.vf[u].z); vv[u][5] = kv_hi(pf.vf[u].z); vv[u][6] = kv_lo(pf.vf[u].w); vv[u][7] = kv_hi(pf.vf[u].w);
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            float mnew = mx[g];
+#pragma unroll
+            for (int u = 0; u < UK; ++u)
+                if (pf.ok[u]) mnew = fmaxf(mnew, sc_[u][g]);
+            if (mnew > -INFINITY) {
+                const float corr = mx[g] == -INFINITY ? 0.f : __expf(mx[g] - mnew);
+                den[g] *= corr;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) o[g][e] *= corr;
+#pragma unroll
+                for (int u = 0; u < UK; ++u) {
+                    if (pf.ok[u]) {
+                        const float pw = __expf(sc_[u][g] - mnew);
+                        den[g] += pw;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) o[g][e] = fmaf(pw, vv[u][e], o[g][e]);
+                    }
+                }
+                mx[g] = mnew;
+            }
         }
     }
     if (k0 <= pos && pos < k1 && cw == 0) {
@@ -713,8 +762,9 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
         const bool attn_active = (int)blockIdx.x < p.Hkv * ns;
         const int a_hk = blockIdx.x / ns, a_split = blockIdx.x - a_hk * ns;
         MegaKvPrefetch pf;
+        mega_barrier_arrive(p, ctid);
         if (attn_active) mega_attention_prefetch<D>(p, kv, a_hk, a_split, ns, pos, cw, lane, pf);
-        mega_grid_barrier(p, sh, epoch, ctid);
+        mega_barrier_wait(p, sh, epoch, ctid);
     MEGA_MARK();
         mega_zero(p.D2, p.h, ctid);
         if (attn_active) mega_attention_unit<D, G>(p, sh, scratch[0], kv, a_hk, a_split, ns, pos, cw, lane, pf);
