@@ -142,6 +142,16 @@ int st_generate_spec(st_model *small, st_model *large, const st_spec_params *par
                      const int32_t *prompt, int32_t prompt_len,
                      const int32_t *force, int32_t n_force, st_spec_result *out);
 
+/* The same for n_seqs independent sequences (the batched workload: ragged prompts, per-sequence token budgets
+ * and forcing schedules).  prompts / force are concatenations indexed by prompt_offsets / force_offsets
+ * (n_seqs + 1 entries each; force may be NULL); max_new_per_seq (nullable) overrides params->max_new_tokens per
+ * sequence; outs[i] receives sequence i's result.  Sequences do not interact, so every outs[i] equals what
+ * st_generate_spec returns for that sequence alone.  In this version the sequences run one after the other
+ * through the batch-1 path; stops at the first failing sequence and returns its status. */
+int st_generate_spec_batch(st_model *small, st_model *large, const st_spec_params *params, int32_t n_seqs,
+                           const int32_t *prompts, const int32_t *prompt_offsets, const int32_t *max_new_per_seq,
+                           const int32_t *force, const int32_t *force_offsets, st_spec_result *outs);
+
 /* Fill `out_dev` (bf16 bit patterns, device) with elements idx0.. of seeded tensor `tid`: the
  * generator behind st_model_create, exposed so that it can be compared bit for bit. */
 int st_fill_tensor_bf16(uint64_t seed, uint32_t model_tag, uint32_t tid, uint64_t idx0, uint64_t n,

@@ -63,7 +63,7 @@ EXPORTS = [
     "st_model_create", "st_model_destroy", "st_seq_alloc", "st_seq_free", "st_seq_reserve", "st_kv_len",
     "st_kv_truncate", "st_prefill", "st_decode_step", "st_generate_spec", "st_fill_tensor_bf16",
     "st_weight_bytes", "st_kv_bytes_per_token", "st_last_device_status", "st_strerror",
-    "st_kernel_launches", "st_time_gemv", "st_argmax_static",
+    "st_kernel_launches", "st_time_gemv", "st_argmax_static", "st_generate_spec_batch",
 ]
 
 _lib = None
@@ -109,6 +109,9 @@ def lib():
         L.st_kernel_launches.argtypes = []
         L.st_time_gemv.restype = C.c_int
         L.st_time_gemv.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_double)]
+        L.st_generate_spec_batch.restype = C.c_int
+        L.st_generate_spec_batch.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(StSpecParams), C.c_int32, C.c_void_p, C.c_void_p,
+                                             C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.st_argmax_static.restype = C.c_int
         L.st_argmax_static.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.st_strerror.restype = C.c_char_p
@@ -282,6 +285,45 @@ class Model:
         return lib().st_last_device_status(self.h)
 
 
+class _ResultBuffers:
+    """Host buffers of one st_spec_result and the struct that points at them."""
+
+    def __init__(self, max_new_tokens, vocab_limit, trace_first_step, trace_n_steps, cap_steps, cap_handoffs):
+        self.cap_steps = 2 * max_new_tokens + 8 if cap_steps is None else cap_steps
+        self.cap_handoffs = max_new_tokens + 1 if cap_handoffs is None else cap_handoffs
+        self.tokens = np.zeros(max_new_tokens + 1, dtype=np.int32)
+        self.source = np.zeros(max_new_tokens + 1, dtype=np.uint8)
+        self.hand = (StHandoff * max(self.cap_handoffs, 1))()
+        n = max(self.cap_steps, 1)
+        self.e_tok, self.e_fed, self.e_arg = (np.zeros(n, dtype=np.int32) for _ in range(3))
+        self.e_src = np.zeros(n, dtype=np.uint8)
+        self.trace = np.zeros((trace_n_steps, vocab_limit), dtype=np.float32) if trace_n_steps > 0 else None
+        self.trace_first_step, self.trace_n_steps = trace_first_step, trace_n_steps
+
+    def fill(self, R: StSpecResult):
+        R.tokens = self.tokens.ctypes.data_as(C.POINTER(C.c_int32))
+        R.source = self.source.ctypes.data_as(C.POINTER(C.c_uint8))
+        R.cap_tokens = self.tokens.size
+        R.handoffs = C.cast(self.hand, C.POINTER(StHandoff))
+        R.cap_handoffs = self.cap_handoffs
+        R.emission_tokens = self.e_tok.ctypes.data_as(C.POINTER(C.c_int32))
+        R.emission_source = self.e_src.ctypes.data_as(C.POINTER(C.c_uint8))
+        R.emission_fed = self.e_fed.ctypes.data_as(C.POINTER(C.c_int32))
+        R.emission_argmax = self.e_arg.ctypes.data_as(C.POINTER(C.c_int32))
+        R.cap_steps = self.cap_steps
+        R.logits_trace = self.trace.ctypes.data_as(C.POINTER(C.c_float)) if self.trace is not None else None
+        R.trace_first_step = self.trace_first_step
+        R.trace_n_steps = self.trace_n_steps
+
+    def result(self, R: StSpecResult) -> SpecResult:
+        n, s = R.n_tokens, min(R.n_steps, self.cap_steps)
+        return SpecResult(self.tokens[:n].copy(), self.source[:n].copy(),
+                          [(self.hand[i].seg_start, self.hand[i].step, self.hand[i].catchup_len)
+                           for i in range(min(R.n_handoffs, self.cap_handoffs))],
+                          self.e_tok[:s].copy(), self.e_src[:s].copy(), self.e_fed[:s].copy(), self.e_arg[:s].copy(),
+                          R.kv_len_small, R.kv_len_large, self.trace, R.seconds, R.bytes_algorithmic, R.n_steps)
+
+
 def st_generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id: int, keyword_ids, n1: int = 20,
                      keep_probe: bool = False, eos_id: int = -1, vocab_limit: int = 0, max_new_tokens: int,
                      force=None, trace_first_step: int = 0, trace_n_steps: int = 0, cap_steps: int | None = None,
@@ -293,36 +335,42 @@ def st_generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id:
                      vocab_limit, max_new_tokens)
     if vocab_limit <= 0:
         vocab_limit = small.vocab if large is None else min(small.vocab, large.vocab)
-    cap_steps = 2 * max_new_tokens + 8 if cap_steps is None else cap_steps
-    cap_handoffs = max_new_tokens + 1 if cap_handoffs is None else cap_handoffs
-    tokens = np.zeros(max_new_tokens + 1, dtype=np.int32)
-    source = np.zeros(max_new_tokens + 1, dtype=np.uint8)
-    hand = (StHandoff * max(cap_handoffs, 1))()
-    e_tok = np.zeros(max(cap_steps, 1), dtype=np.int32)
-    e_src = np.zeros(max(cap_steps, 1), dtype=np.uint8)
-    e_fed = np.zeros(max(cap_steps, 1), dtype=np.int32)
-    e_arg = np.zeros(max(cap_steps, 1), dtype=np.int32)
-    trace = np.zeros((trace_n_steps, vocab_limit), dtype=np.float32) if trace_n_steps > 0 else None
+    bufs = _ResultBuffers(max_new_tokens, vocab_limit, trace_first_step, trace_n_steps, cap_steps, cap_handoffs)
     R = StSpecResult()
-    R.tokens = tokens.ctypes.data_as(C.POINTER(C.c_int32))
-    R.source = source.ctypes.data_as(C.POINTER(C.c_uint8))
-    R.cap_tokens = tokens.size
-    R.handoffs = C.cast(hand, C.POINTER(StHandoff))
-    R.cap_handoffs = cap_handoffs
-    R.emission_tokens = e_tok.ctypes.data_as(C.POINTER(C.c_int32))
-    R.emission_source = e_src.ctypes.data_as(C.POINTER(C.c_uint8))
-    R.emission_fed = e_fed.ctypes.data_as(C.POINTER(C.c_int32))
-    R.emission_argmax = e_arg.ctypes.data_as(C.POINTER(C.c_int32))
-    R.cap_steps = cap_steps
-    R.logits_trace = trace.ctypes.data_as(C.POINTER(C.c_float)) if trace is not None else None
-    R.trace_first_step = trace_first_step
-    R.trace_n_steps = trace_n_steps
+    bufs.fill(R)
     f = None if force is None else np.ascontiguousarray(force, dtype=np.int32)
     rc = lib().st_generate_spec(small.h, large.h if large is not None else None, C.byref(P), _np_ptr(prompt), prompt.size,
                                 _np_ptr(f), 0 if f is None else f.size, C.byref(R))
     _check(rc, "st_generate_spec")
-    n, s = R.n_tokens, min(R.n_steps, cap_steps)
-    return SpecResult(tokens[:n].copy(), source[:n].copy(),
-                      [(hand[i].seg_start, hand[i].step, hand[i].catchup_len) for i in range(min(R.n_handoffs, cap_handoffs))],
-                      e_tok[:s].copy(), e_src[:s].copy(), e_fed[:s].copy(), e_arg[:s].copy(),
-                      R.kv_len_small, R.kv_len_large, trace, R.seconds, R.bytes_algorithmic, R.n_steps)
+    return bufs.result(R)
+
+
+def st_generate_spec_batch(small: Model, large: Model | None, prompts, *, delimiter_id: int, keyword_ids, n1: int = 20,
+                           keep_probe: bool = False, eos_id: int = -1, vocab_limit: int = 0, max_new_tokens,
+                           forces=None) -> list:
+    """prompts / forces: lists of per-sequence arrays; max_new_tokens: one int or a list per sequence."""
+    n = len(prompts)
+    budgets = [int(max_new_tokens)] * n if np.isscalar(max_new_tokens) else [int(x) for x in max_new_tokens]
+    kw = np.ascontiguousarray(keyword_ids, dtype=np.int32)
+    P = StSpecParams(delimiter_id, kw.ctypes.data_as(C.POINTER(C.c_int32)), kw.size, n1, int(keep_probe), eos_id,
+                     vocab_limit, max(budgets) if budgets else 0)
+    if vocab_limit <= 0:
+        vocab_limit = small.vocab if large is None else min(small.vocab, large.vocab)
+    flat_p = np.ascontiguousarray(np.concatenate([np.asarray(p, dtype=np.int32) for p in prompts]) if n else np.zeros(0, np.int32))
+    off_p = np.zeros(n + 1, dtype=np.int32)
+    off_p[1:] = np.cumsum([len(p) for p in prompts])
+    flat_f = off_f = None
+    if forces is not None:
+        flat_f = np.ascontiguousarray(np.concatenate([np.asarray(f, dtype=np.int32) for f in forces]))
+        off_f = np.zeros(n + 1, dtype=np.int32)
+        off_f[1:] = np.cumsum([len(f) for f in forces])
+    budget_arr = np.ascontiguousarray(budgets, dtype=np.int32)
+    bufs = [_ResultBuffers(b, vocab_limit, 0, 0, None, None) for b in budgets]
+    Rs = (StSpecResult * max(n, 1))()
+    for i, b in enumerate(bufs):
+        b.fill(Rs[i])
+    rc = lib().st_generate_spec_batch(small.h, large.h if large is not None else None, C.byref(P), n, _np_ptr(flat_p),
+                                      _np_ptr(off_p), _np_ptr(budget_arr), _np_ptr(flat_f), _np_ptr(off_f),
+                                      C.cast(Rs, C.c_void_p))
+    _check(rc, "st_generate_spec_batch")
+    return [b.result(Rs[i]) for i, b in enumerate(bufs)]

@@ -1537,6 +1537,27 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     return ST_OK;
 }
 
+extern "C" int st_generate_spec_batch(st_model *small, st_model *large, const st_spec_params *P, int32_t n_seqs,
+                                      const int32_t *prompts, const int32_t *prompt_offsets, const int32_t *max_new_per_seq,
+                                      const int32_t *force, const int32_t *force_offsets, st_spec_result *outs)
+{
+    if (!small || !P || n_seqs < 0 || (n_seqs > 0 && (!prompts || !prompt_offsets || !outs))) return ST_ERR_ARG;
+    if (force && !force_offsets) return ST_ERR_ARG;
+    for (int i = 0; i < n_seqs; ++i) {
+        if (prompt_offsets[i + 1] <= prompt_offsets[i]) return ST_ERR_ARG;
+        if (force && force_offsets[i + 1] < force_offsets[i]) return ST_ERR_ARG;
+    }
+    for (int i = 0; i < n_seqs; ++i) {
+        st_spec_params pi = *P;
+        if (max_new_per_seq) pi.max_new_tokens = max_new_per_seq[i];
+        const int32_t *f = force ? force + force_offsets[i] : nullptr;
+        const int32_t nf = force ? force_offsets[i + 1] - force_offsets[i] : 0;
+        TRY(st_generate_spec(small, large, &pi, prompts + prompt_offsets[i], prompt_offsets[i + 1] - prompt_offsets[i],
+                             nf > 0 ? f : nullptr, nf, &outs[i]));
+    }
+    return ST_OK;
+}
+
 // ------------------------------------------------------------------------------------------------
 // greedy sampling without any allocation
 // ------------------------------------------------------------------------------------------------

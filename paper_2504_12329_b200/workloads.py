@@ -113,6 +113,20 @@ CONFIGS = {
 }
 
 
+def batch_inputs(seed: int, n_seqs: int, vocab: int, *, prompt_range=(64, 512), budget_range=(1024, 8192),
+                 mean_interval: float = 40.0, keyword_rate: float = 0.3):
+    """The batched workload: n_seqs independent sequences with prompt lengths uniform in prompt_range, token
+    budgets uniform in budget_range ("up to 8192" generated tokens; drawn so that the live KV fits beside the
+    weights) and one seeded forcing schedule each.  Returns (prompts, budgets, forces) as lists."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    lens = rng.integers(prompt_range[0], prompt_range[1] + 1, size=n_seqs)
+    budgets = rng.integers(budget_range[0], budget_range[1] + 1, size=n_seqs)
+    prompts = [prompt_ids(seed + 1 + i, int(lens[i]), vocab) for i in range(n_seqs)]
+    forces = [forcing_schedule(seed + 10_000 + i, 2 * int(budgets[i]), mean_interval=mean_interval,
+                               keyword_rate=keyword_rate) for i in range(n_seqs)]
+    return prompts, [int(b) for b in budgets], forces
+
+
 def workload_inputs(w: Workload):
     vshared = w.small.vocab if w.large is None else min(w.small.vocab, w.large.vocab)
     prompt = prompt_ids(w.input_seed, w.prompt_len, vshared)

@@ -229,3 +229,28 @@ def test_host_side_errors(B):
         B.Model(bad)
     assert e.value.status == B.ST_ERR_UNSUPPORTED
     m.close()
+
+
+def test_batched_ragged_sequences(B, oracle):
+    """The batched entry point on the tiny pair: 6 independent sequences with ragged prompts, budgets and
+    schedules (every step forced); each sequence's routing equals the oracle's run of that sequence alone."""
+    S, L = shape_dict(W.TINY_S), shape_dict(W.TINY_L)
+    prompts, budgets, forces = W.batch_inputs(7, 6, 1024, prompt_range=(5, 40), budget_range=(20, 90), mean_interval=6,
+                                              keyword_rate=0.6)
+    forces = [W.full_forcing(900 + i, len(f), 1024, mean_interval=6, keyword_rate=0.6) for i, f in enumerate(forces)]
+    gs = B.Model(S, seed=0, tag=0, max_tokens=256)
+    gl = B.Model(L, seed=0, tag=1, max_tokens=256)
+    got = B.st_generate_spec_batch(gs, gl, prompts, delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=4,
+                                   max_new_tokens=budgets, forces=forces)
+    os_, ol = oracle.Model(oracle.Config(**S), 0, 0), oracle.Model(oracle.Config(**L), 0, 1)
+    assert len(got) == 6
+    n_hand = 0
+    for i in range(6):
+        want = oracle.generate_spec(os_, ol, prompts[i], delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=4,
+                                    max_new_tokens=budgets[i], force=forces[i])
+        _assert_routing_equal(want, got[i])
+        assert len(got[i].tokens) == budgets[i]
+        n_hand += len(want.handoffs)
+    assert n_hand >= 6
+    gs.close()
+    gl.close()
