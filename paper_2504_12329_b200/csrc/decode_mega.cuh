@@ -60,7 +60,7 @@ struct MegaParams {
     float *logits;            // [vocab]
     float *part_o, *part_ml;  // attention split partials [Hq][n_splits][D], [Hq][n_splits][2]
     int32_t *tickets;         // [Hkv] attention tickets, zero between launches
-    unsigned *sync;           // [0] barrier counter, [1] exit tickets, [2] abort flag, [3] argmax tickets
+    unsigned *sync;           // [1] exit tickets, [2] abort flag, [3] argmax tickets, [32 * (1 + i)] barrier counter i < 8
     int32_t *status;
     int32_t n_layers, h, Hq, Hkv, f, vocab, n_splits, stages, xarea_bytes;
     float eps, scale;
@@ -177,24 +177,36 @@ struct MegaAttnScratch {   // per attention unit (4 warps)
 // Grid-wide barrier over the consumer warps of all CTAs, in two halves so that work which does not depend on
 // the other CTAs can be slotted between "I am done" and "everybody is done".  When the bounded wait runs out
 // it raises the abort flag (which every later wait honours at once); control flow stays uniform.
+// The arrivals are spread over kMegaBarCounters counters on separate 128-byte lines (CTA c adds to counter
+// c % 8): same-address atomics are served one after the other, and 148 of them in a row were a visible
+// part of the barrier's latency.  Lanes 0..7 of the first consumer warp each watch one counter.
+constexpr int kMegaBarCounters = 8;
+__device__ __forceinline__ unsigned *mega_bar_counter(const MegaParams &p, int i) { return p.sync + 32 * (1 + i); }
+
 __device__ __forceinline__ void mega_barrier_arrive(const MegaParams &p, int ctid)
 {
     consumer_sync();
     // release-add: no return value to wait for
-    if (ctid == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.sync) : "memory");
+    if (ctid == 0)
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(mega_bar_counter(p, blockIdx.x % kMegaBarCounters)) : "memory");
 }
 __device__ __forceinline__ bool mega_barrier_wait(const MegaParams &p, MegaShared &sh, unsigned &epoch, int ctid)
 {
     ++epoch;
-    if (ctid == 0) {
-        const unsigned target = epoch * gridDim.x;
+    if (ctid < 32) {
+        const int i = ctid < kMegaBarCounters ? ctid : 0;
+        // CTAs that add to counter i: those with index congruent to i
+        const unsigned members = (gridDim.x - i + kMegaBarCounters - 1) / kMegaBarCounters;
+        const unsigned target = epoch * members;
+        const unsigned *ctr = mega_bar_counter(p, i);
         bool ok = false;
         for (uint32_t it = 0; it < kMegaSpinLimit; ++it) {
-            if (ld_acquire_u32(&p.sync[0]) >= target) { ok = true; break; }
-            if ((it & 63) == 63 && ld_acquire_u32(&p.sync[2])) break;
+            const bool mine = ctid >= kMegaBarCounters || ld_acquire_u32(ctr) >= target;
+            if (__all_sync(0xffffffffu, mine)) { ok = true; break; }
+            if ((it & 63) == 63 && __any_sync(0xffffffffu, ld_acquire_u32(&p.sync[2]) != 0)) break;
             if (it > 256) __nanosleep(32);
         }
-        if (!ok) {
+        if (!ok && ctid == 0) {
             atomicExch(&p.sync[2], 1u);
             atomicOr(p.status, DEV_WAIT_EXPIRED);
             sh.abort = 1;
@@ -868,7 +880,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
         __threadfence();
         const unsigned t = atomicAdd(&p.sync[1], 1u);
         if (t == gridDim.x - 1) {
-            p.sync[0] = 0;
+            for (int i = 0; i < kMegaBarCounters; ++i) *mega_bar_counter(p, i) = 0;
             p.sync[1] = 0;
             __threadfence();
         }

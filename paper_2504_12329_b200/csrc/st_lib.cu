@@ -132,6 +132,7 @@ struct st_model {
 
 static constexpr int kArgmaxBlocks = 64;
 static constexpr int kGemvWarps = 8;
+static constexpr int kMegaSyncWords = 32 * (1 + kMegaBarCounters);   // ticket/abort words + one 128-byte line per barrier counter
 static constexpr int kMaxKSplits = 8;  // most K splits of a multi-row projection
 static constexpr int kRowSplits = 8;   // most key splits a multi-row pass uses
 
@@ -577,9 +578,9 @@ static int model_build(st_model *m)
         ALLOC(m->X1, float, h);
         ALLOC(m->D1, float, h);
         ALLOC(m->D2, float, h);
-        ALLOC(m->mega_sync, unsigned, 4);
+        ALLOC(m->mega_sync, unsigned, kMegaSyncWords);
         ALLOC(m->mega_tickets, int32_t, c.n_kv_heads);
-        CK(cudaMemsetAsync(m->mega_sync, 0, 4 * sizeof(unsigned), m->stream));
+        CK(cudaMemsetAsync(m->mega_sync, 0, kMegaSyncWords * sizeof(unsigned), m->stream));
         CK(cudaMemsetAsync(m->mega_tickets, 0, c.n_kv_heads * sizeof(int32_t), m->stream));
         int widest = h > qd ? h : qd;
         widest = widest > f ? widest : f;
@@ -1059,7 +1060,7 @@ int st_prefill(st_model *m, int32_t slot, const int32_t *tokens_host, int32_t n,
     for (int i = 0; i < n; ++i)
         if ((unsigned)tokens_host[i] >= (unsigned)m->cfg.vocab) return ST_ERR_VOCAB;
     TRY(seq_reserve(m, slot, m->seq_len[slot] + n));
-    CK(cudaMemsetAsync(m->mega_sync, 0, 4 * sizeof(unsigned), m->stream));
+    CK(cudaMemsetAsync(m->mega_sync, 0, kMegaSyncWords * sizeof(unsigned), m->stream));
     for (int done = 0; done < n;) {
         const int rows = n - done < m->max_rows ? n - done : m->max_rows;
         const bool last = done + rows == n;
@@ -1089,7 +1090,7 @@ int st_decode_step(st_model *m, const int32_t *slots_host, const int32_t *tokens
         for (int j = 0; j < i; ++j)
             if (slots_host[j] == slot) return ST_ERR_ARG;
     }
-    CK(cudaMemsetAsync(m->mega_sync, 0, 4 * sizeof(unsigned), m->stream));
+    CK(cudaMemsetAsync(m->mega_sync, 0, kMegaSyncWords * sizeof(unsigned), m->stream));
     for (int i = 0; i < batch; ++i) {
         const int slot = slots_host[i];
         TRY(seq_reserve(m, slot, m->seq_len[slot] + 1));
@@ -1383,11 +1384,11 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
 
     cudaStream_t s = small->stream;
     CK(cudaMemsetAsync(small->status, 0, sizeof(int32_t), s));
-    CK(cudaMemsetAsync(small->mega_sync, 0, 4 * sizeof(unsigned), s));
+    CK(cudaMemsetAsync(small->mega_sync, 0, kMegaSyncWords * sizeof(unsigned), s));
     CK(cudaMemsetAsync(small->mega_tickets, 0, small->cfg.n_kv_heads * sizeof(int32_t), s));
     if (large) {
         CK(cudaMemsetAsync(large->status, 0, sizeof(int32_t), s));
-        CK(cudaMemsetAsync(large->mega_sync, 0, 4 * sizeof(unsigned), s));
+        CK(cudaMemsetAsync(large->mega_sync, 0, kMegaSyncWords * sizeof(unsigned), s));
         CK(cudaMemsetAsync(large->mega_tickets, 0, large->cfg.n_kv_heads * sizeof(int32_t), s));
     }
     const int total = prompt_len + max_new + 1;
