@@ -319,12 +319,25 @@ static int launch_tc_gemm(const CUtensorMap &tw, const CUtensorMap &ta_hi, const
     auto kern = tc_gemm_kernel<EPI>;
     p.m_pad = (m_upper + 31) / 32 * 32;
     if (p.m_pad > 256) return ST_ERR_INTERNAL;
-    // as many 128-row weight tiles per CTA as TMEM (512 columns) and shared memory (two stages) allow,
-    // but no more than leaves every SM a tile
-    int wt = 512 / p.m_pad;
-    wt = wt > 4 ? 4 : wt;
-    while (wt > 1 && 2 * (wt * kTcWBytes + 2 * p.m_pad * kTcBlockK * 2) > 220 * 1024) --wt;
-    while (wt > 1 && (p.N + kTcTileW * wt - 1) / (kTcTileW * wt) * (EPI == TEPI_SILU ? 1 : 4) < sms) --wt;
+    // 128-row weight tiles per CTA (they share the activation tiles of a stage): bounded by TMEM (512 columns) and
+    // by two pipeline stages of shared memory; among the candidates take the one whose CTA count fills whole waves
+    // of SMs best (a projection with 1.46 waves of CTAs runs as long as one with 2), the larger on a tie.
+    int wt = 1;
+    {
+        double best = -1.0;
+        for (int cand = 4; cand >= 1; --cand) {
+            if (cand * p.m_pad > 512) continue;
+            if (2 * (cand * kTcWBytes + 2 * p.m_pad * kTcBlockK * 2) > 220 * 1024) continue;
+            const int tiles = (p.N + kTcTileW * cand - 1) / (kTcTileW * cand);
+            // projections that may split K fill the machine through the split; the others only through tiles
+            int split = tiles >= sms ? 1 : sms / tiles;   // K splits: as many as still fit one wave
+            split = split > kMaxKSplits ? kMaxKSplits : split;
+            const int ctas = EPI == TEPI_SILU ? tiles : tiles * split;
+            const int waves = (ctas + sms - 1) / sms;
+            const double eff = (double)ctas / ((double)waves * sms);
+            if (eff > best + 0.03) { best = eff; wt = cand; }
+        }
+    }
     p.w_tiles = wt;
     int cols = wt * p.m_pad;
     p.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
@@ -335,7 +348,7 @@ static int launch_tc_gemm(const CUtensorMap &tw, const CUtensorMap &ta_hi, const
     const int kb_total = (p.K + kTcBlockK - 1) / kTcBlockK;
     int ks = 1;
     if (EPI != TEPI_SILU) {
-        ks = (sms + n_tiles - 1) / n_tiles;
+        ks = n_tiles >= sms ? 1 : sms / n_tiles;
         const int ks_max = kb_total / 8 > 1 ? kb_total / 8 : 1;
         ks = ks > ks_max ? ks_max : ks;
         ks = ks > kMaxKSplits ? kMaxKSplits : ks;
