@@ -295,7 +295,7 @@ __global__ void __launch_bounds__(128) attn_kernel(const AttnParams p)
 // from L2 once per 8 rows instead of once per row.  Each warp keeps its row's online softmax for all G
 // query heads exactly as the decode kernel does; rows are causal (row i sees keys 0 .. pos0 + i).
 template <int D, int G>
-__global__ void __launch_bounds__(256) attn_rows_kernel(const AttnParams p)
+__global__ void __launch_bounds__(256, 2) attn_rows_kernel(const AttnParams p)
 {
     constexpr int LPK = D / 8, KPW = 32 / LPK, TK = 64, ROWS = 8;
     __shared__ uint4 s_k[TK * D / 8], s_v[TK * D / 8];
@@ -353,27 +353,60 @@ __global__ void __launch_bounds__(256) attn_rows_kernel(const AttnParams p)
         __syncthreads();
         if (row_live) {
             const int tile_keys = min(TK, k1 - t0);   // may be <= 0 for rows that ended earlier
-            for (int j = 0; j < tile_keys; j += KPW) {
-                const int kj = j + sub;
-                const bool ok = kj < tile_keys;
-                const uint4 kf = s_k[min(kj, TK - 1) * LPK + (lane % LPK)], vf = s_v[min(kj, TK - 1) * LPK + (lane % LPK)];
-                const float kk[8] = {kv_lo(kf.x), kv_hi(kf.x), kv_lo(kf.y), kv_hi(kf.y),
-                                     kv_lo(kf.z), kv_hi(kf.z), kv_lo(kf.w), kv_hi(kf.w)};
-                const float vv[8] = {kv_lo(vf.x), kv_hi(vf.x), kv_lo(vf.y), kv_hi(vf.y),
-                                     kv_lo(vf.z), kv_hi(vf.z), kv_lo(vf.w), kv_hi(vf.w)};
+            constexpr int UB = 4;                      // keys per lane group and softmax update
+            for (int j = 0; j < tile_keys; j += KPW * UB) {
+                // scores of UB keys first (independent chains), then one rescale per head
+                float sc[UB][G];
+                bool ok[UB];
+#pragma unroll
+                for (int u = 0; u < UB; ++u) {
+                    const int kj = j + u * KPW + sub;
+                    ok[u] = kj < tile_keys;
+                    const uint4 kf = s_k[min(kj, TK - 1) * LPK + (lane % LPK)];
+                    const float kk[8] = {kv_lo(kf.x), kv_hi(kf.x), kv_lo(kf.y), kv_hi(kf.y),
+                                         kv_lo(kf.z), kv_hi(kf.z), kv_lo(kf.w), kv_hi(kf.w)};
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        float t = 0.f;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) t = fmaf(q[g][e], kk[e], t);
+                        sc[u][g] = t;
+                    }
+                }
+#pragma unroll
+                for (int off = LPK / 2; off > 0; off >>= 1)
+#pragma unroll
+                    for (int u = 0; u < UB; ++u)
+#pragma unroll
+                        for (int g = 0; g < G; ++g) sc[u][g] += __shfl_xor_sync(0xffffffffu, sc[u][g], off);
+                float vv[UB][8];
+#pragma unroll
+                for (int u = 0; u < UB; ++u) {
+                    const int kj = j + u * KPW + sub;
+                    const uint4 vf = s_v[min(kj, TK - 1) * LPK + (lane % LPK)];
+                    vv[u][0] = kv_lo(vf.x); vv[u][1] = kv_hi(vf.x); vv[u][2] = kv_lo(vf.y); vv[u][3] = kv_hi(vf.y);
+                    vv[u][4] = kv_lo(vf.z); vv[u][5] = kv_hi(vf.z); vv[u][6] = kv_lo(vf.w); vv[u][7] = kv_hi(vf.w);
+                }
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
-                    float s = 0.f;
+                    float mnew = mx[g];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) s = fmaf(q[g][e], kk[e], s);
+                    for (int u = 0; u < UB; ++u)
+                        if (ok[u]) mnew = fmaxf(mnew, sc[u][g]);
+                    if (mnew > -INFINITY) {
+                        const float corr = mx[g] == -INFINITY ? 0.f : __expf(mx[g] - mnew);
+                        den[g] *= corr;
 #pragma unroll
-                    for (int off = LPK / 2; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-                    if (ok) {
-                        const float mnew = fmaxf(mx[g], s);
-                        const float corr = __expf(mx[g] - mnew), pw = __expf(s - mnew);
-                        den[g] = den[g] * corr + pw;
+                        for (int e = 0; e < 8; ++e) o[g][e] *= corr;
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) o[g][e] = fmaf(pw, vv[e], o[g][e] * corr);
+                        for (int u = 0; u < UB; ++u) {
+                            if (ok[u]) {
+                                const float pw = __expf(sc[u][g] - mnew);
+                                den[g] += pw;
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) o[g][e] = fmaf(pw, vv[u][e], o[g][e]);
+                            }
+                        }
                         mx[g] = mnew;
                     }
                 }
