@@ -33,6 +33,7 @@ constexpr int kMegaBoxBytes = kMegaTileRows * 256 * 2;            // one TMA box
 constexpr int kMegaTileBytes = 2 * kMegaBoxBytes;                 // 32 KB: two boxes side by side in K
 constexpr int kMegaMaxStages = 6;
 constexpr uint32_t kMegaSpinLimit = 1u << 22;
+constexpr int kMegaMaxUnitPages = 64;                              // block-table entries of one attention unit kept in shared memory
 constexpr int kMegaAttnWarps = kMegaConsumers;                    // all consumer warps work on one attention unit
 
 struct MegaLayer {
@@ -43,12 +44,13 @@ struct MegaLayer {
 
 // TMA descriptors of the weight matrices for the decode ring: boxes of 256 elements x 32 rows, no
 // swizzle (a tile row is 512 contiguous bytes in shared memory), zero fill outside the matrix.
-// Device array: 4 per layer (QKV, O, gate/up, down), then the LM head.
+// Device array: 4 per layer (QKV, O, gate/up, down), then the LM head; behind them the K and V pools of
+// the paged cache as [all rows][D] matrices in boxes of 16 rows x 64 channels with the 128-byte swizzle.
 constexpr int kMegaBoxK = 256;
 
 struct MegaParams {
     const MegaLayer *layers;
-    const CUtensorMap *maps;   // [4 * n_layers + 1], global memory
+    const CUtensorMap *maps;   // [4 * n_layers + 3], global memory: the weight matrices, then the K and the V pool
     const uint16_t *embed, *lm_head;
     const float *gf;
     const double *inv_freq;
@@ -63,6 +65,7 @@ struct MegaParams {
     unsigned *sync;           // [1] exit tickets, [2] abort flag, [3] argmax tickets, [32 * (1 + i)] barrier counter i < 8
     int32_t *status;
     int32_t n_layers, h, Hq, Hkv, f, vocab, n_splits, stages, xarea_bytes;
+    int32_t kv_off, kv_cap;   // K/V staging area inside the activation area: byte offset, capacity in keys (multiple of 16)
     float eps, scale;
     // sampling
     int32_t want_argmax, limit;
@@ -91,15 +94,6 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
     return v;
 }
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kMegaCT) : "memory"); }
-constexpr int kMegaAttnUK = 4;   // key steps in flight per lane
-
-// First batch of cached keys/values of an attention unit, fetched before the grid barrier that
-// precedes the attention phase (cached K/V do not depend on this layer's QKV).
-struct MegaKvPrefetch {
-    uint4 kf[kMegaAttnUK], vf[kMegaAttnUK];
-    bool ok[kMegaAttnUK];
-};
-
 // The weight matrix of weight phase idx: 4 per layer (QKV, O, gate/up, down), then the LM head.
 struct MegaPhase {
     const uint16_t *W;
@@ -152,12 +146,18 @@ __device__ unsigned long long g_mega_trace[8192];
             g_mega_trace[trace_i++] = t_;                                   \
         }                                                                   \
     } while (0)
+#define MEGA_TRACE_PARAM , int &trace_i, const int ctid
+#define MEGA_TRACE_ARG , trace_i, ctid
 #else
 #define MEGA_MARK() do { } while (0)
+#define MEGA_TRACE_PARAM
+#define MEGA_TRACE_ARG
 #endif
 
 struct MegaShared {
     uint64_t full[kMegaMaxStages], empty[kMegaMaxStages];
+    uint64_t kvfull[2];        // K/V staging buffers of the attention unit
+    int32_t pages[kMegaMaxUnitPages];   // block-table entries of the unit's key range
     float red[kMegaConsumers];
     float2 cs[64];          // rotary table of this step's position
     float s_v[kMegaConsumers];
@@ -361,220 +361,322 @@ __device__ __forceinline__ bool mega_run_tiles(const MegaParams &p, MegaShared &
     return true;
 }
 
-// Key range of split `split` of `n_splits` over keys 0..pos.
-__device__ __forceinline__ void mega_split_range(int pos, int split, int n_splits, int &k0, int &k1)
+// ---------------------------------------------------------------------------------------------
+// Decode attention of one (kv head, key split) unit.
+//
+// The cached keys and values of the unit are staged in shared memory by TMA loads (boxes of 16 keys x 64
+// channels, 128-byte swizzle) that are issued at the very start of the layer (between the arrival at and
+// the wait on the barrier that opens it), so that their DRAM latency -- several microseconds while the
+// weight ring keeps HBM saturated -- is over by the time the QKV projection has been reduced.  The
+// staging rows start at the unit's first key rounded down to a box boundary; with the swizzle ldmatrix reads
+// are free of bank conflicts.  The products run on mma.sync (fp16 inputs, fp32 accumulation) in the
+// transposed form that wastes no accumulator rows on a handful of query heads:
+//     S^T[16 keys x 8 heads]  = K[16 x D] . Q^T[D x 8]        (Q as hi + lo fp16 halves: two MMAs)
+//     O^T[D x 8 heads]       += V^T[D x 16 keys] . P^T[16 x 8] (P^T from the S^T accumulators by movmatrix)
+// Each warp takes groups of 16 keys and keeps its own running maximum / sum / O^T; the warps are merged
+// through shared memory, the key splits by mega_attention_merge.
+// ---------------------------------------------------------------------------------------------
+struct MegaUnit {
+    int hk, split, ns;
+    int k0a;           // first key of the unit rounded down to a multiple of 16: row r of the staging area is key k0a + r
+    int lead;          // rows before the unit's first key (fetched with the first box, masked)
+    int n_rows;        // rows up to and including the unit's last key (this step's own key included)
+    int n_cached;      // rows below this bound hold cached keys
+    int owner;         // the unit holds this step's position (its last row)
+    int CH, nch;       // rows per staging chunk, number of chunks
+    int pg0;           // first block-table entry of the unit
+    uint32_t kbase, vbase;   // shared-memory addresses of the K and V staging areas
+    uint32_t half_bytes;     // one 64-channel half of an area: kv_cap rows of 128 bytes
+    uint8_t *kptr, *vptr;
+};
+
+constexpr int kMegaKvBoxRows = 16;
+constexpr int kMegaKvBoxBytes = kMegaKvBoxRows * 128;
+
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
 {
-    const int n_keys = pos + 1;
-    const int per = (n_keys + n_splits - 1) / n_splits;
-    k0 = split * per;
-    k1 = min(n_keys, k0 + per);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a)
+{
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+__device__ __forceinline__ void mma_f16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi)
+{
+    return (uint32_t)__half_as_ushort(__float2half_rn(lo)) | ((uint32_t)__half_as_ushort(__float2half_rn(hi)) << 16);
 }
 
+// Byte offset of channel d of row `row` inside a staging area (two 64-channel halves of 128-byte rows
+// with the 128-byte swizzle the tensor map writes: 16-byte chunk index xor row mod 8).
+__device__ __forceinline__ uint32_t mega_kv_swz(const MegaUnit &u, int row, int d)
+{
+    const uint32_t cb = (uint32_t)(d & 63) * 2;
+    return (uint32_t)(d >> 6) * u.half_bytes + (uint32_t)row * 128 + (cb ^ ((uint32_t)(row & 7) << 4));
+}
+
+// Geometry of this CTA's unit for the whole step (the same in every layer).
 template <int D>
-__device__ __forceinline__ void mega_attention_prefetch(const MegaParams &p, const KvView &kv, int hk, int split, int n_splits,
-                                                        int pos, int cw, int lane, MegaKvPrefetch &pf)
+__device__ __forceinline__ MegaUnit mega_unit(const MegaParams &p, uint8_t *base_ptr, uint32_t base, int pos, int ns)
 {
-    constexpr int LPK = D / 8, KPW = 32 / LPK;
-    const int sub = lane / LPK, ch = (lane % LPK) * 8;
-    int k0, k1;
-    mega_split_range(pos, split, n_splits, k0, k1);
-    const int k1c = min(k1, pos);
-    const int base = k0 + (cw * kMegaAttnUK) * KPW;
-#pragma unroll
-    for (int u = 0; u < kMegaAttnUK; ++u) {
-        const int key = base + u * KPW + sub;
-        pf.ok[u] = key < k1c;
-        if (pf.ok[u]) {
-            const size_t off = kv_offset(kv, key, hk, D, p.status) + ch;
-            pf.kf[u] = __ldcg(reinterpret_cast<const uint4 *>(kv.k + off));
-            pf.vf[u] = __ldcg(reinterpret_cast<const uint4 *>(kv.v + off));
-        } else {
-            pf.kf[u] = make_uint4(0, 0, 0, 0);
-            pf.vf[u] = make_uint4(0, 0, 0, 0);
+    MegaUnit u;
+    u.ns = ns;
+    u.hk = blockIdx.x / ns;
+    u.split = blockIdx.x - u.hk * ns;
+    const int n_keys = pos + 1;
+    const int per = (n_keys + ns - 1) / ns;
+    const int k0 = u.split * per;
+    const int k1 = min(n_keys, k0 + per);
+    const int n_all = max(0, k1 - k0);
+    u.owner = (k0 <= pos && pos < k1) ? 1 : 0;
+    u.k0a = k0 & ~(kMegaKvBoxRows - 1);
+    u.lead = k0 - u.k0a;
+    u.n_rows = n_all > 0 ? u.lead + n_all : 0;
+    u.n_cached = n_all > 0 ? u.n_rows - u.owner : 0;
+    if (u.n_rows <= p.kv_cap) {
+        u.CH = p.kv_cap;
+        u.nch = u.n_rows > 0 ? 1 : 0;
+    } else {
+        u.CH = (p.kv_cap >> 1) & ~15;
+        u.nch = (u.n_rows + u.CH - 1) / u.CH;
+    }
+    u.pg0 = u.k0a >> p.kv.page_shift;
+    u.half_bytes = (uint32_t)p.kv_cap * 128;
+    u.kbase = base + (uint32_t)p.kv_off;
+    u.vbase = u.kbase + (uint32_t)(D / 64) * u.half_bytes;
+    u.kptr = base_ptr + p.kv_off;
+    u.vptr = u.kptr + (size_t)(D / 64) * u.half_bytes;
+    return u;
+}
+
+// TMA loads of the cached keys/values of chunk ci of layer l into its staging buffer: boxes of 16 keys x 64
+// channels from the pools viewed as [row][D] matrices (a page holds whole boxes), issued by one warp.
+template <int D>
+__device__ __forceinline__ void mega_kv_issue(const MegaParams &p, MegaShared &sh, const MegaUnit &u, int l, int ci, int lane)
+{
+    constexpr int NH = D / 64;
+    const int b = ci & 1;
+    const int r_begin = ci * u.CH;
+    const int r_end = min(u.n_cached, r_begin + u.CH);
+    const int ng = r_end > r_begin ? (r_end - r_begin + kMegaKvBoxRows - 1) / kMegaKvBoxRows : 0;
+    const int boxes = ng * NH * 2;
+    const uint32_t bar = smem_u32(&sh.kvfull[b]);
+    if (lane == 0) mbar_expect_tx(bar, (uint32_t)boxes * kMegaKvBoxBytes);
+    __syncwarp();
+    const CUtensorMap *kmap = p.maps + 4 * p.n_layers + 1;
+    for (int idx = lane; idx < boxes; idx += 32) {
+        const int g = idx / (2 * NH), rem = idx - g * (2 * NH);
+        const int isv = rem / NH, half = rem - isv * NH;
+        const int row = r_begin + g * kMegaKvBoxRows;
+        const int key = u.k0a + row;
+        const int pi = (key >> p.kv.page_shift) - u.pg0;
+        int page = pi < kMegaMaxUnitPages ? sh.pages[pi] : p.kv.block_tab[key >> p.kv.page_shift];
+        if ((unsigned)page >= (unsigned)p.kv.n_pages) {
+            atomicOr(p.status, DEV_BAD_PAGE);
+            page = 0;
         }
+        const int y = ((l * p.kv.n_pages + page) * p.kv.n_kv_heads + u.hk) * p.kv.page_size + (key & (p.kv.page_size - 1));
+        const uint32_t dst = (isv ? u.vbase : u.kbase) + (uint32_t)half * u.half_bytes + (uint32_t)(b * u.CH + row - r_begin) * 128;
+        tma_load_2d(dst, kmap + isv, half * 64, y, bar);
     }
 }
 
-// Attention of one (kv head, key split) unit by the CTA's consumer warps: rotary embedding of q on the
-// fly, cached keys [k0, k1) (the first batch already in registers), and the step's own key/value
-// (position pos) taken from the QKV vector by the split that owns it, which also appends them to the
-// cache.  Partials go to part_o / part_ml; the unit that finishes last for its kv head merges the
-// splits into ATT.
-template <int D, int G>
-__device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaShared &sh, MegaAttnScratch<D, G> &sc,
-                                                    const KvView &kv, int hk, int split, int n_splits, int pos, int cw, int lane,
-                                                    MegaKvPrefetch &pf)
+// The first (up to two) chunks of a layer; called by one consumer warp once the activation area is free.
+template <int D>
+__device__ __forceinline__ void mega_kv_issue_first(const MegaParams &p, MegaShared &sh, const MegaUnit &u, int l, int lane)
 {
-    constexpr int LPK = D / 8, KPW = 32 / LPK, UK = kMegaAttnUK, half = D / 2;
-    const int gt = cw * 32 + lane;                  // thread within the unit
-    const int sub = lane / LPK, ch = (lane % LPK) * 8;
-    int k0, k1;
-    mega_split_range(pos, split, n_splits, k0, k1);
-    const int k1c = min(k1, pos);                   // cached keys only
-    // rotate 8 channels starting at ch of a head vector v (fp32, unrotated) at this step's position
-    auto rotated8 = [&](const float *v, float *out8) {
-        const int other = ch < half ? ch + half : ch - half;
-        const int j0 = ch < half ? ch : ch - half;
-        const float4 m0 = __ldcg(reinterpret_cast<const float4 *>(v + ch)), m1 = __ldcg(reinterpret_cast<const float4 *>(v + ch + 4));
-        const float4 o0 = __ldcg(reinterpret_cast<const float4 *>(v + other)), o1 = __ldcg(reinterpret_cast<const float4 *>(v + other + 4));
-        const float mine[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
-        const float oth[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
+    for (int ci = 0; ci < min(u.nch, 2); ++ci) mega_kv_issue<D>(p, sh, u, l, ci, lane);
+}
+
+template <int D, int G>
+__device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaShared &sh, MegaAttnScratch<D, G> &sc, const MegaUnit &u,
+                                                    const MegaLayer &L, int l, int pos, unsigned (&kvph)[2], int cw, int lane MEGA_TRACE_PARAM)
+{
+    static_assert(G <= 8, "one MMA column per query head of the group");
+    static_assert(D == 64 || D == 128, "staging rows are one or two 64-channel halves");
+    constexpr int KS = D / 16, HALF = D / 2, PER_LANE = (HALF + 31) / 32;
+    const int gt = cw * 32 + lane;
+    const int gq = lane >> 2, t = lane & 3;
+    // ---- Q^T fragments: head gq, channels 16 ks + 2 t + {0, 1, 8, 9}; rotated, scaled, split into hi + lo ----
+    uint32_t qhi[KS][2], qlo[KS][2];
+    {
+        float2 raw[KS][2];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const float2 t = sh.cs[j0 + e];
-            out8[e] = ch < half ? mine[e] * t.x - oth[e] * t.y : mine[e] * t.x + oth[e] * t.y;
+        for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) raw[ks][hf] = make_float2(0.f, 0.f);
+        if (gq < G) {
+            const float *qsrc = p.QKV + (size_t)(u.hk * G + gq) * D + 2 * t;
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) raw[ks][hf] = __ldcg(reinterpret_cast<const float2 *>(qsrc + 16 * ks + 8 * hf));
         }
-    };
-    float q[G][8];
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-        rotated8(p.QKV + (size_t)(hk * G + g) * D, q[g]);
+        for (int ks = 0; ks < KS / 2; ++ks)
 #pragma unroll
-        for (int e = 0; e < 8; ++e) q[g][e] *= p.scale;
+            for (int hf = 0; hf < 2; ++hf) {
+                const int d = 16 * ks + 8 * hf + 2 * t;             // channel in the first half; partner d + HALF
+                const float2 c0 = sh.cs[d], c1 = sh.cs[d + 1];
+                const float2 a = raw[ks][hf], bq = raw[ks + KS / 2][hf];
+                const float x0 = (a.x * c0.x - bq.x * c0.y) * p.scale, y0 = (a.y * c1.x - bq.y * c1.y) * p.scale;
+                const float x1 = (bq.x * c0.x + a.x * c0.y) * p.scale, y1 = (bq.y * c1.x + a.y * c1.y) * p.scale;
+                const uint32_t h0 = pack_half2(x0, y0), h1 = pack_half2(x1, y1);
+                qhi[ks][hf] = h0;
+                qhi[ks + KS / 2][hf] = h1;
+                qlo[ks][hf] = pack_half2(x0 - kv_lo(h0), y0 - kv_hi(h0));
+                qlo[ks + KS / 2][hf] = pack_half2(x1 - kv_lo(h1), y1 - kv_hi(h1));
+            }
     }
-    float mx[G], den[G], o[G][8];
+    // ---- this step's own key/value (owner unit, first warp): rotate k, round both to what the cache holds, append ----
+    uint16_t own_k[PER_LANE][2], own_v[PER_LANE][2];
+    if (u.owner && cw == 0) {
+        const float *ksrc = p.QKV + (size_t)(p.Hq + u.hk) * D, *vsrc = p.QKV + (size_t)(p.Hq + p.Hkv + u.hk) * D;
+        KvView kv = p.kv;
+        const size_t off = kv_offset(kv, pos, u.hk, D, p.status);
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-        mx[g] = -INFINITY;
-        den[g] = 0.f;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) o[g][e] = 0.f;
-    }
-    auto update = [&](const float *kk, const float *vv, bool ok) {
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            float s = 0.f;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) s = fmaf(q[g][e], kk[e], s);
-#pragma unroll
-            for (int off = LPK / 2; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-            if (ok) {
-                const float mnew = fmaxf(mx[g], s);
-                const float corr = __expf(mx[g] - mnew), pw = __expf(s - mnew);
-                den[g] = den[g] * corr + pw;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) o[g][e] = fmaf(pw, vv[e], o[g][e] * corr);
-                mx[g] = mnew;
+        for (int i = 0; i < PER_LANE; ++i) {
+            const int j = lane + 32 * i;
+            if (j < HALF) {
+                const float a = __ldcg(ksrc + j), bk = __ldcg(ksrc + j + HALF);
+                const float2 c = sh.cs[j];
+                own_k[i][0] = kv_bits(a * c.x - bk * c.y);
+                own_k[i][1] = kv_bits(bk * c.x + a * c.y);
+                own_v[i][0] = kv_bits(__ldcg(vsrc + j));
+                own_v[i][1] = kv_bits(__ldcg(vsrc + j + HALF));
+                L.kpool[off + j] = own_k[i][0];
+                L.kpool[off + j + HALF] = own_k[i][1];
+                L.vpool[off + j] = own_v[i][0];
+                L.vpool[off + j + HALF] = own_v[i][1];
             }
         }
-    };
-    for (int base = k0 + (cw * UK) * KPW; base < k1c; base += kMegaAttnWarps * UK * KPW) {
-        if (base != k0 + (cw * UK) * KPW) {   // later batches; the first one was fetched ahead of the barrier
+    }
+    MEGA_MARK();
+    float mrun[2] = {-INFINITY, -INFINITY}, lrun[2] = {0.f, 0.f};
+    float oacc[KS][4];
 #pragma unroll
-            for (int u = 0; u < UK; ++u) {
-                const int key = base + u * KPW + sub;
-                pf.ok[u] = key < k1c;
-                if (pf.ok[u]) {
-                    const size_t off = kv_offset(kv, key, hk, D, p.status) + ch;
-                    pf.kf[u] = __ldcg(reinterpret_cast<const uint4 *>(kv.k + off));
-                    pf.vf[u] = __ldcg(reinterpret_cast<const uint4 *>(kv.v + off));
-                } else {
-                    pf.kf[u] = make_uint4(0, 0, 0, 0);
-                    pf.vf[u] = make_uint4(0, 0, 0, 0);
+    for (int mt = 0; mt < KS; ++mt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) oacc[mt][e] = 0.f;
+
+    for (int ci = 0; ci < u.nch; ++ci) {
+        const int b = ci & 1;
+        const int nr = min(u.n_rows, (ci + 1) * u.CH) - ci * u.CH;   // rows of the chunk, the own key's included
+        mbar_wait(smem_u32(&sh.kvfull[b]), kvph[b] & 1u, &sh.abort, p.status);
+        ++kvph[b];
+        if (ci == u.nch - 1 && u.owner && cw == 0) {
+            const int row = b * u.CH + nr - 1;
+#pragma unroll
+            for (int i = 0; i < PER_LANE; ++i) {
+                const int j = lane + 32 * i;
+                if (j < HALF) {
+                    *reinterpret_cast<uint16_t *>(u.kptr + mega_kv_swz(u, row, j)) = own_k[i][0];
+                    *reinterpret_cast<uint16_t *>(u.kptr + mega_kv_swz(u, row, j + HALF)) = own_k[i][1];
+                    *reinterpret_cast<uint16_t *>(u.vptr + mega_kv_swz(u, row, j)) = own_v[i][0];
+                    *reinterpret_cast<uint16_t *>(u.vptr + mega_kv_swz(u, row, j + HALF)) = own_v[i][1];
                 }
             }
         }
-        // scores of the whole batch first (independent chains), then one softmax update per head
-        float sc_[UK][G];
-#pragma unroll
-        for (int u = 0; u < UK; ++u) {
-            const float kk[8] = {kv_lo(pf.kf[u].x), kv_hi(pf.kf[u].x), kv_lo(pf.kf[u].y), kv_hi(pf.kf[u].y),
-                                 kv_lo(pf.kf[u].z), kv_hi(pf.kf[u].z), kv_lo(pf.kf[u].w), kv_hi(pf.kf[u].w)};
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-                float t = 0.f;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) t = fmaf(q[g][e], kk[e], t);
-                sc_[u][g] = t;
+        {   // value rows behind the last key of the last group of 16 must be finite (their weight is zero)
+            const int pad = ((nr + 15) & ~15) - nr;
+            for (int idx = gt; idx < pad * (D / 8); idx += kMegaCT) {
+                const int r = b * u.CH + nr + idx / (D / 8), c = idx % (D / 8);
+                *reinterpret_cast<uint4 *>(u.vptr + (size_t)(c >> 3) * u.half_bytes + (size_t)r * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
             }
         }
+        consumer_sync();
+        MEGA_MARK();
+        const int ngroups = (nr + 15) >> 4;
+        for (int gi = cw; gi < ngroups; gi += kMegaConsumers) {
+            const int r0 = gi * 16;
+            // S^T = K . Q^T
+            float s[4] = {0.f, 0.f, 0.f, 0.f};
+            const int krow = b * u.CH + r0 + (lane & 7) + ((lane >> 3) & 1) * 8;
+            const uint32_t ka = u.kbase + (uint32_t)krow * 128;
+            const uint32_t kx = (uint32_t)(krow & 7);
 #pragma unroll
-        for (int off = LPK / 2; off > 0; off >>= 1)
+            for (int ks = 0; ks < KS; ++ks) {
+                uint32_t a[4];
+                ldmatrix_x4(a, ka + (uint32_t)(ks >> 2) * u.half_bytes + ((((uint32_t)(ks & 3) * 2 + (uint32_t)(lane >> 4)) ^ kx) << 4));
+                mma_f16_16816(s, a, qhi[ks][0], qhi[ks][1]);
+                mma_f16_16816(s, a, qlo[ks][0], qlo[ks][1]);
+            }
+            // online softmax per head (column): this lane holds rows r0 + gq (+ 8) of heads 2 t, 2 t + 1
+            const int rr = ci * u.CH + r0 + gq;
+            const bool v0 = rr >= u.lead && rr < u.n_rows, v1 = rr + 8 >= u.lead && rr + 8 < u.n_rows;
+            const float s0 = v0 ? s[0] : -INFINITY, s1 = v0 ? s[1] : -INFINITY, s2 = v1 ? s[2] : -INFINITY, s3 = v1 ? s[3] : -INFINITY;
+            float m0 = fmaxf(s0, s2), m1 = fmaxf(s1, s3);
 #pragma unroll
-            for (int u = 0; u < UK; ++u)
+            for (int o = 4; o < 32; o <<= 1) {
+                m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, o));
+                m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, o));
+            }
+            const float n0 = fmaxf(mrun[0], m0), n1 = fmaxf(mrun[1], m1);   // finite: the group holds a live key
+            const float corr0 = mrun[0] == -INFINITY ? 0.f : __expf(mrun[0] - n0);
+            const float corr1 = mrun[1] == -INFINITY ? 0.f : __expf(mrun[1] - n1);
+            const float p0 = v0 ? __expf(s0 - n0) : 0.f, p1 = v0 ? __expf(s1 - n1) : 0.f;
+            const float p2 = v1 ? __expf(s2 - n0) : 0.f, p3 = v1 ? __expf(s3 - n1) : 0.f;
+            mrun[0] = n0;
+            mrun[1] = n1;
+            lrun[0] = lrun[0] * corr0 + p0 + p2;
+            lrun[1] = lrun[1] * corr1 + p1 + p3;
+            const uint32_t pb0 = movmatrix_trans(pack_half2(p0, p1)), pb1 = movmatrix_trans(pack_half2(p2, p3));
+            // O^T += V^T . P^T
+            const int vrow = b * u.CH + r0 + (lane & 7) + (lane >> 4) * 8;
+            const uint32_t va = u.vbase + (uint32_t)vrow * 128;
+            const uint32_t vx = (uint32_t)(vrow & 7);
 #pragma unroll
-                for (int g = 0; g < G; ++g) sc_[u][g] += __shfl_xor_sync(0xffffffffu, sc_[u][g], off);
-        float vv[UK][8];
-#pragma unroll
-        for (int u = 0; u < UK; ++u) {
-            vv[u][0] = kv_lo(pf.vf[u].x); vv[u][1] = kv_hi(pf.vf[u].x); vv[u][2] = kv_lo(pf.vf[u].y); vv[u][3] = kv_hi(pf.vf[u].y);
-            vv[u][4] = kv_lo(pf.vf[u].z); vv[u][5] = kv_hi(pf.vf[u].z); vv[u][6] = kv_lo(pf.vf[u].w); vv[u][7] = kv_hi(pf.vf[u].w);
-        }
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            float mnew = mx[g];
-#pragma unroll
-            for (int u = 0; u < UK; ++u)
-                if (pf.ok[u]) mnew = fmaxf(mnew, sc_[u][g]);
-            if (mnew > -INFINITY) {
-                const float corr = mx[g] == -INFINITY ? 0.f : __expf(mx[g] - mnew);
-                den[g] *= corr;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) o[g][e] *= corr;
-#pragma unroll
-                for (int u = 0; u < UK; ++u) {
-                    if (pf.ok[u]) {
-                        const float pw = __expf(sc_[u][g] - mnew);
-                        den[g] += pw;
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) o[g][e] = fmaf(pw, vv[u][e], o[g][e]);
-                    }
-                }
-                mx[g] = mnew;
+            for (int mt = 0; mt < KS; ++mt) {
+                oacc[mt][0] *= corr0; oacc[mt][1] *= corr1; oacc[mt][2] *= corr0; oacc[mt][3] *= corr1;
+                uint32_t a[4];
+                ldmatrix_x4_trans(a, va + (uint32_t)(mt >> 2) * u.half_bytes + ((((uint32_t)(mt & 3) * 2 + (uint32_t)((lane >> 3) & 1)) ^ vx) << 4));
+                mma_f16_16816(oacc[mt], a, pb0, pb1);
             }
         }
-    }
-    if (k0 <= pos && pos < k1 && cw == 0) {
-        // this step's own key/value: rotate k, round both to fp16 (what the cache holds), append, attend
-        float kk[8], vv[8];
-        rotated8(p.QKV + (size_t)(p.Hq + hk) * D, kk);
-        const float *vsrc = p.QKV + (size_t)(p.Hq + p.Hkv + hk) * D + ch;
-        const float4 v0 = __ldcg(reinterpret_cast<const float4 *>(vsrc)), v1 = __ldcg(reinterpret_cast<const float4 *>(vsrc + 4));
-        const float vraw[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-        uint32_t kb[4], vb[4];
-#pragma unroll
-        for (int e = 0; e < 8; e += 2) {
-            kb[e >> 1] = (uint32_t)kv_bits(kk[e]) | ((uint32_t)kv_bits(kk[e + 1]) << 16);
-            vb[e >> 1] = (uint32_t)kv_bits(vraw[e]) | ((uint32_t)kv_bits(vraw[e + 1]) << 16);
-            kk[e] = kv_lo(kb[e >> 1]); kk[e + 1] = kv_hi(kb[e >> 1]);
-            vv[e] = kv_lo(vb[e >> 1]); vv[e + 1] = kv_hi(vb[e >> 1]);
+        if (ci + 2 < u.nch) {   // refill this buffer with the chunk after next
+            consumer_sync();
+            if (cw == 0) mega_kv_issue<D>(p, sh, u, l, ci + 2, lane);
         }
-        if (sub == 0) {
-            const size_t off = kv_offset(kv, pos, hk, D, p.status) + ch;
-            *reinterpret_cast<uint4 *>(kv.k + off) = make_uint4(kb[0], kb[1], kb[2], kb[3]);
-            *reinterpret_cast<uint4 *>(kv.v + off) = make_uint4(vb[0], vb[1], vb[2], vb[3]);
-        }
-        update(kk, vv, sub == 0);
     }
-    // ---- merge lane groups, then the warps ----
+    MEGA_MARK();
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
+    for (int o = 4; o < 32; o <<= 1) {
+        lrun[0] += __shfl_xor_sync(0xffffffffu, lrun[0], o);
+        lrun[1] += __shfl_xor_sync(0xffffffffu, lrun[1], o);
+    }
+    // ---- merge the warps (the scratch overlays the staging buffers: every warp must be done reading them) ----
+    consumer_sync();
+    MEGA_MARK();
 #pragma unroll
-        for (int off = LPK; off < 32; off <<= 1) {
-            const float m2 = __shfl_xor_sync(0xffffffffu, mx[g], off);
-            const float d2 = __shfl_xor_sync(0xffffffffu, den[g], off);
-            const float mnew = fmaxf(mx[g], m2);
-            const float c1 = mx[g] == -INFINITY ? 0.f : __expf(mx[g] - mnew);
-            const float c2 = m2 == -INFINITY ? 0.f : __expf(m2 - mnew);
-            den[g] = den[g] * c1 + d2 * c2;
+    for (int e = 0; e < 2; ++e) {
+        const int head = 2 * t + e;
+        if (head < G) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const float o2 = __shfl_xor_sync(0xffffffffu, o[g][e], off);
-                o[g][e] = o[g][e] * c1 + o2 * c2;
+            for (int mt = 0; mt < KS; ++mt) {
+                sc.o[cw][head][16 * mt + gq] = oacc[mt][e];
+                sc.o[cw][head][16 * mt + gq + 8] = oacc[mt][2 + e];
             }
-            mx[g] = mnew;
-        }
-    }
-    if (sub == 0) {
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) sc.o[cw][g][ch + e] = o[g][e];
-            if (lane == 0) { sc.m[cw][g] = mx[g]; sc.d[cw][g] = den[g]; }
+            if (gq == 0) { sc.m[cw][head] = mrun[e]; sc.d[cw][head] = lrun[e]; }
         }
     }
     consumer_sync();
-    const int hq0 = hk * G;
+    MEGA_MARK();
+    const int hq0 = u.hk * G;
     for (int idx = gt; idx < G * D; idx += kMegaCT) {
         const int g = idx / D, c = idx - g * D;
         float mnew = -INFINITY;
@@ -583,12 +685,14 @@ __device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaSha
         float dsum = 0.f, osum = 0.f;
 #pragma unroll
         for (int w = 0; w < kMegaAttnWarps; ++w) {
-            const float cw2 = sc.m[w][g] == -INFINITY ? 0.f : __expf(sc.m[w][g] - mnew);
-            dsum += sc.d[w][g] * cw2;
-            osum += sc.o[w][g][c] * cw2;
+            if (sc.m[w][g] != -INFINITY) {   // a warp without keys left its slots untouched
+                const float cw2 = __expf(sc.m[w][g] - mnew);
+                dsum += sc.d[w][g] * cw2;
+                osum += sc.o[w][g][c] * cw2;
+            }
         }
-        const size_t pi = (size_t)(hq0 + g) * n_splits + split;
-        if (n_splits == 1) {
+        const size_t pi = (size_t)(hq0 + g) * u.ns + u.split;
+        if (u.ns == 1) {
             p.ATT[(size_t)(hq0 + g) * D + c] = osum / dsum;   // a single split is the final result
         } else {
             p.part_o[pi * D + c] = osum;
@@ -682,6 +786,8 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
             mbar_init(smem_u32(&sh.full[s]), 1);
             mbar_init(smem_u32(&sh.empty[s]), kMegaConsumers);
         }
+        mbar_init(smem_u32(&sh.kvfull[0]), 1);
+        mbar_init(smem_u32(&sh.kvfull[1]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -734,17 +840,29 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
     MEGA_MARK();
     auto xb_of = [&](int K) { return xa + (K >> 3); };
 
-    // step set-up: rotary table, zeroed accumulation vectors
+    // step set-up: rotary table, zeroed accumulation vectors, this CTA's attention unit
     for (int j = ctid; j < D / 2; j += kMegaCT) {
         double s, c;
         sincos((double)pos * p.inv_freq[j], &s, &c);
         sh.cs[j] = make_float2((float)c, (float)s);
     }
+    // 64 keys per unit while there are CTAs to spare (every CTA derives the same split count)
+    int ns = (pos + 64) / 64;
+    ns = min(ns, min(p.n_splits, max(1, (int)gridDim.x / p.Hkv)));
+    const bool attn_active = (int)blockIdx.x < p.Hkv * ns;
+    const MegaUnit unit = mega_unit<D>(p, base_ptr, base, pos, ns);
+    if (attn_active && unit.n_cached > 0) {
+        const int npg = ((unit.k0a + unit.n_cached - 1) >> p.kv.page_shift) - unit.pg0 + 1;
+        for (int i = ctid; i < min(npg, kMegaMaxUnitPages); i += kMegaCT) sh.pages[i] = p.kv.block_tab[unit.pg0 + i];
+    }
+    unsigned kvph[2] = {0u, 0u};
     mega_zero(p.QKV, qkvd, ctid);
     mega_zero(p.D1, p.h, ctid);
     mega_zero(p.D2, p.h, ctid);
     mega_zero(p.logits, p.vocab, ctid);
-    mega_grid_barrier(p, sh, epoch, ctid);
+    mega_barrier_arrive(p, ctid);
+    if (attn_active && cw == 1) mega_kv_issue_first<D>(p, sh, unit, 0, lane);
+    mega_barrier_wait(p, sh, epoch, ctid);
     MEGA_MARK();
 
     int tokid = p.tok[p.desc->tok_off];
@@ -752,34 +870,29 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
         if (ctid == 0) atomicOr(p.status, DEV_BAD_TOKEN);
         tokid = 0;
     }
-    KvView kv = p.kv;
     MegaAttnScratch<D, G> *scratch = reinterpret_cast<MegaAttnScratch<D, G> *>(base_ptr);
 
     for (int l = 0; l < p.n_layers; ++l) {
         const MegaLayer &L = p.layers[l];
         // ---- QKV: x = (layer 0 ? embedding : x1 + down), normalised ----
-        if (l > 0) mega_grid_barrier(p, sh, epoch, ctid);
+        if (l > 0) {
+            // the down projection is done with the activation area: the unit's cached K/V can start to land
+            fence_proxy_async_smem();
+            mega_barrier_arrive(p, ctid);
+            if (attn_active && cw == 1) mega_kv_issue_first<D>(p, sh, unit, l, lane);
+            mega_barrier_wait(p, sh, epoch, ctid);
+        }
         MEGA_MARK();
         mega_load_x(sh, xa, xb_of(p.h), p.h, p.X1, l > 0 ? p.D2 : nullptr, l == 0 ? p.embed + (size_t)tokid * p.h : nullptr, p.X0,
                     L.g1, p.eps, true, ctid, cw, lane);
     MEGA_MARK();
         mega_run_tiles<MEPI_ADD>(p, sh, mega_phase<D>(p, 4 * l), ring, xa, xb_of(p.h), p.QKV, L.bqkv, it, cw, lane);
     MEGA_MARK();
-        // ---- attention: one (kv head, key split) unit per CTA; its first keys are fetched before the barrier ----
-        kv.k = L.kpool;
-        kv.v = L.vpool;
-        // 64 keys per unit while there are CTAs to spare (every CTA derives the same split count)
-        int ns = (pos + 64) / 64;
-        ns = min(ns, min(p.n_splits, max(1, (int)gridDim.x / p.Hkv)));
-        const bool attn_active = (int)blockIdx.x < p.Hkv * ns;
-        const int a_hk = blockIdx.x / ns, a_split = blockIdx.x - a_hk * ns;
-        MegaKvPrefetch pf;
-        mega_barrier_arrive(p, ctid);
-        if (attn_active) mega_attention_prefetch<D>(p, kv, a_hk, a_split, ns, pos, cw, lane, pf);
-        mega_barrier_wait(p, sh, epoch, ctid);
+        // ---- attention: one (kv head, key split) unit per CTA ----
+        mega_grid_barrier(p, sh, epoch, ctid);
     MEGA_MARK();
         mega_zero(p.D2, p.h, ctid);
-        if (attn_active) mega_attention_unit<D, G>(p, sh, scratch[0], kv, a_hk, a_split, ns, pos, cw, lane, pf);
+        if (attn_active) mega_attention_unit<D, G>(p, sh, scratch[0], unit, L, l, pos, kvph, cw, lane MEGA_TRACE_ARG);
         MEGA_MARK();
         if (ns > 1) {   // uniform over the grid: ns depends on the position only
             mega_grid_barrier(p, sh, epoch, ctid);

@@ -115,7 +115,7 @@ struct st_model {
     float *X0 = nullptr, *X1 = nullptr, *D1 = nullptr, *D2 = nullptr;   // [h] each
     unsigned *mega_sync = nullptr;      // [4]
     int32_t *mega_tickets = nullptr;    // [Hkv]
-    int mega_stages = 0, mega_xarea = 0, mega_splits = 0;
+    int mega_stages = 0, mega_xarea = 0, mega_splits = 0, mega_kv_off = 0, mega_kv_cap = 0;
     size_t mega_smem = 0;
     bool multi_kernel_decode = false;   // debugging aid: one kernel per phase instead
 
@@ -574,7 +574,7 @@ static int model_build(st_model *m)
         CK(cudaMemcpyAsync(m->mega_layers, ml.data(), ml.size() * sizeof(MegaLayer), cudaMemcpyHostToDevice, m->stream));
         CK(cudaStreamSynchronize(m->stream));
         {   // decode-ring TMA descriptors: 256 x 32 boxes without swizzle
-            std::vector<CUtensorMap> maps(4 * c.n_layers + 1);
+            std::vector<CUtensorMap> maps(4 * c.n_layers + 3);
             for (int l = 0; l < c.n_layers; ++l) {
                 const LayerWeights &w = m->layers[l];
                 TRY(make_map_bf16(&maps[4 * l + 0], w.wqkv, qkvd, h, kMegaTileRows, kMegaBoxK, false));
@@ -583,6 +583,11 @@ static int model_build(st_model *m)
                 TRY(make_map_bf16(&maps[4 * l + 3], w.wd, h, f, kMegaTileRows, kMegaBoxK, false));
             }
             TRY(make_map_bf16(&maps[4 * c.n_layers], m->lm_head, c.vocab, h, kMegaTileRows, kMegaBoxK, false));
+            // the K and V pools as [layer][page][kv head][slot] rows of D 16-bit values
+            const uint64_t kv_rows = (uint64_t)c.n_layers * m->n_pages * c.n_kv_heads * c.page_size;
+            if (kv_rows >= (1ull << 31)) return ST_ERR_UNSUPPORTED;   // row coordinates are 32-bit
+            TRY(make_map_bf16(&maps[4 * c.n_layers + 1], m->kpool, kv_rows, D, kMegaKvBoxRows, 64, true));
+            TRY(make_map_bf16(&maps[4 * c.n_layers + 2], m->vpool, kv_rows, D, kMegaKvBoxRows, 64, true));
             ALLOC(m->mega_maps, CUtensorMap, maps.size());
             CK(cudaMemcpyAsync(m->mega_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, m->stream));
             CK(cudaStreamSynchronize(m->stream));
@@ -600,10 +605,21 @@ static int model_build(st_model *m)
         size_t xarea = (size_t)widest * 4;
         const size_t scratch = mega_scratch_bytes(D, c.n_q_heads / c.n_kv_heads);
         if (scratch > xarea) xarea = scratch;
+        // K/V staging of the attention unit: behind the QKV phase's input vector, D 16-bit values per key and pool
+        const size_t kv_row = (size_t)D * 2;
+        const size_t kv_off = ((size_t)h * 4 + 1023) / 1024 * 1024;
+        if (kv_off + 2 * 96 * kv_row > xarea) xarea = kv_off + 2 * 96 * kv_row;
         xarea = (xarea + 1023) / 1024 * 1024;
-        int stages = (int)((226 * 1024 - 1024 - (long long)xarea) / kMegaTileBytes);
+        const long long budget = 226 * 1024 - 1024;
+        int stages = (int)((budget - (long long)xarea) / kMegaTileBytes);
         if (stages < 2) return ST_ERR_UNSUPPORTED;
         m->mega_stages = stages > kMegaMaxStages ? kMegaMaxStages : stages;
+        // shared memory that no ring stage can use enlarges the staging area
+        xarea += (size_t)((budget - (long long)xarea - (long long)m->mega_stages * kMegaTileBytes) / 1024 * 1024);
+        int cap = (int)((xarea - kv_off) / (2 * kv_row)) & ~15;
+        if (cap > 1024) cap = 1024;
+        m->mega_kv_off = (int)kv_off;
+        m->mega_kv_cap = cap;
         m->mega_xarea = (int)xarea;
         m->mega_smem = 1024 + xarea + (size_t)m->mega_stages * kMegaTileBytes;
         m->mega_splits = m->sm_count / c.n_kv_heads > 0 ? m->sm_count / c.n_kv_heads : 1;
@@ -746,6 +762,7 @@ static int pass_decode(st_model *m, const StepDesc *desc, const int32_t *tok, in
     p.part_o = m->part_o; p.part_ml = m->part_ml; p.tickets = m->mega_tickets; p.sync = m->mega_sync; p.status = m->status;
     p.n_layers = c.n_layers; p.h = c.hidden; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.f = c.ffn; p.vocab = c.vocab;
     p.n_splits = m->mega_splits; p.stages = m->mega_stages; p.xarea_bytes = m->mega_xarea;
+    p.kv_off = m->mega_kv_off; p.kv_cap = m->mega_kv_cap;
     p.eps = c.rms_eps; p.scale = 1.f / sqrtf((float)c.head_dim);
     p.want_argmax = sc.want_argmax ? 1 : 0;
     p.limit = sc.vlimit > 0 ? sc.vlimit : c.vocab;
