@@ -183,7 +183,10 @@ class Model:
             self.h = None
 
     def __del__(self):
-        self.close()
+        try:
+            self.close()
+        except TypeError:   # interpreter shutdown: module globals are already gone
+            pass
 
     def set_tensor(self, layer: int, which: int, data):
         a = np.ascontiguousarray(data, dtype=np.float32)
@@ -215,7 +218,10 @@ class KV:
             self.h = None
 
     def __del__(self):
-        self.close()
+        try:
+            self.close()
+        except TypeError:   # interpreter shutdown: module globals are already gone
+            pass
 
     def __len__(self):
         return int(lib().orc_kv_len(self.h))

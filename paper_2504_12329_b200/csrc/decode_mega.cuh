@@ -32,6 +32,7 @@ constexpr int kMegaSeg = 512;                                     // K elements 
 constexpr int kMegaBoxBytes = kMegaTileRows * 256 * 2;            // one TMA box: 32 rows x 256 elements = 16 KB
 constexpr int kMegaTileBytes = 2 * kMegaBoxBytes;                 // 32 KB: two boxes side by side in K
 constexpr int kMegaMaxStages = 6;
+constexpr int kMegaDownSlab = 8;                                  // default K segments per slab of the down projection
 constexpr uint32_t kMegaSpinLimit = 1u << 22;
 constexpr int kMegaMaxUnitPages = 64;                              // block-table entries of one attention unit kept in shared memory
 constexpr int kMegaAttnWarps = kMegaConsumers;                    // all consumer warps work on one attention unit
@@ -65,6 +66,7 @@ struct MegaParams {
     unsigned *sync;           // [1] exit tickets, [2] abort flag, [3] argmax tickets, [32 * (1 + i)] barrier counter i < 8
     int32_t *status;
     int32_t n_layers, h, Hq, Hkv, f, vocab, n_splits, stages, xarea_bytes;
+    int32_t down_slab;        // K segments per slab of the down projection (0: the whole input vector is kept)
     int32_t kv_off, kv_cap;   // K/V staging area inside the activation area: byte offset, capacity in keys (multiple of 16)
     float eps, scale;
     // sampling
@@ -98,7 +100,9 @@ __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;"
 struct MegaPhase {
     const uint16_t *W;
     int N, K;
-    bool whole_blocks;
+    bool whole_blocks;   // split by whole row blocks (the epilogue is not additive)
+    int slab;            // 0: tiles ordered row block first.  s > 0: K is cut into slabs of s segments, tiles ordered slab first,
+                         // then row block, then segment: a CTA's range stays within a slab or two of the input vector
 };
 template <int D>
 __device__ __forceinline__ MegaPhase mega_phase(const MegaParams &p, int idx)
@@ -106,10 +110,13 @@ __device__ __forceinline__ MegaPhase mega_phase(const MegaParams &p, int idx)
     MegaPhase ph;
     const int qd = p.Hq * D, kd = p.Hkv * D;
     if (idx == 4 * p.n_layers) {
-        ph.W = p.lm_head; ph.N = p.vocab; ph.K = p.h; ph.whole_blocks = false;
+        ph.W = p.lm_head; ph.N = p.vocab; ph.K = p.h; ph.whole_blocks = false; ph.slab = 0;
         return ph;
     }
     const MegaLayer &L = p.layers[idx >> 2];
+    // O: one segment per slab (its input load merges the key splits of just those heads); down: slabs of 8 segments
+    // (the activation vector is wide: only a slab of it is kept in shared memory at a time)
+    ph.slab = (idx & 3) == 1 ? 1 : (idx & 3) == 3 ? p.down_slab : 0;
     switch (idx & 3) {
     case 0: ph.W = L.wqkv; ph.N = qd + 2 * kd; ph.K = p.h; ph.whole_blocks = false; break;
     case 1: ph.W = L.wo; ph.N = p.h; ph.K = qd; ph.whole_blocks = false; break;
@@ -119,7 +126,7 @@ __device__ __forceinline__ MegaPhase mega_phase(const MegaParams &p, int idx)
     return ph;
 }
 
-// Tiles [t0, t1) of a phase for this CTA; tile t = (row block t / nseg, K segment t % nseg).
+// Tiles [t0, t1) of a phase for this CTA (MegaTileIter maps tile indices to row blocks and K segments).
 __device__ __forceinline__ void mega_range(const MegaPhase &ph, int cta, int n_cta, int &t0, int &t1, int &nseg)
 {
     const int nblk = (ph.N + kMegaTileRows - 1) / kMegaTileRows;
@@ -133,6 +140,56 @@ __device__ __forceinline__ void mega_range(const MegaPhase &ph, int cta, int n_c
         t1 = (int)((long long)(cta + 1) * T / n_cta);
     }
 }
+
+// Walks the tiles of a phase in order without a division per tile.  The order is slab first (a slab is
+// ph.slab K segments wide; one slab spanning all of K when ph.slab is 0), then row block, then segment.
+struct MegaTileIter {
+    int rb, seg;        // current tile
+    int s_lo, s_hi;     // segments of the current slab
+    int nblk, nseg, slab;
+    __device__ __forceinline__ void init(const MegaPhase &ph, int nseg_, int t)
+    {
+        nseg = nseg_;
+        slab = ph.slab > 0 ? ph.slab : nseg_;
+        nblk = (ph.N + kMegaTileRows - 1) / kMegaTileRows;
+        const int n_slabs = (nseg + slab - 1) / slab;
+        const int sl = min(t / (nblk * slab), n_slabs - 1);
+        s_lo = sl * slab;
+        s_hi = min(nseg, s_lo + slab);   // the last slab may be narrower
+        const int r = t - sl * nblk * slab, width = s_hi - s_lo;
+        rb = r / width;
+        seg = s_lo + (r - rb * width);
+    }
+    // the next tile belongs to another row block (or slab): partial row sums have to be written out
+    __device__ __forceinline__ bool last_of_run() const { return seg + 1 == s_hi; }
+    __device__ __forceinline__ void next()
+    {
+        if (++seg == s_hi) {
+            seg = s_lo;
+            if (++rb == nblk) {
+                rb = 0;
+                s_lo = s_hi;
+                s_hi = min(nseg, s_lo + slab);
+                seg = s_lo;
+            }
+        }
+    }
+};
+
+// Position in the shared-memory ring: slot and the parity of the slot's current use.
+struct MegaRingPos {
+    int slot;
+    unsigned par;
+    bool wrapped;
+    __device__ __forceinline__ void next(int stages)
+    {
+        if (++slot == stages) {
+            slot = 0;
+            par ^= 1u;
+            wrapped = true;
+        }
+    }
+};
 
 // Optional phase timeline (compiled in with -DST_MEGA_TRACE): CTA 0 stamps the global timer at every
 // phase boundary of the step.
@@ -167,11 +224,9 @@ struct MegaShared {
 };
 
 template <int D, int G>
-struct MegaAttnScratch {   // per attention unit (4 warps)
+struct MegaAttnScratch {   // per-warp partial results of an attention unit
     float o[kMegaAttnWarps][G][D];
     float m[kMegaAttnWarps][G], d[kMegaAttnWarps][G];
-    float w[G][kMaxAttnSplits], l[G][kMaxAttnSplits];
-    float den[G];
 };
 
 // Grid-wide barrier over the consumer warps of all CTAs, in two halves so that work which does not depend on
@@ -282,25 +337,33 @@ enum { MEPI_ADD = 0, MEPI_SILU = 1 };
 
 // Consume this CTA's tiles of one weight phase.  out: MEPI_ADD -> out[row] += partial (+ bias with the
 // first K segment); MEPI_SILU -> out[row / 2] = silu(row 2j) * row 2j+1 (whole row blocks only).
+// xa / xb hold the input from element k_base on (phases ordered segment first keep only their segments).
 template <int EPI>
 __device__ __forceinline__ bool mega_run_tiles(const MegaParams &p, MegaShared &sh, const MegaPhase &ph, uint32_t ring,
                                                const float4 *xa, const float4 *xb, float *out, const float *bias,
-                                               unsigned &it, int cw, int lane)
+                                               MegaRingPos &it, int cw, int lane, int k_base = 0, int ta = -1, int tb = -1)
 {
     int t0, t1, nseg;
     mega_range(ph, blockIdx.x, gridDim.x, t0, t1, nseg);
+    if (ta >= 0) {   // a part of this CTA's range
+        t0 = ta;
+        t1 = tb;
+    }
     float acc[kMegaRowsPerWarp], acc2[kMegaRowsPerWarp];
 #pragma unroll
     for (int r = 0; r < kMegaRowsPerWarp; ++r) acc[r] = acc2[r] = 0.f;
     bool first_seg_seen = false;
-    for (int t = t0; t < t1; ++t, ++it) {
-        const int slot = it % p.stages, u = it / p.stages;
-        const int rb = t / nseg, seg = t - rb * nseg;
-        if (seg == 0 || t == t0) first_seg_seen = (seg == 0);
+    MegaTileIter ti;
+    if (t0 < t1) ti.init(ph, nseg, t0);
+    for (int t = t0; t < t1; ++t, ti.next(), it.next(p.stages)) {
+        const int slot = it.slot;
+        const int rb = ti.rb, seg = ti.seg;
+        if (seg == 0) first_seg_seen = true;
+        const bool close = t == t1 - 1 || ti.last_of_run();   // the row block's run of tiles ends here
         const int k0 = seg * kMegaSeg;
         // after an expired wait every later wait returns at once: the step runs to its end (with a
         // status bit set) instead of leaving warps behind at a barrier
-        mbar_wait(smem_u32(&sh.full[slot]), u & 1, &sh.abort, p.status);
+        mbar_wait(smem_u32(&sh.full[slot]), it.par, &sh.abort, p.status);
         const uint32_t tile = ring + (uint32_t)slot * kMegaTileBytes + (uint32_t)(cw * kMegaRowsPerWarp) * (kMegaBoxK * 2);
         // all weight loads of the tile first (8 x 16 bytes per lane), then the multiplies: two
         // independent accumulation chains per row
@@ -316,7 +379,7 @@ __device__ __forceinline__ bool mega_run_tiles(const MegaParams &p, MegaShared &
         for (int c = 0; c < kMegaSeg / kMegaBoxK; ++c) {
             const int e = c * kMegaBoxK + lane * 8;
             if (k0 + e < ph.K) {
-                const float4 a = xa[(k0 + e) >> 3], b = xb[(k0 + e) >> 3];
+                const float4 a = xa[(k0 - k_base + e) >> 3], b = xb[(k0 - k_base + e) >> 3];
 #pragma unroll
                 for (int r = 0; r < kMegaRowsPerWarp; ++r) {
                     const uint4 v = w[c][r];
@@ -332,7 +395,7 @@ __device__ __forceinline__ bool mega_run_tiles(const MegaParams &p, MegaShared &
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&sh.empty[slot]));
-        if (seg == nseg - 1 || t == t1 - 1) {
+        if (close) {
             // close this CTA's share of the row block
 #pragma unroll
             for (int r = 0; r < kMegaRowsPerWarp; ++r) acc[r] = warp_sum(acc[r] + acc2[r]);
@@ -374,7 +437,7 @@ __device__ __forceinline__ bool mega_run_tiles(const MegaParams &p, MegaShared &
 //     S^T[16 keys x 8 heads]  = K[16 x D] . Q^T[D x 8]        (Q as hi + lo fp16 halves: two MMAs)
 //     O^T[D x 8 heads]       += V^T[D x 16 keys] . P^T[16 x 8] (P^T from the S^T accumulators by movmatrix)
 // Each warp takes groups of 16 keys and keeps its own running maximum / sum / O^T; the warps are merged
-// through shared memory, the key splits by mega_attention_merge.
+// through shared memory, the key splits by the O projection's input load (mega_load_att).
 // ---------------------------------------------------------------------------------------------
 struct MegaUnit {
     int hk, split, ns;
@@ -692,66 +755,103 @@ __device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaSha
             }
         }
         const size_t pi = (size_t)(hq0 + g) * u.ns + u.split;
-        if (u.ns == 1) {
-            p.ATT[(size_t)(hq0 + g) * D + c] = osum / dsum;   // a single split is the final result
-        } else {
-            p.part_o[pi * D + c] = osum;
-            if (c == 0) { p.part_ml[pi * 2] = mnew; p.part_ml[pi * 2 + 1] = dsum; }
-        }
+        p.part_o[pi * D + c] = osum;
+        if (c == 0) { p.part_ml[pi * 2] = mnew; p.part_ml[pi * 2 + 1] = dsum; }
     }
 }
 
-// Merge of the key splits, spread over all CTAs (runs between two grid barriers): CTA c owns a
-// contiguous range of the Hq * D output channels; 16 threads share one channel and stride the splits.
-template <int D, int G>
-__device__ __forceinline__ void mega_attention_merge(const MegaParams &p, MegaAttnScratch<D, G> &sc, int n_splits, int ctid)
+// Input of the O projection: the attention output of the K segments this CTA's tiles cover (the phase is
+// ordered segment first, so these are one or two segments = a few heads), merged from the key splits'
+// partial results on the fly: att[h][c] = sum_s w_s o_s[c] / sum_s w_s l_s with w_s = exp(m_s - max m).
+// Warp i computes the weights of the i-th head of the segment; then 128 threads x 2 halves of the splits
+// accumulate 4 channels each.
+template <int D>
+__device__ __forceinline__ void mega_load_att(const MegaParams &p, const MegaPhase &ph, float4 *xa, float4 *xb, float *wbuf, int ns,
+                                              int ctid, int cw, int lane)
 {
-    constexpr int TPO = 16;
-    const int n_out = p.Hq * D;
-    const int per = (n_out + gridDim.x - 1) / gridDim.x;
-    const int o0 = blockIdx.x * per, o1 = min(n_out, o0 + per);
-    if (o0 >= o1) return;   // uniform for the CTA
-    float *w = &sc.w[0][0], *l = &sc.l[0][0];
-    for (int hq = o0 / D; hq <= (o1 - 1) / D; ++hq) {
-        for (int sp = ctid; sp < n_splits; sp += kMegaCT) {
-            const float2 ml = __ldcg(reinterpret_cast<const float2 *>(p.part_ml) + (size_t)hq * n_splits + sp);
-            w[sp] = ml.x;
-            l[sp] = ml.y;
-        }
-        consumer_sync();
-        if (ctid < 32) {
-            float mnew = -INFINITY;
-            for (int sp = ctid; sp < n_splits; sp += 32) mnew = fmaxf(mnew, w[sp]);
+    constexpr int HPS = kMegaSeg / D;   // heads per K segment
+    static_assert(HPS <= kMegaConsumers, "one warp per head of a segment");
+    int t0, t1, nseg;
+    mega_range(ph, blockIdx.x, gridDim.x, t0, t1, nseg);
+    if (t0 >= t1) return;   // uniform for the CTA
+    const int nblk = (ph.N + kMegaTileRows - 1) / kMegaTileRows;
+    float *w = wbuf;                               // [HPS][ns]
+    float *inv_den = wbuf + HPS * kMaxAttnSplits;  // [HPS]
+    float4 *tmp = reinterpret_cast<float4 *>(inv_den + 8);   // [128]
+    for (int seg = t0 / nblk; seg <= (t1 - 1) / nblk; ++seg) {
+        const int hq_first = seg * HPS;
+        if (cw < HPS && hq_first + cw < p.Hq) {
+            const int hq = hq_first + cw;
+            const float2 *ml = reinterpret_cast<const float2 *>(p.part_ml) + (size_t)hq * ns;
+            float mmax = -INFINITY;
+            for (int sp = lane; sp < ns; sp += 32) mmax = fmaxf(mmax, __ldcg(ml + sp).x);
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) mnew = fmaxf(mnew, __shfl_xor_sync(0xffffffffu, mnew, o));
+            for (int o = 16; o > 0; o >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, o));
             float dsum = 0.f;
-            for (int sp = ctid; sp < n_splits; sp += 32) {
-                const float ms = w[sp];
-                const float cw2 = ms == -INFINITY ? 0.f : __expf(ms - mnew);
-                w[sp] = cw2;
-                dsum += l[sp] * cw2;
+            for (int sp = lane; sp < ns; sp += 32) {
+                const float2 v = __ldcg(ml + sp);
+                const float ws = v.x == -INFINITY ? 0.f : __expf(v.x - mmax);
+                w[cw * kMaxAttnSplits + sp] = ws;
+                dsum += v.y * ws;
             }
             dsum = warp_sum(dsum);
-            if (ctid == 0) sc.den[0] = dsum;
+            if (lane == 0) inv_den[cw] = 1.f / dsum;
         }
         consumer_sync();
-        const int lo = max(o0, hq * D), hi = min(o1, (hq + 1) * D);
-        const int j = ctid % TPO;
-        const int n_pass = (hi - lo + kMegaCT / TPO - 1) / (kMegaCT / TPO);   // the same for every thread
-        for (int pass = 0; pass < n_pass; ++pass) {
-            const int oi = lo + pass * (kMegaCT / TPO) + ctid / TPO;
-            const bool live = oi < hi;
-            const int c = (live ? oi : lo) - hq * D;
-            const float *po = p.part_o + (size_t)hq * n_splits * D + c;
-            float acc = 0.f;
-            if (live)
-                for (int sp = j; sp < n_splits; sp += TPO) acc = fmaf(__ldcg(po + (size_t)sp * D), w[sp], acc);
-#pragma unroll
-            for (int o = TPO / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-            if (live && j == 0) p.ATT[(size_t)hq * D + c] = acc / sc.den[0];
+        const int col4 = ctid & 127, part = ctid >> 7;
+        const int c = seg * kMegaSeg + col4 * 4;    // first of this thread's 4 channels (column of the O matrix)
+        const bool live = c < ph.K;
+        const int hl = (col4 * 4) / D, hq = hq_first + hl;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (live) {
+            const float *po = p.part_o + (size_t)hq * ns * D + (c - hq * D);
+            const float *wh = w + hl * kMaxAttnSplits;
+            for (int sp = part; sp < ns; sp += 2) {
+                const float4 o4 = __ldcg(reinterpret_cast<const float4 *>(po + (size_t)sp * D));
+                const float ws = wh[sp];
+                acc.x = fmaf(o4.x, ws, acc.x); acc.y = fmaf(o4.y, ws, acc.y);
+                acc.z = fmaf(o4.z, ws, acc.z); acc.w = fmaf(o4.w, ws, acc.w);
+            }
+        }
+        if (part == 1) tmp[col4] = acc;
+        consumer_sync();
+        if (part == 0 && live) {
+            const float4 o2 = tmp[col4];
+            const float id = inv_den[hl];
+            const float4 r = make_float4((acc.x + o2.x) * id, (acc.y + o2.y) * id, (acc.z + o2.z) * id, (acc.w + o2.w) * id);
+            const int q = c >> 2;
+            ((q & 1) ? xb : xa)[q >> 1] = r;
         }
         consumer_sync();
     }
+}
+
+// The piece of this CTA's tile range [t, t1) that lies within one slab: its end and the slab's segments [s0, s1].
+__device__ __forceinline__ int mega_slab_piece(const MegaPhase &ph, int nseg, int t, int t1, int &s0, int &s1)
+{
+    const int slab = ph.slab > 0 ? ph.slab : nseg;   // no slabs: the whole of K is one
+    const int nblk = (ph.N + kMegaTileRows - 1) / kMegaTileRows;
+    const int n_slabs = (nseg + slab - 1) / slab;
+    const int sl = min(t / (nblk * slab), n_slabs - 1);
+    s0 = sl * slab;
+    s1 = min(nseg, s0 + slab) - 1;
+    return sl == n_slabs - 1 ? t1 : min(t1, (sl + 1) * nblk * slab);
+}
+
+// Input of a slab-ordered phase taken as is from a global fp32 vector: elements [s0 * 512, (s1 + 1) * 512)
+// go to xa / xb (xb = xa + (s1 - s0 + 1) * 64), zero beyond K.
+__device__ __forceinline__ void mega_load_segs(float4 *xa, const float *x, int K, int s0, int s1, int ctid)
+{
+    const int n4 = (s1 - s0 + 1) * (kMegaSeg / 4);
+    float4 *xb = xa + (n4 >> 1);
+    consumer_sync();   // every warp is done with what the area held before
+    const int q_base = s0 * (kMegaSeg / 4);
+    for (int q = ctid; q < n4; q += kMegaCT) {
+        const int qa = q_base + q;
+        const float4 v = qa * 4 < K ? __ldcg(reinterpret_cast<const float4 *>(x) + qa) : make_float4(0.f, 0.f, 0.f, 0.f);
+        ((q & 1) ? xb : xa)[q >> 1] = v;
+    }
+    consumer_sync();
 }
 
 __device__ __forceinline__ void mega_zero(float *buf, int n, int ctid)
@@ -794,21 +894,22 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
 
     if (warp == 0) {
         // ------------------------------ producer ------------------------------
-        unsigned it = 0;
+        MegaRingPos it{0, 0u, false};
         bool ok = true;
         for (int idx = 0; idx < n_phases && ok; ++idx) {
             const MegaPhase ph = mega_phase<D>(p, idx);
             int t0, t1, nseg;
             mega_range(ph, blockIdx.x, gridDim.x, t0, t1, nseg);
-            for (int t = t0; t < t1 && ok; ++t, ++it) {
-                const int slot = it % p.stages, u = it / p.stages;
-                if (u > 0) {
-                    int w_ok = lane == 0 ? (int)mbar_wait(smem_u32(&sh.empty[slot]), (u - 1) & 1, &sh.abort, p.status) : 1;
+            MegaTileIter ti;
+            if (t0 < t1) ti.init(ph, nseg, t0);
+            for (int t = t0; t < t1 && ok; ++t, ti.next(), it.next(p.stages)) {
+                const int slot = it.slot;
+                if (it.wrapped) {
+                    int w_ok = lane == 0 ? (int)mbar_wait(smem_u32(&sh.empty[slot]), it.par ^ 1u, &sh.abort, p.status) : 1;
                     w_ok = __shfl_sync(0xffffffffu, w_ok, 0);
                     if (!w_ok) { ok = false; break; }
                 }
-                const int rb = t / nseg, seg = t - rb * nseg;
-                const int r0 = rb * kMegaTileRows, k0 = seg * kMegaSeg;
+                const int r0 = ti.rb * kMegaTileRows, k0 = ti.seg * kMegaSeg;
                 if (lane == 0) {
                     const uint32_t full = smem_u32(&sh.full[slot]);
                     const uint32_t dst = ring + (uint32_t)slot * kMegaTileBytes;
@@ -834,7 +935,8 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
     float4 *xa = reinterpret_cast<float4 *>(base_ptr);
     const int pos = p.desc->pos0;
     const int qd = p.Hq * D, kd = p.Hkv * D, qkvd = qd + 2 * kd;
-    unsigned epoch = 0, it = 0;
+    unsigned epoch = 0;
+    MegaRingPos it{0, 0u, false};
     int trace_i = 0;
     (void)trace_i;
     MEGA_MARK();
@@ -894,16 +996,14 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
         mega_zero(p.D2, p.h, ctid);
         if (attn_active) mega_attention_unit<D, G>(p, sh, scratch[0], unit, L, l, pos, kvph, cw, lane MEGA_TRACE_ARG);
         MEGA_MARK();
-        if (ns > 1) {   // uniform over the grid: ns depends on the position only
-            mega_grid_barrier(p, sh, epoch, ctid);
-            MEGA_MARK();
-            mega_attention_merge<D, G>(p, scratch[0], ns, ctid);
-            MEGA_MARK();
-        }
         mega_grid_barrier(p, sh, epoch, ctid);
     MEGA_MARK();
-        // ---- O projection into D1 ----
-        mega_load_x(sh, xa, xb_of(qd), qd, p.ATT, nullptr, nullptr, nullptr, nullptr, 0.f, false, ctid, cw, lane);
+        // ---- O projection into D1 (its input load merges the key splits) ----
+        {
+            const MegaPhase pho = mega_phase<D>(p, 4 * l + 1);
+            float *wbuf = reinterpret_cast<float *>(base_ptr) + ((qd + 255) & ~255);
+            mega_load_att<D>(p, pho, xa, xb_of(qd), wbuf, ns, ctid, cw, lane);
+        }
     MEGA_MARK();
         mega_run_tiles<MEPI_ADD>(p, sh, mega_phase<D>(p, 4 * l + 1), ring, xa, xb_of(qd), p.D1, nullptr, it, cw, lane);
     MEGA_MARK();
@@ -917,11 +1017,21 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
     MEGA_MARK();
         mega_grid_barrier(p, sh, epoch, ctid);
     MEGA_MARK();
-        // ---- down projection into D2 ----
-        mega_load_x(sh, xa, xb_of(p.f), p.f, p.ACT, nullptr, nullptr, nullptr, nullptr, 0.f, false, ctid, cw, lane);
-    MEGA_MARK();
-        mega_zero(p.D1, p.h, ctid);
-        mega_run_tiles<MEPI_ADD>(p, sh, mega_phase<D>(p, 4 * l + 3), ring, xa, xb_of(p.f), p.D2, nullptr, it, cw, lane);
+        // ---- down projection into D2, slab by slab of the activation vector ----
+        {
+            const MegaPhase phd = mega_phase<D>(p, 4 * l + 3);
+            int t0, t1, nseg;
+            mega_range(phd, blockIdx.x, gridDim.x, t0, t1, nseg);
+            mega_zero(p.D1, p.h, ctid);
+            for (int t = t0; t < t1;) {
+                int s0, s1;
+                const int te = mega_slab_piece(phd, nseg, t, t1, s0, s1);
+                mega_load_segs(xa, p.ACT, p.f, s0, s1, ctid);
+                mega_run_tiles<MEPI_ADD>(p, sh, phd, ring, xa, xa + (s1 - s0 + 1) * (kMegaSeg / 8), p.D2, nullptr, it, cw, lane,
+                                         s0 * kMegaSeg, t, te);
+                t = te;
+            }
+        }
     MEGA_MARK();
     }
     // ---- LM head ----

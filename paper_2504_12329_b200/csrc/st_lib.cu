@@ -115,7 +115,7 @@ struct st_model {
     float *X0 = nullptr, *X1 = nullptr, *D1 = nullptr, *D2 = nullptr;   // [h] each
     unsigned *mega_sync = nullptr;      // [4]
     int32_t *mega_tickets = nullptr;    // [Hkv]
-    int mega_stages = 0, mega_xarea = 0, mega_splits = 0, mega_kv_off = 0, mega_kv_cap = 0;
+    int mega_stages = 0, mega_xarea = 0, mega_splits = 0, mega_kv_off = 0, mega_kv_cap = 0, mega_down_slab = 0;
     size_t mega_smem = 0;
     bool multi_kernel_decode = false;   // debugging aid: one kernel per phase instead
 
@@ -419,7 +419,7 @@ static int init_kernel_attributes()
 static size_t mega_scratch_bytes(int D, int G)
 {
     // sizeof(MegaAttnScratch<D, G>)
-    return sizeof(float) * ((size_t)kMegaAttnWarps * G * D + 2 * (size_t)kMegaAttnWarps * G + 2 * (size_t)G * kMaxAttnSplits + G);
+    return sizeof(float) * ((size_t)kMegaAttnWarps * G * D + 2 * (size_t)kMegaAttnWarps * G);
 }
 
 static int mega_attr_all();
@@ -600,20 +600,36 @@ static int model_build(st_model *m)
         ALLOC(m->mega_tickets, int32_t, c.n_kv_heads);
         CK(cudaMemsetAsync(m->mega_sync, 0, kMegaSyncWords * sizeof(unsigned), m->stream));
         CK(cudaMemsetAsync(m->mega_tickets, 0, c.n_kv_heads * sizeof(int32_t), m->stream));
-        int widest = h > qd ? h : qd;
-        widest = widest > f ? widest : f;
+        // Activation area: the input vectors of the QKV / gate-up (h floats) and O (Hq*D floats) projections, the
+        // attention scratch, the O projection's merge buffers, and behind the QKV phase's input vector the K/V
+        // staging of the attention unit (D 16-bit values per key and pool).  Few KV heads mean many key splits and
+        // short units: 64 keys of staging are enough; otherwise 128, and more from whatever shared memory no ring
+        // stage can use.
+        const int widest = h > qd ? h : qd;
         size_t xarea = (size_t)widest * 4;
         const size_t scratch = mega_scratch_bytes(D, c.n_q_heads / c.n_kv_heads);
         if (scratch > xarea) xarea = scratch;
-        // K/V staging of the attention unit: behind the QKV phase's input vector, D 16-bit values per key and pool
+        const size_t att_area = ((size_t)qd + 256) * 4 + ((size_t)(kMegaSeg / D) * kMaxAttnSplits + 8) * 4 + 2048;
+        if (att_area > xarea) xarea = att_area;
         const size_t kv_row = (size_t)D * 2;
         const size_t kv_off = ((size_t)h * 4 + 1023) / 1024 * 1024;
-        if (kv_off + 2 * 96 * kv_row > xarea) xarea = kv_off + 2 * 96 * kv_row;
+        const size_t kv_min = (size_t)(c.n_kv_heads <= 2 ? 64 : 128) * 2 * kv_row;
+        if (kv_off + kv_min > xarea) xarea = kv_off + kv_min;
+        // The down projection keeps its whole input vector (ffn floats) when that fits into the area as it is;
+        // otherwise it walks K in slabs of 8 segments and keeps one slab at a time.
+        m->mega_down_slab = ((size_t)f + kMegaSeg) * 4 <= xarea ? 0 : kMegaDownSlab;
+        if (const char *es = getenv("ST_DOWN_SLAB")) m->mega_down_slab = atoi(es) < 0 ? 0 : atoi(es);   // tuning aid
+        const size_t down_x = m->mega_down_slab > 0 ? (size_t)m->mega_down_slab * kMegaSeg * 4 : ((size_t)f + kMegaSeg) * 4;
+        if (down_x > xarea) xarea = down_x;
         xarea = (xarea + 1023) / 1024 * 1024;
         const long long budget = 226 * 1024 - 1024;
         int stages = (int)((budget - (long long)xarea) / kMegaTileBytes);
         if (stages < 2) return ST_ERR_UNSUPPORTED;
         m->mega_stages = stages > kMegaMaxStages ? kMegaMaxStages : stages;
+        if (const char *es = getenv("ST_MEGA_STAGES")) {   // tuning aid: fewer ring stages, more K/V staging
+            const int want = atoi(es);
+            if (want >= 2 && want < m->mega_stages) m->mega_stages = want;
+        }
         // shared memory that no ring stage can use enlarges the staging area
         xarea += (size_t)((budget - (long long)xarea - (long long)m->mega_stages * kMegaTileBytes) / 1024 * 1024);
         int cap = (int)((xarea - kv_off) / (2 * kv_row)) & ~15;
@@ -762,7 +778,7 @@ static int pass_decode(st_model *m, const StepDesc *desc, const int32_t *tok, in
     p.part_o = m->part_o; p.part_ml = m->part_ml; p.tickets = m->mega_tickets; p.sync = m->mega_sync; p.status = m->status;
     p.n_layers = c.n_layers; p.h = c.hidden; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.f = c.ffn; p.vocab = c.vocab;
     p.n_splits = m->mega_splits; p.stages = m->mega_stages; p.xarea_bytes = m->mega_xarea;
-    p.kv_off = m->mega_kv_off; p.kv_cap = m->mega_kv_cap;
+    p.kv_off = m->mega_kv_off; p.kv_cap = m->mega_kv_cap; p.down_slab = m->mega_down_slab;
     p.eps = c.rms_eps; p.scale = 1.f / sqrtf((float)c.head_dim);
     p.want_argmax = sc.want_argmax ? 1 : 0;
     p.limit = sc.vlimit > 0 ? sc.vlimit : c.vocab;
