@@ -299,9 +299,9 @@ def main():
                     "d2h_bytes_per_step": int(5 * len(r.tokens) + 13 * r.n_steps + 12 * len(r.handoffs) + 80 * r.n_steps)},
             "gpu_launches": int(launches),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         # DRAM bytes per launch: ncu measured read+write = 1.006 x the algorithmic bytes on a 4-layer
+                         # DRAM bytes per launch: ncu measured read+write = 1.013 x the algorithmic bytes on a 4-layer
                          # case of this kernel (profiles/decode_mega_kernel_4layer_pair.md); scaled to this launch
-                         "traffic": int(1.006 * kern_bytes),
+                         "traffic": int(1.013 * kern_bytes),
                          "traffic_source": "ncu dram__bytes_read+write on a 4-layer capture, scaled by streamed bytes",
                          "kernel": f"decode_mega_kernel ({shp.name}, one decode step per launch, context {ctx})",
                          "algorithmic_bytes_per_launch": int(kern_bytes),
