@@ -8,6 +8,7 @@
 #include "../../include/st.h"
 #include "attention.cuh"
 #include "decode_mega.cuh"
+#include "attn_rows_mma.cuh"
 #include "gemv.cuh"
 #include "prefill_simt.cuh"
 #include "router.cuh"
@@ -76,6 +77,7 @@ struct st_model {
     std::vector<LayerMaps> maps;
     std::map<int, CUtensorMap> act_maps;   // key: (buffer * 2 + plane) * 1024 + m_pad
     bool simt_gemm = false;                // debugging aid: multi-row projections on the CUDA cores
+    bool simt_attn = false;                // debugging aid: multi-row attention on the CUDA cores
     double *inv_freq = nullptr;
     int64_t weight_bytes = 0;
 
@@ -250,6 +252,41 @@ static cudaError_t launch_attn_rows(const AttnParams &p, int D, int G, dim3 grid
 {
     if (D == 64) return launch_attn_rows_d<64>(p, G, grid, s);
     if (D == 128) return launch_attn_rows_d<128>(p, G, grid, s);
+    return cudaErrorInvalidValue;
+}
+
+// Tensor-core multi-row attention: grid = (key splits, kv heads, ceil(rows / (64 / G))).
+template <int D, int G>
+static cudaError_t launch_attn_rows_mma_dg(const AttnRowsMmaParams &p, dim3 grid, cudaStream_t s, bool attr_only)
+{
+    auto kern = attn_rows_mma_kernel<D, G>;
+    const size_t smem = 1024 + (size_t)kArStages * ar_stage_bytes<D>();
+    if (attr_only) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    kern<<<grid, kArThreads, smem, s>>>(p);
+    ++g_launches;
+    return cudaGetLastError();
+}
+
+template <int D>
+static cudaError_t launch_attn_rows_mma_d(const AttnRowsMmaParams &p, int G, dim3 grid, cudaStream_t s, bool attr_only)
+{
+    switch (G) {
+    case 1: return launch_attn_rows_mma_dg<D, 1>(p, grid, s, attr_only);
+    case 2: return launch_attn_rows_mma_dg<D, 2>(p, grid, s, attr_only);
+    case 3: return launch_attn_rows_mma_dg<D, 3>(p, grid, s, attr_only);
+    case 4: return launch_attn_rows_mma_dg<D, 4>(p, grid, s, attr_only);
+    case 5: return launch_attn_rows_mma_dg<D, 5>(p, grid, s, attr_only);
+    case 6: return launch_attn_rows_mma_dg<D, 6>(p, grid, s, attr_only);
+    case 7: return launch_attn_rows_mma_dg<D, 7>(p, grid, s, attr_only);
+    case 8: return launch_attn_rows_mma_dg<D, 8>(p, grid, s, attr_only);
+    }
+    return cudaErrorInvalidValue;
+}
+
+static cudaError_t launch_attn_rows_mma(const AttnRowsMmaParams &p, int D, int G, dim3 grid, cudaStream_t s, bool attr_only = false)
+{
+    if (D == 64) return launch_attn_rows_mma_d<64>(p, G, grid, s, attr_only);
+    if (D == 128) return launch_attn_rows_mma_d<128>(p, G, grid, s, attr_only);
     return cudaErrorInvalidValue;
 }
 
@@ -506,6 +543,8 @@ static int model_build(st_model *m)
     {
         const char *e = getenv("ST_SIMT_GEMM");
         m->simt_gemm = e && e[0] == '1';
+        const char *ea = getenv("ST_SIMT_ATTN");
+        m->simt_attn = ea && ea[0] == '1';
     }
     {
         const int64_t per_layer = 2ll * ((int64_t)qkvd * h + (int64_t)h * qd + 3ll * f * h) + 4ll * qkvd * (c.qkv_bias ? 1 : 0) + 8ll * h;
@@ -756,7 +795,10 @@ static cudaError_t mega_launch(const MegaParams &p, int D, int G, int grid, size
 static int mega_attr_all()
 {
     for (int D = 64; D <= 128; D += 64)
-        for (int G = 1; G <= 8; ++G) CK(mega_launch(MegaParams{}, D, G, 0, 0, nullptr, true));
+        for (int G = 1; G <= 8; ++G) {
+            CK(mega_launch(MegaParams{}, D, G, 0, 0, nullptr, true));
+            CK(launch_attn_rows_mma(AttnRowsMmaParams{}, D, G, dim3(1, 1, 1), nullptr, true));
+        }
     return ST_OK;
 }
 
@@ -878,8 +920,10 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
     uint16_t *XN_lo = m->XN + (size_t)m->max_rows * h, *ATT_lo = m->ATTb + (size_t)m->max_rows * qd,
              *ACT_lo = m->ACTb + (size_t)m->max_rows * f;
     // few rows over a long context: split the keys so that the pass still fills the GPU
-    const int row_ctas = c.n_kv_heads * ((m_upper + 7) / 8);
-    int row_splits = (2 * m->sm_count + row_ctas - 1) / row_ctas;
+    const int rq = m->simt_attn ? 8 : 64 / G;                    // query rows per CTA
+    const int row_tiles = (m_upper + rq - 1) / rq;
+    const int row_ctas = c.n_kv_heads * row_tiles;
+    int row_splits = ((m->simt_attn ? 2 : 1) * m->sm_count + row_ctas - 1) / row_ctas;
     if (row_splits > ctx_upper / 256) row_splits = ctx_upper / 256;
     row_splits = row_splits < 1 ? 1 : row_splits > kRowSplits ? kRowSplits : row_splits;
     static_assert((int)GEPI_STORE == (int)TEPI_STORE && (int)GEPI_RESADD == (int)TEPI_RESADD && (int)GEPI_SILU == (int)TEPI_SILU, "epilogue ids");
@@ -901,7 +945,16 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
         a.desc = desc; a.qkv = m->QKV; a.kv = kv; a.out_f32 = nullptr; a.out_hi = m->ATTb; a.out_lo = ATT_lo;
         a.part_o = m->part_o; a.part_ml = m->part_ml; a.tickets = m->tickets; a.status = m->status;
         a.Hq = c.n_q_heads; a.n_splits = row_splits; a.scale = 1.f / sqrtf((float)D);
-        CK(launch_attn_rows(a, D, G, dim3(row_splits, c.n_kv_heads, (m_upper + 7) / 8), s));
+        if (m->simt_attn) {
+            CK(launch_attn_rows(a, D, G, dim3(row_splits, c.n_kv_heads, row_tiles), s));
+        } else {
+            AttnRowsMmaParams am{};
+            am.a = a;
+            am.kmap = m->mega_maps + 4 * c.n_layers + 1;
+            am.vmap = m->mega_maps + 4 * c.n_layers + 2;
+            am.row_base = (int32_t)((size_t)l * m->n_pages * c.n_kv_heads * c.page_size);
+            CK(launch_attn_rows_mma(am, D, G, dim3(row_splits, c.n_kv_heads, row_tiles), s));
+        }
         TRY((rows_gemm<TEPI_RESADD>(m, desc, m_upper, 1, m->ATTb, ATT_lo, tm.wo, w.wo, nullptr, m->X, nullptr, nullptr, h, qd)));
         rmsnorm_rows_kernel<<<m_upper, 256, 0, s>>>(desc, m->X, w.g2, c.rms_eps, h, m->XN, XN_lo);
         ++g_launches;
