@@ -57,34 +57,50 @@ __global__ void embed_rope_kernel(const StepDesc *desc, const int32_t *tok, cons
 }
 
 // Rotate q in place (fp32), rotate k and store k, v into the cache (fp16).
-// qkv: [rows][(Hq + 2 Hkv) * D] = q heads, then k heads, then v heads.
-__global__ void rope_append_kernel(const StepDesc *desc, float *qkv, const float2 *cs, int Hq, int Hkv, int D,
-                                   KvView kv, int32_t *status)
+// qkv: [rows][(Hq + 2 Hkv) * D] = q heads, then k heads, then v heads.  With k_splits > 0 the row is not in
+// qkv yet: it is bias + the K-split partial sums Ws[s][row] of the QKV projection (summed in split order).
+__global__ void __launch_bounds__(256) rope_append_kernel(const StepDesc *desc, float *qkv, const float *Ws, int k_splits, int ws_rows,
+                                                          const float *bias, const float2 *cs, int Hq, int Hkv, int D, KvView kv,
+                                                          int32_t *status)
 {
     const int i = blockIdx.x;
     if (i >= desc->m) return;
-    const int half = D >> 1, pos = desc->pos0 + i;
-    float *row = qkv + (size_t)i * (Hq + 2 * Hkv) * D;
+    const int half = D >> 1, pos = desc->pos0 + i, N = (Hq + 2 * Hkv) * D;
+    float *row = qkv + (size_t)i * N;
     const float2 *c = cs + (size_t)i * half;
-    for (int idx = threadIdx.x; idx < (Hq + Hkv) * half; idx += blockDim.x) {
-        const int h = idx / half, j = idx - h * half;
-        float *v = row + h * D;
-        const float a = v[j], b = v[j + half];
-        const float2 t = c[j];
-        const float ra = a * t.x - b * t.y, rb = b * t.x + a * t.y;
+    auto val4 = [&](int n) {   // 4 consecutive features of the row, n a multiple of 4
+        if (k_splits <= 0) return *reinterpret_cast<const float4 *>(row + n);
+        float4 v = bias ? *reinterpret_cast<const float4 *>(bias + n) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s = 0; s < k_splits; ++s) {
+            const float4 w = __ldcg(reinterpret_cast<const float4 *>(Ws + ((size_t)s * ws_rows + i) * N + n));
+            v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
+        }
+        return v;
+    };
+    const int q4 = half >> 2;   // groups of 4 channel pairs per head
+    for (int idx = threadIdx.x; idx < (Hq + Hkv) * q4; idx += blockDim.x) {
+        const int h = idx / q4, j = (idx - h * q4) * 4;
+        const float4 a = val4(h * D + j), b = val4(h * D + j + half);
+        const float2 t0 = c[j], t1 = c[j + 1], t2 = c[j + 2], t3 = c[j + 3];
+        const float4 ra = make_float4(a.x * t0.x - b.x * t0.y, a.y * t1.x - b.y * t1.y, a.z * t2.x - b.z * t2.y, a.w * t3.x - b.w * t3.y);
+        const float4 rb = make_float4(b.x * t0.x + a.x * t0.y, b.y * t1.x + a.y * t1.y, b.z * t2.x + a.z * t2.y, b.w * t3.x + a.w * t3.y);
         if (h < Hq) {
-            v[j] = ra;
-            v[j + half] = rb;
+            *reinterpret_cast<float4 *>(row + h * D + j) = ra;
+            *reinterpret_cast<float4 *>(row + h * D + j + half) = rb;
         } else {
             const size_t o = kv_offset(kv, pos, h - Hq, D, status);
-            kv.k[o + j] = kv_bits(ra);
-            kv.k[o + j + half] = kv_bits(rb);
+            *reinterpret_cast<uint2 *>(kv.k + o + j) = make_uint2((uint32_t)kv_bits(ra.x) | ((uint32_t)kv_bits(ra.y) << 16),
+                                                                  (uint32_t)kv_bits(ra.z) | ((uint32_t)kv_bits(ra.w) << 16));
+            *reinterpret_cast<uint2 *>(kv.k + o + j + half) = make_uint2((uint32_t)kv_bits(rb.x) | ((uint32_t)kv_bits(rb.y) << 16),
+                                                                         (uint32_t)kv_bits(rb.z) | ((uint32_t)kv_bits(rb.w) << 16));
         }
     }
-    const float *vsrc = row + (Hq + Hkv) * D;
-    for (int idx = threadIdx.x; idx < Hkv * D; idx += blockDim.x) {
-        const int h = idx / D, j = idx - h * D;
-        kv.v[kv_offset(kv, pos, h, D, status) + j] = kv_bits(vsrc[idx]);
+    const int v0 = (Hq + Hkv) * D;
+    for (int idx = threadIdx.x; idx < Hkv * (D >> 2); idx += blockDim.x) {
+        const int h = idx / (D >> 2), j = (idx - h * (D >> 2)) * 4;
+        const float4 v = val4(v0 + h * D + j);
+        *reinterpret_cast<uint2 *>(kv.v + kv_offset(kv, pos, h, D, status) + j) =
+            make_uint2((uint32_t)kv_bits(v.x) | ((uint32_t)kv_bits(v.y) << 16), (uint32_t)kv_bits(v.z) | ((uint32_t)kv_bits(v.w) << 16));
     }
 }
 

@@ -10,24 +10,47 @@
 
 namespace st {
 
-// XN[i] = rmsnorm(X[i]) * gain as a hi/lo bf16 pair, one CTA per row.
-__global__ void rmsnorm_rows_kernel(const StepDesc *desc, const float *X, const float *gain, float eps, int hidden,
-                                    uint16_t *XN_hi, uint16_t *XN_lo)
+// XN[i] = rmsnorm(X[i]) * gain as a hi/lo bf16 pair, one CTA per row.  With k_splits > 0 the row first
+// receives the K-split partial sums of the projection that feeds the residual stream,
+// X[i] += sum_s Ws[s][i] (in split order), so that projection needs no reduction pass of its own.
+__global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const StepDesc *desc, float *X, const float *Ws, int k_splits, int ws_rows,
+                                                           const float *gain, float eps, int hidden, uint16_t *XN_hi, uint16_t *XN_lo)
 {
     const int i = blockIdx.x;
     if (i >= desc->m) return;
-    const float *x = X + (size_t)i * hidden;
+    float4 *x4 = reinterpret_cast<float4 *>(X + (size_t)i * hidden);
+    const int n4 = hidden >> 2;
     float ss = 0.f;
-    for (int j = threadIdx.x; j < hidden; j += blockDim.x) ss += x[j] * x[j];
-    __shared__ float s_part[32];
+    for (int j = threadIdx.x; j < n4; j += blockDim.x) {
+        float4 v = x4[j];
+        if (k_splits > 0) {
+            for (int s = 0; s < k_splits; ++s) {
+                const float4 w = __ldcg(reinterpret_cast<const float4 *>(Ws + ((size_t)s * ws_rows + i) * hidden) + j);
+                v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
+            }
+            x4[j] = v;
+        }
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+    __shared__ float s_part[8];
     ss = warp_sum(ss);
     if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
     __syncthreads();
     float tot = 0.f;
     for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += s_part[w];
     const float inv = rsqrtf(tot / (float)hidden + eps);
-    for (int j = threadIdx.x; j < hidden; j += blockDim.x)
-        split_bf16(x[j] * inv * gain[j], XN_hi[(size_t)i * hidden + j], XN_lo[(size_t)i * hidden + j]);
+    uint2 *hi = reinterpret_cast<uint2 *>(XN_hi + (size_t)i * hidden), *lo = reinterpret_cast<uint2 *>(XN_lo + (size_t)i * hidden);
+    for (int j = threadIdx.x; j < n4; j += blockDim.x) {
+        const float4 v = x4[j];   // this thread's own values (just written or read above)
+        const float4 g = reinterpret_cast<const float4 *>(gain)[j];
+        uint16_t h0, h1, h2, h3, l0, l1, l2, l3;
+        split_bf16(v.x * inv * g.x, h0, l0);
+        split_bf16(v.y * inv * g.y, h1, l1);
+        split_bf16(v.z * inv * g.z, h2, l2);
+        split_bf16(v.w * inv * g.w, h3, l3);
+        hi[j] = make_uint2((uint32_t)h0 | ((uint32_t)h1 << 16), (uint32_t)h2 | ((uint32_t)h3 << 16));
+        lo[j] = make_uint2((uint32_t)l0 | ((uint32_t)l1 << 16), (uint32_t)l2 | ((uint32_t)l3 << 16));
+    }
 }
 
 enum { GEPI_STORE = 0, GEPI_RESADD = 1, GEPI_SILU = 2 };

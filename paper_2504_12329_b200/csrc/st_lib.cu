@@ -75,7 +75,7 @@ struct st_model {
     float *gf = nullptr;
     std::vector<LayerWeights> layers;
     std::vector<LayerMaps> maps;
-    std::map<int, CUtensorMap> act_maps;   // key: (buffer * 2 + plane) * 1024 + m_pad
+    CUtensorMap *act_maps = nullptr;       // device [3 buffers][2 planes][8]: activation planes in boxes of 32 (j + 1) rows
     bool simt_gemm = false;                // debugging aid: multi-row projections on the CUDA cores
     bool simt_attn = false;                // debugging aid: multi-row attention on the CUDA cores
     double *inv_freq = nullptr;
@@ -350,8 +350,9 @@ static int make_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint
 }
 
 template <int EPI>
-static int launch_tc_gemm(const CUtensorMap &tw, const CUtensorMap &ta_hi, const CUtensorMap &ta_lo, TcGemmParams p, int m_upper,
-                          int sms, cudaStream_t s)
+// pending_splits: when given, a K-split projection leaves its partial sums in the workspace and reports the split
+// count there (0: the output is complete) -- the kernel that consumes the output adds them up.
+static int launch_tc_gemm(const CUtensorMap &tw, TcGemmParams p, int m_upper, int sms, cudaStream_t s, int *pending_splits = nullptr)
 {
     auto kern = tc_gemm_kernel<EPI>;
     p.m_pad = (m_upper + 31) / 32 * 32;
@@ -395,9 +396,13 @@ static int launch_tc_gemm(const CUtensorMap &tw, const CUtensorMap &ta_hi, const
     if ((p.N & 3) || !p.Ws) ks = 1;
     p.k_splits = ks;
     const size_t smem = (size_t)p.stages * stage_bytes + 1024;
-    kern<<<dim3(n_tiles, ks), 192, smem, s>>>(tw, ta_hi, ta_lo, p);
+    kern<<<dim3(n_tiles, ks), 192, smem, s>>>(tw, p);
     ++g_launches;
     CK(cudaGetLastError());
+    if (pending_splits) {
+        *pending_splits = ks > 1 ? ks : 0;
+        return ST_OK;
+    }
     if (ks > 1) {
         int gx = (p.N / 4 + 255) / 256;
         splitk_reduce_kernel<<<dim3(gx, m_upper), 256, 0, s>>>(p.desc, p.Ws, ks, p.ws_rows, p.N, p.bias, p.Yf, EPI == TEPI_RESADD ? 1 : 0);
@@ -586,6 +591,19 @@ static int model_build(st_model *m)
     ALLOC(m->ACT, float, f);
     ALLOC(m->ACTb, uint16_t, 2 * (size_t)m->max_rows * f);
     ALLOC(m->splitk_ws, float, (size_t)kMaxKSplits * m->max_rows * (qkvd > h ? qkvd : h));
+    {   // TMA descriptors of the GEMM inputs: per buffer and plane, boxes of 32, 64, ... 256 rows
+        std::vector<CUtensorMap> maps(3 * 2 * 8);
+        const uint16_t *bufs[3] = {m->XN, m->ATTb, m->ACTb};
+        const int widths[3] = {h, qd, f};
+        for (int b = 0; b < 3; ++b)
+            for (int plane = 0; plane < 2; ++plane)
+                for (int j = 0; j < 8; ++j)
+                    TRY(make_map_bf16(&maps[(b * 2 + plane) * 8 + j], bufs[b] + (size_t)plane * m->max_rows * widths[b],
+                                      (uint64_t)m->max_rows, (uint64_t)widths[b], (uint32_t)(32 * (j + 1))));
+        ALLOC(m->act_maps, CUtensorMap, maps.size());
+        CK(cudaMemcpyAsync(m->act_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, m->stream));
+        CK(cudaStreamSynchronize(m->stream));
+    }
     ALLOC(m->cs, float2, (size_t)m->max_rows * (D / 2));
     ALLOC(m->logits, float, c.vocab);
     {   // split-KV partials: one decode row with up to max_splits splits, or max_rows rows with up to kRowSplits
@@ -851,7 +869,7 @@ static int pass_decode_multi(st_model *m, const StepDesc *desc, const int32_t *t
         g.N = qd + 2 * kd; g.K = h; g.x_row = 0; g.eps = c.rms_eps;
         CK((launch_gemv<PRO_NORM, EPI_STORE>(g, s, m->sm_count)));
         const KvView kv = kv_view(m, l, slot);
-        rope_append_kernel<<<1, 256, 0, s>>>(desc, m->QKV, m->cs, c.n_q_heads, c.n_kv_heads, D, kv, m->status);
+        rope_append_kernel<<<1, 256, 0, s>>>(desc, m->QKV, nullptr, 0, 0, nullptr, m->cs, c.n_q_heads, c.n_kv_heads, D, kv, m->status);
         ++g_launches;
         CK(cudaGetLastError());
         AttnParams a{};
@@ -872,26 +890,13 @@ static int pass_decode_multi(st_model *m, const StepDesc *desc, const int32_t *t
     return sample_tail(m, desc, sc);
 }
 
-// TMA descriptor of one activation plane ([max_rows][K] bf16) with a box of m_pad rows; cached per model.
-static int act_map(st_model *m, int buffer, int plane, const uint16_t *base, int K, int m_pad, const CUtensorMap **out)
-{
-    const int key = (buffer * 2 + plane) * 1024 + m_pad;
-    auto it = m->act_maps.find(key);
-    if (it == m->act_maps.end()) {
-        CUtensorMap map;
-        TRY(make_map_bf16(&map, base, (uint64_t)m->max_rows, (uint64_t)K, (uint32_t)m_pad));
-        it = m->act_maps.emplace(key, map).first;
-    }
-    *out = &it->second;
-    return ST_OK;
-}
-
 // One multi-row projection: tensor cores (default) or the CUDA-core tiled GEMM (debugging aid).
 template <int EPI>
 static int rows_gemm(st_model *m, const StepDesc *desc, int m_upper, int buffer, const uint16_t *A_hi, const uint16_t *A_lo,
                      const CUtensorMap &tw, const uint16_t *W, const float *bias, float *Yf, uint16_t *Yb_hi, uint16_t *Yb_lo,
-                     int N, int K)
+                     int N, int K, int *pending_splits = nullptr)
 {
+    if (pending_splits) *pending_splits = 0;
     if (m->simt_gemm) {
         GemmParams g{};
         g.desc = desc; g.A_hi = A_hi; g.A_lo = A_lo; g.W = W; g.bias = bias; g.Yf = Yf; g.Yb_hi = Yb_hi; g.Yb_lo = Yb_lo;
@@ -899,14 +904,14 @@ static int rows_gemm(st_model *m, const StepDesc *desc, int m_upper, int buffer,
         CK(launch_gemm<EPI>(g, m_upper, m->stream));
         return ST_OK;
     }
-    const int m_pad = (m_upper + 31) / 32 * 32;
-    const CUtensorMap *ta_hi, *ta_lo;
-    TRY(act_map(m, buffer, 0, A_hi, K, m_pad, &ta_hi));
-    TRY(act_map(m, buffer, 1, A_lo, K, m_pad, &ta_lo));
+    (void)A_hi;
+    (void)A_lo;
     TcGemmParams p{};
+    p.act_hi = m->act_maps + (buffer * 2 + 0) * 8;
+    p.act_lo = m->act_maps + (buffer * 2 + 1) * 8;
     p.desc = desc; p.bias = bias; p.Yf = Yf; p.Yb_hi = Yb_hi; p.Yb_lo = Yb_lo; p.status = m->status; p.N = N; p.K = K;
     p.Ws = m->splitk_ws; p.ws_rows = m->max_rows;
-    return launch_tc_gemm<EPI>(tw, *ta_hi, *ta_lo, p, m_upper, m->sm_count, m->stream);
+    return launch_tc_gemm<EPI>(tw, p, m_upper, m->sm_count, m->stream, pending_splits);
 }
 
 // Multi-row pass: up to m_upper rows (the exact count is desc->m on the device).
@@ -930,15 +935,19 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
     embed_rope_kernel<<<m_upper, 256, 0, s>>>(desc, tok, m->embed, h, c.vocab, m->X, m->inv_freq, D / 2, m->cs, m->status);
     ++g_launches;
     CK(cudaGetLastError());
+    int pend_down = 0;   // K splits of the previous layer's down projection still to be added to X
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerWeights &w = m->layers[l];
         const LayerMaps &tm = m->maps[l];
-        rmsnorm_rows_kernel<<<m_upper, 256, 0, s>>>(desc, m->X, w.g1, c.rms_eps, h, m->XN, XN_lo);
+        // the previous layer's down projection may have left its K-split partial sums for this kernel to add
+        rmsnorm_rows_kernel<<<m_upper, 256, 0, s>>>(desc, m->X, m->splitk_ws, pend_down, m->max_rows, w.g1, c.rms_eps, h, m->XN, XN_lo);
         ++g_launches;
         CK(cudaGetLastError());
-        TRY((rows_gemm<TEPI_STORE>(m, desc, m_upper, 0, m->XN, XN_lo, tm.wqkv, w.wqkv, w.bqkv, m->QKV, nullptr, nullptr, qd + 2 * kd, h)));
+        int pend = 0;
+        TRY((rows_gemm<TEPI_STORE>(m, desc, m_upper, 0, m->XN, XN_lo, tm.wqkv, w.wqkv, w.bqkv, m->QKV, nullptr, nullptr, qd + 2 * kd, h, &pend)));
         const KvView kv = kv_view(m, l, slot);
-        rope_append_kernel<<<m_upper, 256, 0, s>>>(desc, m->QKV, m->cs, c.n_q_heads, c.n_kv_heads, D, kv, m->status);
+        rope_append_kernel<<<m_upper, 256, 0, s>>>(desc, m->QKV, m->splitk_ws, pend, m->max_rows, w.bqkv, m->cs, c.n_q_heads, c.n_kv_heads, D, kv,
+                                                   m->status);
         ++g_launches;
         CK(cudaGetLastError());
         AttnParams a{};
@@ -955,12 +964,14 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
             am.row_base = (int32_t)((size_t)l * m->n_pages * c.n_kv_heads * c.page_size);
             CK(launch_attn_rows_mma(am, D, G, dim3(row_splits, c.n_kv_heads, row_tiles), s));
         }
-        TRY((rows_gemm<TEPI_RESADD>(m, desc, m_upper, 1, m->ATTb, ATT_lo, tm.wo, w.wo, nullptr, m->X, nullptr, nullptr, h, qd)));
-        rmsnorm_rows_kernel<<<m_upper, 256, 0, s>>>(desc, m->X, w.g2, c.rms_eps, h, m->XN, XN_lo);
+        TRY((rows_gemm<TEPI_RESADD>(m, desc, m_upper, 1, m->ATTb, ATT_lo, tm.wo, w.wo, nullptr, m->X, nullptr, nullptr, h, qd, &pend)));
+        rmsnorm_rows_kernel<<<m_upper, 256, 0, s>>>(desc, m->X, m->splitk_ws, pend, m->max_rows, w.g2, c.rms_eps, h, m->XN, XN_lo);
         ++g_launches;
         CK(cudaGetLastError());
         TRY((rows_gemm<TEPI_SILU>(m, desc, m_upper, 0, m->XN, XN_lo, tm.wgu, w.wgu, nullptr, nullptr, m->ACTb, ACT_lo, 2 * f, h)));
-        TRY((rows_gemm<TEPI_RESADD>(m, desc, m_upper, 2, m->ACTb, ACT_lo, tm.wd, w.wd, nullptr, m->X, nullptr, nullptr, h, f)));
+        // the last layer's down projection reduces its own splits: the final norm belongs to the LM head
+        TRY((rows_gemm<TEPI_RESADD>(m, desc, m_upper, 2, m->ACTb, ACT_lo, tm.wd, w.wd, nullptr, m->X, nullptr, nullptr, h, f,
+                                    l + 1 < c.n_layers ? &pend_down : nullptr)));
     }
     if (emit) return sample_tail(m, desc, sc);
     return ST_OK;

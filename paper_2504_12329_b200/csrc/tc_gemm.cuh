@@ -31,7 +31,9 @@ struct TcGemmParams {
     uint16_t *Yb_hi, *Yb_lo;  // TEPI_SILU: [rows][N / 2] hi/lo planes of silu(row 2j) * row 2j+1
     int32_t *status;
     int32_t N, K;
-    int32_t m_pad;            // MMA N: activation rows padded to a multiple of 32, <= 256
+    const CUtensorMap *act_hi, *act_lo;   // global memory, [8] each: the hi / lo activation plane in boxes of 32 (j + 1) rows
+    int32_t m_pad;            // upper bound of the MMA N of this launch (multiple of 32, <= 256): shared-memory and TMEM
+                              // layout follow it; the rows actually loaded and multiplied are desc->m rounded up to 32
     int32_t stages;           // shared-memory pipeline depth
     int32_t k_splits;
     int32_t tmem_cols;        // power of two >= max(32, w_tiles * m_pad)
@@ -153,9 +155,7 @@ __global__ void splitk_reduce_kernel(const StepDesc *desc, const float *Ws, int 
 }
 
 template <int EPI>
-__global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW,
-                                                      const __grid_constant__ CUtensorMap tmAhi,
-                                                      const __grid_constant__ CUtensorMap tmAlo, const TcGemmParams p)
+__global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW,                                                       const TcGemmParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t s_full[8], s_empty[8], s_acc;
@@ -174,6 +174,10 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
     if (n_kb <= 0) return;   // uniform for the CTA
 
     const uint32_t a_bytes = (uint32_t)p.m_pad * kTcBlockK * 2;
+    // the pass may hold fewer rows than the launch was sized for: load and multiply only those (rounded up to 32)
+    const int m_eff = min(p.m_pad, (m + 31) & ~31);
+    const uint32_t a_bytes_eff = (uint32_t)m_eff * kTcBlockK * 2;
+    const CUtensorMap *tmAhi = p.act_hi + (m_eff / 32 - 1), *tmAlo = p.act_lo + (m_eff / 32 - 1);
     const uint32_t w_bytes = (uint32_t)p.w_tiles * kTcWBytes;
     const uint32_t stage_bytes = w_bytes + 2 * a_bytes;
     const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 1024-byte aligned tile area
@@ -205,11 +209,11 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
                 if (u > 0 && !mbar_wait(smem_u32(&s_empty[s]), (u - 1) & 1, &s_abort, p.status)) break;
                 const uint32_t full = smem_u32(&s_full[s]);
                 const uint32_t base = tiles + (uint32_t)s * stage_bytes;
-                mbar_expect_tx(full, stage_bytes);
+                mbar_expect_tx(full, w_bytes + 2 * a_bytes_eff);
                 const int kx = (kb0 + i) * kTcBlockK;
                 for (int t = 0; t < p.w_tiles; ++t) tma_load_2d(base + (uint32_t)t * kTcWBytes, &tmW, kx, n0 + t * kTcTileW, full);
-                tma_load_2d(base + w_bytes, &tmAhi, kx, 0, full);
-                tma_load_2d(base + w_bytes + a_bytes, &tmAlo, kx, 0, full);
+                tma_load_2d(base + w_bytes, tmAhi, kx, 0, full);
+                tma_load_2d(base + w_bytes + a_bytes, tmAlo, kx, 0, full);
                 armed = i + 1;
             }
             if (s_abort) {
@@ -223,7 +227,7 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_bf16(p.m_pad);
+            const uint32_t idesc = umma_idesc_bf16(m_eff);
             bool ok = true;
             for (int i = 0; i < n_kb && ok; ++i) {
                 const int s = i % p.stages, u = i / p.stages;
