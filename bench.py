@@ -33,6 +33,56 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def measured_tensor_peak():
+    """Dense bf16 TFLOP/s of a long-running GEMM (the multi-row passes run for tens of milliseconds)."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "measured (sustained)"
+    return 1400.0, "fallback (sustained)"
+
+
+def time_multi_row_passes(torch, model, shape, ctx, row_counts, hbm_peak):
+    """Catch-up / prefill passes of one model on their own: `rows` new tokens over `ctx` cached ones, timed with
+    CUDA events on the launching stream.  Every pass streams the model's weights once (larger than L2)."""
+    tensor_peak, tensor_kind = measured_tensor_peak()
+    lm_head_bytes = 2 * shape.vocab * shape.hidden
+    layer_params = (model.st_weight_bytes() - lm_head_bytes) / 2
+    out = []
+    for rows in row_counts:
+        best = None
+        for rep in range(3):
+            slot = model.st_seq_alloc()
+            i = 0
+            while i < ctx:
+                c = min(256, ctx - i)
+                model.st_prefill(slot, W.prompt_ids(7 + i, c, shape.vocab))
+                i += c
+            toks = W.prompt_ids(99, rows, shape.vocab)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            model.st_prefill(slot, toks)
+            e1.record()
+            torch.cuda.synchronize()
+            t = e0.elapsed_time(e1) * 1e-3
+            model.st_seq_free(slot)
+            if rep > 0:
+                best = t if best is None else min(best, t)
+        flops = 2.0 * rows * layer_params + 2.0 * lm_head_bytes / 2 \
+            + 4.0 * rows * (ctx + rows / 2) * shape.n_q_heads * shape.head_dim * shape.n_layers
+        gbs = (model.st_weight_bytes() + model.st_kv_bytes_per_token() * (ctx + rows)) / best / 1e9
+        useful = flops / best / 1e12
+        hbm_time = (model.st_weight_bytes() / 1e9) / hbm_peak
+        tensor_time = 2.0 * flops / 1e12 / tensor_peak      # hi and lo activation planes: two MMAs per product
+        out.append({"model": shape.name, "rows": rows, "context": ctx, "ms": best * 1e3, "tokens_per_s": rows / best,
+                    "hbm_gbs": gbs, "frac_hbm": gbs / hbm_peak, "tflops_useful": useful, "tflops_issued": 2 * useful,
+                    "frac_tensor_useful": useful / tensor_peak, "frac_tensor_issued": 2 * useful / tensor_peak,
+                    "bound": "hbm" if hbm_time >= tensor_time else "tensor", "tensor_peak": tensor_peak,
+                    "tensor_peak_source": tensor_kind})
+    return out
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -277,6 +327,26 @@ def main():
     kern_bytes = dom.st_weight_bytes() + dom.st_kv_bytes_per_token() * (ctx + 3 + n_k // 2)
     achieved = kern_bytes / kern_s / 1e9
     dom.st_seq_free(slot)
+    # multi-row passes (handoff catch-up and prompt prefill) of the same model, and the small model's decode step
+    mean_catchup = int(np.mean([h[2] for h in r.handoffs])) if len(r.handoffs) else 128
+    prefill = time_multi_row_passes(torch, dom, shp, max(0, min(1024, cap - 64 - 256)), [min(256, max(2, mean_catchup)), 256], peak)
+    small_step = None
+    if large is not None:
+        sslot = small.st_seq_alloc()
+        small.st_prefill(sslot, W.prompt_ids(7, ctx, wl.small.vocab))
+        for _ in range(3):
+            small.st_decode_step([sslot], tok_dev, None, amax_dev)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(n_k):
+            small.st_decode_step([sslot], tok_dev, None, amax_dev)
+        e1.record()
+        torch.cuda.synchronize()
+        s_s = e0.elapsed_time(e1) * 1e-3 / n_k
+        s_bytes = small.st_weight_bytes() + small.st_kv_bytes_per_token() * (ctx + 3 + n_k // 2)
+        small_step = {"kernel": f"decode_mega_kernel ({wl.small.name}, context {ctx})", "us_per_launch": s_s * 1e6,
+                      "achieved": s_bytes / s_s / 1e9, "frac": s_bytes / s_s / 1e9 / peak, "unit": "GB/s"}
+        small.st_seq_free(sslot)
     path_gbs = sum(x.bytes_algorithmic for x in results) / sum(x.seconds for x in results) / 1e9
     steps_small = int((r.emission_source == 0).sum())
     steps_large = int((r.emission_source == 1).sum())
@@ -309,6 +379,8 @@ def main():
             "path_roofline": {"achieved_gbs": path_gbs, "frac_of_measured_hbm": path_gbs / peak,
                               "frac_of_nominal_8tbs": path_gbs / 8000.0,
                               "note": "algorithmic bytes of every pass (weights + KV) / device time of the generation"},
+            "prefill": prefill,
+            "small_model_decode": small_step,
             "wall_s_timed_region": t_region,
         }
         if not args.no_cpu_baseline:

@@ -91,6 +91,14 @@ def test_full_width_two_layers(B, oracle, shape):
     _teacher_forced(B, oracle, shape_dict(shape, n_layers=2), 0, 3, chunks=[19], n_decode=3)
 
 
+@pytest.mark.parametrize("shape", [W.QWEN_1P5B, W.QWEN_32B])
+def test_full_width_two_layers_longer_context(B, oracle, shape):
+    """head_dim 128 with a context that needs several key splits and K/V pages in the decode kernel (the splits'
+    first keys are not multiples of the staging box), a catch-up sized chunk over that context (multi-row
+    attention with key splits) and a 256-row prompt chunk; vocabulary cut to keep the oracle fast."""
+    _teacher_forced(B, oracle, shape_dict(shape, n_layers=2, vocab=4096), 0, 3, chunks=[256, 256, 45, 20, 130], n_decode=6)
+
+
 def test_qwen1p5b_full_depth(B, oracle):
     """All 28 layers of the 1.5B shape: prompt prefill, a catch-up sized chunk and decode steps."""
     _teacher_forced(B, oracle, shape_dict(W.QWEN_1P5B), 0, 0, chunks=[24, 20], n_decode=4)
