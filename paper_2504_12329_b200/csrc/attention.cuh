@@ -32,8 +32,10 @@ __device__ __forceinline__ size_t kv_offset(const KvView &kv, int pos, int head,
 
 // x[i] = E[token_i] (fp32) and the rotary table of row i: cs[i][j] = (cos, sin)(pos_i * inv_freq[j]),
 // evaluated in double so that long positions lose nothing.
+// row_pos (nullable): the rows belong to different sequences (batched decode), row i sits at position row_pos[i].
 __global__ void embed_rope_kernel(const StepDesc *desc, const int32_t *tok, const uint16_t *E, int hidden, int vocab,
-                                  float *X, const double *inv_freq, int half, float2 *cs, int32_t *status)
+                                  float *X, const double *inv_freq, int half, float2 *cs, int32_t *status,
+                                  const int32_t *row_pos = nullptr)
 {
     const int i = blockIdx.x;
     if (i >= desc->m) return;
@@ -48,7 +50,7 @@ __global__ void embed_rope_kernel(const StepDesc *desc, const int32_t *tok, cons
         const uint32_t v = e[j];
         x2[j] = make_float2(bf16_lo(v), bf16_hi(v));
     }
-    const double pos = (double)(desc->pos0 + i);
+    const double pos = (double)(row_pos ? row_pos[i] : desc->pos0 + i);
     for (int j = threadIdx.x; j < half; j += blockDim.x) {
         double s, c;
         sincos(pos * inv_freq[j], &s, &c);
@@ -57,15 +59,18 @@ __global__ void embed_rope_kernel(const StepDesc *desc, const int32_t *tok, cons
 }
 
 // Rotate q in place (fp32), rotate k and store k, v into the cache (fp16).
+// With row_slot / row_pos the rows belong to different sequences (batched decode).
 // qkv: [rows][(Hq + 2 Hkv) * D] = q heads, then k heads, then v heads.  With k_splits > 0 the row is not in
 // qkv yet: it is bias + the K-split partial sums Ws[s][row] of the QKV projection (summed in split order).
 __global__ void __launch_bounds__(256) rope_append_kernel(const StepDesc *desc, float *qkv, const float *Ws, int k_splits, int ws_rows,
                                                           const float *bias, const float2 *cs, int Hq, int Hkv, int D, KvView kv,
-                                                          int32_t *status)
+                                                          int32_t *status, const int32_t *row_slot = nullptr,
+                                                          const int32_t *row_pos = nullptr, int pages_per_seq = 0)
 {
     const int i = blockIdx.x;
     if (i >= desc->m) return;
-    const int half = D >> 1, pos = desc->pos0 + i, N = (Hq + 2 * Hkv) * D;
+    if (row_slot) kv.block_tab += (size_t)row_slot[i] * pages_per_seq;   // batched decode: kv.block_tab is sequence 0's table
+    const int half = D >> 1, pos = row_pos ? row_pos[i] : desc->pos0 + i, N = (Hq + 2 * Hkv) * D;
     float *row = qkv + (size_t)i * N;
     const float2 *c = cs + (size_t)i * half;
     auto val4 = [&](int n) {   // 4 consecutive features of the row, n a multiple of 4

@@ -265,4 +265,201 @@ __global__ void __launch_bounds__(kArThreads, 1) attn_rows_mma_kernel(const Attn
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Batched decode attention: every row is the newest token of a different sequence.  One CTA per (kv head, row)
+// walks that sequence's keys 0 .. pos in tiles of 128 keys (TMA, three tiles in flight); warp w takes the w-th
+// group of 16 keys of every tile for the G query heads of the group, and the warps are merged through shared
+// memory at the end.  The row's own key/value is already in the cache (the rope kernel appended it).
+// ---------------------------------------------------------------------------------------------
+constexpr int kAbTileKeys = 128;
+constexpr int kAbStages = 3;
+
+struct AttnBatchParams {
+    AttnParams a;                     // a.kv.block_tab: the block table of sequence 0
+    const CUtensorMap *kmap, *vmap;
+    int32_t row_base;                 // first pool row of this layer
+    const int32_t *row_slot, *row_pos;
+    int32_t pages_per_seq;
+};
+
+template <int D>
+__host__ __device__ constexpr int ab_stage_bytes() { return 2 * kAbTileKeys * D * 2; }
+
+template <int D, int G>
+__global__ void __launch_bounds__(kArThreads, 1) attn_batch_mma_kernel(const AttnBatchParams pp)
+{
+    static_assert(G >= 1 && G <= 8, "one MMA column per head of the group");
+    constexpr int KS = D / 16, NH = D / 64, HALF_BYTES = kAbTileKeys * 128, STAGE = ab_stage_bytes<D>();
+    extern __shared__ uint8_t ab_smem[];
+    __shared__ uint64_t s_full[kAbStages];
+    __shared__ int s_abort;
+    const AttnParams &p = pp.a;
+    const int row = blockIdx.y;
+    if (row >= p.desc->m) return;   // uniform for the CTA
+    const int hk = blockIdx.x, Hkv = p.kv.n_kv_heads;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int gq = lane >> 2, t = lane & 3;
+    const uint32_t base = (smem_u32(ab_smem) + 1023u) & ~1023u;
+    uint8_t *base_ptr = ab_smem + (base - smem_u32(ab_smem));
+    if (tid == 0) {
+        s_abort = 0;
+        for (int s = 0; s < kAbStages; ++s) mbar_init(smem_u32(&s_full[s]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const int pos = pp.row_pos[row];
+    const int n_keys = pos + 1;
+    const int32_t *tab = p.kv.block_tab + (size_t)pp.row_slot[row] * pp.pages_per_seq;
+    const int ntiles = (n_keys + kAbTileKeys - 1) / kAbTileKeys;
+
+    auto issue = [&](int i) {
+        const int s = i % kAbStages;
+        const int key0 = i * kAbTileKeys;
+        const int ng = (min(kAbTileKeys, n_keys - key0) + 15) >> 4;
+        const int boxes = ng * NH * 2;
+        const uint32_t bar = smem_u32(&s_full[s]);
+        if (lane == 0) mbar_expect_tx(bar, (uint32_t)boxes * kMegaKvBoxBytes);
+        __syncwarp();
+        if (lane < boxes) {
+            const int g = lane / (2 * NH), rem = lane - g * (2 * NH);
+            const int isv = rem / NH, half = rem - isv * NH;
+            const int key = key0 + g * 16;
+            int page = tab[key >> p.kv.page_shift];
+            if ((unsigned)page >= (unsigned)p.kv.n_pages) {
+                atomicOr(p.status, DEV_BAD_PAGE);
+                page = 0;
+            }
+            const int y = pp.row_base + (page * Hkv + hk) * p.kv.page_size + (key & (p.kv.page_size - 1));
+            const uint32_t dst = base + (uint32_t)s * STAGE + (uint32_t)(isv * NH + half) * HALF_BYTES + (uint32_t)g * kMegaKvBoxBytes;
+            tma_load_2d(dst, isv ? pp.vmap : pp.kmap, half * 64, y, bar);
+        }
+    };
+    if (warp == 0)
+        for (int i = 0; i < min(ntiles, kAbStages); ++i) issue(i);
+
+    uint32_t qhi[KS][2], qlo[KS][2];
+    {
+        const bool live = gq < G;
+        const float *qsrc = p.qkv + (size_t)row * (p.Hq + 2 * Hkv) * D + (size_t)(hk * G + (live ? gq : 0)) * D + 2 * t;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                float2 v = make_float2(0.f, 0.f);
+                if (live) v = *reinterpret_cast<const float2 *>(qsrc + 16 * ks + 8 * hf);
+                const float x = v.x * p.scale, y = v.y * p.scale;
+                const uint32_t h = pack_half2(x, y);
+                qhi[ks][hf] = h;
+                qlo[ks][hf] = pack_half2(x - kv_lo(h), y - kv_hi(h));
+            }
+    }
+    float mrun[2] = {-INFINITY, -INFINITY}, lrun[2] = {0.f, 0.f};
+    float oacc[KS][4];
+#pragma unroll
+    for (int mt = 0; mt < KS; ++mt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) oacc[mt][e] = 0.f;
+
+    for (int i = 0; i < ntiles; ++i) {
+        const int s = i % kAbStages;
+        const int key0 = i * kAbTileKeys;
+        const int nk = min(kAbTileKeys, n_keys - key0);
+        mbar_wait(smem_u32(&s_full[s]), (uint32_t)(i / kAbStages) & 1u, &s_abort, p.status);
+        const uint32_t kst = base + (uint32_t)s * STAGE, vst = kst + (uint32_t)NH * HALF_BYTES;
+        if (nk < kAbTileKeys) {   // last tile: value rows behind the last key of its group must be finite
+            uint8_t *vptr = base_ptr + (size_t)s * STAGE + (size_t)NH * HALF_BYTES;
+            const int pad = ((nk + 15) & ~15) - nk;
+            for (int idx = tid; idx < pad * (D / 8); idx += kArThreads) {
+                const int r = nk + idx / (D / 8), c = idx % (D / 8);
+                *reinterpret_cast<uint4 *>(vptr + (size_t)(c >> 3) * HALF_BYTES + (size_t)r * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
+            }
+            __syncthreads();
+        }
+        const int r0 = warp * 16;
+        if (r0 < nk) {
+            float sacc[4] = {0.f, 0.f, 0.f, 0.f};
+            const int krow = r0 + (lane & 7) + ((lane >> 3) & 1) * 8;
+            const uint32_t ka = kst + (uint32_t)krow * 128;
+            const uint32_t kx = (uint32_t)(krow & 7);
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                uint32_t a[4];
+                ldmatrix_x4(a, ka + (uint32_t)(ks >> 2) * HALF_BYTES + ((((uint32_t)(ks & 3) * 2 + (uint32_t)(lane >> 4)) ^ kx) << 4));
+                mma_f16_16816(sacc, a, qhi[ks][0], qhi[ks][1]);
+                mma_f16_16816(sacc, a, qlo[ks][0], qlo[ks][1]);
+            }
+            const bool v0 = r0 + gq < nk, v1 = r0 + gq + 8 < nk;
+            const float s0 = v0 ? sacc[0] : -INFINITY, s1 = v0 ? sacc[1] : -INFINITY;
+            const float s2 = v1 ? sacc[2] : -INFINITY, s3 = v1 ? sacc[3] : -INFINITY;
+            float m0 = fmaxf(s0, s2), m1 = fmaxf(s1, s3);
+#pragma unroll
+            for (int o = 4; o < 32; o <<= 1) {
+                m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, o));
+                m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, o));
+            }
+            const float n0 = fmaxf(mrun[0], m0), n1 = fmaxf(mrun[1], m1);   // finite: the group holds a live key
+            const float corr0 = mrun[0] == -INFINITY ? 0.f : __expf(mrun[0] - n0);
+            const float corr1 = mrun[1] == -INFINITY ? 0.f : __expf(mrun[1] - n1);
+            const float p0 = v0 ? __expf(s0 - n0) : 0.f, p1 = v0 ? __expf(s1 - n1) : 0.f;
+            const float p2 = v1 ? __expf(s2 - n0) : 0.f, p3 = v1 ? __expf(s3 - n1) : 0.f;
+            mrun[0] = n0;
+            mrun[1] = n1;
+            lrun[0] = lrun[0] * corr0 + p0 + p2;
+            lrun[1] = lrun[1] * corr1 + p1 + p3;
+            const uint32_t pb0 = movmatrix_trans(pack_half2(p0, p1)), pb1 = movmatrix_trans(pack_half2(p2, p3));
+            const int vrow = r0 + (lane & 7) + (lane >> 4) * 8;
+            const uint32_t va = vst + (uint32_t)vrow * 128;
+            const uint32_t vx = (uint32_t)(vrow & 7);
+#pragma unroll
+            for (int mt = 0; mt < KS; ++mt) {
+                oacc[mt][0] *= corr0; oacc[mt][1] *= corr1; oacc[mt][2] *= corr0; oacc[mt][3] *= corr1;
+                uint32_t a[4];
+                ldmatrix_x4_trans(a, va + (uint32_t)(mt >> 2) * HALF_BYTES + ((((uint32_t)(mt & 3) * 2 + (uint32_t)((lane >> 3) & 1)) ^ vx) << 4));
+                mma_f16_16816(oacc[mt], a, pb0, pb1);
+            }
+        }
+        __syncthreads();   // every warp is done with the stage
+        if (warp == 0 && i + kAbStages < ntiles) issue(i + kAbStages);
+    }
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) {
+        lrun[0] += __shfl_xor_sync(0xffffffffu, lrun[0], o);
+        lrun[1] += __shfl_xor_sync(0xffffffffu, lrun[1], o);
+    }
+    // ---- merge the warps through shared memory (the tiles are no longer needed) ----
+    float *so = reinterpret_cast<float *>(base_ptr);                 // [8 warps][G][D]
+    float *sm = so + 8 * G * D, *sd = sm + 8 * G;                    // [8][G] each
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+        const int head = 2 * t + e;
+        if (head < G) {
+#pragma unroll
+            for (int mt = 0; mt < KS; ++mt) {
+                so[(warp * G + head) * D + 16 * mt + gq] = oacc[mt][e];
+                so[(warp * G + head) * D + 16 * mt + gq + 8] = oacc[mt][2 + e];
+            }
+            if (gq == 0) { sm[warp * G + head] = mrun[e]; sd[warp * G + head] = lrun[e]; }
+        }
+    }
+    __syncthreads();
+    const int hq0 = hk * G;
+    for (int idx = tid; idx < G * D; idx += kArThreads) {
+        const int g = idx / D, c = idx - g * D;
+        float mnew = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) mnew = fmaxf(mnew, sm[w * G + g]);
+        float dsum = 0.f, osum = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+            const float mw = sm[w * G + g];
+            if (mw != -INFINITY) {
+                const float cw = __expf(mw - mnew);
+                dsum += sd[w * G + g] * cw;
+                osum += so[(w * G + g) * D + c] * cw;
+            }
+        }
+        attn_store(p, ((size_t)row * p.Hq + hq0 + g) * D + c, osum / dsum);
+    }
+}
+
 }  // namespace st

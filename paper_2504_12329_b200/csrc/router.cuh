@@ -187,6 +187,31 @@ __device__ __forceinline__ void argmax_merge(float &v, int &i, float v2, int i2)
     if (v2 > v || (v2 == v && i2 < i)) { v = v2; i = i2; }
 }
 
+// Batched decode: lowest-id argmax of every row of logits [rows][vocab] over ids < limit, one CTA per row.
+__global__ void __launch_bounds__(256) argmax_rows_kernel(const StepDesc *desc, const float *logits, int vocab, int limit, int32_t *argmax_out)
+{
+    __shared__ float s_v[8];
+    __shared__ int s_i[8];
+    const int row = blockIdx.x;
+    if (row >= desc->m) return;
+    const float *z = logits + (size_t)row * vocab;
+    float v = -INFINITY;
+    int idx = 0x7fffffff;
+    for (int i = threadIdx.x; i < limit; i += blockDim.x) argmax_merge(v, idx, __ldcg(z + i), i);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float v2 = __shfl_xor_sync(0xffffffffu, v, o);
+        const int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
+        argmax_merge(v, idx, v2, i2);
+    }
+    if ((threadIdx.x & 31) == 0) { s_v[threadIdx.x >> 5] = v; s_i[threadIdx.x >> 5] = idx; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w) argmax_merge(v, idx, s_v[w], s_i[w]);
+        argmax_out[row] = idx == 0x7fffffff ? 0 : idx;
+    }
+}
+
 __global__ void __launch_bounds__(256) argmax_router_kernel(const ArgmaxParams p)
 {
     __shared__ float s_v[8];

@@ -75,6 +75,9 @@ struct st_model {
     float *gf = nullptr;
     std::vector<LayerWeights> layers;
     std::vector<LayerMaps> maps;
+    CUtensorMap map_lm{};                  // LM head in 128-row tiles (batched decode)
+    int32_t *row_slot = nullptr, *row_pos = nullptr;   // device [max_rows]: sequence and position of every row of a batched decode pass
+    float *batch_logits = nullptr;         // [max_rows][vocab], allocated on first use
     CUtensorMap *act_maps = nullptr;       // device [3 buffers][2 planes][8]: activation planes in boxes of 32 (j + 1) rows
     bool simt_gemm = false;                // debugging aid: multi-row projections on the CUDA cores
     bool simt_attn = false;                // debugging aid: multi-row attention on the CUDA cores
@@ -287,6 +290,41 @@ static cudaError_t launch_attn_rows_mma(const AttnRowsMmaParams &p, int D, int G
 {
     if (D == 64) return launch_attn_rows_mma_d<64>(p, G, grid, s, attr_only);
     if (D == 128) return launch_attn_rows_mma_d<128>(p, G, grid, s, attr_only);
+    return cudaErrorInvalidValue;
+}
+
+// Batched decode attention: grid = (kv heads, rows).
+template <int D, int G>
+static cudaError_t launch_attn_batch_dg(const AttnBatchParams &p, dim3 grid, cudaStream_t s, bool attr_only)
+{
+    auto kern = attn_batch_mma_kernel<D, G>;
+    const size_t smem = 1024 + (size_t)kAbStages * ab_stage_bytes<D>();
+    if (attr_only) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    kern<<<grid, kArThreads, smem, s>>>(p);
+    ++g_launches;
+    return cudaGetLastError();
+}
+
+template <int D>
+static cudaError_t launch_attn_batch_d(const AttnBatchParams &p, int G, dim3 grid, cudaStream_t s, bool attr_only)
+{
+    switch (G) {
+    case 1: return launch_attn_batch_dg<D, 1>(p, grid, s, attr_only);
+    case 2: return launch_attn_batch_dg<D, 2>(p, grid, s, attr_only);
+    case 3: return launch_attn_batch_dg<D, 3>(p, grid, s, attr_only);
+    case 4: return launch_attn_batch_dg<D, 4>(p, grid, s, attr_only);
+    case 5: return launch_attn_batch_dg<D, 5>(p, grid, s, attr_only);
+    case 6: return launch_attn_batch_dg<D, 6>(p, grid, s, attr_only);
+    case 7: return launch_attn_batch_dg<D, 7>(p, grid, s, attr_only);
+    case 8: return launch_attn_batch_dg<D, 8>(p, grid, s, attr_only);
+    }
+    return cudaErrorInvalidValue;
+}
+
+static cudaError_t launch_attn_batch(const AttnBatchParams &p, int D, int G, dim3 grid, cudaStream_t s, bool attr_only = false)
+{
+    if (D == 64) return launch_attn_batch_d<64>(p, G, grid, s, attr_only);
+    if (D == 128) return launch_attn_batch_d<128>(p, G, grid, s, attr_only);
     return cudaErrorInvalidValue;
 }
 
@@ -538,6 +576,7 @@ static int model_build(st_model *m)
         TRY(fill_const(m, w.g2, 1.f, h));
     }
     m->maps.resize(c.n_layers);
+    TRY(make_map_bf16(&m->map_lm, m->lm_head, c.vocab, h, kTcTileW));
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerWeights &w = m->layers[l];
         TRY(make_map_bf16(&m->maps[l].wqkv, w.wqkv, qkvd, h, kTcTileW));
@@ -605,6 +644,8 @@ static int model_build(st_model *m)
         CK(cudaStreamSynchronize(m->stream));
     }
     ALLOC(m->cs, float2, (size_t)m->max_rows * (D / 2));
+    ALLOC(m->row_slot, int32_t, m->max_rows);
+    ALLOC(m->row_pos, int32_t, m->max_rows);
     ALLOC(m->logits, float, c.vocab);
     {   // split-KV partials: one decode row with up to max_splits splits, or max_rows rows with up to kRowSplits
         size_t n = (size_t)m->max_splits > (size_t)m->max_rows * kRowSplits ? (size_t)m->max_splits : (size_t)m->max_rows * kRowSplits;
@@ -816,6 +857,7 @@ static int mega_attr_all()
         for (int G = 1; G <= 8; ++G) {
             CK(mega_launch(MegaParams{}, D, G, 0, 0, nullptr, true));
             CK(launch_attn_rows_mma(AttnRowsMmaParams{}, D, G, dim3(1, 1, 1), nullptr, true));
+            CK(launch_attn_batch(AttnBatchParams{}, D, G, dim3(1, 1, 1), nullptr, true));
         }
     return ST_OK;
 }
@@ -915,7 +957,10 @@ static int rows_gemm(st_model *m, const StepDesc *desc, int m_upper, int buffer,
 }
 
 // Multi-row pass: up to m_upper rows (the exact count is desc->m on the device).
-static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int slot, int m_upper, int ctx_upper, bool emit, const SampleCtx &sc)
+// batch: the rows are the newest tokens of different sequences (m->row_slot / m->row_pos, `slot` unused); the pass
+// then ends with the LM head over all rows (logits [rows][vocab] to sc.logits_out) and one argmax per row.
+static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int slot, int m_upper, int ctx_upper, bool emit, const SampleCtx &sc,
+                     bool batch = false)
 {
     const st_config &c = m->cfg;
     const int h = c.hidden, D = c.head_dim, qd = c.n_q_heads * D, kd = c.n_kv_heads * D, f = c.ffn;
@@ -932,7 +977,8 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
     if (row_splits > ctx_upper / 256) row_splits = ctx_upper / 256;
     row_splits = row_splits < 1 ? 1 : row_splits > kRowSplits ? kRowSplits : row_splits;
     static_assert((int)GEPI_STORE == (int)TEPI_STORE && (int)GEPI_RESADD == (int)TEPI_RESADD && (int)GEPI_SILU == (int)TEPI_SILU, "epilogue ids");
-    embed_rope_kernel<<<m_upper, 256, 0, s>>>(desc, tok, m->embed, h, c.vocab, m->X, m->inv_freq, D / 2, m->cs, m->status);
+    embed_rope_kernel<<<m_upper, 256, 0, s>>>(desc, tok, m->embed, h, c.vocab, m->X, m->inv_freq, D / 2, m->cs, m->status,
+                                              batch ? m->row_pos : nullptr);
     ++g_launches;
     CK(cudaGetLastError());
     int pend_down = 0;   // K splits of the previous layer's down projection still to be added to X
@@ -945,16 +991,26 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
         CK(cudaGetLastError());
         int pend = 0;
         TRY((rows_gemm<TEPI_STORE>(m, desc, m_upper, 0, m->XN, XN_lo, tm.wqkv, w.wqkv, w.bqkv, m->QKV, nullptr, nullptr, qd + 2 * kd, h, &pend)));
-        const KvView kv = kv_view(m, l, slot);
+        const KvView kv = kv_view(m, l, batch ? 0 : slot);
         rope_append_kernel<<<m_upper, 256, 0, s>>>(desc, m->QKV, m->splitk_ws, pend, m->max_rows, w.bqkv, m->cs, c.n_q_heads, c.n_kv_heads, D, kv,
-                                                   m->status);
+                                                   m->status, batch ? m->row_slot : nullptr, batch ? m->row_pos : nullptr, m->pages_per_seq);
         ++g_launches;
         CK(cudaGetLastError());
         AttnParams a{};
         a.desc = desc; a.qkv = m->QKV; a.kv = kv; a.out_f32 = nullptr; a.out_hi = m->ATTb; a.out_lo = ATT_lo;
         a.part_o = m->part_o; a.part_ml = m->part_ml; a.tickets = m->tickets; a.status = m->status;
         a.Hq = c.n_q_heads; a.n_splits = row_splits; a.scale = 1.f / sqrtf((float)D);
-        if (m->simt_attn) {
+        if (batch) {
+            AttnBatchParams ab{};
+            ab.a = a;
+            ab.kmap = m->mega_maps + 4 * c.n_layers + 1;
+            ab.vmap = m->mega_maps + 4 * c.n_layers + 2;
+            ab.row_base = (int32_t)((size_t)l * m->n_pages * c.n_kv_heads * c.page_size);
+            ab.row_slot = m->row_slot;
+            ab.row_pos = m->row_pos;
+            ab.pages_per_seq = m->pages_per_seq;
+            CK(launch_attn_batch(ab, D, G, dim3(c.n_kv_heads, m_upper), s));
+        } else if (m->simt_attn) {
             CK(launch_attn_rows(a, D, G, dim3(row_splits, c.n_kv_heads, row_tiles), s));
         } else {
             AttnRowsMmaParams am{};
@@ -972,6 +1028,19 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
         // the last layer's down projection reduces its own splits: the final norm belongs to the LM head
         TRY((rows_gemm<TEPI_RESADD>(m, desc, m_upper, 2, m->ACTb, ACT_lo, tm.wd, w.wd, nullptr, m->X, nullptr, nullptr, h, f,
                                     l + 1 < c.n_layers ? &pend_down : nullptr)));
+    }
+    if (batch) {
+        // final norm of every row, LM head on the tensor cores, one lowest-id argmax per row
+        rmsnorm_rows_kernel<<<m_upper, 256, 0, s>>>(desc, m->X, m->splitk_ws, 0, m->max_rows, m->gf, c.rms_eps, h, m->XN, XN_lo);
+        ++g_launches;
+        CK(cudaGetLastError());
+        TRY((rows_gemm<TEPI_STORE>(m, desc, m_upper, 0, m->XN, XN_lo, m->map_lm, m->lm_head, nullptr, sc.logits_out, nullptr, nullptr, c.vocab, h)));
+        if (sc.want_argmax) {
+            argmax_rows_kernel<<<m_upper, 256, 0, s>>>(desc, sc.logits_out, c.vocab, sc.vlimit > 0 ? sc.vlimit : c.vocab, sc.argmax_out);
+            ++g_launches;
+            CK(cudaGetLastError());
+        }
+        return ST_OK;
     }
     if (emit) return sample_tail(m, desc, sc);
     return ST_OK;
@@ -1199,6 +1268,42 @@ int st_decode_step(st_model *m, const int32_t *slots_host, const int32_t *tokens
         if (slot < 0 || slot >= m->cfg.max_seqs || !m->seq_used[slot]) return ST_ERR_ARG;
         for (int j = 0; j < i; ++j)
             if (slots_host[j] == slot) return ST_ERR_ARG;
+    }
+    if (batch >= 2 && !m->multi_kernel_decode) {
+        // several sequences: one pass over the weights for all of them, projections on the tensor cores
+        float *logits = logits_dev;
+        if (!logits) {
+            if (!m->batch_logits) {
+                m->batch_logits = (float *)m->dalloc((size_t)m->max_rows * m->cfg.vocab * sizeof(float));
+                if (!m->batch_logits) return ST_ERR_OOM;
+            }
+            logits = m->batch_logits;
+        }
+        for (int i0 = 0; i0 < batch; i0 += m->max_rows) {
+            const int n = batch - i0 < m->max_rows ? batch - i0 : m->max_rows;
+            std::vector<int32_t> rows(2 * (size_t)n);
+            int ctx_upper = 1;
+            for (int i = 0; i < n; ++i) {
+                const int slot = slots_host[i0 + i];
+                TRY(seq_reserve(m, slot, m->seq_len[slot] + 1));
+                rows[i] = slot;
+                rows[n + i] = m->seq_len[slot];
+                if (m->seq_len[slot] + 1 > ctx_upper) ctx_upper = m->seq_len[slot] + 1;
+            }
+            CK(cudaMemcpyAsync(m->row_slot, rows.data(), (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, m->stream));
+            CK(cudaMemcpyAsync(m->row_pos, rows.data() + n, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, m->stream));
+            StepDesc d{0, n, i0, 1};
+            CK(cudaMemcpyAsync(m->desc, &d, sizeof d, cudaMemcpyHostToDevice, m->stream));
+            SampleCtx sc{};
+            sc.logits_out = logits + (logits_dev ? (size_t)i0 * m->cfg.vocab : 0);
+            sc.argmax_out = argmax_dev ? argmax_dev + i0 : nullptr;
+            sc.want_argmax = argmax_dev != nullptr;
+            TRY(pass_rows(m, m->desc, tokens_dev, -1, (n + 31) / 32 * 32 > m->max_rows ? m->max_rows : (n + 31) / 32 * 32, ctx_upper, true, sc, true));
+            for (int i = 0; i < n; ++i) m->seq_len[slots_host[i0 + i]] += 1;
+            // the row tables and the descriptor are rewritten for the next chunk
+            CK(cudaStreamSynchronize(m->stream));
+        }
+        return ST_OK;
     }
     CK(cudaMemsetAsync(m->mega_sync, 0, kMegaSyncWords * sizeof(unsigned), m->stream));
     for (int i = 0; i < batch; ++i) {

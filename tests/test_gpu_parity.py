@@ -99,6 +99,56 @@ def test_full_width_two_layers_longer_context(B, oracle, shape):
     _teacher_forced(B, oracle, shape_dict(shape, n_layers=2, vocab=4096), 0, 3, chunks=[256, 256, 45, 20, 130], n_decode=6)
 
 
+def _batched_decode(B, oracle, shape, lengths, n_steps):
+    """Sequences of different cached lengths decoded together (one st_decode_step call per step, all rows through
+    the tensor-core pass); every row's logits are compared with the oracle run on that sequence alone."""
+    rng = np.random.default_rng(11)
+    n = len(lengths)
+    om = oracle.Model(oracle.Config(**shape), 0, 2)
+    gm = B.Model(shape, seed=0, tag=2, max_seqs=n, max_tokens=sum(lengths) + n * (n_steps + 64))
+    okvs, slots, toks = [], [], []
+    for ln in lengths:
+        t = rng.integers(0, shape["vocab"], size=ln + n_steps).astype(np.int32)
+        okv = oracle.KV(om, ln + n_steps + 1)
+        okv.forward(t[:ln])
+        slot = gm.st_seq_alloc()
+        for i in range(0, ln, 256):
+            gm.st_prefill(slot, t[i:min(ln, i + 256)])
+        okvs.append(okv)
+        slots.append(slot)
+        toks.append(t)
+    logits = torch.empty((n, shape["vocab"]), dtype=torch.float32, device="cuda")
+    amax = torch.empty(n, dtype=torch.int32, device="cuda")
+    worst = 0.0
+    for k in range(n_steps):
+        step_toks = np.array([toks[i][lengths[i] + k] for i in range(n)], dtype=np.int32)
+        gm.st_decode_step(slots, torch.from_numpy(step_toks).cuda(), logits, amax)
+        torch.cuda.synchronize()
+        got = logits.cpu().numpy()
+        for i in range(n):
+            want = okvs[i].forward(step_toks[i:i + 1])
+            e, _ = assert_logits_close(got[i], want, f"step {k}, sequence {i} (cached {lengths[i] + k})")
+            worst = max(worst, e)
+            gi, margin = oracle.argmax(want)
+            if margin >= MARGIN:
+                assert int(amax[i].item()) == gi
+            assert int(amax[i].item()) == int(np.argmax(got[i]))
+            assert gm.st_kv_len(slots[i]) == lengths[i] + k + 1
+    assert gm.st_last_device_status() == 0
+    gm.close()
+    return worst
+
+
+def test_batched_decode_tiny(B, oracle):
+    # ragged lengths: empty-ish, inside a page, page boundaries, several 128-key tiles
+    _batched_decode(B, oracle, shape_dict(W.TINY_L), [1, 15, 16, 63, 64, 127, 128, 300, 517], 3)
+
+
+@pytest.mark.parametrize("shape", [W.QWEN_1P5B, W.QWEN_32B])
+def test_batched_decode_full_width_two_layers(B, oracle, shape):
+    _batched_decode(B, oracle, shape_dict(shape, n_layers=2, vocab=4096), [5, 70, 129, 260], 2)
+
+
 def test_qwen1p5b_full_depth(B, oracle):
     """All 28 layers of the 1.5B shape: prompt prefill, a catch-up sized chunk and decode steps."""
     _teacher_forced(B, oracle, shape_dict(W.QWEN_1P5B), 0, 0, chunks=[24, 20], n_decode=4)
