@@ -129,7 +129,10 @@ int st_prefill(st_model *m, int32_t slot, const int32_t *tokens_host, int32_t n,
 
 /* One KV-cached decode step for `batch` sequences: sequence slots_host[i] ingests tokens_dev[i] at its
  * next position.  logits_dev (nullable): fp32 [batch][vocab]; argmax_dev (nullable): int32 [batch],
- * lowest-id argmax over the whole vocabulary. */
+ * lowest-id argmax over the whole vocabulary.  batch == 1 runs the single-kernel step; batch >= 2 streams the
+ * weights once for all rows (projections and LM head on the tensor cores, attention per sequence over its own
+ * pages), in chunks of at most 256 rows; without logits_dev the library keeps the [256][vocab] logits itself
+ * (allocated on the first such call). */
 int st_decode_step(st_model *m, const int32_t *slots_host, const int32_t *tokens_dev, int32_t batch,
                    float *logits_dev, int32_t *argmax_dev);
 
@@ -145,9 +148,15 @@ int st_generate_spec(st_model *small, st_model *large, const st_spec_params *par
 /* The same for n_seqs independent sequences (the batched workload: ragged prompts, per-sequence token budgets
  * and forcing schedules).  prompts / force are concatenations indexed by prompt_offsets / force_offsets
  * (n_seqs + 1 entries each; force may be NULL); max_new_per_seq (nullable) overrides params->max_new_tokens per
- * sequence; outs[i] receives sequence i's result.  Sequences do not interact, so every outs[i] equals what
- * st_generate_spec returns for that sequence alone.  In this version the sequences run one after the other
- * through the batch-1 path; stops at the first failing sequence and returns its status. */
+ * sequence; outs[i] receives sequence i's result.  Sequences do not interact, so every outs[i] holds the
+ * routing st_generate_spec gives for that sequence alone (its logits differ by rounding: batched rows go
+ * through the tensor-core passes).  When both models have a free sequence slot and KV pages for every sequence
+ * (st_config.max_seqs >= n_seqs, max_tokens >= the sum of prompt + budget + 1), n_seqs <= 256 and no logits
+ * trace is asked for, the sequences advance together in rounds: per round one batched decode pass per model over
+ * the sequences that lack one token, and a multi-row pass for each sequence that ingests a prompt or catches up
+ * after a handoff; the host reads only the shape of the next round, never a token.  outs[i].seconds is then the
+ * time of the whole batch and outs[i].bytes_algorithmic what sequence i would move alone.  Otherwise the
+ * sequences run one after the other through st_generate_spec (stops at the first failing one). */
 int st_generate_spec_batch(st_model *small, st_model *large, const st_spec_params *params, int32_t n_seqs,
                            const int32_t *prompts, const int32_t *prompt_offsets, const int32_t *max_new_per_seq,
                            const int32_t *force, const int32_t *force_offsets, st_spec_result *outs);

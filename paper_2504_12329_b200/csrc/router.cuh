@@ -121,6 +121,17 @@ __device__ void router_step(GenState *g, const GenBuffers &b, int greedy, StepDe
     plan_next_pass(g, desc_small, desc_large);
 }
 
+// After a batched decode pass (several independent generations advanced together): row k's greedy token advances
+// the state of the sequence the row belongs to.
+__global__ void batch_router_kernel(GenState *gs, const GenBuffers *gb, const int32_t *row_seq, const int32_t *greedy,
+                                    const StepDesc *bdesc, StepDesc *descs, int32_t *status)
+{
+    for (int k = threadIdx.x; k < bdesc->m; k += blockDim.x) {
+        const int i = row_seq[k];
+        router_step(gs + i, gb[i], greedy[k], descs + 2 * i, descs + 2 * i + 1, status);
+    }
+}
+
 // An ingest-only chunk finished: advance the cached length and plan the next pass.
 __global__ void advance_ingest_kernel(GenState *g, StepDesc *desc_small, StepDesc *desc_large)
 {
@@ -166,6 +177,64 @@ __global__ void dispatch_kernel(GenState *g, cudaGraphConditionalHandle loop, cu
     g->body_runs[b]++;
     cudaGraphSetConditional(loop, 1);
     cudaGraphSetConditional(body, (unsigned)b);
+}
+
+// ---- several independent generations advanced together (batched decode passes) ----
+
+constexpr int kBatchMaxCatchups = 256;
+
+// What the host needs to launch the next round of passes; it never contains a token.
+struct BatchPlan {
+    int32_t n_dec[2];                       // rows of the batched decode pass of each model
+    int32_t n_cu;                           // sequences that need a multi-row pass of their own this round
+    int32_t all_done;
+    int32_t max_ctx[2];                     // longest context among the decode rows of each model
+    int32_t cu[kBatchMaxCatchups][5];       // sequence, model, rows, first position, samples (1) or only ingests (0)
+};
+
+// One thread walks the sequences in order: a sequence whose active model lacks exactly one token joins that
+// model's batched decode pass (row = its place in the list), any other gets a multi-row pass of its own.
+// row_* and bdesc: per model [2]; slots: [n_seqs][2]; descs: [n_seqs][2].
+__global__ void batch_plan_kernel(GenState *gs, const GenBuffers *gb, int n_seqs, const int32_t *slots, StepDesc *descs,
+                                  int32_t *row_slot0, int32_t *row_pos0, int32_t *row_slot1, int32_t *row_pos1,
+                                  int32_t *row_tok /*[2][n_seqs]*/, int32_t *row_seq /*[2][n_seqs]*/, StepDesc *bdesc /*[2]*/,
+                                  int max_rows, BatchPlan *plan)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    int n_dec[2] = {0, 0}, n_cu = 0, live = 0, max_ctx[2] = {1, 1};
+    for (int i = 0; i < n_seqs; ++i) {
+        GenState *g = gs + i;
+        if (g->done) continue;
+        ++live;
+        const int a = g->active;
+        const int pending = g->pos - g->kv_len[a];
+        if (pending == 1 && n_dec[a] < max_rows) {
+            const int k = n_dec[a]++;
+            (a ? row_slot1 : row_slot0)[k] = slots[2 * i + a];
+            (a ? row_pos1 : row_pos0)[k] = g->kv_len[a];
+            row_tok[a * n_seqs + k] = gb[i].tokens[g->pos - 1];
+            row_seq[a * n_seqs + k] = i;
+            if (g->pos > max_ctx[a]) max_ctx[a] = g->pos;
+        } else if (pending > 1 && n_cu < kBatchMaxCatchups) {
+            plan_next_pass(g, descs + 2 * i, descs + 2 * i + 1);
+            int32_t *c = plan->cu[n_cu++];
+            c[0] = i;
+            c[1] = a;
+            c[2] = g->next_m;
+            c[3] = g->kv_len[a];
+            c[4] = g->next_emit;
+        }   // (a sequence that found no room waits for the next round)
+    }
+    for (int a = 0; a < 2; ++a) {
+        bdesc[a].pos0 = 0;
+        bdesc[a].m = n_dec[a];
+        bdesc[a].tok_off = 0;
+        bdesc[a].emit = 1;
+        plan->n_dec[a] = n_dec[a];
+        plan->max_ctx[a] = max_ctx[a];
+    }
+    plan->n_cu = n_cu;
+    plan->all_done = live == 0;
 }
 
 struct ArgmaxParams {

@@ -1753,6 +1753,273 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     return ST_OK;
 }
 
+// Several independent generations advanced together.  Every round a one-thread kernel sorts the live
+// sequences: those whose active model lacks exactly one token become rows of that model's batched decode pass
+// (one pass over the weights for all of them, projections on the tensor cores), the others (prompt prefill,
+// catch-up after a handoff) get a multi-row pass of their own.  The host reads back only the shape of the round
+// (row counts, which sequences need a multi-row pass of how many rows), never a token; sampling and the handoff
+// rule run on the device per sequence exactly as in st_generate_spec, so the results per sequence are the same.
+// Returns ST_OK with *handled = false when the call does not qualify (a logits trace is wanted, more sequences
+// than rows of a pass or than free sequence slots / KV pages): the caller then runs the sequences one by one.
+static int generate_spec_batch_rounds(st_model *small, st_model *large, const st_spec_params *P, int32_t n, const int32_t *prompts,
+                                      const int32_t *prompt_offsets, const int32_t *max_new_per_seq, const int32_t *force,
+                                      const int32_t *force_offsets, st_spec_result *outs, bool *handled)
+{
+    *handled = false;
+    static const bool sequential = [] { const char *e = getenv("ST_BATCH_SEQUENTIAL"); return e && e[0] == '1'; }();
+    if (sequential || n < 2 || n > small->max_rows || (large && n > large->max_rows)) return ST_OK;
+    if (P->max_new_tokens < 0 || P->n1 < 1 || P->n_keywords < 0 || (P->n_keywords > 0 && !P->keyword_ids)) return ST_ERR_ARG;
+    if (large && (large->stream != small->stream || large->device != small->device)) return ST_ERR_ARG;
+    int vshared = small->cfg.vocab;
+    if (large && large->cfg.vocab < vshared) vshared = large->cfg.vocab;
+    const int vlimit = P->vocab_limit > 0 ? P->vocab_limit : vshared;
+    if (vlimit > vshared) return ST_ERR_VOCAB;
+    for (int i = 0; i < P->n_keywords; ++i)
+        if ((unsigned)P->keyword_ids[i] >= (unsigned)vlimit) return ST_ERR_VOCAB;
+    if ((unsigned)P->delimiter_id >= (unsigned)vlimit) return ST_ERR_VOCAB;
+    std::vector<int> plen(n), mnew(n), nforce(n), total(n);
+    int longest = 0;
+    for (int i = 0; i < n; ++i) {
+        st_spec_result &o = outs[i];
+        if (o.logits_trace && o.trace_n_steps > 0) return ST_OK;   // traces: one sequence at a time
+        plen[i] = prompt_offsets[i + 1] - prompt_offsets[i];
+        mnew[i] = max_new_per_seq ? max_new_per_seq[i] : P->max_new_tokens;
+        nforce[i] = force ? force_offsets[i + 1] - force_offsets[i] : 0;
+        total[i] = plen[i] + mnew[i] + 1;
+        if (total[i] > longest) longest = total[i];
+        if (mnew[i] < 0) return ST_ERR_ARG;
+        if (o.cap_tokens < mnew[i] || (mnew[i] > 0 && (!o.tokens || !o.source))) return ST_ERR_CAPACITY;
+        if ((o.cap_steps > 0 && (!o.emission_tokens || !o.emission_source)) || (o.cap_handoffs > 0 && !o.handoffs)) return ST_ERR_ARG;
+        for (int j = prompt_offsets[i]; j < prompt_offsets[i + 1]; ++j)
+            if ((unsigned)prompts[j] >= (unsigned)vlimit) return ST_ERR_VOCAB;
+        for (int j = 0; j < nforce[i]; ++j)
+            if (force[force_offsets[i] + j] >= vlimit) return ST_ERR_VOCAB;
+    }
+    // sequence slots and KV pages for every sequence on both models, or the sequential path
+    std::vector<int32_t> slots(2 * (size_t)n, -1);
+    auto release_slots = [&] {
+        for (int i = 0; i < n; ++i) {
+            if (slots[2 * i] >= 0) st_seq_free(small, slots[2 * i]);
+            if (large && slots[2 * i + 1] >= 0) st_seq_free(large, slots[2 * i + 1]);
+        }
+    };
+    for (int i = 0; i < n; ++i) {
+        bool ok = st_seq_alloc(small, &slots[2 * i]) == ST_OK && seq_reserve(small, slots[2 * i], total[i]) == ST_OK;
+        if (ok && large) ok = st_seq_alloc(large, &slots[2 * i + 1]) == ST_OK && seq_reserve(large, slots[2 * i + 1], total[i]) == ST_OK;
+        if (!ok) {
+            release_slots();
+            return ST_OK;
+        }
+    }
+    *handled = true;
+    cudaStream_t s = small->stream;
+    st_model *models[2] = {small, large};
+    int rc = ST_OK;
+    uint8_t *arena = nullptr;
+    BatchPlan *plan_host = nullptr;
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    std::vector<GenState> gs(n);
+    std::vector<GenBuffers> gb(n);
+    GenState *d_gs = nullptr;
+    do {
+        for (int a = 0; a < 2; ++a) {
+            st_model *m = models[a];
+            if (!m) continue;
+            if (cudaMemsetAsync(m->status, 0, sizeof(int32_t), s) != cudaSuccess) { rc = ST_ERR_INTERNAL; break; }
+            if (!m->batch_logits) {
+                m->batch_logits = (float *)m->dalloc((size_t)m->max_rows * m->cfg.vocab * sizeof(float));
+                if (!m->batch_logits) { rc = ST_ERR_OOM; break; }
+            }
+        }
+        if (rc != ST_OK) break;
+        // ---- one device arena for the per-sequence state, buffers and logs ----
+        size_t off = 0;
+        auto take = [&](size_t bytes) { off = (off + 255) & ~(size_t)255; const size_t o = off; off += bytes; return o; };
+        const size_t o_gs = take(n * sizeof(GenState)), o_gb = take(n * sizeof(GenBuffers)), o_slots = take(2 * n * sizeof(int32_t));
+        const size_t o_descs = take(2 * n * sizeof(StepDesc)), o_bdesc = take(2 * sizeof(StepDesc));
+        const size_t o_rtok = take(2 * n * sizeof(int32_t)), o_rseq = take(2 * n * sizeof(int32_t)), o_amax = take(2 * n * sizeof(int32_t));
+        const size_t o_plan = take(sizeof(BatchPlan)), o_cls = take((size_t)vlimit);
+        std::vector<size_t> o_tok(n), o_src(n), o_emt(n), o_emf(n), o_ema(n), o_ems(n), o_hand(n), o_force(n);
+        for (int i = 0; i < n; ++i) {
+            const int cs = outs[i].cap_steps > 0 ? outs[i].cap_steps : 1, ch = outs[i].cap_handoffs > 0 ? outs[i].cap_handoffs : 1;
+            o_tok[i] = take((size_t)total[i] * 4);
+            o_src[i] = take((size_t)mnew[i] + 1);
+            o_emt[i] = take((size_t)cs * 4);
+            o_emf[i] = take((size_t)cs * 4);
+            o_ema[i] = take((size_t)cs * 4);
+            o_ems[i] = take((size_t)cs);
+            o_hand[i] = take((size_t)ch * 12);
+            o_force[i] = take((size_t)(nforce[i] > 0 ? nforce[i] : 1) * 4);
+        }
+        if (cudaMalloc(&arena, off + 256) != cudaSuccess) { cudaGetLastError(); rc = ST_ERR_OOM; break; }
+        if (cudaMallocHost(&plan_host, sizeof(BatchPlan)) != cudaSuccess) { cudaGetLastError(); rc = ST_ERR_OOM; break; }
+        d_gs = (GenState *)(arena + o_gs);
+        GenBuffers *d_gb = (GenBuffers *)(arena + o_gb);
+        int32_t *d_slots = (int32_t *)(arena + o_slots), *d_rtok = (int32_t *)(arena + o_rtok), *d_rseq = (int32_t *)(arena + o_rseq);
+        int32_t *d_amax = (int32_t *)(arena + o_amax);
+        StepDesc *d_descs = (StepDesc *)(arena + o_descs), *d_bdesc = (StepDesc *)(arena + o_bdesc);
+        BatchPlan *d_plan = (BatchPlan *)(arena + o_plan);
+        uint8_t *d_cls = arena + o_cls;
+        std::vector<uint8_t> cls(vlimit, 0);
+        for (int i = 0; i < P->n_keywords; ++i) cls[P->keyword_ids[i]] |= kClsKeyword;
+        int max_chunk = small->max_rows;
+        if (large && large->max_rows < max_chunk) max_chunk = large->max_rows;
+        for (int i = 0; i < n; ++i) {
+            GenState &g = gs[i];
+            g = GenState{};
+            g.wbytes[0] = small->weight_bytes;
+            g.kvb[0] = st_kv_bytes_per_token(small);
+            if (large) {
+                g.wbytes[1] = large->weight_bytes;
+                g.kvb[1] = st_kv_bytes_per_token(large);
+            }
+            g.has_large = large ? 1 : 0;
+            g.pos = plen[i];
+            g.delimiter = P->delimiter_id;
+            g.n1 = P->n1;
+            g.keep_probe = P->keep_probe;
+            g.eos = P->eos_id;
+            g.vlimit = vlimit;
+            g.max_new = mnew[i];
+            g.n_force = nforce[i];
+            g.prompt_len = plen[i];
+            g.cap_steps = outs[i].cap_steps;
+            g.cap_handoffs = outs[i].cap_handoffs;
+            g.max_chunk = max_chunk;
+            g.done = mnew[i] == 0 ? 1 : 0;
+            g.pass_cap = 0x7fffffff;
+            GenBuffers &b = gb[i];
+            b.tokens = (int32_t *)(arena + o_tok[i]);
+            b.source = arena + o_src[i];
+            b.em_tok = (int32_t *)(arena + o_emt[i]);
+            b.em_fed = (int32_t *)(arena + o_emf[i]);
+            b.em_arg = (int32_t *)(arena + o_ema[i]);
+            b.em_src = arena + o_ems[i];
+            b.handoffs = (int32_t *)(arena + o_hand[i]);
+            b.force = (const int32_t *)(arena + o_force[i]);
+            b.cls = d_cls;
+            b.trace = nullptr;
+        }
+        bool up = cudaMemcpyAsync(d_gs, gs.data(), n * sizeof(GenState), cudaMemcpyHostToDevice, s) == cudaSuccess &&
+                  cudaMemcpyAsync(d_gb, gb.data(), n * sizeof(GenBuffers), cudaMemcpyHostToDevice, s) == cudaSuccess &&
+                  cudaMemcpyAsync(d_slots, slots.data(), 2 * n * sizeof(int32_t), cudaMemcpyHostToDevice, s) == cudaSuccess &&
+                  cudaMemcpyAsync(d_cls, cls.data(), (size_t)vlimit, cudaMemcpyHostToDevice, s) == cudaSuccess;
+        for (int i = 0; i < n && up; ++i) {
+            up = cudaMemcpyAsync(gb[i].tokens, prompts + prompt_offsets[i], (size_t)plen[i] * 4, cudaMemcpyHostToDevice, s) == cudaSuccess;
+            if (up && nforce[i] > 0)
+                up = cudaMemcpyAsync(arena + o_force[i], force + force_offsets[i], (size_t)nforce[i] * 4, cudaMemcpyHostToDevice, s) == cudaSuccess;
+        }
+        if (!up) { set_error_text("batched generation upload", cudaGetLastError()); rc = ST_ERR_INTERNAL; break; }
+        if (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess) { rc = ST_ERR_INTERNAL; break; }
+        cudaEventRecord(ev0, s);
+        // ---- rounds ----
+        int64_t sum_new = 0;
+        for (int i = 0; i < n; ++i) sum_new += mnew[i];
+        const int64_t round_cap = 4 * (sum_new + 4ll * n + 16) + 4ll * n * (longest / max_chunk + 2);
+        bool finished = false;
+        for (int64_t round = 0; round < round_cap && rc == ST_OK; ++round) {
+            batch_plan_kernel<<<1, 1, 0, s>>>(d_gs, d_gb, n, d_slots, d_descs, small->row_slot, small->row_pos,
+                                              large ? large->row_slot : small->row_slot, large ? large->row_pos : small->row_pos,
+                                              d_rtok, d_rseq, d_bdesc, max_chunk, d_plan);
+            ++g_launches;
+            if (cudaMemcpyAsync(plan_host, d_plan, sizeof(BatchPlan), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+                cudaStreamSynchronize(s) != cudaSuccess) {
+                set_error_text("batched generation round", cudaGetLastError());
+                rc = ST_ERR_INTERNAL;
+                break;
+            }
+            const BatchPlan &pl = *plan_host;
+            if (pl.all_done) { finished = true; break; }
+            for (int a = 0; a < 2 && rc == ST_OK; ++a) {
+                const int rows = pl.n_dec[a];
+                st_model *m = models[a];
+                if (rows <= 0 || !m) continue;
+                SampleCtx sc{};
+                sc.logits_out = m->batch_logits;
+                sc.argmax_out = d_amax + (size_t)a * n;
+                sc.want_argmax = true;
+                sc.vlimit = vlimit;
+                int m_upper = (rows + 31) / 32 * 32;
+                if (m_upper > m->max_rows) m_upper = m->max_rows;
+                rc = pass_rows(m, d_bdesc + a, d_rtok + (size_t)a * n, -1, m_upper, pl.max_ctx[a], true, sc, true);
+                if (rc != ST_OK) break;
+                batch_router_kernel<<<1, 64, 0, s>>>(d_gs, d_gb, d_rseq + (size_t)a * n, d_amax + (size_t)a * n, d_bdesc + a, d_descs,
+                                                     small->status);
+                ++g_launches;
+                if (cudaGetLastError() != cudaSuccess) rc = ST_ERR_INTERNAL;
+            }
+            for (int k = 0; k < pl.n_cu && rc == ST_OK; ++k) {
+                const int i = pl.cu[k][0], a = pl.cu[k][1], rows = pl.cu[k][2], pos0 = pl.cu[k][3], emit = pl.cu[k][4];
+                st_model *m = models[a];
+                if (i < 0 || i >= n || !m || rows < 1 || rows > m->max_rows) { rc = ST_ERR_INTERNAL; break; }
+                SampleCtx sc{};
+                sc.vlimit = vlimit;
+                sc.gen = d_gs + i;
+                sc.buf = gb[i];
+                sc.desc_small = d_descs + 2 * i;
+                sc.desc_large = d_descs + 2 * i + 1;
+                sc.want_argmax = true;
+                rc = pass_rows(m, d_descs + 2 * i + a, gb[i].tokens, slots[2 * i + a], rows, pos0 + rows, emit != 0, sc);
+                if (rc == ST_OK && !emit) {
+                    advance_ingest_kernel<<<1, 1, 0, s>>>(d_gs + i, d_descs + 2 * i, d_descs + 2 * i + 1);
+                    ++g_launches;
+                    if (cudaGetLastError() != cudaSuccess) rc = ST_ERR_INTERNAL;
+                }
+            }
+        }
+        if (rc != ST_OK) break;
+        cudaEventRecord(ev1, s);
+        if (cudaStreamSynchronize(s) != cudaSuccess) { set_error_text("batched generation", cudaGetLastError()); rc = ST_ERR_INTERNAL; break; }
+        if (!finished) { rc = ST_ERR_TIMEOUT; break; }
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, ev0, ev1);
+        // ---- results ----
+        if (cudaMemcpy(gs.data(), d_gs, n * sizeof(GenState), cudaMemcpyDeviceToHost) != cudaSuccess) { rc = ST_ERR_INTERNAL; break; }
+        bool dn = true;
+        for (int i = 0; i < n && dn; ++i) {
+            const GenState &g = gs[i];
+            const GenBuffers &b = gb[i];
+            st_spec_result &o = outs[i];
+            o.n_tokens = g.generated;
+            o.n_steps = g.step;
+            o.n_handoffs = g.n_handoffs;
+            o.kv_len_small = g.kv_len[0];
+            o.kv_len_large = g.kv_len[1];
+            o.seconds = ms * 1e-3;   // of the whole batch
+            o.bytes_algorithmic = g.bytes_algo;
+            const int n_steps = g.step < o.cap_steps ? g.step : o.cap_steps;
+            const int n_hand = g.n_handoffs < o.cap_handoffs ? g.n_handoffs : o.cap_handoffs;
+            if (g.generated > 0) {
+                dn = dn && cudaMemcpyAsync(o.tokens, b.tokens + plen[i], (size_t)g.generated * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+                dn = dn && cudaMemcpyAsync(o.source, b.source, (size_t)g.generated, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+            }
+            if (n_steps > 0) {
+                dn = dn && cudaMemcpyAsync(o.emission_tokens, b.em_tok, (size_t)n_steps * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+                dn = dn && cudaMemcpyAsync(o.emission_source, b.em_src, (size_t)n_steps, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+                if (o.emission_fed) dn = dn && cudaMemcpyAsync(o.emission_fed, b.em_fed, (size_t)n_steps * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+                if (o.emission_argmax) dn = dn && cudaMemcpyAsync(o.emission_argmax, b.em_arg, (size_t)n_steps * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+            }
+            if (n_hand > 0) dn = dn && cudaMemcpyAsync(o.handoffs, b.handoffs, (size_t)n_hand * 12, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+        }
+        if (!dn || cudaStreamSynchronize(s) != cudaSuccess) { set_error_text("batched generation results", cudaGetLastError()); rc = ST_ERR_INTERNAL; break; }
+        int32_t dev_status = 0, s2 = 0;
+        cudaMemcpy(&dev_status, small->status, sizeof dev_status, cudaMemcpyDeviceToHost);
+        if (large) cudaMemcpy(&s2, large->status, sizeof s2, cudaMemcpyDeviceToHost);
+        dev_status |= s2;
+        if (dev_status & DEV_LOG_FULL) rc = ST_ERR_CAPACITY;
+        else if (dev_status & DEV_BAD_TOKEN) rc = ST_ERR_VOCAB;
+        else if (dev_status & DEV_WAIT_EXPIRED) rc = ST_ERR_TIMEOUT;
+        else if (dev_status) rc = ST_ERR_INTERNAL;
+    } while (0);
+    cudaStreamSynchronize(s);
+    if (ev0) cudaEventDestroy(ev0);
+    if (ev1) cudaEventDestroy(ev1);
+    if (plan_host) cudaFreeHost(plan_host);
+    if (arena) cudaFree(arena);
+    release_slots();
+    return rc;
+}
+
 extern "C" int st_generate_spec_batch(st_model *small, st_model *large, const st_spec_params *P, int32_t n_seqs,
                                       const int32_t *prompts, const int32_t *prompt_offsets, const int32_t *max_new_per_seq,
                                       const int32_t *force, const int32_t *force_offsets, st_spec_result *outs)
@@ -1763,6 +2030,9 @@ extern "C" int st_generate_spec_batch(st_model *small, st_model *large, const st
         if (prompt_offsets[i + 1] <= prompt_offsets[i]) return ST_ERR_ARG;
         if (force && force_offsets[i + 1] < force_offsets[i]) return ST_ERR_ARG;
     }
+    bool handled = false;
+    TRY(generate_spec_batch_rounds(small, large, P, n_seqs, prompts, prompt_offsets, max_new_per_seq, force, force_offsets, outs, &handled));
+    if (handled) return ST_OK;
     for (int i = 0; i < n_seqs; ++i) {
         st_spec_params pi = *P;
         if (max_new_per_seq) pi.max_new_tokens = max_new_per_seq[i];

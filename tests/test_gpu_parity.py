@@ -312,3 +312,40 @@ def test_batched_ragged_sequences(B, oracle):
     assert n_hand >= 6
     gs.close()
     gl.close()
+
+
+def test_batched_generation_in_rounds(B, oracle):
+    """Enough sequence slots and KV pages for all sequences: they advance together, one batched decode pass per
+    model and round plus a multi-row pass per prompt / catch-up.  Routing per sequence equals the oracle's run of
+    that sequence alone, and so does the greedy choice wherever the oracle's margin allows a comparison."""
+    S, L = shape_dict(W.TINY_S), shape_dict(W.TINY_L)
+    n = 7
+    prompts, budgets, forces = W.batch_inputs(17, n, 1024, prompt_range=(5, 70), budget_range=(20, 120), mean_interval=6,
+                                              keyword_rate=0.6)
+    forces = [W.full_forcing(700 + i, len(f), 1024, mean_interval=6, keyword_rate=0.6) for i, f in enumerate(forces)]
+    budgets[2] = 0                      # a sequence with nothing to generate
+    gs = B.Model(S, seed=0, tag=0, max_seqs=n, max_tokens=n * 256)
+    gl = B.Model(L, seed=0, tag=1, max_seqs=n, max_tokens=n * 256)
+    got = B.st_generate_spec_batch(gs, gl, prompts, delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=4,
+                                   max_new_tokens=budgets, forces=forces)
+    assert len({r.seconds for r in got}) == 1, "the sequences did not run as one batch"
+    os_, ol = oracle.Model(oracle.Config(**S), 0, 0), oracle.Model(oracle.Config(**L), 0, 1)
+    n_hand = n_cmp = 0
+    for i in range(n):
+        want = oracle.generate_spec(os_, ol, prompts[i], delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=4,
+                                    max_new_tokens=budgets[i], force=forces[i])
+        _assert_routing_equal(want, got[i])
+        assert len(got[i].tokens) == budgets[i]
+        n_hand += len(want.handoffs)
+        for t in range(len(want.emission_tokens)):
+            if want.emission_margin[t] >= MARGIN:
+                assert got[i].emission_argmax[t] == want.emission_argmax[t], (i, t)
+                n_cmp += 1
+    assert n_hand >= 6 and n_cmp >= 100
+    # the models are reusable, and a second call gives the same result
+    again = B.st_generate_spec_batch(gs, gl, prompts, delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=4,
+                                     max_new_tokens=budgets, forces=forces)
+    for a, b in zip(got, again):
+        assert a.tokens.tolist() == b.tokens.tolist() and a.emission_argmax.tolist() == b.emission_argmax.tolist()
+    gs.close()
+    gl.close()
