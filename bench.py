@@ -267,8 +267,11 @@ def main():
     wl = rank_workload(w, rank)
     prompt, force = W.workload_inputs(wl)
     cap = wl.prompt_len + wl.max_new_tokens + 64
+    # room for the batched decode measurement at the end: BATCH more sequences of BATCH_CTX + 64 tokens on the large model
+    BATCH, BATCH_CTX = 64, 512
     small = B.Model(wl.small.as_dict(), seed=wl.weight_seed, tag=0, max_tokens=cap)
-    large = B.Model(wl.large.as_dict(), seed=wl.weight_seed, tag=1, max_tokens=cap) if wl.large else None
+    large = B.Model(wl.large.as_dict(), seed=wl.weight_seed, tag=1, max_seqs=BATCH + 1,
+                    max_tokens=cap + BATCH * (BATCH_CTX + 64)) if wl.large else None
     kw = dict(delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=W.N1, max_new_tokens=wl.max_new_tokens, force=force)
 
     def barrier():
@@ -347,6 +350,31 @@ def main():
         small_step = {"kernel": f"decode_mega_kernel ({wl.small.name}, context {ctx})", "us_per_launch": s_s * 1e6,
                       "achieved": s_bytes / s_s / 1e9, "frac": s_bytes / s_s / 1e9 / peak, "unit": "GB/s"}
         small.st_seq_free(sslot)
+    # batched decode of the same model (the 64-sequence workload's step): one pass over the weights for all rows
+    batched = None
+    if large is not None:
+        bslots = [large.st_seq_alloc() for _ in range(BATCH)]
+        for i, sl in enumerate(bslots):
+            for j in range(0, BATCH_CTX, 256):
+                large.st_prefill(sl, W.prompt_ids(50 + i, min(256, BATCH_CTX - j), shp.vocab))
+        btok = torch.zeros(BATCH, dtype=torch.int32, device="cuda")
+        bamax = torch.zeros(BATCH, dtype=torch.int32, device="cuda")
+        for _ in range(3):
+            large.st_decode_step(bslots, btok, None, bamax)
+        torch.cuda.synchronize()
+        n_b = 10
+        e0.record()
+        for _ in range(n_b):
+            large.st_decode_step(bslots, btok, None, bamax)
+        e1.record()
+        torch.cuda.synchronize()
+        b_s = e0.elapsed_time(e1) * 1e-3 / n_b
+        b_bytes = large.st_weight_bytes() + large.st_kv_bytes_per_token() * BATCH * (BATCH_CTX + 3 + n_b // 2)
+        batched = {"model": shp.name, "batch": BATCH, "context": BATCH_CTX, "ms_per_step": b_s * 1e3, "tokens_per_s": BATCH / b_s,
+                   "hbm_gbs": b_bytes / b_s / 1e9, "frac_hbm": b_bytes / b_s / 1e9 / peak,
+                   "note": "st_decode_step with 64 sequences: tcgen05 projections, per-sequence attention over paged K/V"}
+        for sl in bslots:
+            large.st_seq_free(sl)
     path_gbs = sum(x.bytes_algorithmic for x in results) / sum(x.seconds for x in results) / 1e9
     steps_small = int((r.emission_source == 0).sum())
     steps_large = int((r.emission_source == 1).sum())
@@ -381,6 +409,7 @@ def main():
                               "note": "algorithmic bytes of every pass (weights + KV) / device time of the generation"},
             "prefill": prefill,
             "small_model_decode": small_step,
+            "batched_decode": batched,
             "wall_s_timed_region": t_region,
         }
         if not args.no_cpu_baseline:
