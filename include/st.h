@@ -78,6 +78,11 @@ typedef struct {
     int32_t eos_id;         /* -1: none */
     int32_t vocab_limit;    /* tokens are chosen among ids < vocab_limit; 0 = min of the two vocabularies */
     int32_t max_new_tokens;
+    /* Variant for a speculative model that emits no reflective cues (Section 4, "Modification for speculative
+     * thinking applied to non-reasoning models"); both 0 for the rule above. */
+    int32_t takeover_every_delimiter; /* 1: no keyword test -- whenever the speculative model writes the delimiter,
+                                         the target writes the next n1 tokens */
+    int32_t target_first_n;           /* > 0: the target writes the first target_first_n tokens (paper: 100) */
 } st_spec_params;
 
 typedef struct {

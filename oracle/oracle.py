@@ -40,6 +40,7 @@ class _SpecParams(C.Structure):
         ("delimiter_id", C.c_int32), ("keyword_ids", C.POINTER(C.c_int32)), ("n_keywords", C.c_int32),
         ("n1", C.c_int32), ("keep_probe", C.c_int32), ("eos_id", C.c_int32), ("vocab_limit", C.c_int32),
         ("max_new_tokens", C.c_int32),
+        ("takeover_every_delimiter", C.c_int32), ("target_first_n", C.c_int32),
     ]
 
 
@@ -258,13 +259,14 @@ class SpecResult:
 
 def generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id: int, keyword_ids, n1: int = 20,
                   keep_probe: bool = False, eos_id: int = -1, vocab_limit: int = 0, max_new_tokens: int,
-                  force=None, trace_first_step: int = 0, trace_n_steps: int = 0) -> SpecResult:
+                  force=None, trace_first_step: int = 0, trace_n_steps: int = 0,
+                  takeover_every_delimiter: bool = False, target_first_n: int = 0) -> SpecResult:
     prompt = np.ascontiguousarray(prompt, dtype=np.int32)
     kw = np.ascontiguousarray(keyword_ids, dtype=np.int32)
     if vocab_limit <= 0:
         vocab_limit = small.cfg.vocab if large is None else min(small.cfg.vocab, large.cfg.vocab)
     P = _SpecParams(delimiter_id, kw.ctypes.data_as(C.POINTER(C.c_int32)), kw.size, n1, int(keep_probe), eos_id,
-                    vocab_limit, max_new_tokens)
+                    vocab_limit, max_new_tokens, int(takeover_every_delimiter), int(target_first_n))
     cap_steps = 2 * max_new_tokens + 8
     tokens = np.zeros(max_new_tokens + 1, dtype=np.int32)
     source = np.zeros(max_new_tokens + 1, dtype=np.uint8)

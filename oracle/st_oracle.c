@@ -481,6 +481,11 @@ typedef struct {
     int32_t eos_id;      /* -1: none */
     int32_t vocab_limit; /* sample over ids < vocab_limit */
     int32_t max_new_tokens;
+    /* Variant for a speculative model without reflective cues (Section "Reasoning Models Monitor
+     * Non-Reasoning Models", paragraph "Modification ..."): */
+    int32_t takeover_every_delimiter; /* 1: no keyword test; the target writes the n1 tokens after every
+                                         delimiter the speculative model writes */
+    int32_t target_first_n;           /* > 0: the target writes the first target_first_n tokens (paper: 100) */
 } orc_spec_params;
 
 typedef struct { int32_t seg_start, step, catchup_len; } orc_handoff;
@@ -523,6 +528,10 @@ int orc_generate_spec(const orc_model *small, const orc_model *large, const orc_
     int active = 0, remaining = 0, rc = 0;
     int32_t pos = prompt_len, t = 0, generated = 0;
     R->n_tokens = R->n_handoffs = R->n_steps = 0;
+    if (large && P->target_first_n > 0) {   /* the target opens the answer */
+        active = 1;
+        remaining = P->target_first_n;
+    }
     while (generated < P->max_new_tokens) {
         int a = active;
         int32_t fed = pos - (int32_t)kv[a]->len;
@@ -542,7 +551,7 @@ int orc_generate_spec(const orc_model *small, const orc_model *large, const orc_
         R->n_steps = t;
         int is_kw = 0;
         for (int i = 0; i < P->n_keywords; ++i) is_kw |= (P->keyword_ids[i] == tok);
-        if (large && a == 0 && tokens[pos - 1] == P->delimiter_id && is_kw) {
+        if (large && a == 0 && !P->takeover_every_delimiter && tokens[pos - 1] == P->delimiter_id && is_kw) {
             if (P->keep_probe) {
                 tokens[pos] = tok;
                 if (generated >= R->cap_tokens) { rc = -3; break; }
@@ -569,6 +578,16 @@ int orc_generate_spec(const orc_model *small, const orc_model *large, const orc_
         R->n_tokens = generated;
         if (tok == P->eos_id) break;
         if (a == 1 && --remaining == 0) active = 0;
+        if (large && a == 0 && P->takeover_every_delimiter && tok == P->delimiter_id && generated < P->max_new_tokens) {
+            /* the speculative model closed a paragraph: the target writes the next n1 tokens */
+            if (R->n_handoffs >= R->cap_handoffs) { rc = -3; break; }
+            R->handoffs[R->n_handoffs].seg_start = pos;
+            R->handoffs[R->n_handoffs].step = t - 1;
+            R->handoffs[R->n_handoffs].catchup_len = pos - (int32_t)kv[1]->len;
+            R->n_handoffs++;
+            active = 1;
+            remaining = P->n1;
+        }
     }
     R->kv_len_small = (int32_t)kv[0]->len;
     R->kv_len_large = kv[1] ? (int32_t)kv[1]->len : 0;

@@ -37,7 +37,7 @@ class StSpecParams(C.Structure):
     _fields_ = [
         ("delimiter_id", C.c_int32), ("keyword_ids", C.POINTER(C.c_int32)), ("n_keywords", C.c_int32),
         ("n1", C.c_int32), ("keep_probe", C.c_int32), ("eos_id", C.c_int32), ("vocab_limit", C.c_int32),
-        ("max_new_tokens", C.c_int32),
+        ("max_new_tokens", C.c_int32), ("takeover_every_delimiter", C.c_int32), ("target_first_n", C.c_int32),
     ]
 
 
@@ -327,12 +327,13 @@ class _ResultBuffers:
 def st_generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id: int, keyword_ids, n1: int = 20,
                      keep_probe: bool = False, eos_id: int = -1, vocab_limit: int = 0, max_new_tokens: int,
                      force=None, trace_first_step: int = 0, trace_n_steps: int = 0, cap_steps: int | None = None,
-                     cap_handoffs: int | None = None) -> SpecResult:
+                     cap_handoffs: int | None = None, takeover_every_delimiter: bool = False,
+                     target_first_n: int = 0) -> SpecResult:
     """Host buffers in, host buffers out: marshals the arguments of st_generate_spec."""
     prompt = np.ascontiguousarray(prompt, dtype=np.int32)
     kw = np.ascontiguousarray(keyword_ids, dtype=np.int32)
     P = StSpecParams(delimiter_id, kw.ctypes.data_as(C.POINTER(C.c_int32)), kw.size, n1, int(keep_probe), eos_id,
-                     vocab_limit, max_new_tokens)
+                     vocab_limit, max_new_tokens, int(takeover_every_delimiter), int(target_first_n))
     if vocab_limit <= 0:
         vocab_limit = small.vocab if large is None else min(small.vocab, large.vocab)
     bufs = _ResultBuffers(max_new_tokens, vocab_limit, trace_first_step, trace_n_steps, cap_steps, cap_handoffs)
@@ -347,13 +348,13 @@ def st_generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id:
 
 def st_generate_spec_batch(small: Model, large: Model | None, prompts, *, delimiter_id: int, keyword_ids, n1: int = 20,
                            keep_probe: bool = False, eos_id: int = -1, vocab_limit: int = 0, max_new_tokens,
-                           forces=None) -> list:
+                           forces=None, takeover_every_delimiter: bool = False, target_first_n: int = 0) -> list:
     """prompts / forces: lists of per-sequence arrays; max_new_tokens: one int or a list per sequence."""
     n = len(prompts)
     budgets = [int(max_new_tokens)] * n if np.isscalar(max_new_tokens) else [int(x) for x in max_new_tokens]
     kw = np.ascontiguousarray(keyword_ids, dtype=np.int32)
     P = StSpecParams(delimiter_id, kw.ctypes.data_as(C.POINTER(C.c_int32)), kw.size, n1, int(keep_probe), eos_id,
-                     vocab_limit, max(budgets) if budgets else 0)
+                     vocab_limit, max(budgets) if budgets else 0, int(takeover_every_delimiter), int(target_first_n))
     if vocab_limit <= 0:
         vocab_limit = small.vocab if large is None else min(small.vocab, large.vocab)
     flat_p = np.ascontiguousarray(np.concatenate([np.asarray(p, dtype=np.int32) for p in prompts]) if n else np.zeros(0, np.int32))

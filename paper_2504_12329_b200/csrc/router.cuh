@@ -35,6 +35,7 @@ struct GenState {
     int32_t pass_cap;    // hard bound on passes (the device loop stops there)
     // --- parameters ---
     int32_t has_large, delimiter, n1, keep_probe, eos, vlimit, max_new, n_force;
+    int32_t every_delim;   // 1: no keyword test; the target takes over after every delimiter the speculative model writes
     int32_t prompt_len, cap_steps, cap_handoffs, max_chunk;
     int32_t trace_first, trace_n;
 };
@@ -89,7 +90,7 @@ __device__ void router_step(GenState *g, const GenBuffers &b, int greedy, StepDe
     }
     g->step = t + 1;
     if ((unsigned)tok >= (unsigned)g->vlimit) { atomicOr(status, DEV_BAD_TOKEN); tok = 0; }
-    const bool trigger = g->has_large && a == 0 && b.tokens[g->pos - 1] == g->delimiter && (b.cls[tok] & kClsKeyword);
+    const bool trigger = g->has_large && a == 0 && !g->every_delim && b.tokens[g->pos - 1] == g->delimiter && (b.cls[tok] & kClsKeyword);
     if (trigger) {
         if (g->keep_probe) {
             b.tokens[g->pos] = tok;
@@ -116,6 +117,20 @@ __device__ void router_step(GenState *g, const GenBuffers &b, int greedy, StepDe
         g->generated++;
         if (tok == g->eos) g->done = 1;
         if (a == 1 && --g->remaining == 0) g->active = 0;
+        if (g->has_large && a == 0 && g->every_delim && tok == g->delimiter && !g->done && g->generated < g->max_new) {
+            // the speculative model closed a paragraph: the target writes the next n1 tokens
+            if (g->n_handoffs < g->cap_handoffs) {
+                int32_t *h = b.handoffs + 3 * g->n_handoffs;
+                h[0] = g->pos;
+                h[1] = t;
+                h[2] = g->pos - g->kv_len[1];
+            } else {
+                atomicOr(status, DEV_LOG_FULL);
+            }
+            g->n_handoffs++;
+            g->active = 1;
+            g->remaining = g->n1;
+        }
     }
     if (g->generated >= g->max_new) g->done = 1;
     plan_next_pass(g, desc_small, desc_large);

@@ -1573,7 +1573,7 @@ static int ensure_gen_context(st_model *small, st_model *large, int slot_s, int 
 extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_params *P, const int32_t *prompt,
                                 int32_t prompt_len, const int32_t *force, int32_t n_force, st_spec_result *out)
 {
-    if (!small || !P || !prompt || !out || prompt_len < 1 || P->max_new_tokens < 0 || P->n1 < 1 || n_force < 0) return ST_ERR_ARG;
+    if (!small || !P || !prompt || !out || prompt_len < 1 || P->max_new_tokens < 0 || P->n1 < 1 || n_force < 0 || P->target_first_n < 0) return ST_ERR_ARG;
     if (P->n_keywords < 0 || (P->n_keywords > 0 && !P->keyword_ids) || (n_force > 0 && !force)) return ST_ERR_ARG;
     if (large && (large->stream != small->stream || large->device != small->device)) return ST_ERR_ARG;
     int vshared = small->cfg.vocab;
@@ -1637,6 +1637,11 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     g0.delimiter = P->delimiter_id;
     g0.n1 = P->n1;
     g0.keep_probe = P->keep_probe;
+    g0.every_delim = P->takeover_every_delimiter ? 1 : 0;
+    if (large && P->target_first_n > 0) {   // the target opens the answer
+        g0.active = 1;
+        g0.remaining = P->target_first_n;
+    }
     g0.eos = P->eos_id;
     g0.vlimit = vlimit;
     g0.max_new = max_new;
@@ -1878,6 +1883,11 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
             g.delimiter = P->delimiter_id;
             g.n1 = P->n1;
             g.keep_probe = P->keep_probe;
+            g.every_delim = P->takeover_every_delimiter ? 1 : 0;
+            if (large && P->target_first_n > 0) {
+                g.active = 1;
+                g.remaining = P->target_first_n;
+            }
             g.eos = P->eos_id;
             g.vlimit = vlimit;
             g.max_new = mnew[i];

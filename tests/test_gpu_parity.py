@@ -349,3 +349,33 @@ def test_batched_generation_in_rounds(B, oracle):
         assert a.tokens.tolist() == b.tokens.tolist() and a.emission_argmax.tolist() == b.emission_argmax.tolist()
     gs.close()
     gl.close()
+
+
+def test_every_delimiter_variant_on_device(B, oracle):
+    """The variant for a speculative model without reflective cues: the target opens the answer and takes over
+    after every delimiter the small model writes.  Routing bit-exact against the oracle (hand-traced stream and a
+    longer forced run), greedy choices wherever the margin allows, alone and through the batched rounds."""
+    S, L = shape_dict(W.TINY_S), shape_dict(W.TINY_L)
+    os_, ol = oracle.Model(oracle.Config(**S), 0, 0), oracle.Model(oracle.Config(**L), 0, 1)
+    gs = B.Model(S, seed=0, tag=0, max_seqs=3, max_tokens=1024)
+    gl = B.Model(L, seed=0, tag=1, max_seqs=3, max_tokens=1024)
+    kw = dict(delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, takeover_every_delimiter=True)
+    hand = [5, 6, 7, 10, 20, 21, 22, 8, 10, 30, 31, 32, 9]
+    got = B.st_generate_spec(gs, gl, [1, 2, 3], n1=3, target_first_n=2, max_new_tokens=12, force=hand, **kw)
+    assert got.tokens.tolist() == [5, 6, 7, 10, 20, 21, 22, 8, 10, 30, 31, 32]
+    assert got.source.tolist() == [1, 1, 0, 0, 1, 1, 1, 0, 0, 1, 1, 1]
+    assert got.handoffs == [(7, 3, 3), (12, 8, 3)]
+    prompts = [W.prompt_ids(300 + i, 20 + 9 * i, 1024) for i in range(3)]
+    forces = [W.full_forcing(310 + i, 300, 1024, mean_interval=7, keyword_rate=0.3) for i in range(3)]
+    wants = [oracle.generate_spec(os_, ol, prompts[i], n1=5, target_first_n=10, max_new_tokens=100, force=forces[i], **kw)
+             for i in range(3)]
+    alone = B.st_generate_spec(gs, gl, prompts[0], n1=5, target_first_n=10, max_new_tokens=100, force=forces[0], **kw)
+    batch = B.st_generate_spec_batch(gs, gl, prompts, n1=5, target_first_n=10, max_new_tokens=100, forces=forces, **kw)
+    for want, got in [(wants[0], alone)] + list(zip(wants, batch)):
+        _assert_routing_equal(want, got)
+        assert len(want.handoffs) >= 4 and want.source[:10].tolist() == [1] * 10
+        for t in range(len(want.emission_tokens)):
+            if want.emission_margin[t] >= MARGIN:
+                assert got.emission_argmax[t] == want.emission_argmax[t]
+    gs.close()
+    gl.close()

@@ -48,6 +48,44 @@ def test_hand_traced_streams(oracle, tiny, name, keep):
     assert (r.kv_len_small, r.kv_len_large) == (T["kv_len_small"], T["kv_len_large"])
 
 
+def test_hand_traced_stream_every_delimiter(oracle, tiny):
+    T = _trace("handoff_trace_every_delimiter.txt")
+    r = oracle.generate_spec(tiny[0], tiny[1], [1, 2, 3], delimiter_id=10, keyword_ids=[11, 12, 13], n1=3,
+                             max_new_tokens=12, force=T["force"], takeover_every_delimiter=True, target_first_n=2)
+    assert r.rc == 0
+    assert r.tokens.tolist() == T["tokens"]
+    assert r.source.tolist() == T["source"]
+    assert r.handoffs == T["handoffs"]
+    assert r.emission_source.tolist() == T["emission_source"]
+    assert r.emission_fed.tolist() == T["emission_fed"]
+    assert (r.kv_len_small, r.kv_len_large) == (T["kv_len_small"], T["kv_len_large"])
+
+
+def test_every_delimiter_edge_cases(oracle, tiny):
+    kw = dict(delimiter_id=10, keyword_ids=[11, 12, 13], n1=2, takeover_every_delimiter=True)
+    # keywords mean nothing in this mode; a delimiter written by the target or standing in the prompt hands nothing over
+    r = oracle.generate_spec(tiny[0], tiny[1], [4, 10], max_new_tokens=8, force=[11, 10, 10, 21, 12, 10, 30, 31], **kw)
+    assert r.source.tolist() == [0, 0, 1, 1, 0, 0, 1, 1]
+    assert r.handoffs == [(4, 1, 4), (8, 5, 3)]      # the target cached 5 tokens by its second turn: it ingests positions 5..7
+    # the budget ends on the delimiter: no handoff is logged for a segment that cannot start
+    r = oracle.generate_spec(tiny[0], tiny[1], [4], max_new_tokens=2, force=[5, 10], **kw)
+    assert r.handoffs == [] and r.source.tolist() == [0, 0]
+    # the opening segment alone; without a target both switches are ignored
+    r = oracle.generate_spec(tiny[0], tiny[1], [4], max_new_tokens=5, force=[5, 6, 7, 8, 9], delimiter_id=10, keyword_ids=[],
+                             n1=2, target_first_n=3)
+    assert r.source.tolist() == [1, 1, 1, 0, 0] and r.handoffs == []
+    r = oracle.generate_spec(tiny[0], None, [4], max_new_tokens=4, force=[5, 10, 7, 8], target_first_n=3, **kw)
+    assert r.source.tolist() == [0, 0, 0, 0] and r.handoffs == []
+    # every target segment has exactly n1 tokens unless the budget cuts it
+    force = W.full_forcing(5, 200, 1024, mean_interval=5, keyword_rate=0.0)
+    r = oracle.generate_spec(tiny[0], tiny[1], [1, 2, 3], max_new_tokens=90, force=force, **kw)
+    src = r.source.tolist()
+    runs = [len(x) for x in "".join(map(str, src)).split("0") if x]
+    assert len(r.handoffs) >= 5 and all(n == 2 for n in runs[:-1]) and runs[-1] <= 2
+    for (seg, step, cu) in r.handoffs:
+        assert r.tokens[seg - 3 - 1] == 10 and src[seg - 3 - 1] == 0     # the token before the segment is a small-model delimiter
+
+
 def _run(oracle, tiny, prompt, force, n1=3, max_new=10, keep=False, eos=-1, large=True):
     return oracle.generate_spec(tiny[0], tiny[1] if large else None, prompt, delimiter_id=10,
                                 keyword_ids=[11, 12, 13], n1=n1, keep_probe=keep, eos_id=eos,
