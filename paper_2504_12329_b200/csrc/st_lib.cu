@@ -78,6 +78,17 @@ struct st_model {
     CUtensorMap map_lm{};                  // LM head in 128-row tiles (batched decode)
     int32_t *row_slot = nullptr, *row_pos = nullptr;   // device [max_rows]: sequence and position of every row of a batched decode pass
     float *batch_logits = nullptr;         // [max_rows][vocab], allocated on first use
+    struct BatchGraph {                    // a captured batched decode pass, keyed by everything baked into its nodes
+        int m_upper, vlimit;
+        const int32_t *tok;
+        const StepDesc *desc;
+        float *logits;
+        int32_t *argmax;
+        cudaGraphExec_t exec;
+        int64_t launches;
+    };
+    std::vector<BatchGraph> batch_graphs;
+    cudaStream_t cap_stream = nullptr;     // side stream the batched pass is captured on (the model's own may be the legacy stream)
     CUtensorMap *act_maps = nullptr;       // device [3 buffers][2 planes][8]: activation planes in boxes of 32 (j + 1) rows
     bool simt_gemm = false;                // debugging aid: multi-row projections on the CUDA cores
     bool simt_attn = false;                // debugging aid: multi-row attention on the CUDA cores
@@ -1046,6 +1057,54 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
     return ST_OK;
 }
 
+// A batched decode pass through a CUDA graph: the pass is ~13 kernels per layer whose arguments depend only on
+// device arrays (row tables, descriptor) and on the pointers in the key, so it is captured once per key and
+// replayed; the launch gaps between its short kernels go away.
+static int pass_rows_batch_graphed(st_model *m, const StepDesc *desc, const int32_t *tok, int m_upper, int ctx_upper, const SampleCtx &sc)
+{
+    static const bool off = [] { const char *e = getenv("ST_BATCH_GRAPH"); return e && e[0] == '0'; }();
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (off || cudaStreamIsCapturing(m->stream, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone)
+        return pass_rows(m, desc, tok, -1, m_upper, ctx_upper, true, sc, true);
+    for (auto &g : m->batch_graphs)
+        if (g.m_upper == m_upper && g.vlimit == sc.vlimit && g.tok == tok && g.desc == desc && g.logits == sc.logits_out &&
+            g.argmax == (sc.want_argmax ? sc.argmax_out : nullptr)) {
+            CK(cudaGraphLaunch(g.exec, m->stream));
+            g_launches += g.launches;
+            return ST_OK;
+        }
+    if (m->batch_graphs.size() >= 16) {
+        CK(cudaStreamSynchronize(m->stream));
+        for (auto &g : m->batch_graphs) cudaGraphExecDestroy(g.exec);
+        m->batch_graphs.clear();
+    }
+    const int64_t before = g_launches;
+    // captured on a side stream: the model's own stream may be the legacy default stream, which cannot be captured
+    if (!m->cap_stream) CK(cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking));
+    if (cudaStreamBeginCapture(m->cap_stream, cudaStreamCaptureModeRelaxed) != cudaSuccess) {
+        cudaGetLastError();
+        return pass_rows(m, desc, tok, -1, m_upper, ctx_upper, true, sc, true);
+    }
+    cudaStream_t own = m->stream;
+    m->stream = m->cap_stream;
+    const int rc = pass_rows(m, desc, tok, -1, m_upper, ctx_upper, true, sc, true);
+    m->stream = own;
+    cudaGraph_t graph = nullptr;
+    const cudaError_t e = cudaStreamEndCapture(m->cap_stream, &graph);
+    if (rc != ST_OK) {
+        if (graph) cudaGraphDestroy(graph);
+        return rc;
+    }
+    CK(e);
+    st_model::BatchGraph g{m_upper, sc.vlimit, tok, desc, sc.logits_out, sc.want_argmax ? sc.argmax_out : nullptr, nullptr, g_launches - before};
+    const cudaError_t ei = cudaGraphInstantiate(&g.exec, graph, 0);
+    cudaGraphDestroy(graph);
+    CK(ei);
+    m->batch_graphs.push_back(g);
+    CK(cudaGraphLaunch(g.exec, m->stream));
+    return ST_OK;
+}
+
 // ------------------------------------------------------------------------------------------------
 // C ABI
 // ------------------------------------------------------------------------------------------------
@@ -1103,6 +1162,8 @@ void st_model_destroy(st_model *m)
     if (!m) return;
     cudaStreamSynchronize(m->stream);
     destroy_gen_context(m);
+    for (auto &g : m->batch_graphs) cudaGraphExecDestroy(g.exec);
+    if (m->cap_stream) cudaStreamDestroy(m->cap_stream);
     for (void *p : m->allocations) {
         if (m->cfg.free) m->cfg.free(p, m->cfg.alloc_user);
         else cudaFree(p);
@@ -1298,7 +1359,7 @@ int st_decode_step(st_model *m, const int32_t *slots_host, const int32_t *tokens
             sc.logits_out = logits + (logits_dev ? (size_t)i0 * m->cfg.vocab : 0);
             sc.argmax_out = argmax_dev ? argmax_dev + i0 : nullptr;
             sc.want_argmax = argmax_dev != nullptr;
-            TRY(pass_rows(m, m->desc, tokens_dev, -1, (n + 31) / 32 * 32 > m->max_rows ? m->max_rows : (n + 31) / 32 * 32, ctx_upper, true, sc, true));
+            TRY(pass_rows_batch_graphed(m, m->desc, tokens_dev, (n + 31) / 32 * 32 > m->max_rows ? m->max_rows : (n + 31) / 32 * 32, ctx_upper, sc));
             for (int i = 0; i < n; ++i) m->seq_len[slots_host[i0 + i]] += 1;
             // the row tables and the descriptor are rewritten for the next chunk
             CK(cudaStreamSynchronize(m->stream));
@@ -1951,7 +2012,7 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
                 sc.vlimit = vlimit;
                 int m_upper = (rows + 31) / 32 * 32;
                 if (m_upper > m->max_rows) m_upper = m->max_rows;
-                rc = pass_rows(m, d_bdesc + a, d_rtok + (size_t)a * n, -1, m_upper, pl.max_ctx[a], true, sc, true);
+                rc = pass_rows_batch_graphed(m, d_bdesc + a, d_rtok + (size_t)a * n, m_upper, pl.max_ctx[a], sc);
                 if (rc != ST_OK) break;
                 batch_router_kernel<<<1, 64, 0, s>>>(d_gs, d_gb, d_rseq + (size_t)a * n, d_amax + (size_t)a * n, d_bdesc + a, d_descs,
                                                      small->status);
