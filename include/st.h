@@ -157,9 +157,10 @@ int st_generate_spec(st_model *small, st_model *large, const st_spec_params *par
  * routing st_generate_spec gives for that sequence alone (its logits differ by rounding: batched rows go
  * through the tensor-core passes).  When both models have a free sequence slot and KV pages for every sequence
  * (st_config.max_seqs >= n_seqs, max_tokens >= the sum of prompt + budget + 1), n_seqs <= 256 and no logits
- * trace is asked for, the sequences advance together in rounds: per round one batched decode pass per model over
- * the sequences that lack one token, and a multi-row pass for each sequence that ingests a prompt or catches up
- * after a handoff; the host reads only the shape of the next round, never a token.  outs[i].seconds is then the
+ * trace is asked for, the sequences advance together in rounds: per round one ragged pass per model whose rows are
+ * all the tokens its sequences lack (one per sequence in steady decode, a whole catch-up or prompt of up to 256
+ * tokens after a handoff or at the start; each row attends to its own sequence's pages), and chunked passes of
+ * its own for a sequence that lacks more than 256; the host reads only the shape of the next round, never a token.  outs[i].seconds is then the
  * time of the whole batch and outs[i].bytes_algorithmic what sequence i would move alone.  Otherwise the
  * sequences run one after the other through st_generate_spec (stops at the first failing one). */
 int st_generate_spec_batch(st_model *small, st_model *large, const st_spec_params *params, int32_t n_seqs,

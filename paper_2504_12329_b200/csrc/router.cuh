@@ -136,14 +136,14 @@ __device__ void router_step(GenState *g, const GenBuffers &b, int greedy, StepDe
     plan_next_pass(g, desc_small, desc_large);
 }
 
-// After a batched decode pass (several independent generations advanced together): row k's greedy token advances
-// the state of the sequence the row belongs to.
-__global__ void batch_router_kernel(GenState *gs, const GenBuffers *gb, const int32_t *row_seq, const int32_t *greedy,
-                                    const StepDesc *bdesc, StepDesc *descs, int32_t *status)
+// After a ragged pass (several independent generations advanced together): the greedy token of a sequence's
+// last row advances that sequence's state.
+__global__ void batch_router_kernel(GenState *gs, const GenBuffers *gb, const int32_t *pass_seq, const int32_t *pass_last,
+                                    const int32_t *n_pass_seq, const int32_t *greedy, StepDesc *descs, int32_t *status)
 {
-    for (int k = threadIdx.x; k < bdesc->m; k += blockDim.x) {
-        const int i = row_seq[k];
-        router_step(gs + i, gb[i], greedy[k], descs + 2 * i, descs + 2 * i + 1, status);
+    for (int k = threadIdx.x; k < *n_pass_seq; k += blockDim.x) {
+        const int i = pass_seq[k];
+        router_step(gs + i, gb[i], greedy[pass_last[k]], descs + 2 * i, descs + 2 * i + 1, status);
     }
 }
 
@@ -200,52 +200,70 @@ constexpr int kBatchMaxCatchups = 256;
 
 // What the host needs to launch the next round of passes; it never contains a token.
 struct BatchPlan {
-    int32_t n_dec[2];                       // rows of the batched decode pass of each model
+    int32_t n_dec[2];                       // rows of this round's ragged pass of each model
     int32_t n_cu;                           // sequences that need a multi-row pass of their own this round
     int32_t all_done;
-    int32_t max_ctx[2];                     // longest context among the decode rows of each model
+    int32_t max_ctx[2];                     // longest context among the rows of each model
     int32_t cu[kBatchMaxCatchups][5];       // sequence, model, rows, first position, samples (1) or only ingests (0)
 };
 
-// One thread walks the sequences in order: a sequence whose active model lacks exactly one token joins that
-// model's batched decode pass (row = its place in the list), any other gets a multi-row pass of its own.
-// row_* and bdesc: per model [2]; slots: [n_seqs][2]; descs: [n_seqs][2].
+// One thread builds the round.  Every live sequence lacks `pending` tokens on its active model (1 in steady
+// decode, more after a handoff or at the start).  Its tokens become consecutive rows of that model's ragged pass
+// -- row j sits at position kv_len + j of the sequence's own cache, the last of them is the one that samples --
+// as long as the pass has room; sequences that ingest more than one token are placed first so that the single
+// rows cannot crowd them out, and one that does not fit waits for the next round.  More pending tokens than a
+// pass has rows (a long prompt) go through the sequence's own chunked multi-row passes instead.
+// row_* and bdesc: per model [2]; slots: [n_seqs][2]; descs: [n_seqs][2]; row_tok: [2][max_rows];
+// pass_seq / pass_last: [2][n_seqs] sequences of each pass and their sampling rows; n_pass_seq: [2].
 __global__ void batch_plan_kernel(GenState *gs, const GenBuffers *gb, int n_seqs, const int32_t *slots, StepDesc *descs,
                                   int32_t *row_slot0, int32_t *row_pos0, int32_t *row_slot1, int32_t *row_pos1,
-                                  int32_t *row_tok /*[2][n_seqs]*/, int32_t *row_seq /*[2][n_seqs]*/, StepDesc *bdesc /*[2]*/,
+                                  int32_t *row_tok, int32_t *pass_seq, int32_t *pass_last, int32_t *n_pass_seq, StepDesc *bdesc,
                                   int max_rows, BatchPlan *plan)
 {
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
-    int n_dec[2] = {0, 0}, n_cu = 0, live = 0, max_ctx[2] = {1, 1};
-    for (int i = 0; i < n_seqs; ++i) {
-        GenState *g = gs + i;
-        if (g->done) continue;
-        ++live;
-        const int a = g->active;
-        const int pending = g->pos - g->kv_len[a];
-        if (pending == 1 && n_dec[a] < max_rows) {
-            const int k = n_dec[a]++;
-            (a ? row_slot1 : row_slot0)[k] = slots[2 * i + a];
-            (a ? row_pos1 : row_pos0)[k] = g->kv_len[a];
-            row_tok[a * n_seqs + k] = gb[i].tokens[g->pos - 1];
-            row_seq[a * n_seqs + k] = i;
+    int n_rows[2] = {0, 0}, n_in[2] = {0, 0}, n_cu = 0, live = 0, max_ctx[2] = {1, 1};
+    for (int round = 0; round < 2; ++round) {   // 0: sequences with several pending tokens, 1: with one
+        for (int i = 0; i < n_seqs; ++i) {
+            GenState *g = gs + i;
+            if (g->done) continue;
+            const int a = g->active;
+            const int pending = g->pos - g->kv_len[a];
+            if ((pending > 1) != (round == 0)) continue;
+            ++live;
+            if (pending > max_rows) {
+                if (n_cu < kBatchMaxCatchups) {
+                    plan_next_pass(g, descs + 2 * i, descs + 2 * i + 1);
+                    int32_t *c = plan->cu[n_cu++];
+                    c[0] = i;
+                    c[1] = a;
+                    c[2] = g->next_m;
+                    c[3] = g->kv_len[a];
+                    c[4] = g->next_emit;
+                }
+                continue;
+            }
+            if (pending < 1 || n_rows[a] + pending > max_rows) continue;   // no room this round
+            const int r0 = n_rows[a];
+            int32_t *rs = a ? row_slot1 : row_slot0, *rp = a ? row_pos1 : row_pos0;
+            for (int j = 0; j < pending; ++j) {
+                rs[r0 + j] = slots[2 * i + a];
+                rp[r0 + j] = g->kv_len[a] + j;
+                row_tok[a * max_rows + r0 + j] = gb[i].tokens[g->kv_len[a] + j];
+            }
+            n_rows[a] += pending;
+            pass_seq[a * n_seqs + n_in[a]] = i;
+            pass_last[a * n_seqs + n_in[a]] = r0 + pending - 1;
+            ++n_in[a];
             if (g->pos > max_ctx[a]) max_ctx[a] = g->pos;
-        } else if (pending > 1 && n_cu < kBatchMaxCatchups) {
-            plan_next_pass(g, descs + 2 * i, descs + 2 * i + 1);
-            int32_t *c = plan->cu[n_cu++];
-            c[0] = i;
-            c[1] = a;
-            c[2] = g->next_m;
-            c[3] = g->kv_len[a];
-            c[4] = g->next_emit;
-        }   // (a sequence that found no room waits for the next round)
+        }
     }
     for (int a = 0; a < 2; ++a) {
         bdesc[a].pos0 = 0;
-        bdesc[a].m = n_dec[a];
+        bdesc[a].m = n_rows[a];
         bdesc[a].tok_off = 0;
         bdesc[a].emit = 1;
-        plan->n_dec[a] = n_dec[a];
+        n_pass_seq[a] = n_in[a];
+        plan->n_dec[a] = n_rows[a];
         plan->max_ctx[a] = max_ctx[a];
     }
     plan->n_cu = n_cu;

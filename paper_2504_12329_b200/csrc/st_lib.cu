@@ -1903,7 +1903,10 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
         auto take = [&](size_t bytes) { off = (off + 255) & ~(size_t)255; const size_t o = off; off += bytes; return o; };
         const size_t o_gs = take(n * sizeof(GenState)), o_gb = take(n * sizeof(GenBuffers)), o_slots = take(2 * n * sizeof(int32_t));
         const size_t o_descs = take(2 * n * sizeof(StepDesc)), o_bdesc = take(2 * sizeof(StepDesc));
-        const size_t o_rtok = take(2 * n * sizeof(int32_t)), o_rseq = take(2 * n * sizeof(int32_t)), o_amax = take(2 * n * sizeof(int32_t));
+        int max_chunk = small->max_rows;   // rows of one pass
+        if (large && large->max_rows < max_chunk) max_chunk = large->max_rows;
+        const size_t o_rtok = take(2 * (size_t)max_chunk * sizeof(int32_t)), o_amax = take(2 * (size_t)max_chunk * sizeof(int32_t));
+        const size_t o_pseq = take(2 * n * sizeof(int32_t)), o_plast = take(2 * n * sizeof(int32_t)), o_npass = take(2 * sizeof(int32_t));
         const size_t o_plan = take(sizeof(BatchPlan)), o_cls = take((size_t)vlimit);
         std::vector<size_t> o_tok(n), o_src(n), o_emt(n), o_emf(n), o_ema(n), o_ems(n), o_hand(n), o_force(n);
         for (int i = 0; i < n; ++i) {
@@ -1921,15 +1924,14 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
         if (cudaMallocHost(&plan_host, sizeof(BatchPlan)) != cudaSuccess) { cudaGetLastError(); rc = ST_ERR_OOM; break; }
         d_gs = (GenState *)(arena + o_gs);
         GenBuffers *d_gb = (GenBuffers *)(arena + o_gb);
-        int32_t *d_slots = (int32_t *)(arena + o_slots), *d_rtok = (int32_t *)(arena + o_rtok), *d_rseq = (int32_t *)(arena + o_rseq);
+        int32_t *d_slots = (int32_t *)(arena + o_slots), *d_rtok = (int32_t *)(arena + o_rtok), *d_pseq = (int32_t *)(arena + o_pseq);
+        int32_t *d_plast = (int32_t *)(arena + o_plast), *d_npass = (int32_t *)(arena + o_npass);
         int32_t *d_amax = (int32_t *)(arena + o_amax);
         StepDesc *d_descs = (StepDesc *)(arena + o_descs), *d_bdesc = (StepDesc *)(arena + o_bdesc);
         BatchPlan *d_plan = (BatchPlan *)(arena + o_plan);
         uint8_t *d_cls = arena + o_cls;
         std::vector<uint8_t> cls(vlimit, 0);
         for (int i = 0; i < P->n_keywords; ++i) cls[P->keyword_ids[i]] |= kClsKeyword;
-        int max_chunk = small->max_rows;
-        if (large && large->max_rows < max_chunk) max_chunk = large->max_rows;
         for (int i = 0; i < n; ++i) {
             GenState &g = gs[i];
             g = GenState{};
@@ -1991,7 +1993,7 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
         for (int64_t round = 0; round < round_cap && rc == ST_OK; ++round) {
             batch_plan_kernel<<<1, 1, 0, s>>>(d_gs, d_gb, n, d_slots, d_descs, small->row_slot, small->row_pos,
                                               large ? large->row_slot : small->row_slot, large ? large->row_pos : small->row_pos,
-                                              d_rtok, d_rseq, d_bdesc, max_chunk, d_plan);
+                                              d_rtok, d_pseq, d_plast, d_npass, d_bdesc, max_chunk, d_plan);
             ++g_launches;
             if (cudaMemcpyAsync(plan_host, d_plan, sizeof(BatchPlan), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
                 cudaStreamSynchronize(s) != cudaSuccess) {
@@ -2007,15 +2009,15 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
                 if (rows <= 0 || !m) continue;
                 SampleCtx sc{};
                 sc.logits_out = m->batch_logits;
-                sc.argmax_out = d_amax + (size_t)a * n;
+                sc.argmax_out = d_amax + (size_t)a * max_chunk;
                 sc.want_argmax = true;
                 sc.vlimit = vlimit;
                 int m_upper = (rows + 31) / 32 * 32;
                 if (m_upper > m->max_rows) m_upper = m->max_rows;
-                rc = pass_rows_batch_graphed(m, d_bdesc + a, d_rtok + (size_t)a * n, m_upper, pl.max_ctx[a], sc);
+                rc = pass_rows_batch_graphed(m, d_bdesc + a, d_rtok + (size_t)a * max_chunk, m_upper, pl.max_ctx[a], sc);
                 if (rc != ST_OK) break;
-                batch_router_kernel<<<1, 64, 0, s>>>(d_gs, d_gb, d_rseq + (size_t)a * n, d_amax + (size_t)a * n, d_bdesc + a, d_descs,
-                                                     small->status);
+                batch_router_kernel<<<1, 64, 0, s>>>(d_gs, d_gb, d_pseq + (size_t)a * n, d_plast + (size_t)a * n, d_npass + a,
+                                                     d_amax + (size_t)a * max_chunk, d_descs, small->status);
                 ++g_launches;
                 if (cudaGetLastError() != cudaSuccess) rc = ST_ERR_INTERNAL;
             }
