@@ -213,12 +213,14 @@ struct BatchPlan {
 // as long as the pass has room; sequences that ingest more than one token are placed first so that the single
 // rows cannot crowd them out, and one that does not fit waits for the next round.  More pending tokens than a
 // pass has rows (a long prompt) go through the sequence's own chunked multi-row passes instead.
+// min_target_rows: the target's pass is skipped this round when it would hold fewer rows and the speculative model
+// has work (sequences do not interact, so the order in which they advance does not change any result).
 // row_* and bdesc: per model [2]; slots: [n_seqs][2]; descs: [n_seqs][2]; row_tok: [2][max_rows];
 // pass_seq / pass_last: [2][n_seqs] sequences of each pass and their sampling rows; n_pass_seq: [2].
 __global__ void batch_plan_kernel(GenState *gs, const GenBuffers *gb, int n_seqs, const int32_t *slots, StepDesc *descs,
                                   int32_t *row_slot0, int32_t *row_pos0, int32_t *row_slot1, int32_t *row_pos1,
                                   int32_t *row_tok, int32_t *pass_seq, int32_t *pass_last, int32_t *n_pass_seq, StepDesc *bdesc,
-                                  int max_rows, BatchPlan *plan)
+                                  int max_rows, int min_target_rows, BatchPlan *plan)
 {
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     int n_rows[2] = {0, 0}, n_in[2] = {0, 0}, n_cu = 0, live = 0, max_ctx[2] = {1, 1};
@@ -257,6 +259,9 @@ __global__ void batch_plan_kernel(GenState *gs, const GenBuffers *gb, int n_seqs
             if (g->pos > max_ctx[a]) max_ctx[a] = g->pos;
         }
     }
+    // A pass of the target costs several passes of the speculative model whatever its row count: while the
+    // speculative model has rows and the target only a few, the target's sequences wait and their rows accumulate.
+    if (n_rows[1] > 0 && n_rows[1] < min_target_rows && n_rows[0] > 0) n_rows[1] = n_in[1] = 0;
     for (int a = 0; a < 2; ++a) {
         bdesc[a].pos0 = 0;
         bdesc[a].m = n_rows[a];

@@ -1989,11 +1989,14 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
         int64_t sum_new = 0;
         for (int i = 0; i < n; ++i) sum_new += mnew[i];
         const int64_t round_cap = 4 * (sum_new + 4ll * n + 16) + 4ll * n * (longest / max_chunk + 2);
+        // rows the target's pass waits for while the speculative model has work: an eighth of the sequences
+        int min_target_rows = n / 8;
+        if (const char *e = getenv("ST_BATCH_TARGET_MIN")) min_target_rows = atoi(e);   // tuning aid
         bool finished = false;
         for (int64_t round = 0; round < round_cap && rc == ST_OK; ++round) {
             batch_plan_kernel<<<1, 1, 0, s>>>(d_gs, d_gb, n, d_slots, d_descs, small->row_slot, small->row_pos,
                                               large ? large->row_slot : small->row_slot, large ? large->row_pos : small->row_pos,
-                                              d_rtok, d_pseq, d_plast, d_npass, d_bdesc, max_chunk, d_plan);
+                                              d_rtok, d_pseq, d_plast, d_npass, d_bdesc, max_chunk, min_target_rows, d_plan);
             ++g_launches;
             if (cudaMemcpyAsync(plan_host, d_plan, sizeof(BatchPlan), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
                 cudaStreamSynchronize(s) != cudaSuccess) {
