@@ -379,3 +379,32 @@ def test_every_delimiter_variant_on_device(B, oracle):
                 assert got.emission_argmax[t] == want.emission_argmax[t]
     gs.close()
     gl.close()
+
+
+def test_batched_generation_fallbacks_and_edges(B, oracle):
+    """Calls that do not qualify for the rounds (too few sequence slots or KV pages) run the sequences one by one with
+    the same results; an empty batch and a single sequence are fine; a prompt longer than a pass takes its own chunks."""
+    S, L = shape_dict(W.TINY_S), shape_dict(W.TINY_L)
+    kw = dict(delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=4)
+    prompts = [W.prompt_ids(40 + i, n, 1024) for i, n in enumerate([300, 7, 33])]       # 300 > 256 rows of a pass
+    forces = [W.full_forcing(50 + i, 120, 1024, mean_interval=6, keyword_rate=0.6) for i in range(3)]
+    os_, ol = oracle.Model(oracle.Config(**S), 0, 0), oracle.Model(oracle.Config(**L), 0, 1)
+    wants = [oracle.generate_spec(os_, ol, prompts[i], max_new_tokens=50, force=forces[i], **kw) for i in range(3)]
+    roomy = (B.Model(S, seed=0, tag=0, max_seqs=3, max_tokens=2048), B.Model(L, seed=0, tag=1, max_seqs=3, max_tokens=2048))
+    one_slot = (B.Model(S, seed=0, tag=0, max_seqs=1, max_tokens=2048), B.Model(L, seed=0, tag=1, max_seqs=1, max_tokens=2048))
+    few_pages = (B.Model(S, seed=0, tag=0, max_seqs=3, max_tokens=512), B.Model(L, seed=0, tag=1, max_seqs=3, max_tokens=512))
+    for gs, gl in (roomy, one_slot, few_pages):
+        got = B.st_generate_spec_batch(gs, gl, prompts, max_new_tokens=50, forces=forces, **kw)
+        for want, g in zip(wants, got):
+            _assert_routing_equal(want, g)
+        assert B.st_generate_spec_batch(gs, gl, [], max_new_tokens=5, **kw) == []
+        single = B.st_generate_spec_batch(gs, gl, prompts[1:2], max_new_tokens=50, forces=forces[1:2], **kw)
+        _assert_routing_equal(wants[1], single[0])
+        # every slot is free again
+        for m in (gs, gl):
+            slots = [m.st_seq_alloc() for _ in range(1)]
+            m.st_seq_free(slots[0])
+    assert len({r.seconds for r in B.st_generate_spec_batch(*roomy, prompts, max_new_tokens=50, forces=forces, **kw)}) == 1
+    for gs, gl in (roomy, one_slot, few_pages):
+        gs.close()
+        gl.close()
