@@ -155,7 +155,7 @@ __global__ void splitk_reduce_kernel(const StepDesc *desc, const float *Ws, int 
 }
 
 template <int EPI>
-__global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW,                                                       const TcGemmParams p)
+__global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const TcGemmParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t s_full[8], s_empty[8], s_acc;
