@@ -41,6 +41,10 @@ class _SpecParams(C.Structure):
         ("n1", C.c_int32), ("keep_probe", C.c_int32), ("eos_id", C.c_int32), ("vocab_limit", C.c_int32),
         ("max_new_tokens", C.c_int32),
         ("takeover_every_delimiter", C.c_int32), ("target_first_n", C.c_int32),
+        ("affirmation_ids", C.POINTER(C.c_int32)), ("n_affirmation", C.c_int32),
+        ("verification_ids", C.POINTER(C.c_int32)), ("n_verification", C.c_int32),
+        ("n2", C.c_int32), ("neg_threshold", C.c_int32), ("n3", C.c_int32),
+        ("aux_ids", C.POINTER(C.c_int32)), ("n_aux", C.c_int32),
     ]
 
 
@@ -59,6 +63,7 @@ class _SpecResult(C.Structure):
         ("cap_steps", C.c_int32), ("n_steps", C.c_int32),
         ("kv_len_small", C.c_int32), ("kv_len_large", C.c_int32),
         ("logits_trace", C.POINTER(C.c_double)), ("trace_first_step", C.c_int32), ("trace_n_steps", C.c_int32),
+        ("handoff_kinds", C.POINTER(C.c_uint8)),
     ]
 
 
@@ -255,18 +260,25 @@ class SpecResult:
     kv_len_large: int
     logits_trace: np.ndarray | None
     rc: int
+    handoff_kinds: list = None   # 1 reflection / affirmation, 2 verification, 3 excessive reflection
 
 
 def generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id: int, keyword_ids, n1: int = 20,
                   keep_probe: bool = False, eos_id: int = -1, vocab_limit: int = 0, max_new_tokens: int,
                   force=None, trace_first_step: int = 0, trace_n_steps: int = 0,
-                  takeover_every_delimiter: bool = False, target_first_n: int = 0) -> SpecResult:
+                  takeover_every_delimiter: bool = False, target_first_n: int = 0, affirmation_ids=(),
+                  verification_ids=(), n2: int = 125, neg_threshold: int = -1, n3: int = 125, aux_ids=()) -> SpecResult:
     prompt = np.ascontiguousarray(prompt, dtype=np.int32)
+    aff = np.ascontiguousarray(affirmation_ids, dtype=np.int32)
+    ver = np.ascontiguousarray(verification_ids, dtype=np.int32)
+    aux = np.ascontiguousarray(aux_ids, dtype=np.int32)
+    ip = lambda a: a.ctypes.data_as(C.POINTER(C.c_int32))
     kw = np.ascontiguousarray(keyword_ids, dtype=np.int32)
     if vocab_limit <= 0:
         vocab_limit = small.cfg.vocab if large is None else min(small.cfg.vocab, large.cfg.vocab)
     P = _SpecParams(delimiter_id, kw.ctypes.data_as(C.POINTER(C.c_int32)), kw.size, n1, int(keep_probe), eos_id,
-                    vocab_limit, max_new_tokens, int(takeover_every_delimiter), int(target_first_n))
+                    vocab_limit, max_new_tokens, int(takeover_every_delimiter), int(target_first_n),
+                    ip(aff), aff.size, ip(ver), ver.size, n2, neg_threshold, n3, ip(aux), aux.size)
     cap_steps = 2 * max_new_tokens + 8
     tokens = np.zeros(max_new_tokens + 1, dtype=np.int32)
     source = np.zeros(max_new_tokens + 1, dtype=np.uint8)
@@ -292,6 +304,8 @@ def generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id: in
     R.logits_trace = trace.ctypes.data_as(C.POINTER(C.c_double)) if trace is not None else None
     R.trace_first_step = trace_first_step
     R.trace_n_steps = trace_n_steps
+    kinds = np.zeros(max_new_tokens + 1, dtype=np.uint8)
+    R.handoff_kinds = kinds.ctypes.data_as(C.POINTER(C.c_uint8))
     f = None if force is None else np.ascontiguousarray(force, dtype=np.int32)
     rc = lib().orc_generate_spec(small.h, large.h if large is not None else None, C.byref(P), _p(prompt), prompt.size,
                                  None if f is None else _p(f), 0 if f is None else f.size, C.byref(R))
@@ -299,4 +313,4 @@ def generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id: in
     return SpecResult(tokens[:n].copy(), source[:n].copy(),
                       [(hand[i].seg_start, hand[i].step, hand[i].catchup_len) for i in range(R.n_handoffs)],
                       e_tok[:s].copy(), e_src[:s].copy(), e_fed[:s].copy(), e_arg[:s].copy(), e_mar[:s].copy(),
-                      R.kv_len_small, R.kv_len_large, trace, rc)
+                      R.kv_len_small, R.kv_len_large, trace, rc, kinds[:R.n_handoffs].tolist())

@@ -486,6 +486,18 @@ typedef struct {
     int32_t takeover_every_delimiter; /* 1: no keyword test; the target writes the n1 tokens after every
                                          delimiter the speculative model writes */
     int32_t target_first_n;           /* > 0: the target writes the first target_first_n tokens (paper: 100) */
+    /* Section 3, takeovers (1)-(3) in token-id form (the token sampled right after a delimiter stands for
+     * the sentence that follows it).  All off when the sets are empty and neg_threshold < 0. */
+    const int32_t *affirmation_ids;   /* (1): an affirmation cue hands over n1 tokens like a reflection cue */
+    int32_t n_affirmation;
+    const int32_t *verification_ids;  /* (2): a verification cue after a delimiter, whoever samples it: n2 target tokens */
+    int32_t n_verification;
+    int32_t n2;                       /* paper: 125 */
+    int32_t neg_threshold;            /* (3): once more than this many reflection cues were sampled by the speculative
+                                         model (paper: 15), aux_ids are inserted and the target writes n3 tokens; < 0: off */
+    int32_t n3;                       /* paper: 125 */
+    const int32_t *aux_ids;           /* the auxiliary sentence of (3) */
+    int32_t n_aux;
 } orc_spec_params;
 
 typedef struct { int32_t seg_start, step, catchup_len; } orc_handoff;
@@ -505,6 +517,7 @@ typedef struct {
     int32_t kv_len_small, kv_len_large;
     double *logits_trace;       /* optional [trace_n_steps][vocab_limit] */
     int32_t trace_first_step, trace_n_steps;
+    uint8_t *handoff_kinds;     /* optional [cap_handoffs]: 1 reflection/affirmation, 2 verification, 3 excessive reflection */
 } orc_spec_result;
 
 /* The speculative model writes until it samples a reflection keyword right
@@ -517,6 +530,7 @@ int orc_generate_spec(const orc_model *small, const orc_model *large, const orc_
                       orc_spec_result *R)
 {
     if (prompt_len < 1 || P->max_new_tokens < 0) return -1;
+    if ((P->n_verification > 0 && P->n2 < 1) || (P->neg_threshold >= 0 && P->n3 < 1)) return -1;
     int64_t cap = (int64_t)prompt_len + P->max_new_tokens + 1;
     const orc_model *M[2] = {small, large};
     orc_kv *kv[2] = {orc_kv_create(small, cap), large ? orc_kv_create(large, cap) : NULL};
@@ -525,7 +539,7 @@ int orc_generate_spec(const orc_model *small, const orc_model *large, const orc_
     int vmax = small->c.vocab;
     if (large && large->c.vocab > vmax) vmax = large->c.vocab;
     double *z = (double *)malloc((size_t)vmax * sizeof(double));
-    int active = 0, remaining = 0, rc = 0;
+    int active = 0, remaining = 0, rc = 0, neg_count = 0;
     int32_t pos = prompt_len, t = 0, generated = 0;
     R->n_tokens = R->n_handoffs = R->n_steps = 0;
     if (large && P->target_first_n > 0) {   /* the target opens the answer */
@@ -549,26 +563,62 @@ int orc_generate_spec(const orc_model *small, const orc_model *large, const orc_
             memcpy(R->logits_trace + (size_t)(t - R->trace_first_step) * P->vocab_limit, z, (size_t)P->vocab_limit * sizeof(double));
         ++t;
         R->n_steps = t;
-        int is_kw = 0;
+        int is_kw = 0, is_aff = 0, is_ver = 0;
         for (int i = 0; i < P->n_keywords; ++i) is_kw |= (P->keyword_ids[i] == tok);
-        if (large && a == 0 && !P->takeover_every_delimiter && tokens[pos - 1] == P->delimiter_id && is_kw) {
-            if (P->keep_probe) {
-                tokens[pos] = tok;
-                if (generated >= R->cap_tokens) { rc = -3; break; }
-                R->tokens[generated] = tok;
-                R->source[generated] = 0;
-                ++pos; ++generated;
-                R->n_tokens = generated;
+        for (int i = 0; i < P->n_affirmation; ++i) is_aff |= (P->affirmation_ids[i] == tok);
+        for (int i = 0; i < P->n_verification; ++i) is_ver |= (P->verification_ids[i] == tok);
+        const int after_delim = tokens[pos - 1] == P->delimiter_id;
+        if (large && a == 0 && !P->takeover_every_delimiter && after_delim) {
+            /* the speculative model opened a sentence: classify its first token */
+            if (is_kw && P->neg_threshold >= 0) ++neg_count;
+            int kind = 0, len = 0;
+            if (P->neg_threshold >= 0 && neg_count > P->neg_threshold) { kind = 3; len = P->n3; }   /* (3) */
+            else if (is_ver) { kind = 2; len = P->n2; }                                             /* (2) */
+            else if (is_kw || is_aff) { kind = 1; len = P->n1; }                                    /* (1) */
+            if (kind) {
+                int stop = 0;
+                if (P->keep_probe) {
+                    if (generated >= R->cap_tokens) { rc = -3; break; }
+                    tokens[pos] = tok;
+                    R->tokens[generated] = tok;
+                    R->source[generated] = 0;
+                    ++pos; ++generated;
+                    R->n_tokens = generated;
+                    if (tok == P->eos_id) stop = 1;
+                }
+                if (kind == 3) {   /* the auxiliary sentence goes into the output, then the target continues */
+                    for (int i = 0; i < P->n_aux && generated < P->max_new_tokens && !stop; ++i) {
+                        if (generated >= R->cap_tokens) { rc = -3; break; }
+                        tokens[pos] = P->aux_ids[i];
+                        R->tokens[generated] = P->aux_ids[i];
+                        R->source[generated] = 2;
+                        ++pos; ++generated;
+                        R->n_tokens = generated;
+                    }
+                    if (rc) break;
+                    neg_count = 0;
+                }
+                if (R->n_handoffs >= R->cap_handoffs) { rc = -3; break; }
+                R->handoffs[R->n_handoffs].seg_start = pos;
+                R->handoffs[R->n_handoffs].step = t - 1;
+                R->handoffs[R->n_handoffs].catchup_len = pos - (int32_t)kv[1]->len;
+                if (R->handoff_kinds) R->handoff_kinds[R->n_handoffs] = (uint8_t)kind;
+                R->n_handoffs++;
+                active = 1;
+                remaining = len;
+                if (stop) break;
+                continue;
             }
+        }
+        if (large && a == 1 && after_delim && is_ver && remaining < P->n2) {
+            /* (2) applies to the target's own sentences too: from this token on it writes n2 tokens */
             if (R->n_handoffs >= R->cap_handoffs) { rc = -3; break; }
             R->handoffs[R->n_handoffs].seg_start = pos;
             R->handoffs[R->n_handoffs].step = t - 1;
-            R->handoffs[R->n_handoffs].catchup_len = pos - (int32_t)kv[1]->len;
+            R->handoffs[R->n_handoffs].catchup_len = 0;
+            if (R->handoff_kinds) R->handoff_kinds[R->n_handoffs] = 2;
             R->n_handoffs++;
-            active = 1;
-            remaining = P->n1;
-            if (P->keep_probe && tok == P->eos_id) break;
-            continue;
+            remaining = P->n2;
         }
         if (generated >= R->cap_tokens) { rc = -3; break; }
         tokens[pos] = tok;

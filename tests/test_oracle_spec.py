@@ -17,7 +17,9 @@ def _trace(name):
             if not line or line.startswith("#"):
                 continue
             k, v = line.split("=")
-            if k == "handoffs":
+            if k == "handoff_kinds":
+                out[k] = [int(x) for x in v.split(",")]
+            elif k == "handoffs":
                 out[k] = [tuple(int(x) for x in h.split(":")) for h in v.split(",")]
             elif "," in v:
                 out[k] = [int(x) for x in v.split(",")]
@@ -59,6 +61,56 @@ def test_hand_traced_stream_every_delimiter(oracle, tiny):
     assert r.emission_source.tolist() == T["emission_source"]
     assert r.emission_fed.tolist() == T["emission_fed"]
     assert (r.kv_len_small, r.kv_len_large) == (T["kv_len_small"], T["kv_len_large"])
+
+
+RULES = dict(delimiter_id=10, keyword_ids=[11, 12, 13], affirmation_ids=[14], verification_ids=[13, 15], n1=2, n2=3, n3=2,
+             neg_threshold=1, aux_ids=[40, 41])
+
+
+def test_hand_traced_stream_three_takeovers(oracle, tiny):
+    T = _trace("handoff_trace_three_takeovers.txt")
+    r = oracle.generate_spec(tiny[0], tiny[1], [1, 2, 3], max_new_tokens=15, force=T["force"], **RULES)
+    assert r.rc == 0
+    assert r.tokens.tolist() == T["tokens"]
+    assert r.source.tolist() == T["source"]
+    assert r.handoffs == T["handoffs"]
+    assert r.handoff_kinds == T["handoff_kinds"]
+    assert r.emission_source.tolist() == T["emission_source"]
+    assert r.emission_fed.tolist() == T["emission_fed"]
+    assert (r.kv_len_small, r.kv_len_large) == (T["kv_len_small"], T["kv_len_large"])
+
+
+def test_three_takeovers_reduce_and_hold_invariants(oracle, tiny):
+    base = dict(delimiter_id=10, keyword_ids=[11, 12, 13], n1=3)
+    force = W.full_forcing(77, 400, 1024, mean_interval=5, keyword_rate=0.7)
+    plain = oracle.generate_spec(tiny[0], tiny[1], [1, 2, 3], max_new_tokens=150, force=force, **base)
+    # empty extra sets and a switched-off counter are the plain rule
+    same = oracle.generate_spec(tiny[0], tiny[1], [1, 2, 3], max_new_tokens=150, force=force, affirmation_ids=[],
+                                verification_ids=[], neg_threshold=-1, aux_ids=[40], **base)
+    assert same.tokens.tolist() == plain.tokens.tolist() and same.handoffs == plain.handoffs
+    assert set(plain.handoff_kinds) == {1}
+    # with the counter on, every (3) follows exactly neg_threshold + 1 reflection cues of the small model since the last (3)
+    r = oracle.generate_spec(tiny[0], tiny[1], [1, 2, 3], max_new_tokens=150, force=force, neg_threshold=2, n3=4,
+                             aux_ids=[40, 41, 42], **base)
+    assert 3 in r.handoff_kinds and r.rc == 0
+    cues = 0
+    hk = dict(zip([h[1] for h in r.handoffs], r.handoff_kinds))
+    for t, (tok, src) in enumerate(zip(r.emission_tokens.tolist(), r.emission_source.tolist())):
+        if t in hk and src == 0:
+            if tok in (11, 12, 13):
+                cues += 1
+            if hk[t] == 3:
+                assert cues == 3
+                cues = 0
+    src = r.source.tolist()
+    toks = r.tokens.tolist()
+    for (seg, step, cu), kind in zip(r.handoffs, r.handoff_kinds):
+        i = seg - 3                      # index into the generated tokens
+        if kind == 3 and i + 4 <= len(src):
+            assert toks[i - 3:i] == [40, 41, 42] and src[i - 3:i] == [2, 2, 2]
+            assert src[i:i + 4] == [1, 1, 1, 1]
+    # n_steps = tokens written by a model + dropped cues
+    assert len(r.emission_tokens) == sum(1 for x in src if x != 2) + sum(1 for k, h in zip(r.handoff_kinds, r.handoffs) if h[2] > 0 or k != 2)
 
 
 def test_every_delimiter_edge_cases(oracle, tiny):
