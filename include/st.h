@@ -83,6 +83,22 @@ typedef struct {
     int32_t takeover_every_delimiter; /* 1: no keyword test -- whenever the speculative model writes the delimiter,
                                          the target writes the next n1 tokens */
     int32_t target_first_n;           /* > 0: the target writes the first target_first_n tokens (paper: 100) */
+    /* The other takeovers of Section 3, in token-id form: the token sampled right after a delimiter stands for
+     * the sentence that follows it.  All off with empty sets and neg_threshold < 0.  Precedence when several
+     * apply to one token: (3), then (2), then (1). */
+    const int32_t *affirmation_ids;   /* (1) Affirmation cues: hand over n1 tokens like reflection keywords */
+    int32_t n_affirmation;
+    const int32_t *verification_ids;  /* (2) Verification cues: sampled after a delimiter by the speculative model -> the
+                                         target writes n2 tokens; sampled by the target -> it writes n2 tokens from there */
+    int32_t n_verification;
+    int32_t n2;                       /* paper: 125; >= 1 when verification_ids is not empty */
+    int32_t neg_threshold;            /* (3) Excessive reflection: < 0 off; else, once the speculative model has sampled
+                                         more than this many reflection keywords after delimiters (paper: 15), aux_ids
+                                         are written into the output (source 2), the target writes n3 tokens and the
+                                         count restarts */
+    int32_t n3;                       /* paper: 125; >= 1 when neg_threshold >= 0 */
+    const int32_t *aux_ids;           /* host, the auxiliary sentence, at most 64 ids */
+    int32_t n_aux;
 } st_spec_params;
 
 typedef struct {
@@ -96,7 +112,7 @@ typedef struct {
  * forced) token; a dropped keyword still counts as a step. */
 typedef struct {
     int32_t *tokens;          /* [cap_tokens] tokens written after the prompt */
-    uint8_t *source;          /* [cap_tokens] 0 = speculative model, 1 = target model */
+    uint8_t *source;          /* [cap_tokens] 0 = speculative model, 1 = target model, 2 = inserted auxiliary token */
     int32_t cap_tokens, n_tokens;
     st_handoff *handoffs;     /* [cap_handoffs] */
     int32_t cap_handoffs, n_handoffs;
@@ -110,6 +126,8 @@ typedef struct {
     int32_t trace_first_step, trace_n_steps;
     double seconds;           /* device time of the generation (CUDA events) */
     int64_t bytes_algorithmic; /* weights + KV bytes the passes had to move (sum over steps) */
+    uint8_t *handoff_kinds;   /* optional [cap_handoffs]: which takeover each handoff was (1 reflection / affirmation or
+                                 every-delimiter, 2 verification, 3 excessive reflection) */
 } st_spec_result;
 
 /* Create a model with seeded random-init weights: element idx of tensor tid of model `tag` is

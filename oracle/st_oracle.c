@@ -634,6 +634,7 @@ int orc_generate_spec(const orc_model *small, const orc_model *large, const orc_
             R->handoffs[R->n_handoffs].seg_start = pos;
             R->handoffs[R->n_handoffs].step = t - 1;
             R->handoffs[R->n_handoffs].catchup_len = pos - (int32_t)kv[1]->len;
+            if (R->handoff_kinds) R->handoff_kinds[R->n_handoffs] = 1;
             R->n_handoffs++;
             active = 1;
             remaining = P->n1;

@@ -38,6 +38,10 @@ class StSpecParams(C.Structure):
         ("delimiter_id", C.c_int32), ("keyword_ids", C.POINTER(C.c_int32)), ("n_keywords", C.c_int32),
         ("n1", C.c_int32), ("keep_probe", C.c_int32), ("eos_id", C.c_int32), ("vocab_limit", C.c_int32),
         ("max_new_tokens", C.c_int32), ("takeover_every_delimiter", C.c_int32), ("target_first_n", C.c_int32),
+        ("affirmation_ids", C.POINTER(C.c_int32)), ("n_affirmation", C.c_int32),
+        ("verification_ids", C.POINTER(C.c_int32)), ("n_verification", C.c_int32),
+        ("n2", C.c_int32), ("neg_threshold", C.c_int32), ("n3", C.c_int32),
+        ("aux_ids", C.POINTER(C.c_int32)), ("n_aux", C.c_int32),
     ]
 
 
@@ -56,6 +60,7 @@ class StSpecResult(C.Structure):
         ("kv_len_small", C.c_int32), ("kv_len_large", C.c_int32),
         ("logits_trace", C.POINTER(C.c_float)), ("trace_first_step", C.c_int32), ("trace_n_steps", C.c_int32),
         ("seconds", C.c_double), ("bytes_algorithmic", C.c_int64),
+        ("handoff_kinds", C.POINTER(C.c_uint8)),
     ]
 
 
@@ -201,6 +206,7 @@ class SpecResult:
     seconds: float
     bytes_algorithmic: int
     n_steps: int
+    handoff_kinds: list = None   # 1 reflection / affirmation / every-delimiter, 2 verification, 3 excessive reflection
 
 
 class Model:
@@ -294,6 +300,7 @@ class _ResultBuffers:
         self.tokens = np.zeros(max_new_tokens + 1, dtype=np.int32)
         self.source = np.zeros(max_new_tokens + 1, dtype=np.uint8)
         self.hand = (StHandoff * max(self.cap_handoffs, 1))()
+        self.kinds = np.zeros(max(self.cap_handoffs, 1), dtype=np.uint8)
         n = max(self.cap_steps, 1)
         self.e_tok, self.e_fed, self.e_arg = (np.zeros(n, dtype=np.int32) for _ in range(3))
         self.e_src = np.zeros(n, dtype=np.uint8)
@@ -306,6 +313,7 @@ class _ResultBuffers:
         R.cap_tokens = self.tokens.size
         R.handoffs = C.cast(self.hand, C.POINTER(StHandoff))
         R.cap_handoffs = self.cap_handoffs
+        R.handoff_kinds = self.kinds.ctypes.data_as(C.POINTER(C.c_uint8))
         R.emission_tokens = self.e_tok.ctypes.data_as(C.POINTER(C.c_int32))
         R.emission_source = self.e_src.ctypes.data_as(C.POINTER(C.c_uint8))
         R.emission_fed = self.e_fed.ctypes.data_as(C.POINTER(C.c_int32))
@@ -321,19 +329,32 @@ class _ResultBuffers:
                           [(self.hand[i].seg_start, self.hand[i].step, self.hand[i].catchup_len)
                            for i in range(min(R.n_handoffs, self.cap_handoffs))],
                           self.e_tok[:s].copy(), self.e_src[:s].copy(), self.e_fed[:s].copy(), self.e_arg[:s].copy(),
-                          R.kv_len_small, R.kv_len_large, self.trace, R.seconds, R.bytes_algorithmic, R.n_steps)
+                          R.kv_len_small, R.kv_len_large, self.trace, R.seconds, R.bytes_algorithmic, R.n_steps,
+                          self.kinds[:min(R.n_handoffs, self.cap_handoffs)].tolist())
+
+
+def _spec_params(delimiter_id, keyword_ids, n1, keep_probe, eos_id, vocab_limit, max_new_tokens, takeover_every_delimiter,
+                 target_first_n, affirmation_ids=(), verification_ids=(), n2=125, neg_threshold=-1, n3=125, aux_ids=()):
+    """st_spec_params and the arrays it points at (keep both alive during the call)."""
+    arrs = [np.ascontiguousarray(a, dtype=np.int32) for a in (keyword_ids, affirmation_ids, verification_ids, aux_ids)]
+    ip = lambda a: a.ctypes.data_as(C.POINTER(C.c_int32))
+    kw, aff, ver, aux = arrs
+    P = StSpecParams(delimiter_id, ip(kw), kw.size, n1, int(keep_probe), eos_id, vocab_limit, max_new_tokens,
+                     int(takeover_every_delimiter), int(target_first_n), ip(aff), aff.size, ip(ver), ver.size, n2,
+                     neg_threshold, n3, ip(aux), aux.size)
+    return P, arrs
 
 
 def st_generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id: int, keyword_ids, n1: int = 20,
                      keep_probe: bool = False, eos_id: int = -1, vocab_limit: int = 0, max_new_tokens: int,
                      force=None, trace_first_step: int = 0, trace_n_steps: int = 0, cap_steps: int | None = None,
                      cap_handoffs: int | None = None, takeover_every_delimiter: bool = False,
-                     target_first_n: int = 0) -> SpecResult:
-    """Host buffers in, host buffers out: marshals the arguments of st_generate_spec."""
+                     target_first_n: int = 0, **rules) -> SpecResult:
+    """Host buffers in, host buffers out: marshals the arguments of st_generate_spec.  rules: affirmation_ids,
+    verification_ids, n2, neg_threshold, n3, aux_ids (the other takeovers of the paper's Section 3)."""
     prompt = np.ascontiguousarray(prompt, dtype=np.int32)
-    kw = np.ascontiguousarray(keyword_ids, dtype=np.int32)
-    P = StSpecParams(delimiter_id, kw.ctypes.data_as(C.POINTER(C.c_int32)), kw.size, n1, int(keep_probe), eos_id,
-                     vocab_limit, max_new_tokens, int(takeover_every_delimiter), int(target_first_n))
+    P, _keep = _spec_params(delimiter_id, keyword_ids, n1, keep_probe, eos_id, vocab_limit, max_new_tokens,
+                            takeover_every_delimiter, target_first_n, **rules)
     if vocab_limit <= 0:
         vocab_limit = small.vocab if large is None else min(small.vocab, large.vocab)
     bufs = _ResultBuffers(max_new_tokens, vocab_limit, trace_first_step, trace_n_steps, cap_steps, cap_handoffs)
@@ -348,13 +369,12 @@ def st_generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id:
 
 def st_generate_spec_batch(small: Model, large: Model | None, prompts, *, delimiter_id: int, keyword_ids, n1: int = 20,
                            keep_probe: bool = False, eos_id: int = -1, vocab_limit: int = 0, max_new_tokens,
-                           forces=None, takeover_every_delimiter: bool = False, target_first_n: int = 0) -> list:
+                           forces=None, takeover_every_delimiter: bool = False, target_first_n: int = 0, **rules) -> list:
     """prompts / forces: lists of per-sequence arrays; max_new_tokens: one int or a list per sequence."""
     n = len(prompts)
     budgets = [int(max_new_tokens)] * n if np.isscalar(max_new_tokens) else [int(x) for x in max_new_tokens]
-    kw = np.ascontiguousarray(keyword_ids, dtype=np.int32)
-    P = StSpecParams(delimiter_id, kw.ctypes.data_as(C.POINTER(C.c_int32)), kw.size, n1, int(keep_probe), eos_id,
-                     vocab_limit, max(budgets) if budgets else 0, int(takeover_every_delimiter), int(target_first_n))
+    P, _keep = _spec_params(delimiter_id, keyword_ids, n1, keep_probe, eos_id, vocab_limit, max(budgets) if budgets else 0,
+                            takeover_every_delimiter, target_first_n, **rules)
     if vocab_limit <= 0:
         vocab_limit = small.vocab if large is None else min(small.vocab, large.vocab)
     flat_p = np.ascontiguousarray(np.concatenate([np.asarray(p, dtype=np.int32) for p in prompts]) if n else np.zeros(0, np.int32))

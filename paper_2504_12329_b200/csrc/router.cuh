@@ -11,6 +11,8 @@
 namespace st {
 
 constexpr int kClsKeyword = 2;  // class-table bit of a reflection keyword
+constexpr int kClsAffirm = 4;   // ... of an affirmation cue
+constexpr int kClsVerify = 8;   // ... of a verification cue
 
 struct GenState {
     // --- accounting (64-bit fields first) ---
@@ -35,6 +37,8 @@ struct GenState {
     int32_t pass_cap;    // hard bound on passes (the device loop stops there)
     // --- parameters ---
     int32_t has_large, delimiter, n1, keep_probe, eos, vlimit, max_new, n_force;
+    int32_t n2, n3, neg_threshold, n_aux;   // takeovers (2) and (3): segment lengths, counter bound (< 0: off), auxiliary tokens
+    int32_t neg_count;                      // reflection cues the speculative model sampled since the last takeover (3)
     int32_t every_delim;   // 1: no keyword test; the target takes over after every delimiter the speculative model writes
     int32_t prompt_len, cap_steps, cap_handoffs, max_chunk;
     int32_t trace_first, trace_n;
@@ -46,6 +50,8 @@ struct GenBuffers {
     int32_t *em_tok, *em_fed, *em_arg;  // [cap_steps]
     uint8_t *em_src;           // [cap_steps]
     int32_t *handoffs;         // [cap_handoffs][3]
+    uint8_t *hand_kind;        // [cap_handoffs] 1 reflection/affirmation, 2 verification, 3 excessive reflection
+    const int32_t *aux;        // [n_aux] auxiliary sentence of takeover (3)
     const int32_t *force;      // [n_force]
     const uint8_t *cls;        // [vlimit] class bits per token id
     float *trace;              // [trace_n][vlimit] or null
@@ -90,8 +96,29 @@ __device__ void router_step(GenState *g, const GenBuffers &b, int greedy, StepDe
     }
     g->step = t + 1;
     if ((unsigned)tok >= (unsigned)g->vlimit) { atomicOr(status, DEV_BAD_TOKEN); tok = 0; }
-    const bool trigger = g->has_large && a == 0 && !g->every_delim && b.tokens[g->pos - 1] == g->delimiter && (b.cls[tok] & kClsKeyword);
-    if (trigger) {
+    // Takeovers of Section 3 in token-id form: the token sampled right after a delimiter stands for the sentence.
+    const int cls = b.cls[tok];
+    const bool after_delim = b.tokens[g->pos - 1] == g->delimiter;
+    int kind = 0, len = 0;
+    if (g->has_large && a == 0 && !g->every_delim && after_delim) {
+        if ((cls & kClsKeyword) && g->neg_threshold >= 0) g->neg_count++;
+        if (g->neg_threshold >= 0 && g->neg_count > g->neg_threshold) { kind = 3; len = g->n3; }   // (3) excessive reflection
+        else if (cls & kClsVerify) { kind = 2; len = g->n2; }                                       // (2) verification
+        else if (cls & (kClsKeyword | kClsAffirm)) { kind = 1; len = g->n1; }                       // (1) reflection / affirmation
+    }
+    auto log_handoff = [&](int seg_start, int catchup, int k) {
+        if (g->n_handoffs < g->cap_handoffs) {
+            int32_t *h = b.handoffs + 3 * g->n_handoffs;
+            h[0] = seg_start;
+            h[1] = t;
+            h[2] = catchup;
+            if (b.hand_kind) b.hand_kind[g->n_handoffs] = (uint8_t)k;
+        } else {
+            atomicOr(status, DEV_LOG_FULL);
+        }
+        g->n_handoffs++;
+    };
+    if (kind) {
         if (g->keep_probe) {
             b.tokens[g->pos] = tok;
             b.source[g->generated] = 0;
@@ -99,18 +126,24 @@ __device__ void router_step(GenState *g, const GenBuffers &b, int greedy, StepDe
             g->generated++;
             if (tok == g->eos) g->done = 1;
         }
-        if (g->n_handoffs < g->cap_handoffs) {
-            int32_t *h = b.handoffs + 3 * g->n_handoffs;
-            h[0] = g->pos;
-            h[1] = t;
-            h[2] = g->pos - g->kv_len[1];
-        } else {
-            atomicOr(status, DEV_LOG_FULL);
+        if (kind == 3) {   // the auxiliary sentence goes into the output, then the target continues
+            for (int i = 0; i < g->n_aux && g->generated < g->max_new && !g->done; ++i) {
+                b.tokens[g->pos] = b.aux[i];
+                b.source[g->generated] = 2;
+                g->pos++;
+                g->generated++;
+            }
+            g->neg_count = 0;
         }
-        g->n_handoffs++;
+        log_handoff(g->pos, g->pos - g->kv_len[1], kind);
         g->active = 1;
-        g->remaining = g->n1;
+        g->remaining = len;
     } else {
+        if (g->has_large && a == 1 && after_delim && (cls & kClsVerify) && g->remaining < g->n2) {
+            // (2) applies to the target's own sentences too: from this token on it writes n2 tokens
+            log_handoff(g->pos, 0, 2);
+            g->remaining = g->n2;
+        }
         b.tokens[g->pos] = tok;
         b.source[g->generated] = (uint8_t)a;
         g->pos++;
@@ -119,15 +152,7 @@ __device__ void router_step(GenState *g, const GenBuffers &b, int greedy, StepDe
         if (a == 1 && --g->remaining == 0) g->active = 0;
         if (g->has_large && a == 0 && g->every_delim && tok == g->delimiter && !g->done && g->generated < g->max_new) {
             // the speculative model closed a paragraph: the target writes the next n1 tokens
-            if (g->n_handoffs < g->cap_handoffs) {
-                int32_t *h = b.handoffs + 3 * g->n_handoffs;
-                h[0] = g->pos;
-                h[1] = t;
-                h[2] = g->pos - g->kv_len[1];
-            } else {
-                atomicOr(status, DEV_LOG_FULL);
-            }
-            g->n_handoffs++;
+            log_handoff(g->pos, g->pos - g->kv_len[1], 1);
             g->active = 1;
             g->remaining = g->n1;
         }

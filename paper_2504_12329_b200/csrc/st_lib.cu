@@ -150,6 +150,7 @@ static constexpr int kArgmaxBlocks = 64;
 static constexpr int kGemvWarps = 8;
 static constexpr int kMegaSyncWords = 32 * (1 + kMegaBarCounters);   // ticket/abort words + one 128-byte line per barrier counter
 static constexpr int kMaxKSplits = 8;  // most K splits of a multi-row projection
+static constexpr int kMaxAuxTokens = 64;   // longest auxiliary sentence of takeover (3)
 static constexpr int kRowSplits = 8;   // most key splits a multi-row pass uses
 
 // ------------------------------------------------------------------------------------------------
@@ -1406,6 +1407,7 @@ struct GenContext {
     StepDesc *desc2 = nullptr;
     GenBuffers b{};
     int32_t *d_force = nullptr;
+    int32_t *d_aux = nullptr;
     uint8_t *d_cls = nullptr;
     float *d_trace = nullptr;
     std::vector<void *> ptrs;
@@ -1610,11 +1612,14 @@ static int ensure_gen_context(st_model *small, st_model *large, int slot_s, int 
     c->b.em_arg = c->get<int32_t>(g_steps);
     c->b.em_src = c->get<uint8_t>(g_steps);
     c->b.handoffs = c->get<int32_t>(3 * (size_t)g_hand);
+    c->b.hand_kind = c->get<uint8_t>((size_t)g_hand);
+    c->d_aux = c->get<int32_t>(kMaxAuxTokens);
+    c->b.aux = c->d_aux;
     c->d_force = c->get<int32_t>(g_force);
     c->d_cls = c->get<uint8_t>(vlimit);
     c->d_trace = g_trace ? c->get<float>(g_trace) : nullptr;
     if (!c->gen || !c->desc2 || !c->b.tokens || !c->b.source || !c->b.em_tok || !c->b.em_fed || !c->b.em_arg || !c->b.em_src ||
-        !c->b.handoffs || !c->d_force || !c->d_cls || (g_trace && !c->d_trace)) {
+        !c->b.handoffs || !c->b.hand_kind || !c->d_aux || !c->d_force || !c->d_cls || (g_trace && !c->d_trace)) {
         destroy_gen_context(small);
         return ST_ERR_OOM;
     }
@@ -1629,6 +1634,31 @@ static int ensure_gen_context(st_model *small, st_model *large, int slot_s, int 
         }
     }
     return ST_OK;
+}
+
+// Takeover parameters beyond the keyword set: ids inside the shared vocabulary, positive segment lengths where a
+// rule is on, an auxiliary sentence that fits the device buffer.
+static int check_rule_params(const st_spec_params *P, int vlimit)
+{
+    if (P->n_affirmation < 0 || P->n_verification < 0 || P->n_aux < 0) return ST_ERR_ARG;
+    if ((P->n_affirmation > 0 && !P->affirmation_ids) || (P->n_verification > 0 && !P->verification_ids) || (P->n_aux > 0 && !P->aux_ids))
+        return ST_ERR_ARG;
+    if ((P->n_verification > 0 && P->n2 < 1) || (P->neg_threshold >= 0 && P->n3 < 1)) return ST_ERR_ARG;
+    if (P->n_aux > kMaxAuxTokens) return ST_ERR_CAPACITY;
+    for (int i = 0; i < P->n_affirmation; ++i)
+        if ((unsigned)P->affirmation_ids[i] >= (unsigned)vlimit) return ST_ERR_VOCAB;
+    for (int i = 0; i < P->n_verification; ++i)
+        if ((unsigned)P->verification_ids[i] >= (unsigned)vlimit) return ST_ERR_VOCAB;
+    for (int i = 0; i < P->n_aux; ++i)
+        if ((unsigned)P->aux_ids[i] >= (unsigned)vlimit) return ST_ERR_VOCAB;
+    return ST_OK;
+}
+
+static void fill_class_table(const st_spec_params *P, std::vector<uint8_t> &cls)
+{
+    for (int i = 0; i < P->n_keywords; ++i) cls[P->keyword_ids[i]] |= kClsKeyword;
+    for (int i = 0; i < P->n_affirmation; ++i) cls[P->affirmation_ids[i]] |= kClsAffirm;
+    for (int i = 0; i < P->n_verification; ++i) cls[P->verification_ids[i]] |= kClsVerify;
 }
 
 extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_params *P, const int32_t *prompt,
@@ -1648,6 +1678,7 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     for (int i = 0; i < P->n_keywords; ++i)
         if ((unsigned)P->keyword_ids[i] >= (unsigned)vlimit) return ST_ERR_VOCAB;
     if ((unsigned)P->delimiter_id >= (unsigned)vlimit) return ST_ERR_VOCAB;
+    TRY(check_rule_params(P, vlimit));
     const int max_new = P->max_new_tokens;
     if (out->cap_tokens < max_new || (max_new > 0 && (!out->tokens || !out->source))) return ST_ERR_CAPACITY;
     const int cap_steps = out->cap_steps, cap_handoffs = out->cap_handoffs;
@@ -1685,7 +1716,7 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     StepDesc *desc_small = C.desc2, *desc_large = C.desc2 + 1;
 
     std::vector<uint8_t> cls(vlimit, 0);
-    for (int i = 0; i < P->n_keywords; ++i) cls[P->keyword_ids[i]] |= kClsKeyword;
+    fill_class_table(P, cls);
     GenState g0{};
     g0.wbytes[0] = small->weight_bytes;
     g0.kvb[0] = st_kv_bytes_per_token(small);
@@ -1699,6 +1730,10 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     g0.n1 = P->n1;
     g0.keep_probe = P->keep_probe;
     g0.every_delim = P->takeover_every_delimiter ? 1 : 0;
+    g0.n2 = P->n2;
+    g0.n3 = P->n3;
+    g0.neg_threshold = P->neg_threshold;
+    g0.n_aux = P->n_aux;
     if (large && P->target_first_n > 0) {   // the target opens the answer
         g0.active = 1;
         g0.remaining = P->target_first_n;
@@ -1721,6 +1756,7 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     CK(cudaMemcpyAsync(b.tokens, prompt, (size_t)prompt_len * sizeof(int32_t), cudaMemcpyHostToDevice, s));
     if (n_force) CK(cudaMemcpyAsync(C.d_force, force, (size_t)n_force * sizeof(int32_t), cudaMemcpyHostToDevice, s));
     CK(cudaMemcpyAsync(C.d_cls, cls.data(), (size_t)vlimit, cudaMemcpyHostToDevice, s));
+    if (P->n_aux > 0) CK(cudaMemcpyAsync(C.d_aux, P->aux_ids, (size_t)P->n_aux * sizeof(int32_t), cudaMemcpyHostToDevice, s));
     plan_first_pass_kernel<<<1, 1, 0, s>>>(gen, desc_small, desc_large);
     ++g_launches;
     CK(cudaGetLastError());
@@ -1803,6 +1839,7 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
         if (out->emission_argmax) CK(cudaMemcpyAsync(out->emission_argmax, b.em_arg, (size_t)n_steps * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
     }
     if (n_hand > 0) CK(cudaMemcpyAsync(out->handoffs, b.handoffs, (size_t)n_hand * 3 * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    if (n_hand > 0 && out->handoff_kinds) CK(cudaMemcpyAsync(out->handoff_kinds, b.hand_kind, (size_t)n_hand, cudaMemcpyDeviceToHost, s));
     if (trace_n > 0) CK(cudaMemcpyAsync(out->logits_trace, C.d_trace, (size_t)trace_n * vlimit * sizeof(float), cudaMemcpyDeviceToHost, s));
     CK(cudaStreamSynchronize(s));
     int32_t dev_status = 0;
@@ -1843,6 +1880,7 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
     for (int i = 0; i < P->n_keywords; ++i)
         if ((unsigned)P->keyword_ids[i] >= (unsigned)vlimit) return ST_ERR_VOCAB;
     if ((unsigned)P->delimiter_id >= (unsigned)vlimit) return ST_ERR_VOCAB;
+    TRY(check_rule_params(P, vlimit));
     std::vector<int> plen(n), mnew(n), nforce(n), total(n);
     int longest = 0;
     for (int i = 0; i < n; ++i) {
@@ -1907,8 +1945,8 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
         if (large && large->max_rows < max_chunk) max_chunk = large->max_rows;
         const size_t o_rtok = take(2 * (size_t)max_chunk * sizeof(int32_t)), o_amax = take(2 * (size_t)max_chunk * sizeof(int32_t));
         const size_t o_pseq = take(2 * n * sizeof(int32_t)), o_plast = take(2 * n * sizeof(int32_t)), o_npass = take(2 * sizeof(int32_t));
-        const size_t o_plan = take(sizeof(BatchPlan)), o_cls = take((size_t)vlimit);
-        std::vector<size_t> o_tok(n), o_src(n), o_emt(n), o_emf(n), o_ema(n), o_ems(n), o_hand(n), o_force(n);
+        const size_t o_plan = take(sizeof(BatchPlan)), o_cls = take((size_t)vlimit), o_aux = take(kMaxAuxTokens * sizeof(int32_t));
+        std::vector<size_t> o_tok(n), o_src(n), o_emt(n), o_emf(n), o_ema(n), o_ems(n), o_hand(n), o_hkind(n), o_force(n);
         for (int i = 0; i < n; ++i) {
             const int cs = outs[i].cap_steps > 0 ? outs[i].cap_steps : 1, ch = outs[i].cap_handoffs > 0 ? outs[i].cap_handoffs : 1;
             o_tok[i] = take((size_t)total[i] * 4);
@@ -1918,6 +1956,7 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
             o_ema[i] = take((size_t)cs * 4);
             o_ems[i] = take((size_t)cs);
             o_hand[i] = take((size_t)ch * 12);
+            o_hkind[i] = take((size_t)ch);
             o_force[i] = take((size_t)(nforce[i] > 0 ? nforce[i] : 1) * 4);
         }
         if (cudaMalloc(&arena, off + 256) != cudaSuccess) { cudaGetLastError(); rc = ST_ERR_OOM; break; }
@@ -1931,7 +1970,7 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
         BatchPlan *d_plan = (BatchPlan *)(arena + o_plan);
         uint8_t *d_cls = arena + o_cls;
         std::vector<uint8_t> cls(vlimit, 0);
-        for (int i = 0; i < P->n_keywords; ++i) cls[P->keyword_ids[i]] |= kClsKeyword;
+        fill_class_table(P, cls);
         for (int i = 0; i < n; ++i) {
             GenState &g = gs[i];
             g = GenState{};
@@ -1947,6 +1986,10 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
             g.n1 = P->n1;
             g.keep_probe = P->keep_probe;
             g.every_delim = P->takeover_every_delimiter ? 1 : 0;
+            g.n2 = P->n2;
+            g.n3 = P->n3;
+            g.neg_threshold = P->neg_threshold;
+            g.n_aux = P->n_aux;
             if (large && P->target_first_n > 0) {
                 g.active = 1;
                 g.remaining = P->target_first_n;
@@ -1969,6 +2012,8 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
             b.em_arg = (int32_t *)(arena + o_ema[i]);
             b.em_src = arena + o_ems[i];
             b.handoffs = (int32_t *)(arena + o_hand[i]);
+            b.hand_kind = arena + o_hkind[i];
+            b.aux = (const int32_t *)(arena + o_aux);
             b.force = (const int32_t *)(arena + o_force[i]);
             b.cls = d_cls;
             b.trace = nullptr;
@@ -1976,7 +2021,9 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
         bool up = cudaMemcpyAsync(d_gs, gs.data(), n * sizeof(GenState), cudaMemcpyHostToDevice, s) == cudaSuccess &&
                   cudaMemcpyAsync(d_gb, gb.data(), n * sizeof(GenBuffers), cudaMemcpyHostToDevice, s) == cudaSuccess &&
                   cudaMemcpyAsync(d_slots, slots.data(), 2 * n * sizeof(int32_t), cudaMemcpyHostToDevice, s) == cudaSuccess &&
-                  cudaMemcpyAsync(d_cls, cls.data(), (size_t)vlimit, cudaMemcpyHostToDevice, s) == cudaSuccess;
+                  cudaMemcpyAsync(d_cls, cls.data(), (size_t)vlimit, cudaMemcpyHostToDevice, s) == cudaSuccess &&
+                  (P->n_aux == 0 ||
+                   cudaMemcpyAsync(arena + o_aux, P->aux_ids, (size_t)P->n_aux * sizeof(int32_t), cudaMemcpyHostToDevice, s) == cudaSuccess);
         for (int i = 0; i < n && up; ++i) {
             up = cudaMemcpyAsync(gb[i].tokens, prompts + prompt_offsets[i], (size_t)plen[i] * 4, cudaMemcpyHostToDevice, s) == cudaSuccess;
             if (up && nforce[i] > 0)
@@ -2076,6 +2123,8 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
                 if (o.emission_argmax) dn = dn && cudaMemcpyAsync(o.emission_argmax, b.em_arg, (size_t)n_steps * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
             }
             if (n_hand > 0) dn = dn && cudaMemcpyAsync(o.handoffs, b.handoffs, (size_t)n_hand * 12, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+            if (n_hand > 0 && o.handoff_kinds)
+                dn = dn && cudaMemcpyAsync(o.handoff_kinds, b.hand_kind, (size_t)n_hand, cudaMemcpyDeviceToHost, s) == cudaSuccess;
         }
         if (!dn || cudaStreamSynchronize(s) != cudaSuccess) { set_error_text("batched generation results", cudaGetLastError()); rc = ST_ERR_INTERNAL; break; }
         int32_t dev_status = 0, s2 = 0;

@@ -408,3 +408,41 @@ def test_batched_generation_fallbacks_and_edges(B, oracle):
     for gs, gl in (roomy, one_slot, few_pages):
         gs.close()
         gl.close()
+
+
+@pytest.mark.parametrize("keep", [False, True])
+def test_three_takeovers_on_device(B, oracle, keep):
+    """Takeovers (1)-(3) of the paper's Section 3 in token-id form (reflection / affirmation, verification by either
+    model, excessive reflection with the inserted auxiliary sentence): the hand-traced stream, and a longer forced
+    run against the oracle -- routing, handoff kinds and inserted tokens bit-exact, alone and in batched rounds."""
+    S, L = shape_dict(W.TINY_S), shape_dict(W.TINY_L)
+    os_, ol = oracle.Model(oracle.Config(**S), 0, 0), oracle.Model(oracle.Config(**L), 0, 1)
+    gs = B.Model(S, seed=0, tag=0, max_seqs=3, max_tokens=1536)
+    gl = B.Model(L, seed=0, tag=1, max_seqs=3, max_tokens=1536)
+    rules = dict(delimiter_id=10, keyword_ids=[11, 12, 13], affirmation_ids=[14], verification_ids=[13, 15], n1=2, n2=3, n3=2,
+                 neg_threshold=1, aux_ids=[40, 41])
+    if not keep:
+        hand = [10, 14, 20, 10, 11, 21, 10, 13, 10, 15, 22, 10, 15, 23, 24, 25, 26]
+        got = B.st_generate_spec(gs, gl, [1, 2, 3], max_new_tokens=15, force=hand, **rules)
+        assert got.tokens.tolist() == [10, 20, 10, 21, 10, 40, 41, 10, 15, 22, 10, 23, 24, 25, 26]
+        assert got.source.tolist() == [0, 1, 1, 1, 1, 2, 2, 1, 1, 1, 1, 1, 1, 1, 0]
+        assert got.handoffs == [(4, 1, 4), (6, 4, 1), (10, 7, 3), (11, 9, 0), (14, 12, 1)]
+        assert got.handoff_kinds == [1, 1, 3, 2, 2]
+    rules.update(n1=4, n2=9, n3=6, neg_threshold=2, aux_ids=[40, 41, 42], keep_probe=keep)
+    prompts = [W.prompt_ids(500 + i, 12 + 20 * i, 1024) for i in range(3)]
+    # forced streams over a small alphabet so that every class of cue follows delimiters often
+    rng = np.random.default_rng(9)
+    forces = [rng.choice([10, 10, 11, 13, 14, 15, 30, 31, 32, 33], size=400).astype(np.int32) for _ in range(3)]
+    wants = [oracle.generate_spec(os_, ol, prompts[i], max_new_tokens=160, force=forces[i], **rules) for i in range(3)]
+    assert {1, 2, 3} <= set(k for w in wants for k in w.handoff_kinds)
+    alone = B.st_generate_spec(gs, gl, prompts[0], max_new_tokens=160, force=forces[0], **rules)
+    batch = B.st_generate_spec_batch(gs, gl, prompts, max_new_tokens=160, forces=forces, **rules)
+    for want, got in [(wants[0], alone)] + list(zip(wants, batch)):
+        assert want.rc == 0
+        _assert_routing_equal(want, got)
+        assert got.handoff_kinds == want.handoff_kinds
+        for t in range(len(want.emission_tokens)):
+            if want.emission_margin[t] >= MARGIN:
+                assert got.emission_argmax[t] == want.emission_argmax[t]
+    gs.close()
+    gl.close()
