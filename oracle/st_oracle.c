@@ -498,6 +498,8 @@ typedef struct {
     int32_t n3;                       /* paper: 125 */
     const int32_t *aux_ids;           /* the auxiliary sentence of (3) */
     int32_t n_aux;
+    int32_t probe_len;                /* tokens of the speculative model's sentence after a delimiter that are classified
+                                         (paper: "one full sentence (i.e. n1 tokens)"); <= 1: only its first token */
 } orc_spec_params;
 
 typedef struct { int32_t seg_start, step, catchup_len; } orc_handoff;
@@ -540,6 +542,8 @@ int orc_generate_spec(const orc_model *small, const orc_model *large, const orc_
     if (large && large->c.vocab > vmax) vmax = large->c.vocab;
     double *z = (double *)malloc((size_t)vmax * sizeof(double));
     int active = 0, remaining = 0, rc = 0, neg_count = 0;
+    int probing = 0, probe_n = 0, n_refl = 0, n_aff = 0, n_ver = 0;
+    int32_t probe_start = 0;
     int32_t pos = prompt_len, t = 0, generated = 0;
     R->n_tokens = R->n_handoffs = R->n_steps = 0;
     if (large && P->target_first_n > 0) {   /* the target opens the answer */
@@ -568,13 +572,25 @@ int orc_generate_spec(const orc_model *small, const orc_model *large, const orc_
         for (int i = 0; i < P->n_affirmation; ++i) is_aff |= (P->affirmation_ids[i] == tok);
         for (int i = 0; i < P->n_verification; ++i) is_ver |= (P->verification_ids[i] == tok);
         const int after_delim = tokens[pos - 1] == P->delimiter_id;
-        if (large && a == 0 && !P->takeover_every_delimiter && after_delim) {
-            /* the speculative model opened a sentence: classify its first token */
-            if (is_kw && P->neg_threshold >= 0) ++neg_count;
+        if (large && a == 0 && !P->takeover_every_delimiter && !probing && after_delim) {
+            /* the speculative model opens a sentence: its next probe_len tokens are classified by cue counts */
+            probing = 1;
+            probe_start = pos;
+            probe_n = n_refl = n_aff = n_ver = 0;
+        }
+        if (probing) {
+            n_refl += is_kw; n_aff += is_aff; n_ver += is_ver;
+            ++probe_n;
+        }
+        if (probing && probe_n >= (P->probe_len > 1 ? P->probe_len : 1)) {
+            probing = 0;
+            /* Affirmation and Reflection cues in one sentence: the majority decides, a tie is a Reflection */
+            const int reflection = n_refl > 0 && n_refl >= n_aff;
+            if (reflection && P->neg_threshold >= 0) ++neg_count;
             int kind = 0, len = 0;
             if (P->neg_threshold >= 0 && neg_count > P->neg_threshold) { kind = 3; len = P->n3; }   /* (3) */
-            else if (is_ver) { kind = 2; len = P->n2; }                                             /* (2) */
-            else if (is_kw || is_aff) { kind = 1; len = P->n1; }                                    /* (1) */
+            else if (n_ver > 0) { kind = 2; len = P->n2; }                                          /* (2) */
+            else if (n_refl + n_aff > 0) { kind = 1; len = P->n1; }                                 /* (1) */
             if (kind) {
                 int stop = 0;
                 if (P->keep_probe) {
@@ -585,6 +601,13 @@ int orc_generate_spec(const orc_model *small, const orc_model *large, const orc_
                     ++pos; ++generated;
                     R->n_tokens = generated;
                     if (tok == P->eos_id) stop = 1;
+                } else {
+                    /* the target's segment replaces the whole probe sentence: the speculative model's cache
+                     * and the output go back to where the sentence began */
+                    generated -= pos - probe_start;
+                    pos = probe_start;
+                    kv[0]->len = probe_start;
+                    R->n_tokens = generated;
                 }
                 if (kind == 3) {   /* the auxiliary sentence goes into the output, then the target continues */
                     for (int i = 0; i < P->n_aux && generated < P->max_new_tokens && !stop; ++i) {

@@ -113,6 +113,49 @@ def test_three_takeovers_reduce_and_hold_invariants(oracle, tiny):
     assert len(r.emission_tokens) == sum(1 for x in src if x != 2) + sum(1 for k, h in zip(r.handoff_kinds, r.handoffs) if h[2] > 0 or k != 2)
 
 
+PROBE = dict(delimiter_id=10, keyword_ids=[11, 12], affirmation_ids=[14], verification_ids=[15], n1=3, n2=4, probe_len=3)
+
+
+def test_hand_traced_stream_sentence_probe(oracle, tiny):
+    T = _trace("handoff_trace_sentence_probe.txt")
+    r = oracle.generate_spec(tiny[0], tiny[1], [1, 2, 3], max_new_tokens=14, force=T["force"], **PROBE)
+    assert r.rc == 0
+    assert r.tokens.tolist() == T["tokens"]
+    assert r.source.tolist() == T["source"]
+    assert r.handoffs == T["handoffs"] and r.handoff_kinds == T["handoff_kinds"]
+    assert r.emission_source.tolist() == T["emission_source"]
+    assert r.emission_fed.tolist() == T["emission_fed"]
+    assert r.emission_tokens.tolist() == T["force"]
+    assert (r.kv_len_small, r.kv_len_large) == (T["kv_len_small"], T["kv_len_large"])
+
+
+def test_sentence_probe_invariants(oracle, tiny):
+    rng = np.random.default_rng(4)
+    force = rng.choice([10, 10, 11, 12, 14, 15, 30, 31, 32, 33, 34, 35], size=900).astype(np.int32)
+    for keep in (False, True):
+        r = oracle.generate_spec(tiny[0], tiny[1], [1, 2, 3], max_new_tokens=200, force=force, keep_probe=keep,
+                                 neg_threshold=3, n3=5, aux_ids=[40, 41], **PROBE)
+        assert r.rc == 0 and {1, 2, 3} <= set(r.handoff_kinds) and len(r.tokens) == 200
+        toks, src = r.tokens.tolist(), r.source.tolist()
+        for (seg, step, cu), kind in zip(r.handoffs, r.handoff_kinds):
+            i = seg - 3
+            if cu == 0:
+                continue                                     # the target extended its own segment (verification)
+            back = 3 if kind == 3 else 1                      # two auxiliary tokens sit before the segment of a (3)
+            if keep:
+                assert src[i - back] == 0                    # the probe sentence stays, the segment follows it
+            else:
+                assert toks[i - back] == 10                  # the segment (or the auxiliary sentence) starts right after the delimiter
+        # the speculative model's cache never runs ahead of the text, and every step is accounted for
+        assert r.kv_len_small <= 3 + 200 and r.kv_len_large <= 3 + 200
+    # a probe of one token is the rule with the first-token test
+    one = oracle.generate_spec(tiny[0], tiny[1], [1, 2, 3], max_new_tokens=120, force=force, neg_threshold=3, n3=5, aux_ids=[40, 41],
+                               **dict(PROBE, probe_len=1))
+    ref = oracle.generate_spec(tiny[0], tiny[1], [1, 2, 3], max_new_tokens=120, force=force, neg_threshold=3, n3=5, aux_ids=[40, 41],
+                               **{k: v for k, v in PROBE.items() if k != "probe_len"})
+    assert one.tokens.tolist() == ref.tokens.tolist() and one.handoffs == ref.handoffs
+
+
 def test_every_delimiter_edge_cases(oracle, tiny):
     kw = dict(delimiter_id=10, keyword_ids=[11, 12, 13], n1=2, takeover_every_delimiter=True)
     # keywords mean nothing in this mode; a delimiter written by the target or standing in the prompt hands nothing over
