@@ -99,6 +99,12 @@ typedef struct {
     int32_t n3;                       /* paper: 125; >= 1 when neg_threshold >= 0 */
     const int32_t *aux_ids;           /* host, the auxiliary sentence, at most 64 ids */
     int32_t n_aux;
+    int32_t probe_len;                /* <= 1: the first token after a delimiter is classified.  k > 1 (paper: n1): the
+                                         speculative model writes k tokens after the delimiter, the sentence is classified
+                                         by cue counts (affirmation vs reflection: majority, tie = reflection) and on a
+                                         takeover the target's segment replaces the whole sentence (keep_probe 0: output
+                                         and the speculative model's cached length go back to the sentence's start) or
+                                         follows it (keep_probe 1).  Size emission logs for (1 + k) * max_new_tokens steps */
 } st_spec_params;
 
 typedef struct {

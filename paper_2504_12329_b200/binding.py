@@ -41,7 +41,7 @@ class StSpecParams(C.Structure):
         ("affirmation_ids", C.POINTER(C.c_int32)), ("n_affirmation", C.c_int32),
         ("verification_ids", C.POINTER(C.c_int32)), ("n_verification", C.c_int32),
         ("n2", C.c_int32), ("neg_threshold", C.c_int32), ("n3", C.c_int32),
-        ("aux_ids", C.POINTER(C.c_int32)), ("n_aux", C.c_int32),
+        ("aux_ids", C.POINTER(C.c_int32)), ("n_aux", C.c_int32), ("probe_len", C.c_int32),
     ]
 
 
@@ -334,14 +334,15 @@ class _ResultBuffers:
 
 
 def _spec_params(delimiter_id, keyword_ids, n1, keep_probe, eos_id, vocab_limit, max_new_tokens, takeover_every_delimiter,
-                 target_first_n, affirmation_ids=(), verification_ids=(), n2=125, neg_threshold=-1, n3=125, aux_ids=()):
+                 target_first_n, affirmation_ids=(), verification_ids=(), n2=125, neg_threshold=-1, n3=125, aux_ids=(),
+                 probe_len=1):
     """st_spec_params and the arrays it points at (keep both alive during the call)."""
     arrs = [np.ascontiguousarray(a, dtype=np.int32) for a in (keyword_ids, affirmation_ids, verification_ids, aux_ids)]
     ip = lambda a: a.ctypes.data_as(C.POINTER(C.c_int32))
     kw, aff, ver, aux = arrs
     P = StSpecParams(delimiter_id, ip(kw), kw.size, n1, int(keep_probe), eos_id, vocab_limit, max_new_tokens,
                      int(takeover_every_delimiter), int(target_first_n), ip(aff), aff.size, ip(ver), ver.size, n2,
-                     neg_threshold, n3, ip(aux), aux.size)
+                     neg_threshold, n3, ip(aux), aux.size, probe_len)
     return P, arrs
 
 
@@ -357,6 +358,8 @@ def st_generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id:
                             takeover_every_delimiter, target_first_n, **rules)
     if vocab_limit <= 0:
         vocab_limit = small.vocab if large is None else min(small.vocab, large.vocab)
+    if cap_steps is None:   # replaced probe sentences are steps that leave no token
+        cap_steps = (1 + max(1, int(rules.get("probe_len", 1)))) * max_new_tokens + 8
     bufs = _ResultBuffers(max_new_tokens, vocab_limit, trace_first_step, trace_n_steps, cap_steps, cap_handoffs)
     R = StSpecResult()
     bufs.fill(R)
@@ -386,7 +389,8 @@ def st_generate_spec_batch(small: Model, large: Model | None, prompts, *, delimi
         off_f = np.zeros(n + 1, dtype=np.int32)
         off_f[1:] = np.cumsum([len(f) for f in forces])
     budget_arr = np.ascontiguousarray(budgets, dtype=np.int32)
-    bufs = [_ResultBuffers(b, vocab_limit, 0, 0, None, None) for b in budgets]
+    k = 1 + max(1, int(rules.get("probe_len", 1)))
+    bufs = [_ResultBuffers(b, vocab_limit, 0, 0, k * b + 8, None) for b in budgets]
     Rs = (StSpecResult * max(n, 1))()
     for i, b in enumerate(bufs):
         b.fill(Rs[i])

@@ -38,6 +38,8 @@ struct GenState {
     // --- parameters ---
     int32_t has_large, delimiter, n1, keep_probe, eos, vlimit, max_new, n_force;
     int32_t n2, n3, neg_threshold, n_aux;   // takeovers (2) and (3): segment lengths, counter bound (< 0: off), auxiliary tokens
+    int32_t probe_len;                      // tokens of the speculative model's sentence after a delimiter that are classified
+    int32_t probing, probe_start, probe_n, n_refl, n_aff, n_ver;   // the probe in progress
     int32_t neg_count;                      // reflection cues the speculative model sampled since the last takeover (3)
     int32_t every_delim;   // 1: no keyword test; the target takes over after every delimiter the speculative model writes
     int32_t prompt_len, cap_steps, cap_handoffs, max_chunk;
@@ -100,11 +102,26 @@ __device__ void router_step(GenState *g, const GenBuffers &b, int greedy, StepDe
     const int cls = b.cls[tok];
     const bool after_delim = b.tokens[g->pos - 1] == g->delimiter;
     int kind = 0, len = 0;
-    if (g->has_large && a == 0 && !g->every_delim && after_delim) {
-        if ((cls & kClsKeyword) && g->neg_threshold >= 0) g->neg_count++;
-        if (g->neg_threshold >= 0 && g->neg_count > g->neg_threshold) { kind = 3; len = g->n3; }   // (3) excessive reflection
-        else if (cls & kClsVerify) { kind = 2; len = g->n2; }                                       // (2) verification
-        else if (cls & (kClsKeyword | kClsAffirm)) { kind = 1; len = g->n1; }                       // (1) reflection / affirmation
+    if (g->has_large && a == 0 && !g->every_delim && !g->probing && after_delim) {
+        // the speculative model opens a sentence: its next probe_len tokens are classified by cue counts
+        g->probing = 1;
+        g->probe_start = g->pos;
+        g->probe_n = g->n_refl = g->n_aff = g->n_ver = 0;
+    }
+    if (g->probing) {
+        g->n_refl += (cls & kClsKeyword) != 0;
+        g->n_aff += (cls & kClsAffirm) != 0;
+        g->n_ver += (cls & kClsVerify) != 0;
+        g->probe_n++;
+        if (g->probe_n >= (g->probe_len > 1 ? g->probe_len : 1)) {
+            g->probing = 0;
+            // affirmation and reflection cues in one sentence: the majority decides, a tie is a reflection
+            const bool reflection = g->n_refl > 0 && g->n_refl >= g->n_aff;
+            if (reflection && g->neg_threshold >= 0) g->neg_count++;
+            if (g->neg_threshold >= 0 && g->neg_count > g->neg_threshold) { kind = 3; len = g->n3; }   // (3) excessive reflection
+            else if (g->n_ver > 0) { kind = 2; len = g->n2; }                                           // (2) verification
+            else if (g->n_refl + g->n_aff > 0) { kind = 1; len = g->n1; }                               // (1) reflection / affirmation
+        }
     }
     auto log_handoff = [&](int seg_start, int catchup, int k) {
         if (g->n_handoffs < g->cap_handoffs) {
@@ -125,6 +142,12 @@ __device__ void router_step(GenState *g, const GenBuffers &b, int greedy, StepDe
             g->pos++;
             g->generated++;
             if (tok == g->eos) g->done = 1;
+        } else {
+            // the target's segment replaces the whole probe sentence: the output and the speculative model's cached
+            // length go back to where the sentence began (the stale cache rows are overwritten by the next catch-up)
+            g->generated -= g->pos - g->probe_start;
+            g->pos = g->probe_start;
+            g->kv_len[0] = g->probe_start;
         }
         if (kind == 3) {   // the auxiliary sentence goes into the output, then the target continues
             for (int i = 0; i < g->n_aux && g->generated < g->max_new && !g->done; ++i) {

@@ -1734,6 +1734,7 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     g0.n3 = P->n3;
     g0.neg_threshold = P->neg_threshold;
     g0.n_aux = P->n_aux;
+    g0.probe_len = P->probe_len > 1 ? P->probe_len : 1;
     if (large && P->target_first_n > 0) {   // the target opens the answer
         g0.active = 1;
         g0.remaining = P->target_first_n;
@@ -1750,7 +1751,8 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     g0.trace_first = out->trace_first_step;
     g0.trace_n = trace_n;
     g0.done = max_new == 0 ? 1 : 0;
-    const int64_t pass_cap = 2ll * (max_new + 2) + 2ll * (total / g0.max_chunk + 2) * (max_new / P->n1 + 2);
+    // every token costs a pass; a replaced probe sentence costs probe_len passes more per takeover
+    const int64_t pass_cap = (1ll + g0.probe_len) * (max_new + 2) + 2ll * (total / g0.max_chunk + 2) * (max_new / P->n1 + 2);
     g0.pass_cap = pass_cap > 0x7fffffff ? 0x7fffffff : (int32_t)pass_cap;
     CK(cudaMemcpyAsync(gen, &g0, sizeof g0, cudaMemcpyHostToDevice, s));
     CK(cudaMemcpyAsync(b.tokens, prompt, (size_t)prompt_len * sizeof(int32_t), cudaMemcpyHostToDevice, s));
@@ -1990,6 +1992,7 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
             g.n3 = P->n3;
             g.neg_threshold = P->neg_threshold;
             g.n_aux = P->n_aux;
+            g.probe_len = P->probe_len > 1 ? P->probe_len : 1;
             if (large && P->target_first_n > 0) {
                 g.active = 1;
                 g.remaining = P->target_first_n;
@@ -2035,7 +2038,7 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
         // ---- rounds ----
         int64_t sum_new = 0;
         for (int i = 0; i < n; ++i) sum_new += mnew[i];
-        const int64_t round_cap = 4 * (sum_new + 4ll * n + 16) + 4ll * n * (longest / max_chunk + 2);
+        const int64_t round_cap = (3ll + (P->probe_len > 1 ? P->probe_len : 1)) * (sum_new + 4ll * n + 16) + 4ll * n * (longest / max_chunk + 2);
         // rows the target's pass waits for while the speculative model has work: an eighth of the sequences
         int min_target_rows = n / 8;
         if (const char *e = getenv("ST_BATCH_TARGET_MIN")) min_target_rows = atoi(e);   // tuning aid

@@ -446,3 +446,39 @@ def test_three_takeovers_on_device(B, oracle, keep):
                 assert got.emission_argmax[t] == want.emission_argmax[t]
     gs.close()
     gl.close()
+
+
+@pytest.mark.parametrize("keep", [False, True])
+def test_sentence_probe_on_device(B, oracle, keep):
+    """The n1-token probe sentence (paper Section 3 (1)): classified by cue counts, replaced as a whole by the target's
+    segment (or kept).  The hand-traced stream, then a longer forced run with all three takeovers against the oracle:
+    routing, rolled-back cache lengths, handoff kinds and greedy choices, alone and in batched rounds."""
+    S, L = shape_dict(W.TINY_S), shape_dict(W.TINY_L)
+    os_, ol = oracle.Model(oracle.Config(**S), 0, 0), oracle.Model(oracle.Config(**L), 0, 1)
+    gs = B.Model(S, seed=0, tag=0, max_seqs=3, max_tokens=2048)
+    gl = B.Model(L, seed=0, tag=1, max_seqs=3, max_tokens=2048)
+    rules = dict(delimiter_id=10, keyword_ids=[11, 12], affirmation_ids=[14], verification_ids=[15], n1=3, n2=4, probe_len=3)
+    if not keep:
+        hand = [10, 30, 11, 14, 20, 21, 10, 14, 31, 14, 22, 23, 10, 32, 10, 33, 15, 10, 15, 34]
+        got = B.st_generate_spec(gs, gl, [1, 2, 3], max_new_tokens=14, force=hand, **rules)
+        assert got.tokens.tolist() == [10, 20, 21, 10, 22, 23, 10, 32, 10, 33, 15, 10, 15, 34]
+        assert got.source.tolist() == [0, 1, 1, 1, 1, 1, 1, 0, 0, 0, 0, 0, 0, 0]
+        assert got.handoffs == [(4, 3, 4), (7, 9, 1)] and got.handoff_kinds == [1, 1]
+        assert (got.kv_len_small, got.kv_len_large) == (16, 9)
+    rules.update(neg_threshold=3, n3=5, aux_ids=[40, 41], keep_probe=keep)
+    rng = np.random.default_rng(4)
+    forces = [rng.choice([10, 10, 11, 12, 14, 15, 30, 31, 32, 33, 34, 35], size=900).astype(np.int32) for _ in range(3)]
+    prompts = [W.prompt_ids(600 + i, 9 + 30 * i, 1024) for i in range(3)]
+    wants = [oracle.generate_spec(os_, ol, prompts[i], max_new_tokens=180, force=forces[i], **rules) for i in range(3)]
+    assert {1, 2, 3} <= set(k for w in wants for k in w.handoff_kinds)
+    alone = B.st_generate_spec(gs, gl, prompts[1], max_new_tokens=180, force=forces[1], **rules)
+    batch = B.st_generate_spec_batch(gs, gl, prompts, max_new_tokens=180, forces=forces, **rules)
+    for want, got in [(wants[1], alone)] + list(zip(wants, batch)):
+        assert want.rc == 0
+        _assert_routing_equal(want, got)
+        assert got.handoff_kinds == want.handoff_kinds
+        for t in range(len(want.emission_tokens)):
+            if want.emission_margin[t] >= MARGIN:
+                assert got.emission_argmax[t] == want.emission_argmax[t]
+    gs.close()
+    gl.close()
