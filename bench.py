@@ -42,6 +42,15 @@ def measured_tensor_peak():
     return 1400.0, "fallback (sustained)"
 
 
+def paper_accounting(r, wl):
+    """The paper's own figures for this run, as context: share of target tokens and its FLOP-model speed estimate
+    (formulas as printed, capacity constant 3.12e10 FLOP/s -- accounting, not a measurement)."""
+    from paper_2504_12329_b200 import accounting as A
+    return {"modify_ratio": A.modify_ratio(r.source),
+            "estimated_speed_tokens_per_s": A.estimated_speed(r, wl.prompt_len, wl.small.as_dict(), wl.large.as_dict() if wl.large else None),
+            "note": "paper's FLOP model and capacity constant; context only"}
+
+
 def time_multi_row_passes(torch, model, shape, ctx, row_counts, hbm_peak):
     """Catch-up / prefill passes of one model on their own: `rows` new tokens over `ctx` cached ones, timed with
     CUDA events on the launching stream.  Every pass streams the model's weights once (larger than L2)."""
@@ -407,6 +416,7 @@ def main():
             "path_roofline": {"achieved_gbs": path_gbs, "frac_of_measured_hbm": path_gbs / peak,
                               "frac_of_nominal_8tbs": path_gbs / 8000.0,
                               "note": "algorithmic bytes of every pass (weights + KV) / device time of the generation"},
+            "paper_accounting": paper_accounting(r, wl),
             "prefill": prefill,
             "small_model_decode": small_step,
             "batched_decode": batched,
