@@ -14,7 +14,8 @@ torch = pytest.importorskip("torch")
 def B():
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
-    from paper_2504_12329_b200 import binding
+    from paper_2504_12329_b200 import binding, build
+    build.build()   # no-op when the in-tree library is newer than its sources
     binding.lib()
     return binding
 

@@ -18,7 +18,8 @@ torch = pytest.importorskip("torch")
 def test_static_argmax_matches_decode_step_twice():
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
-    from paper_2504_12329_b200 import binding as B
+    from paper_2504_12329_b200 import binding as B, build
+    build.build()   # no-op when the in-tree library is newer than its sources
     shape = W.TINY_L.as_dict()
     m = B.Model(shape, seed=0, tag=1, max_tokens=128)
     slot = m.st_seq_alloc()
