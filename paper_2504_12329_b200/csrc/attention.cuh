@@ -62,11 +62,12 @@ __global__ void embed_rope_kernel(const StepDesc *desc, const int32_t *tok, cons
 // With row_slot / row_pos the rows belong to different sequences (batched decode).
 // qkv: [rows][(Hq + 2 Hkv) * D] = q heads, then k heads, then v heads.  With k_splits > 0 the row is not in
 // qkv yet: it is bias + the K-split partial sums Ws[s][row] of the QKV projection (summed in split order).
-__global__ void __launch_bounds__(256) rope_append_kernel(const StepDesc *desc, float *qkv, const float *Ws, int k_splits, int ws_rows,
+__global__ void __launch_bounds__(512) rope_append_kernel(const StepDesc *desc, float *qkv, const float *Ws, int k_splits, int ws_rows,
                                                           const float *bias, const float2 *cs, int Hq, int Hkv, int D, KvView kv,
                                                           int32_t *status, const int32_t *row_slot = nullptr,
                                                           const int32_t *row_pos = nullptr, int pages_per_seq = 0)
 {
+    pdl_launch();
     const int i = blockIdx.x;
     if (i >= desc->m) return;
     if (row_slot) kv.block_tab += (size_t)row_slot[i] * pages_per_seq;   // batched decode: kv.block_tab is sequence 0's table
@@ -76,11 +77,7 @@ __global__ void __launch_bounds__(256) rope_append_kernel(const StepDesc *desc, 
     auto val4 = [&](int n) {   // 4 consecutive features of the row, n a multiple of 4
         if (k_splits <= 0) return *reinterpret_cast<const float4 *>(row + n);
         float4 v = bias ? *reinterpret_cast<const float4 *>(bias + n) : make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s = 0; s < k_splits; ++s) {
-            const float4 w = __ldcg(reinterpret_cast<const float4 *>(Ws + ((size_t)s * ws_rows + i) * N + n));
-            v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
-        }
-        return v;
+        return add_splits4(v, Ws + (size_t)i * N + n, (size_t)ws_rows * N, k_splits);
     };
     const int q4 = half >> 2;   // groups of 4 channel pairs per head
     for (int idx = threadIdx.x; idx < (Hq + Hkv) * q4; idx += blockDim.x) {

@@ -34,6 +34,7 @@ __global__ void __launch_bounds__(kArThreads, 1) attn_rows_mma_kernel(const Attn
 {
     static_assert(G >= 1 && G <= 8, "one MMA column per (row, head)");
     constexpr int KS = D / 16, NH = D / 64, RQ = 64 / G, HALF_BYTES = kArTileKeys * 128, STAGE = ar_stage_bytes<D>();
+    pdl_launch();
     extern __shared__ uint8_t ar_smem[];
     __shared__ uint64_t s_full[kArStages];
     __shared__ int s_abort, s_last;
@@ -290,6 +291,7 @@ __global__ void __launch_bounds__(kArThreads, 1) attn_batch_mma_kernel(const Att
 {
     static_assert(G >= 1 && G <= 8, "one MMA column per head of the group");
     constexpr int KS = D / 16, NH = D / 64, HALF_BYTES = kAbTileKeys * 128, STAGE = ab_stage_bytes<D>();
+    pdl_launch();
     extern __shared__ uint8_t ab_smem[];
     __shared__ uint64_t s_full[kAbStages];
     __shared__ int s_abort;

@@ -30,11 +30,6 @@ struct GemvParams {
     float eps;
 };
 
-// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may
-// start while its predecessor still runs; it must not touch the predecessor's results before wait().
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-
 template <int NW, int S, int R, int U, int PRO, int EPI>
 __global__ void __launch_bounds__(NW * 32) gemv_kernel(const GemvParams p)
 {
@@ -78,7 +73,7 @@ __global__ void __launch_bounds__(NW * 32) gemv_kernel(const GemvParams p)
     issue(0, wa);   // weights do not depend on the previous kernel: fetch before waiting for it
 
     pdl_wait();
-    pdl_launch_dependents();
+    pdl_launch();
     if (p.desc && p.desc->m <= 0) return;
     const int xrow = p.x_row >= 0 ? p.x_row : p.desc->m - 1;
     const float4 *xin = reinterpret_cast<const float4 *>(p.x + (size_t)xrow * K);

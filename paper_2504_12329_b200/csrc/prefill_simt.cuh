@@ -13,9 +13,10 @@ namespace st {
 // XN[i] = rmsnorm(X[i]) * gain as a hi/lo bf16 pair, one CTA per row.  With k_splits > 0 the row first
 // receives the K-split partial sums of the projection that feeds the residual stream,
 // X[i] += sum_s Ws[s][i] (in split order), so that projection needs no reduction pass of its own.
-__global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const StepDesc *desc, float *X, const float *Ws, int k_splits, int ws_rows,
+__global__ void __launch_bounds__(1024) rmsnorm_rows_kernel(const StepDesc *desc, float *X, const float *Ws, int k_splits, int ws_rows,
                                                            const float *gain, float eps, int hidden, uint16_t *XN_hi, uint16_t *XN_lo)
 {
+    pdl_launch();   // the projection that follows may fetch its weights meanwhile
     const int i = blockIdx.x;
     if (i >= desc->m) return;
     float4 *x4 = reinterpret_cast<float4 *>(X + (size_t)i * hidden);
@@ -24,15 +25,12 @@ __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const StepDesc *desc,
     for (int j = threadIdx.x; j < n4; j += blockDim.x) {
         float4 v = x4[j];
         if (k_splits > 0) {
-            for (int s = 0; s < k_splits; ++s) {
-                const float4 w = __ldcg(reinterpret_cast<const float4 *>(Ws + ((size_t)s * ws_rows + i) * hidden) + j);
-                v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
-            }
+            v = add_splits4(v, Ws + (size_t)i * hidden + 4 * (size_t)j, (size_t)ws_rows * hidden, k_splits);
             x4[j] = v;
         }
         ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
     }
-    __shared__ float s_part[8];
+    __shared__ float s_part[32];
     ss = warp_sum(ss);
     if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
     __syncthreads();

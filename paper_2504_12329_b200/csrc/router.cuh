@@ -261,8 +261,9 @@ struct BatchPlan {
 // as long as the pass has room; sequences that ingest more than one token are placed first so that the single
 // rows cannot crowd them out, and one that does not fit waits for the next round.  More pending tokens than a
 // pass has rows (a long prompt) go through the sequence's own chunked multi-row passes instead.
-// min_target_rows: the target's pass is skipped this round when it would hold fewer rows and the speculative model
-// has work (sequences do not interact, so the order in which they advance does not change any result).
+// min_target_rows (r >= 0: r rows; r < 0: |r| percent of the sequences still running): the target's pass is skipped this
+// round when it would hold fewer rows and the speculative model has work (sequences do not interact, so the
+// order in which they advance does not change any result).
 // row_* and bdesc: per model [2]; slots: [n_seqs][2]; descs: [n_seqs][2]; row_tok: [2][max_rows];
 // pass_seq / pass_last: [2][n_seqs] sequences of each pass and their sampling rows; n_pass_seq: [2].
 __global__ void batch_plan_kernel(GenState *gs, const GenBuffers *gb, int n_seqs, const int32_t *slots, StepDesc *descs,
@@ -309,6 +310,7 @@ __global__ void batch_plan_kernel(GenState *gs, const GenBuffers *gb, int n_seqs
     }
     // A pass of the target costs several passes of the speculative model whatever its row count: while the
     // speculative model has rows and the target only a few, the target's sequences wait and their rows accumulate.
+    if (min_target_rows < 0) min_target_rows = live * -min_target_rows / 100;   // a share of the sequences still running
     if (n_rows[1] > 0 && n_rows[1] < min_target_rows && n_rows[0] > 0) n_rows[1] = n_in[1] = 0;
     for (int a = 0; a < 2; ++a) {
         bdesc[a].pos0 = 0;
@@ -343,16 +345,35 @@ __device__ __forceinline__ void argmax_merge(float &v, int &i, float v2, int i2)
 }
 
 // Batched decode: lowest-id argmax of every row of logits [rows][vocab] over ids < limit, one CTA per row.
-__global__ void __launch_bounds__(256) argmax_rows_kernel(const StepDesc *desc, const float *logits, int vocab, int limit, int32_t *argmax_out)
+__global__ void __launch_bounds__(1024) argmax_rows_kernel(const StepDesc *desc, const float *logits, int vocab, int limit, int32_t *argmax_out)
 {
-    __shared__ float s_v[8];
-    __shared__ int s_i[8];
+    __shared__ float s_v[32];
+    __shared__ int s_i[32];
     const int row = blockIdx.x;
     if (row >= desc->m) return;
     const float *z = logits + (size_t)row * vocab;
     float v = -INFINITY;
     int idx = 0x7fffffff;
-    for (int i = threadIdx.x; i < limit; i += blockDim.x) argmax_merge(v, idx, __ldcg(z + i), i);
+    // 16-byte loads where the rows are 16-byte aligned, four in flight per thread; the ragged end one by one
+    const int lim4 = (vocab & 3) == 0 ? limit >> 2 : 0;
+    const float4 *z4 = reinterpret_cast<const float4 *>(z);
+    for (int i0 = threadIdx.x; i0 < lim4; i0 += 4 * blockDim.x) {
+        float4 w[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (i0 + u * (int)blockDim.x < lim4) w[u] = __ldcg(z4 + i0 + u * blockDim.x);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = i0 + u * (int)blockDim.x;
+            if (i < lim4) {
+                argmax_merge(v, idx, w[u].x, 4 * i);
+                argmax_merge(v, idx, w[u].y, 4 * i + 1);
+                argmax_merge(v, idx, w[u].z, 4 * i + 2);
+                argmax_merge(v, idx, w[u].w, 4 * i + 3);
+            }
+        }
+    }
+    for (int i = 4 * lim4 + threadIdx.x; i < limit; i += blockDim.x) argmax_merge(v, idx, __ldcg(z + i), i);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         const float v2 = __shfl_xor_sync(0xffffffffu, v, o);
@@ -362,7 +383,7 @@ __global__ void __launch_bounds__(256) argmax_rows_kernel(const StepDesc *desc, 
     if ((threadIdx.x & 31) == 0) { s_v[threadIdx.x >> 5] = v; s_i[threadIdx.x >> 5] = idx; }
     __syncthreads();
     if (threadIdx.x == 0) {
-        for (int w = 1; w < 8; ++w) argmax_merge(v, idx, s_v[w], s_i[w]);
+        for (int w = 1; w < (int)(blockDim.x >> 5); ++w) argmax_merge(v, idx, s_v[w], s_i[w]);
         argmax_out[row] = idx == 0x7fffffff ? 0 : idx;
     }
 }

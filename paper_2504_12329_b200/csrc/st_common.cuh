@@ -56,6 +56,27 @@ __device__ __forceinline__ uint16_t kv_bits(float f) { return __half_as_ushort(_
 __device__ __forceinline__ float kv_lo(uint32_t v) { return __half2float(__ushort_as_half((unsigned short)(v & 0xffffu))); }
 __device__ __forceinline__ float kv_hi(uint32_t v) { return __half2float(__ushort_as_half((unsigned short)(v >> 16))); }
 
+// Programmatic dependent launch.  pdl_launch: the next kernel of the stream, if it was launched with programmatic
+// stream serialization, may become resident once every CTA of this grid has got here (or exited).  pdl_wait: block
+// until the grids before this one have completed and their writes are visible; a thread calls it before its first
+// access to memory they produce.  Both do nothing in a launch without the attribute.
+__device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// v + the K-split partial sums ws[s * split_stride .. +3], s < k_splits <= 8, added in split order.  All loads are
+// issued before the first addition, so a row costs one trip to L2 instead of one per split.
+__device__ __forceinline__ float4 add_splits4(float4 v, const float *ws, size_t split_stride, int k_splits)
+{
+    float4 w[8];
+#pragma unroll
+    for (int s = 0; s < 8; ++s)
+        if (s < k_splits) w[s] = __ldcg(reinterpret_cast<const float4 *>(ws + (size_t)s * split_stride));
+#pragma unroll
+    for (int s = 0; s < 8; ++s)
+        if (s < k_splits) { v.x += w[s].x; v.y += w[s].y; v.z += w[s].z; v.w += w[s].w; }
+    return v;
+}
+
 // a = hi + lo with hi = bf16(a), lo = bf16(a - hi): 16 significand bits in two bf16 values.
 __device__ __forceinline__ void split_bf16(float a, uint16_t &hi, uint16_t &lo)
 {

@@ -149,7 +149,16 @@ struct st_model {
 static constexpr int kArgmaxBlocks = 64;
 static constexpr int kGemvWarps = 8;
 static constexpr int kMegaSyncWords = 32 * (1 + kMegaBarCounters);   // ticket/abort words + one 128-byte line per barrier counter
-static constexpr int kMaxKSplits = 8;  // most K splits of a multi-row projection
+static constexpr int kMaxKSplits = 8;  // most K splits of a multi-row projection (add_splits4 holds as many loads)
+
+// Threads of a one-CTA-per-row kernel with `items` independent work items: the fewest passes over the row that
+// `cap` threads allow, spread evenly (a row is latency bound, so as many loads as possible should be in flight).
+static int row_threads(int items, int cap)
+{
+    const int passes = (items + cap - 1) / cap;
+    const int t = ((items + passes - 1) / passes + 31) / 32 * 32;
+    return t < 128 ? 128 : t;
+}
 static constexpr int kMaxAuxTokens = 64;   // longest auxiliary sentence of takeover (3)
 static constexpr int kRowSplits = 8;   // most key splits a multi-row pass uses
 
@@ -399,6 +408,11 @@ static int make_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint
     return ST_OK;
 }
 
+// Whether the multi-row projections are launched with programmatic stream serialization: not inside the bodies of
+// the generation graph's conditional nodes (g_pdl_off > 0), and never with ST_PDL=0.
+static int g_pdl_off = 0;
+static bool pdl_enabled() { return use_pdl() && g_pdl_off == 0; }
+
 template <int EPI>
 // pending_splits: when given, a K-split projection leaves its partial sums in the workspace and reports the split
 // count there (0: the output is complete) -- the kernel that consumes the output adds them up.
@@ -446,9 +460,20 @@ static int launch_tc_gemm(const CUtensorMap &tw, TcGemmParams p, int m_upper, in
     if ((p.N & 3) || !p.Ws) ks = 1;
     p.k_splits = ks;
     const size_t smem = (size_t)p.stages * stage_bytes + 1024;
-    kern<<<dim3(n_tiles, ks), 192, smem, s>>>(tw, p);
+    // programmatic dependent launch: the CTAs may become resident, set up and fetch their first weight tiles while
+    // the kernel before this one is still running (it reads that kernel's output only after griddepcontrol.wait)
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(n_tiles, ks);
+    cfg.blockDim = dim3(192);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    CK(cudaLaunchKernelEx(&cfg, kern, tw, p));
     ++g_launches;
-    CK(cudaGetLastError());
     if (pending_splits) {
         *pending_splits = ks > 1 ? ks : 0;
         return ST_OK;
@@ -998,13 +1023,13 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
         const LayerWeights &w = m->layers[l];
         const LayerMaps &tm = m->maps[l];
         // the previous layer's down projection may have left its K-split partial sums for this kernel to add
-        rmsnorm_rows_kernel<<<m_upper, 256, 0, s>>>(desc, m->X, m->splitk_ws, pend_down, m->max_rows, w.g1, c.rms_eps, h, m->XN, XN_lo);
+        rmsnorm_rows_kernel<<<m_upper, row_threads(h / 4, 1024), 0, s>>>(desc, m->X, m->splitk_ws, pend_down, m->max_rows, w.g1, c.rms_eps, h, m->XN, XN_lo);
         ++g_launches;
         CK(cudaGetLastError());
         int pend = 0;
         TRY((rows_gemm<TEPI_STORE>(m, desc, m_upper, 0, m->XN, XN_lo, tm.wqkv, w.wqkv, w.bqkv, m->QKV, nullptr, nullptr, qd + 2 * kd, h, &pend)));
         const KvView kv = kv_view(m, l, batch ? 0 : slot);
-        rope_append_kernel<<<m_upper, 256, 0, s>>>(desc, m->QKV, m->splitk_ws, pend, m->max_rows, w.bqkv, m->cs, c.n_q_heads, c.n_kv_heads, D, kv,
+        rope_append_kernel<<<m_upper, row_threads((c.n_q_heads + c.n_kv_heads) * D / 8, 512), 0, s>>>(desc, m->QKV, m->splitk_ws, pend, m->max_rows, w.bqkv, m->cs, c.n_q_heads, c.n_kv_heads, D, kv,
                                                    m->status, batch ? m->row_slot : nullptr, batch ? m->row_pos : nullptr, m->pages_per_seq);
         ++g_launches;
         CK(cudaGetLastError());
@@ -1033,7 +1058,7 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
             CK(launch_attn_rows_mma(am, D, G, dim3(row_splits, c.n_kv_heads, row_tiles), s));
         }
         TRY((rows_gemm<TEPI_RESADD>(m, desc, m_upper, 1, m->ATTb, ATT_lo, tm.wo, w.wo, nullptr, m->X, nullptr, nullptr, h, qd, &pend)));
-        rmsnorm_rows_kernel<<<m_upper, 256, 0, s>>>(desc, m->X, m->splitk_ws, pend, m->max_rows, w.g2, c.rms_eps, h, m->XN, XN_lo);
+        rmsnorm_rows_kernel<<<m_upper, row_threads(h / 4, 1024), 0, s>>>(desc, m->X, m->splitk_ws, pend, m->max_rows, w.g2, c.rms_eps, h, m->XN, XN_lo);
         ++g_launches;
         CK(cudaGetLastError());
         TRY((rows_gemm<TEPI_SILU>(m, desc, m_upper, 0, m->XN, XN_lo, tm.wgu, w.wgu, nullptr, nullptr, m->ACTb, ACT_lo, 2 * f, h)));
@@ -1043,12 +1068,12 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
     }
     if (batch) {
         // final norm of every row, LM head on the tensor cores, one lowest-id argmax per row
-        rmsnorm_rows_kernel<<<m_upper, 256, 0, s>>>(desc, m->X, m->splitk_ws, 0, m->max_rows, m->gf, c.rms_eps, h, m->XN, XN_lo);
+        rmsnorm_rows_kernel<<<m_upper, row_threads(h / 4, 1024), 0, s>>>(desc, m->X, m->splitk_ws, 0, m->max_rows, m->gf, c.rms_eps, h, m->XN, XN_lo);
         ++g_launches;
         CK(cudaGetLastError());
         TRY((rows_gemm<TEPI_STORE>(m, desc, m_upper, 0, m->XN, XN_lo, m->map_lm, m->lm_head, nullptr, sc.logits_out, nullptr, nullptr, c.vocab, h)));
         if (sc.want_argmax) {
-            argmax_rows_kernel<<<m_upper, 256, 0, s>>>(desc, sc.logits_out, c.vocab, sc.vlimit > 0 ? sc.vlimit : c.vocab, sc.argmax_out);
+            argmax_rows_kernel<<<m_upper, 1024, 0, s>>>(desc, sc.logits_out, c.vocab, sc.vlimit > 0 ? sc.vlimit : c.vocab, sc.argmax_out);
             ++g_launches;
             CK(cudaGetLastError());
         }
@@ -1493,6 +1518,7 @@ static int capture_body(GenContext &c, st_model *small, cudaStream_t cap, cudaGr
     const SampleCtx sc = gen_sample_ctx(c);
     CK(cudaStreamBeginCaptureToGraph(cap, body, nullptr, nullptr, 0, cudaStreamCaptureModeRelaxed));
     int rc;
+    ++g_pdl_off;
     {
         StreamSwap swap(small, c.large, cap);
         int rows = kRowsOf[kind];
@@ -1505,6 +1531,7 @@ static int capture_body(GenContext &c, st_model *small, cudaStream_t cap, cudaGr
             if (cudaGetLastError() != cudaSuccess) rc = ST_ERR_INTERNAL;
         }
     }
+    --g_pdl_off;
     cudaGraph_t g = nullptr;
     const cudaError_t e = cudaStreamEndCapture(cap, &g);
     if (rc != ST_OK) return rc;
@@ -2039,8 +2066,8 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
         int64_t sum_new = 0;
         for (int i = 0; i < n; ++i) sum_new += mnew[i];
         const int64_t round_cap = (3ll + (P->probe_len > 1 ? P->probe_len : 1)) * (sum_new + 4ll * n + 16) + 4ll * n * (longest / max_chunk + 2);
-        // rows the target's pass waits for while the speculative model has work: an eighth of the sequences
-        int min_target_rows = n / 8;
+        // rows the target's pass waits for while the speculative model has work: 45 % of the sequences still running
+        int min_target_rows = -45;
         if (const char *e = getenv("ST_BATCH_TARGET_MIN")) min_target_rows = atoi(e);   // tuning aid
         bool finished = false;
         for (int64_t round = 0; round < round_cap && rc == ST_OK; ++round) {

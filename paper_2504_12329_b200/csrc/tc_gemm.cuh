@@ -162,7 +162,8 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
-    const int m = p.desc->m;
+    pdl_launch();
+    const int m = p.desc->m;   // set before the kernel that precedes this one was launched
     if (m <= 0) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n0 = blockIdx.x * kTcTileW * p.w_tiles;
@@ -204,14 +205,28 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             int armed = 0;
-            for (int i = 0; i < n_kb; ++i) {
-                const int s = i % p.stages, u = i / p.stages;
-                if (u > 0 && !mbar_wait(smem_u32(&s_empty[s]), (u - 1) & 1, &s_abort, p.status)) break;
+            auto load_w = [&](int i) {   // arm the stage of K block i and fetch its weight tiles
+                const int s = i % p.stages;
                 const uint32_t full = smem_u32(&s_full[s]);
                 const uint32_t base = tiles + (uint32_t)s * stage_bytes;
                 mbar_expect_tx(full, w_bytes + 2 * a_bytes_eff);
                 const int kx = (kb0 + i) * kTcBlockK;
                 for (int t = 0; t < p.w_tiles; ++t) tma_load_2d(base + (uint32_t)t * kTcWBytes, &tmW, kx, n0 + t * kTcTileW, full);
+            };
+            // the weights do not depend on the kernel before this one: the first trip round the ring fetches them
+            // while that kernel may still be running; the activations follow once it is complete
+            const int pre = min(n_kb, p.stages);
+            for (int i = 0; i < pre; ++i) load_w(i);
+            pdl_wait();
+            for (int i = 0; i < n_kb; ++i) {
+                const int s = i % p.stages, u = i / p.stages;
+                if (u > 0) {
+                    if (!mbar_wait(smem_u32(&s_empty[s]), (u - 1) & 1, &s_abort, p.status)) break;
+                    load_w(i);
+                }
+                const uint32_t full = smem_u32(&s_full[s]);
+                const uint32_t base = tiles + (uint32_t)s * stage_bytes;
+                const int kx = (kb0 + i) * kTcBlockK;
                 tma_load_2d(base + w_bytes, tmAhi, kx, 0, full);
                 tma_load_2d(base + w_bytes + a_bytes, tmAlo, kx, 0, full);
                 armed = i + 1;
@@ -254,6 +269,7 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
     } else {
         // ---------------- epilogue: TMEM -> registers -> global ----------------
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
+        pdl_wait();                             // the residual and the outputs belong to the kernels before this one
         int ok_i = lane == 0 ? (int)mbar_wait(smem_u32(&s_acc), 0, &s_abort, p.status) : 1;
         const bool ok = __shfl_sync(0xffffffffu, ok_i, 0) != 0;   // one poller per warp, uniform outcome
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
