@@ -1950,7 +1950,9 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
     int rc = ST_OK;
     uint8_t *arena = nullptr;
     BatchPlan *plan_host = nullptr;
-    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr, ev_fork = nullptr, ev_join = nullptr;
+    cudaStream_t side = nullptr;   // the speculative model's pass of a round that also has a target pass
+    static const bool overlap = [] { const char *e = getenv("ST_BATCH_OVERLAP"); return !(e && e[0] == '0'); }();
     std::vector<GenState> gs(n);
     std::vector<GenBuffers> gb(n);
     GenState *d_gs = nullptr;
@@ -2061,6 +2063,9 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
         }
         if (!up) { set_error_text("batched generation upload", cudaGetLastError()); rc = ST_ERR_INTERNAL; break; }
         if (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess) { rc = ST_ERR_INTERNAL; break; }
+        if (overlap && (cudaStreamCreateWithFlags(&side, cudaStreamNonBlocking) != cudaSuccess ||
+                        cudaEventCreateWithFlags(&ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+                        cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming) != cudaSuccess)) { rc = ST_ERR_INTERNAL; break; }
         cudaEventRecord(ev0, s);
         // ---- rounds ----
         int64_t sum_new = 0;
@@ -2083,10 +2088,19 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
             }
             const BatchPlan &pl = *plan_host;
             if (pl.all_done) { finished = true; break; }
+            // The two models' passes of a round hold different sequences and touch nothing in common: when both
+            // have rows, the speculative model's pass and routing run on a side stream beside the target's pass
+            // (its short kernels fill the gaps of the target's weight streaming) and join before the next step.
+            const bool both = overlap && large && pl.n_dec[0] > 0 && pl.n_dec[1] > 0;
+            if (both && (cudaEventRecord(ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(side, ev_fork, 0) != cudaSuccess)) {
+                rc = ST_ERR_INTERNAL;
+                break;
+            }
             for (int a = 0; a < 2 && rc == ST_OK; ++a) {
                 const int rows = pl.n_dec[a];
                 st_model *m = models[a];
                 if (rows <= 0 || !m) continue;
+                cudaStream_t ps = both && a == 0 ? side : s;
                 SampleCtx sc{};
                 sc.logits_out = m->batch_logits;
                 sc.argmax_out = d_amax + (size_t)a * max_chunk;
@@ -2094,13 +2108,17 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
                 sc.vlimit = vlimit;
                 int m_upper = (rows + 31) / 32 * 32;
                 if (m_upper > m->max_rows) m_upper = m->max_rows;
+                m->stream = ps;
                 rc = pass_rows_batch_graphed(m, d_bdesc + a, d_rtok + (size_t)a * max_chunk, m_upper, pl.max_ctx[a], sc);
+                m->stream = s;
                 if (rc != ST_OK) break;
-                batch_router_kernel<<<1, 64, 0, s>>>(d_gs, d_gb, d_pseq + (size_t)a * n, d_plast + (size_t)a * n, d_npass + a,
-                                                     d_amax + (size_t)a * max_chunk, d_descs, small->status);
+                batch_router_kernel<<<1, 64, 0, ps>>>(d_gs, d_gb, d_pseq + (size_t)a * n, d_plast + (size_t)a * n, d_npass + a,
+                                                      d_amax + (size_t)a * max_chunk, d_descs, small->status);
                 ++g_launches;
                 if (cudaGetLastError() != cudaSuccess) rc = ST_ERR_INTERNAL;
             }
+            // joined even after an error, so that nothing is still running on the side stream when the arena is freed
+            if (both && (cudaEventRecord(ev_join, side) != cudaSuccess || cudaStreamWaitEvent(s, ev_join, 0) != cudaSuccess)) rc = ST_ERR_INTERNAL;
             for (int k = 0; k < pl.n_cu && rc == ST_OK; ++k) {
                 const int i = pl.cu[k][0], a = pl.cu[k][1], rows = pl.cu[k][2], pos0 = pl.cu[k][3], emit = pl.cu[k][4];
                 st_model *m = models[a];
@@ -2167,8 +2185,14 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
         else if (dev_status) rc = ST_ERR_INTERNAL;
     } while (0);
     cudaStreamSynchronize(s);
+    if (side) {
+        cudaStreamSynchronize(side);
+        cudaStreamDestroy(side);
+    }
     if (ev0) cudaEventDestroy(ev0);
     if (ev1) cudaEventDestroy(ev1);
+    if (ev_fork) cudaEventDestroy(ev_fork);
+    if (ev_join) cudaEventDestroy(ev_join);
     if (plan_host) cudaFreeHost(plan_host);
     if (arena) cudaFree(arena);
     release_slots();
