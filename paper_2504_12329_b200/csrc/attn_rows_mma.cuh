@@ -268,11 +268,12 @@ __global__ void __launch_bounds__(kArThreads, 1) attn_rows_mma_kernel(const Attn
 
 // ---------------------------------------------------------------------------------------------
 // Batched decode attention: every row is the newest token of a different sequence.  One CTA per (kv head, row)
-// walks that sequence's keys 0 .. pos in tiles of 128 keys (TMA, three tiles in flight); warp w takes the w-th
-// group of 16 keys of every tile for the G query heads of the group, and the warps are merged through shared
-// memory at the end.  The row's own key/value is already in the cache (the rope kernel appended it).
+// walks that sequence's keys 0 .. pos in tiles of TK keys (TMA, three tiles in flight); warp w of the TK / 16 warps
+// takes the w-th group of 16 keys of every tile for the G query heads of the group, and the warps are merged
+// through shared memory at the end.  The row's own key/value is already in the cache (the rope kernel appended
+// it).  TK = 64 (four warps, two CTAs per SM: one CTA's loads cover the other's prologue, tile hand-overs and
+// merge) is what the host launches; TK = 128 (eight warps, one CTA per SM) is kept as an alternative.
 // ---------------------------------------------------------------------------------------------
-constexpr int kAbTileKeys = 128;
 constexpr int kAbStages = 3;
 
 struct AttnBatchParams {
@@ -283,14 +284,17 @@ struct AttnBatchParams {
     int32_t pages_per_seq;
 };
 
-template <int D>
-__host__ __device__ constexpr int ab_stage_bytes() { return 2 * kAbTileKeys * D * 2; }
+template <int D, int TK>
+__host__ __device__ constexpr int ab_stage_bytes() { return 2 * TK * D * 2; }
 
-template <int D, int G>
-__global__ void __launch_bounds__(kArThreads, 1) attn_batch_mma_kernel(const AttnBatchParams pp)
+template <int D, int G, int TK>
+__global__ void __launch_bounds__(2 * TK, 1) attn_batch_mma_kernel(const AttnBatchParams pp)
 {
     static_assert(G >= 1 && G <= 8, "one MMA column per head of the group");
-    constexpr int KS = D / 16, NH = D / 64, HALF_BYTES = kAbTileKeys * 128, STAGE = ab_stage_bytes<D>();
+    static_assert(TK == 64 || TK == 128, "one warp per 16 keys of a tile");
+    constexpr int kAbTileKeys = TK, NT = 2 * TK, NW = TK / 16;
+    constexpr int KS = D / 16, NH = D / 64, HALF_BYTES = kAbTileKeys * 128, STAGE = ab_stage_bytes<D, TK>();
+    static_assert(NW * G * (D + 2) * 4 <= kAbStages * STAGE, "the merge area reuses the tile ring");
     pdl_launch();
     extern __shared__ uint8_t ab_smem[];
     __shared__ uint64_t s_full[kAbStages];
@@ -371,7 +375,7 @@ __global__ void __launch_bounds__(kArThreads, 1) attn_batch_mma_kernel(const Att
         if (nk < kAbTileKeys) {   // last tile: value rows behind the last key of its group must be finite
             uint8_t *vptr = base_ptr + (size_t)s * STAGE + (size_t)NH * HALF_BYTES;
             const int pad = ((nk + 15) & ~15) - nk;
-            for (int idx = tid; idx < pad * (D / 8); idx += kArThreads) {
+            for (int idx = tid; idx < pad * (D / 8); idx += NT) {
                 const int r = nk + idx / (D / 8), c = idx % (D / 8);
                 *reinterpret_cast<uint4 *>(vptr + (size_t)(c >> 3) * HALF_BYTES + (size_t)r * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
             }
@@ -429,8 +433,8 @@ __global__ void __launch_bounds__(kArThreads, 1) attn_batch_mma_kernel(const Att
         lrun[1] += __shfl_xor_sync(0xffffffffu, lrun[1], o);
     }
     // ---- merge the warps through shared memory (the tiles are no longer needed) ----
-    float *so = reinterpret_cast<float *>(base_ptr);                 // [8 warps][G][D]
-    float *sm = so + 8 * G * D, *sd = sm + 8 * G;                    // [8][G] each
+    float *so = reinterpret_cast<float *>(base_ptr);                 // [NW warps][G][D]
+    float *sm = so + NW * G * D, *sd = sm + NW * G;                  // [NW][G] each
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
         const int head = 2 * t + e;
@@ -445,14 +449,14 @@ __global__ void __launch_bounds__(kArThreads, 1) attn_batch_mma_kernel(const Att
     }
     __syncthreads();
     const int hq0 = hk * G;
-    for (int idx = tid; idx < G * D; idx += kArThreads) {
+    for (int idx = tid; idx < G * D; idx += NT) {
         const int g = idx / D, c = idx - g * D;
         float mnew = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < 8; ++w) mnew = fmaxf(mnew, sm[w * G + g]);
+        for (int w = 0; w < NW; ++w) mnew = fmaxf(mnew, sm[w * G + g]);
         float dsum = 0.f, osum = 0.f;
 #pragma unroll
-        for (int w = 0; w < 8; ++w) {
+        for (int w = 0; w < NW; ++w) {
             const float mw = sm[w * G + g];
             if (mw != -INFINITY) {
                 const float cw = __expf(mw - mnew);

@@ -79,7 +79,7 @@ struct st_model {
     int32_t *row_slot = nullptr, *row_pos = nullptr;   // device [max_rows]: sequence and position of every row of a batched decode pass
     float *batch_logits = nullptr;         // [max_rows][vocab], allocated on first use
     struct BatchGraph {                    // a captured batched decode pass, keyed by everything baked into its nodes
-        int m_upper, vlimit;
+        int m_upper, vlimit, tile;         // tile: keys per attention tile (chosen from the context bound)
         const int32_t *tok;
         const StepDesc *desc;
         float *logits;
@@ -314,39 +314,58 @@ static cudaError_t launch_attn_rows_mma(const AttnRowsMmaParams &p, int D, int G
     return cudaErrorInvalidValue;
 }
 
-// Batched decode attention: grid = (kv heads, rows).
-template <int D, int G>
-static cudaError_t launch_attn_batch_dg(const AttnBatchParams &p, dim3 grid, cudaStream_t s, bool attr_only)
+// Batched decode attention: grid = (kv heads, rows); tk = keys per tile (64 or 128).
+template <int D, int G, int TK>
+static cudaError_t launch_attn_batch_dgt(const AttnBatchParams &p, dim3 grid, cudaStream_t s, bool attr_only)
 {
-    auto kern = attn_batch_mma_kernel<D, G>;
-    const size_t smem = 1024 + (size_t)kAbStages * ab_stage_bytes<D>();
+    auto kern = attn_batch_mma_kernel<D, G, TK>;
+    const size_t smem = 1024 + (size_t)kAbStages * ab_stage_bytes<D, TK>();
     if (attr_only) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    kern<<<grid, kArThreads, smem, s>>>(p);
+    kern<<<grid, 2 * TK, smem, s>>>(p);
     ++g_launches;
     return cudaGetLastError();
 }
 
+template <int D, int G>
+static cudaError_t launch_attn_batch_dg(const AttnBatchParams &p, dim3 grid, cudaStream_t s, int tk, bool attr_only)
+{
+    if (attr_only) {
+        const cudaError_t e = launch_attn_batch_dgt<D, G, 64>(p, grid, s, true);
+        return e != cudaSuccess ? e : launch_attn_batch_dgt<D, G, 128>(p, grid, s, true);
+    }
+    return tk == 64 ? launch_attn_batch_dgt<D, G, 64>(p, grid, s, false) : launch_attn_batch_dgt<D, G, 128>(p, grid, s, false);
+}
+
 template <int D>
-static cudaError_t launch_attn_batch_d(const AttnBatchParams &p, int G, dim3 grid, cudaStream_t s, bool attr_only)
+static cudaError_t launch_attn_batch_d(const AttnBatchParams &p, int G, dim3 grid, cudaStream_t s, int tk, bool attr_only)
 {
     switch (G) {
-    case 1: return launch_attn_batch_dg<D, 1>(p, grid, s, attr_only);
-    case 2: return launch_attn_batch_dg<D, 2>(p, grid, s, attr_only);
-    case 3: return launch_attn_batch_dg<D, 3>(p, grid, s, attr_only);
-    case 4: return launch_attn_batch_dg<D, 4>(p, grid, s, attr_only);
-    case 5: return launch_attn_batch_dg<D, 5>(p, grid, s, attr_only);
-    case 6: return launch_attn_batch_dg<D, 6>(p, grid, s, attr_only);
-    case 7: return launch_attn_batch_dg<D, 7>(p, grid, s, attr_only);
-    case 8: return launch_attn_batch_dg<D, 8>(p, grid, s, attr_only);
+    case 1: return launch_attn_batch_dg<D, 1>(p, grid, s, tk, attr_only);
+    case 2: return launch_attn_batch_dg<D, 2>(p, grid, s, tk, attr_only);
+    case 3: return launch_attn_batch_dg<D, 3>(p, grid, s, tk, attr_only);
+    case 4: return launch_attn_batch_dg<D, 4>(p, grid, s, tk, attr_only);
+    case 5: return launch_attn_batch_dg<D, 5>(p, grid, s, tk, attr_only);
+    case 6: return launch_attn_batch_dg<D, 6>(p, grid, s, tk, attr_only);
+    case 7: return launch_attn_batch_dg<D, 7>(p, grid, s, tk, attr_only);
+    case 8: return launch_attn_batch_dg<D, 8>(p, grid, s, tk, attr_only);
     }
     return cudaErrorInvalidValue;
 }
 
-static cudaError_t launch_attn_batch(const AttnBatchParams &p, int D, int G, dim3 grid, cudaStream_t s, bool attr_only = false)
+static cudaError_t launch_attn_batch(const AttnBatchParams &p, int D, int G, dim3 grid, cudaStream_t s, int tk, bool attr_only = false)
 {
-    if (D == 64) return launch_attn_batch_d<64>(p, G, grid, s, attr_only);
-    if (D == 128) return launch_attn_batch_d<128>(p, G, grid, s, attr_only);
+    if (D == 64) return launch_attn_batch_d<64>(p, G, grid, s, tk, attr_only);
+    if (D == 128) return launch_attn_batch_d<128>(p, G, grid, s, tk, attr_only);
     return cudaErrorInvalidValue;
+}
+
+// Keys per tile of the batched attention: 64 (two CTAs per SM) was the faster one at every context measured,
+// 512 to 4000 keys; ST_AB_TILE=128 selects the 128-key kernel.
+static int attn_batch_tile(int ctx_upper)
+{
+    (void)ctx_upper;
+    static const int forced = [] { const char *e = getenv("ST_AB_TILE"); return e ? atoi(e) : 0; }();
+    return forced == 128 ? 128 : 64;
 }
 
 static cudaError_t launch_attn(const AttnParams &p, int D, int G, dim3 grid, cudaStream_t s)
@@ -894,7 +913,7 @@ static int mega_attr_all()
         for (int G = 1; G <= 8; ++G) {
             CK(mega_launch(MegaParams{}, D, G, 0, 0, nullptr, true));
             CK(launch_attn_rows_mma(AttnRowsMmaParams{}, D, G, dim3(1, 1, 1), nullptr, true));
-            CK(launch_attn_batch(AttnBatchParams{}, D, G, dim3(1, 1, 1), nullptr, true));
+            CK(launch_attn_batch(AttnBatchParams{}, D, G, dim3(1, 1, 1), nullptr, 128, true));
         }
     return ST_OK;
 }
@@ -929,7 +948,7 @@ static int pass_decode(st_model *m, const StepDesc *desc, const int32_t *tok, in
     return ST_OK;
 }
 
-// Decode pass, one kernel per phase (debugging aid).  ctx_upper bounds the number of keys (chooses the key split).  ctx_upper bounds the number of keys (chooses the key split).
+// Decode pass, one kernel per phase (debugging aid).  ctx_upper bounds the number of keys (chooses the key split).
 static int pass_decode_multi(st_model *m, const StepDesc *desc, const int32_t *tok, int slot, int ctx_upper, const SampleCtx &sc)
 {
     const st_config &c = m->cfg;
@@ -1046,7 +1065,7 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
             ab.row_slot = m->row_slot;
             ab.row_pos = m->row_pos;
             ab.pages_per_seq = m->pages_per_seq;
-            CK(launch_attn_batch(ab, D, G, dim3(c.n_kv_heads, m_upper), s));
+            CK(launch_attn_batch(ab, D, G, dim3(c.n_kv_heads, m_upper), s, attn_batch_tile(ctx_upper)));
         } else if (m->simt_attn) {
             CK(launch_attn_rows(a, D, G, dim3(row_splits, c.n_kv_heads, row_tiles), s));
         } else {
@@ -1093,7 +1112,7 @@ static int pass_rows_batch_graphed(st_model *m, const StepDesc *desc, const int3
     if (off || cudaStreamIsCapturing(m->stream, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone)
         return pass_rows(m, desc, tok, -1, m_upper, ctx_upper, true, sc, true);
     for (auto &g : m->batch_graphs)
-        if (g.m_upper == m_upper && g.vlimit == sc.vlimit && g.tok == tok && g.desc == desc && g.logits == sc.logits_out &&
+        if (g.m_upper == m_upper && g.vlimit == sc.vlimit && g.tile == attn_batch_tile(ctx_upper) && g.tok == tok && g.desc == desc && g.logits == sc.logits_out &&
             g.argmax == (sc.want_argmax ? sc.argmax_out : nullptr)) {
             CK(cudaGraphLaunch(g.exec, m->stream));
             g_launches += g.launches;
@@ -1122,7 +1141,7 @@ static int pass_rows_batch_graphed(st_model *m, const StepDesc *desc, const int3
         return rc;
     }
     CK(e);
-    st_model::BatchGraph g{m_upper, sc.vlimit, tok, desc, sc.logits_out, sc.want_argmax ? sc.argmax_out : nullptr, nullptr, g_launches - before};
+    st_model::BatchGraph g{m_upper, sc.vlimit, attn_batch_tile(ctx_upper), tok, desc, sc.logits_out, sc.want_argmax ? sc.argmax_out : nullptr, nullptr, g_launches - before};
     const cudaError_t ei = cudaGraphInstantiate(&g.exec, graph, 0);
     cudaGraphDestroy(graph);
     CK(ei);
