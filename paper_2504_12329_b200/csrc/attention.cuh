@@ -68,6 +68,7 @@ __global__ void __launch_bounds__(512) rope_append_kernel(const StepDesc *desc, 
                                                           const int32_t *row_pos = nullptr, int pages_per_seq = 0)
 {
     pdl_launch();
+    pdl_wait();
     const int i = blockIdx.x;
     if (i >= desc->m) return;
     if (row_slot) kv.block_tab += (size_t)row_slot[i] * pages_per_seq;   // batched decode: kv.block_tab is sequence 0's table

@@ -17,6 +17,7 @@ __global__ void __launch_bounds__(1024) rmsnorm_rows_kernel(const StepDesc *desc
                                                            const float *gain, float eps, int hidden, uint16_t *XN_hi, uint16_t *XN_lo)
 {
     pdl_launch();   // the projection that follows may fetch its weights meanwhile
+    pdl_wait();     // the row and its partial sums come from the kernels before this one
     const int i = blockIdx.x;
     if (i >= desc->m) return;
     float4 *x4 = reinterpret_cast<float4 *>(X + (size_t)i * hidden);

@@ -432,6 +432,24 @@ static int make_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint
 static int g_pdl_off = 0;
 static bool pdl_enabled() { return use_pdl() && g_pdl_off == 0; }
 
+// Launch of a kernel that begins with pdl_launch(); pdl_wait(): with programmatic stream serialization its CTAs are
+// scheduled while the kernel before it drains.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, cudaStream_t s, Args... args)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    ++g_launches;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 template <int EPI>
 // pending_splits: when given, a K-split projection leaves its partial sums in the workspace and reports the split
 // count there (0: the output is complete) -- the kernel that consumes the output adds them up.
@@ -1042,16 +1060,14 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
         const LayerWeights &w = m->layers[l];
         const LayerMaps &tm = m->maps[l];
         // the previous layer's down projection may have left its K-split partial sums for this kernel to add
-        rmsnorm_rows_kernel<<<m_upper, row_threads(h / 4, 1024), 0, s>>>(desc, m->X, m->splitk_ws, pend_down, m->max_rows, w.g1, c.rms_eps, h, m->XN, XN_lo);
-        ++g_launches;
-        CK(cudaGetLastError());
+        CK(launch_dependent(rmsnorm_rows_kernel, dim3(m_upper), dim3(row_threads(h / 4, 1024)), s, desc, m->X, m->splitk_ws, pend_down, m->max_rows,
+                            w.g1, c.rms_eps, h, m->XN, XN_lo));
         int pend = 0;
         TRY((rows_gemm<TEPI_STORE>(m, desc, m_upper, 0, m->XN, XN_lo, tm.wqkv, w.wqkv, w.bqkv, m->QKV, nullptr, nullptr, qd + 2 * kd, h, &pend)));
         const KvView kv = kv_view(m, l, batch ? 0 : slot);
-        rope_append_kernel<<<m_upper, row_threads((c.n_q_heads + c.n_kv_heads) * D / 8, 512), 0, s>>>(desc, m->QKV, m->splitk_ws, pend, m->max_rows, w.bqkv, m->cs, c.n_q_heads, c.n_kv_heads, D, kv,
-                                                   m->status, batch ? m->row_slot : nullptr, batch ? m->row_pos : nullptr, m->pages_per_seq);
-        ++g_launches;
-        CK(cudaGetLastError());
+        CK(launch_dependent(rope_append_kernel, dim3(m_upper), dim3(row_threads((c.n_q_heads + c.n_kv_heads) * D / 8, 512)), s, desc, m->QKV,
+                            m->splitk_ws, pend, m->max_rows, w.bqkv, m->cs, c.n_q_heads, c.n_kv_heads, D, kv, m->status,
+                            batch ? m->row_slot : nullptr, batch ? m->row_pos : nullptr, m->pages_per_seq));
         AttnParams a{};
         a.desc = desc; a.qkv = m->QKV; a.kv = kv; a.out_f32 = nullptr; a.out_hi = m->ATTb; a.out_lo = ATT_lo;
         a.part_o = m->part_o; a.part_ml = m->part_ml; a.tickets = m->tickets; a.status = m->status;
@@ -1077,9 +1093,8 @@ static int pass_rows(st_model *m, const StepDesc *desc, const int32_t *tok, int 
             CK(launch_attn_rows_mma(am, D, G, dim3(row_splits, c.n_kv_heads, row_tiles), s));
         }
         TRY((rows_gemm<TEPI_RESADD>(m, desc, m_upper, 1, m->ATTb, ATT_lo, tm.wo, w.wo, nullptr, m->X, nullptr, nullptr, h, qd, &pend)));
-        rmsnorm_rows_kernel<<<m_upper, row_threads(h / 4, 1024), 0, s>>>(desc, m->X, m->splitk_ws, pend, m->max_rows, w.g2, c.rms_eps, h, m->XN, XN_lo);
-        ++g_launches;
-        CK(cudaGetLastError());
+        CK(launch_dependent(rmsnorm_rows_kernel, dim3(m_upper), dim3(row_threads(h / 4, 1024)), s, desc, m->X, m->splitk_ws, pend, m->max_rows,
+                            w.g2, c.rms_eps, h, m->XN, XN_lo));
         TRY((rows_gemm<TEPI_SILU>(m, desc, m_upper, 0, m->XN, XN_lo, tm.wgu, w.wgu, nullptr, nullptr, m->ACTb, ACT_lo, 2 * f, h)));
         // the last layer's down projection reduces its own splits: the final norm belongs to the LM head
         TRY((rows_gemm<TEPI_RESADD>(m, desc, m_upper, 2, m->ACTb, ACT_lo, tm.wd, w.wd, nullptr, m->X, nullptr, nullptr, h, f,
