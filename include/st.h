@@ -208,6 +208,15 @@ int64_t st_kv_bytes_per_token(const st_model *m);
 int64_t st_kernel_launches(void);
 int st_time_gemv(st_model *m, int32_t which, int32_t iters, double *seconds_out);
 
+/* How the single-kernel decode step lays out its attention phase (Section 3 names no kernel; this describes the
+ * split-KV decode attention of the hot path) when `ctx` tokens are cached: key splits per kv head, the capacity in
+ * keys of a CTA's K/V staging area, the most staging chunks any (kv head, split) unit streams through it, and
+ * whether the unit that holds the step's own key reaches its last chunk with no cached key left for it.  Host
+ * arithmetic only (the same function the kernel evaluates); every output pointer may be NULL.  Tests use it to
+ * prove that a case really takes the multi-chunk path. */
+int st_decode_geometry(const st_model *m, int32_t ctx, int32_t *n_splits, int32_t *kv_cap, int32_t *max_chunks,
+                       int32_t *own_chunk_empty);
+
 /* Greedy sampling that allocates nothing (the paper has no counterpart: this is a service entry point).
  * For callers that must not call cudaMalloc -- code running while another component owns the whole
  * device memory pool, or inside a region where allocation is forbidden or would synchronise the device.

@@ -110,6 +110,8 @@ def lib():
         L.orc_kv_truncate.argtypes = [C.c_void_p, C.c_int64]
         L.orc_forward.restype = C.c_int
         L.orc_forward.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]
+        L.orc_forward_last.restype = C.c_int
+        L.orc_forward_last.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
         L.orc_forward_full.restype = C.c_int
         L.orc_forward_full.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
         L.orc_argmax.restype = C.c_int32
@@ -243,6 +245,16 @@ class KV:
         rc = lib().orc_forward(self.model.h, self.h, _p(t), t.size, int(all_rows), _p(out))
         if rc != 0:
             raise RuntimeError(f"orc_forward rc={rc}")
+        return out
+
+    def forward_last(self, tokens) -> np.ndarray:
+        """forward(tokens) with the last layer's attention and FFN evaluated only for the last row (the only row
+        the returned logits depend on); keys and values of every row are cached as usual."""
+        t = np.ascontiguousarray(tokens, dtype=np.int32)
+        out = np.empty((self.model.cfg.vocab,), dtype=np.float64)
+        rc = lib().orc_forward_last(self.model.h, self.h, _p(t), t.size, _p(out))
+        if rc != 0:
+            raise RuntimeError(f"orc_forward_last rc={rc}")
         return out
 
 

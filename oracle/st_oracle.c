@@ -340,7 +340,7 @@ static void lm_head(const orc_model *m, const double *X, int rows, int all_rows,
  * and including itself.  logits: [rows][vocab] if all_rows, else [vocab] for
  * the last fed position; may be NULL.  Returns 0, or -1 when the cache is
  * too small. */
-int orc_forward(const orc_model *m, orc_kv *kv, const int32_t *tokens, int rows, int all_rows, double *logits)
+static int forward_rows(const orc_model *m, orc_kv *kv, const int32_t *tokens, int rows, int all_rows, double *logits, int skip_unread)
 {
     const orc_config *c = &m->c;
     int h = c->hidden, d = c->head_dim, Hq = c->n_q_heads, Hkv = c->n_kv_heads, f = c->ffn;
@@ -359,35 +359,55 @@ int orc_forward(const orc_model *m, orc_kv *kv, const int32_t *tokens, int rows,
     embed_rows(m, tokens, rows, X);
     for (int l = 0; l < c->n_layers; ++l) {
         double *kl = kv->k + (size_t)l * kv->cap * kd, *vl = kv->v + (size_t)l * kv->cap * kd;
+        /* r0: first row whose attention / FFN result anything reads.  Keys and values are needed for every
+         * row; with skip_unread the last layer's remaining work is done for the last row only (the only row
+         * the returned logits depend on). */
+        int r0 = (skip_unread && !all_rows && l == c->n_layers - 1) ? rows - 1 : 0;
+        int nr = rows - r0;
         for (int i = 0; i < rows; ++i) orc_rmsnorm(X + (int64_t)i * h, m->gain[layer_tid(l, 0)], h, c->rms_eps, XN + (int64_t)i * h);
-        linear(m, layer_tid(l, T_WQ), qd, h, layer_tid(l, T_BQ), c->qkv_bias, XN, rows, Q);
+        linear(m, layer_tid(l, T_WQ), qd, h, layer_tid(l, T_BQ), c->qkv_bias, XN + (int64_t)r0 * h, nr, Q + (int64_t)r0 * qd);
         linear(m, layer_tid(l, T_WK), kd, h, layer_tid(l, T_BK), c->qkv_bias, XN, rows, Kn);
         linear(m, layer_tid(l, T_WV), kd, h, layer_tid(l, T_BV), c->qkv_bias, XN, rows, Vn);
         for (int i = 0; i < rows; ++i) {
-            for (int hq = 0; hq < Hq; ++hq) orc_rope(Q + (int64_t)i * qd + hq * d, d, p0 + i, c->rope_theta);
+            if (i >= r0)
+                for (int hq = 0; hq < Hq; ++hq) orc_rope(Q + (int64_t)i * qd + hq * d, d, p0 + i, c->rope_theta);
             for (int hk = 0; hk < Hkv; ++hk) orc_rope(Kn + (int64_t)i * kd + hk * d, d, p0 + i, c->rope_theta);
             memcpy(kl + (p0 + i) * kd, Kn + (int64_t)i * kd, (size_t)kd * sizeof(double));
             memcpy(vl + (p0 + i) * kd, Vn + (int64_t)i * kd, (size_t)kd * sizeof(double));
         }
 #pragma omp parallel for collapse(2) schedule(dynamic)
-        for (int i = 0; i < rows; ++i)
+        for (int i = r0; i < rows; ++i)
             for (int hq = 0; hq < Hq; ++hq) {
                 int hk = hq / grp; /* consecutive q heads share a kv head */
                 orc_attend(Q + (int64_t)i * qd + hq * d, kl + hk * d, vl + hk * d, p0 + i + 1, d, kd, A + (int64_t)i * qd + hq * d);
             }
-        linear(m, layer_tid(l, T_WO), h, qd, 0, 0, A, rows, D);
-        for (int64_t i = 0; i < (int64_t)rows * h; ++i) X[i] += D[i];
-        for (int i = 0; i < rows; ++i) orc_rmsnorm(X + (int64_t)i * h, m->gain[layer_tid(l, 8)], h, c->rms_eps, XN + (int64_t)i * h);
-        linear(m, layer_tid(l, T_WG), f, h, 0, 0, XN, rows, G);
-        linear(m, layer_tid(l, T_WU), f, h, 0, 0, XN, rows, U);
-        for (int64_t i = 0; i < (int64_t)rows * f; ++i) G[i] = orc_silu(G[i]) * U[i];
-        linear(m, layer_tid(l, T_WD), h, f, 0, 0, G, rows, D);
-        for (int64_t i = 0; i < (int64_t)rows * h; ++i) X[i] += D[i];
+        linear(m, layer_tid(l, T_WO), h, qd, 0, 0, A + (int64_t)r0 * qd, nr, D + (int64_t)r0 * h);
+        for (int64_t i = (int64_t)r0 * h; i < (int64_t)rows * h; ++i) X[i] += D[i];
+        for (int i = r0; i < rows; ++i) orc_rmsnorm(X + (int64_t)i * h, m->gain[layer_tid(l, 8)], h, c->rms_eps, XN + (int64_t)i * h);
+        linear(m, layer_tid(l, T_WG), f, h, 0, 0, XN + (int64_t)r0 * h, nr, G + (int64_t)r0 * f);
+        linear(m, layer_tid(l, T_WU), f, h, 0, 0, XN + (int64_t)r0 * h, nr, U + (int64_t)r0 * f);
+        for (int64_t i = (int64_t)r0 * f; i < (int64_t)rows * f; ++i) G[i] = orc_silu(G[i]) * U[i];
+        linear(m, layer_tid(l, T_WD), h, f, 0, 0, G + (int64_t)r0 * f, nr, D + (int64_t)r0 * h);
+        for (int64_t i = (int64_t)r0 * h; i < (int64_t)rows * h; ++i) X[i] += D[i];
     }
     kv->len += rows;
     if (logits) lm_head(m, X, rows, all_rows, logits);
     free(X); free(XN); free(Q); free(Kn); free(Vn); free(A); free(D); free(G); free(U);
     return 0;
+}
+
+int orc_forward(const orc_model *m, orc_kv *kv, const int32_t *tokens, int rows, int all_rows, double *logits)
+{
+    return forward_rows(m, kv, tokens, rows, all_rows, logits, 0);
+}
+
+/* The same pass with the work nothing reads left out: when only the last row's logits are returned, the last
+ * layer's attention, output projection and FFN are evaluated for that row alone (keys and values are still stored
+ * for every row).  No result changes; long contexts get affordable (a one-layer model's pass becomes linear in
+ * the number of rows).  Pinned to orc_forward by equality in tests/test_oracle_model.py. */
+int orc_forward_last(const orc_model *m, orc_kv *kv, const int32_t *tokens, int rows, double *logits)
+{
+    return forward_rows(m, kv, tokens, rows, 0, logits, 1);
 }
 
 /* Full recompute without any cache: the reference definition of the causal

@@ -68,7 +68,7 @@ EXPORTS = [
     "st_model_create", "st_model_destroy", "st_seq_alloc", "st_seq_free", "st_seq_reserve", "st_kv_len",
     "st_kv_truncate", "st_prefill", "st_decode_step", "st_generate_spec", "st_fill_tensor_bf16",
     "st_weight_bytes", "st_kv_bytes_per_token", "st_last_device_status", "st_strerror",
-    "st_kernel_launches", "st_time_gemv", "st_argmax_static", "st_generate_spec_batch",
+    "st_kernel_launches", "st_time_gemv", "st_argmax_static", "st_generate_spec_batch", "st_decode_geometry",
 ]
 
 _lib = None
@@ -119,6 +119,8 @@ def lib():
                                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.st_argmax_static.restype = C.c_int
         L.st_argmax_static.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+        L.st_decode_geometry.restype = C.c_int
+        L.st_decode_geometry.argtypes = [C.c_void_p, C.c_int32] + [C.POINTER(C.c_int32)] * 4
         L.st_strerror.restype = C.c_char_p
         L.st_strerror.argtypes = [C.c_int]
         _lib = L
@@ -265,6 +267,12 @@ class Model:
 
     def st_kv_truncate(self, slot: int, new_len: int):
         _check(lib().st_kv_truncate(self.h, slot, new_len), "st_kv_truncate")
+
+    def st_decode_geometry(self, ctx: int) -> dict:
+        """Attention layout of the single-kernel decode step with ctx tokens cached (host arithmetic)."""
+        v = [C.c_int32() for _ in range(4)]
+        _check(lib().st_decode_geometry(self.h, ctx, *[C.byref(x) for x in v]), "st_decode_geometry")
+        return dict(n_splits=v[0].value, kv_cap=v[1].value, max_chunks=v[2].value, own_chunk_empty=bool(v[3].value))
 
     # --- passes ----------------------------------------------------------------------------
     def st_prefill(self, slot: int, tokens, last_logits=None):

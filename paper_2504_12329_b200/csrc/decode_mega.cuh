@@ -493,31 +493,59 @@ __device__ __forceinline__ uint32_t mega_kv_swz(const MegaUnit &u, int row, int 
     return (uint32_t)(d >> 6) * u.half_bytes + (uint32_t)row * 128 + (cb ^ ((uint32_t)(row & 7) << 4));
 }
 
+// Key splits of a decode step at position pos: 64 keys per unit while there are CTAs to spare.
+__host__ __device__ __forceinline__ int mega_key_splits(int pos, int n_splits_max, int n_cta, int Hkv)
+{
+    int ns = (pos + 64) / 64;
+    const int fit = n_cta / Hkv > 1 ? n_cta / Hkv : 1;
+    const int cap = n_splits_max < fit ? n_splits_max : fit;
+    return ns < cap ? ns : cap;
+}
+
+// Rows and staging chunks of key split `split` of `ns` at position pos (kv_cap: staging capacity in keys).
+struct MegaUnitShape {
+    int k0a, lead, n_rows, n_cached, owner, CH, nch;
+};
+__host__ __device__ __forceinline__ MegaUnitShape mega_unit_shape(int pos, int ns, int split, int kv_cap)
+{
+    MegaUnitShape u;
+    const int n_keys = pos + 1;
+    const int per = (n_keys + ns - 1) / ns;
+    const int k0 = split * per;
+    const int k1 = n_keys < k0 + per ? n_keys : k0 + per;
+    const int n_all = k1 > k0 ? k1 - k0 : 0;
+    u.owner = (k0 <= pos && pos < k1) ? 1 : 0;
+    u.k0a = k0 & ~15;   // staging boxes hold 16 keys
+    u.lead = k0 - u.k0a;
+    u.n_rows = n_all > 0 ? u.lead + n_all : 0;
+    u.n_cached = n_all > 0 ? u.n_rows - u.owner : 0;
+    if (u.n_rows <= kv_cap) {
+        u.CH = kv_cap;
+        u.nch = u.n_rows > 0 ? 1 : 0;
+    } else {
+        u.CH = (kv_cap >> 1) & ~15;
+        u.nch = (u.n_rows + u.CH - 1) / u.CH;
+    }
+    return u;
+}
+
 // Geometry of this CTA's unit for the whole step (the same in every layer).
 template <int D>
 __device__ __forceinline__ MegaUnit mega_unit(const MegaParams &p, uint8_t *base_ptr, uint32_t base, int pos, int ns)
 {
+    static_assert(kMegaKvBoxRows == 16, "mega_unit_shape rounds to boxes of 16 keys");
     MegaUnit u;
     u.ns = ns;
     u.hk = blockIdx.x / ns;
     u.split = blockIdx.x - u.hk * ns;
-    const int n_keys = pos + 1;
-    const int per = (n_keys + ns - 1) / ns;
-    const int k0 = u.split * per;
-    const int k1 = min(n_keys, k0 + per);
-    const int n_all = max(0, k1 - k0);
-    u.owner = (k0 <= pos && pos < k1) ? 1 : 0;
-    u.k0a = k0 & ~(kMegaKvBoxRows - 1);
-    u.lead = k0 - u.k0a;
-    u.n_rows = n_all > 0 ? u.lead + n_all : 0;
-    u.n_cached = n_all > 0 ? u.n_rows - u.owner : 0;
-    if (u.n_rows <= p.kv_cap) {
-        u.CH = p.kv_cap;
-        u.nch = u.n_rows > 0 ? 1 : 0;
-    } else {
-        u.CH = (p.kv_cap >> 1) & ~15;
-        u.nch = (u.n_rows + u.CH - 1) / u.CH;
-    }
+    const MegaUnitShape sh = mega_unit_shape(pos, ns, u.split, p.kv_cap);
+    u.owner = sh.owner;
+    u.k0a = sh.k0a;
+    u.lead = sh.lead;
+    u.n_rows = sh.n_rows;
+    u.n_cached = sh.n_cached;
+    u.CH = sh.CH;
+    u.nch = sh.nch;
     u.pg0 = u.k0a >> p.kv.page_shift;
     u.half_bytes = (uint32_t)p.kv_cap * 128;
     u.kbase = base + (uint32_t)p.kv_off;
@@ -948,9 +976,8 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
         sincos((double)pos * p.inv_freq[j], &s, &c);
         sh.cs[j] = make_float2((float)c, (float)s);
     }
-    // 64 keys per unit while there are CTAs to spare (every CTA derives the same split count)
-    int ns = (pos + 64) / 64;
-    ns = min(ns, min(p.n_splits, max(1, (int)gridDim.x / p.Hkv)));
+    // every CTA derives the same split count
+    const int ns = mega_key_splits(pos, p.n_splits, (int)gridDim.x, p.Hkv);
     const bool attn_active = (int)blockIdx.x < p.Hkv * ns;
     const MegaUnit unit = mega_unit<D>(p, base_ptr, base, pos, ns);
     if (attn_active && unit.n_cached > 0) {

@@ -806,6 +806,10 @@ static int model_build(st_model *m)
         xarea += (size_t)((budget - (long long)xarea - (long long)m->mega_stages * kMegaTileBytes) / 1024 * 1024);
         int cap = (int)((xarea - kv_off) / (2 * kv_row)) & ~15;
         if (cap > 1024) cap = 1024;
+        if (const char *ec = getenv("ST_MEGA_KV_CAP")) {   // test aid: a small staging area makes short contexts stream in chunks
+            const int want = atoi(ec) & ~15;
+            if (want >= 32 && want < cap) cap = want;
+        }
         m->mega_kv_off = (int)kv_off;
         m->mega_kv_cap = cap;
         m->mega_xarea = (int)xarea;
@@ -1239,6 +1243,23 @@ int64_t st_kv_bytes_per_token(const st_model *m)
 }
 
 int64_t st_kernel_launches(void) { return g_launches; }
+
+int st_decode_geometry(const st_model *m, int32_t ctx, int32_t *n_splits, int32_t *kv_cap, int32_t *max_chunks, int32_t *own_chunk_empty)
+{
+    if (!m || ctx < 0) return ST_ERR_ARG;
+    const int ns = mega_key_splits(ctx, m->mega_splits, m->sm_count, m->cfg.n_kv_heads);
+    int most = 0, empty = 0;
+    for (int sp = 0; sp < ns; ++sp) {
+        const MegaUnitShape u = mega_unit_shape(ctx, ns, sp, m->mega_kv_cap);
+        if (u.nch > most) most = u.nch;
+        if (u.owner && u.nch > 1 && u.n_cached == (u.nch - 1) * u.CH) empty = 1;
+    }
+    if (n_splits) *n_splits = ns;
+    if (kv_cap) *kv_cap = m->mega_kv_cap;
+    if (max_chunks) *max_chunks = most;
+    if (own_chunk_empty) *own_chunk_empty = empty;
+    return ST_OK;
+}
 
 #ifdef ST_MEGA_TRACE
 int st_debug_trace(unsigned long long *out, int n) { return (int)cudaMemcpyFromSymbol(out, g_mega_trace, (size_t)n * 8); }

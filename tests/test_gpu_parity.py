@@ -483,3 +483,29 @@ def test_sentence_probe_on_device(B, oracle, keep):
                 assert got.emission_argmax[t] == want.emission_argmax[t]
     gs.close()
     gl.close()
+
+
+def test_hand_traced_rule_cases_on_device(B):
+    """The hand-traced streams of tests/golden (cue precedence inside a probe sentence, the reflection counter
+    crossing its threshold and restarting, probe sentences cut by end-of-sequence or the budget in both probe
+    readings, a delimiter inside a probe, verification cues in the target's own sentences): the device's
+    routing must reproduce every one of them bit for bit, alone and in batched rounds.  No oracle is involved:
+    the expected values were traced by hand from the paper's rules."""
+    from test_oracle_spec import RULE_TRACES, assert_matches_trace, load_rule_trace
+    S, L = shape_dict(W.TINY_S), shape_dict(W.TINY_L)
+    gs = B.Model(S, seed=0, tag=0, max_seqs=2, max_tokens=512)
+    gl = B.Model(L, seed=0, tag=1, max_seqs=2, max_tokens=512)
+    for name in RULE_TRACES:
+        T, params = load_rule_trace(name)
+        got = B.st_generate_spec(gs, gl, T["prompt"], max_new_tokens=T["max_new"], force=T["force"], **params)
+        assert_matches_trace(got, T)
+        twice = B.st_generate_spec_batch(gs, gl, [T["prompt"], T["prompt"]], max_new_tokens=T["max_new"],
+                                         forces=[T["force"], T["force"]], **params)
+        for r in twice:
+            assert_matches_trace(r, T)
+        if "budget" in T:
+            cut = B.st_generate_spec(gs, gl, T["prompt"], max_new_tokens=T["budget"], force=T["force"], **dict(params, eos_id=-1))
+            assert cut.tokens.tolist() == T["budget_tokens"] and len(cut.emission_tokens) == T["budget_steps"]
+            assert cut.handoffs == T["handoffs"]
+    gs.close()
+    gl.close()

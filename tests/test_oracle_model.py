@@ -114,6 +114,26 @@ def test_cached_decode_equals_full_recompute(oracle):
     assert np.allclose(om.forward_full(tokens[:8]), full[:8], atol=1e-12)
 
 
+def test_last_row_only_pass_equals_full_pass(oracle):
+    """forward_last leaves out work nothing reads; its logits and its cache must equal forward's, for one and
+    several layers, from an empty and from a filled cache, and later steps on top of either cache must agree."""
+    rng = np.random.default_rng(4)
+    for n_layers in (1, 2, 3):
+        cfg = _cfg(oracle, n_layers=n_layers)
+        om = oracle.Model(cfg, 2, 0)
+        tokens = rng.integers(0, cfg.vocab, size=23).astype(np.int32)
+        full = om.forward_full(tokens)
+        a, b = oracle.KV(om, 32), oracle.KV(om, 32)
+        for lo, hi in ((0, 9), (9, 10), (10, 21)):
+            za, zb = a.forward(tokens[lo:hi]), b.forward_last(tokens[lo:hi])
+            assert np.array_equal(za, zb)
+            assert np.allclose(zb, full[hi - 1], atol=1e-12)
+            assert len(a) == len(b) == hi
+        # the caches are interchangeable afterwards
+        assert np.array_equal(a.forward(tokens[21:22]), b.forward(tokens[21:22]))
+        assert np.allclose(b.forward(tokens[22:23]), full[22], atol=1e-12)
+
+
 def test_gqa_equals_mha_with_repeated_kv(oracle):
     cfg_g = _cfg(oracle, n_layers=1, n_q_heads=4, n_kv_heads=2)
     cfg_m = _cfg(oracle, n_layers=1, n_q_heads=4, n_kv_heads=4)

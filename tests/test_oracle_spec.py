@@ -28,6 +28,43 @@ def _trace(name):
     return out
 
 
+LIST_PARAMS = ("keyword_ids", "affirmation_ids", "verification_ids", "aux_ids")
+RULE_TRACES = ["handoff_trace_verify_in_probe.txt", "handoff_trace_counter_reset.txt", "handoff_trace_probe_cut_replace.txt",
+               "handoff_trace_probe_cut_keep.txt", "handoff_trace_delimiter_in_probe.txt", "handoff_trace_target_verification.txt"]
+
+
+def load_rule_trace(name):
+    """A self-describing hand-traced stream: `p.<name>=` lines are the rule parameters, the rest the expected logs."""
+    T, params = {}, {}
+    with open(os.path.join(HERE, "golden", name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            k, v = line.split("=")
+            if k.startswith("p."):
+                k = k[2:]
+                params[k] = [int(x) for x in v.split(",")] if k in LIST_PARAMS else int(v)
+            elif k == "handoffs":
+                T[k] = [tuple(int(x) for x in h.split(":")) for h in v.split(",")]
+            elif k in ("max_new", "kv_len_small", "kv_len_large", "budget", "budget_steps"):
+                T[k] = int(v)
+            else:
+                T[k] = [int(x) for x in v.split(",")]
+    params.setdefault("keyword_ids", [])
+    return T, params
+
+
+def assert_matches_trace(r, T):
+    assert r.tokens.tolist() == T["tokens"]
+    assert r.source.tolist() == T["source"]
+    assert r.handoffs == T["handoffs"] and r.handoff_kinds == T["handoff_kinds"]
+    assert r.emission_tokens.tolist() == T["force"]
+    assert r.emission_source.tolist() == T["emission_source"]
+    assert r.emission_fed.tolist() == T["emission_fed"]
+    assert (r.kv_len_small, r.kv_len_large) == (T["kv_len_small"], T["kv_len_large"])
+
+
 @pytest.fixture(scope="module")
 def tiny(oracle):
     cfg_s = oracle.Config(**W.TINY_S.as_dict())
@@ -78,6 +115,23 @@ def test_hand_traced_stream_three_takeovers(oracle, tiny):
     assert r.emission_source.tolist() == T["emission_source"]
     assert r.emission_fed.tolist() == T["emission_fed"]
     assert (r.kv_len_small, r.kv_len_large) == (T["kv_len_small"], T["kv_len_large"])
+
+
+@pytest.mark.parametrize("name", RULE_TRACES)
+def test_hand_traced_rule_cases(oracle, tiny, name):
+    """One hand-traced stream per reading that a transcription of the rule could get wrong: cue precedence inside
+    one probe sentence, the reflection counter crossing its threshold and restarting, a probe sentence cut by
+    end-of-sequence or by the budget (both probe readings), a delimiter inside a probe, a verification cue in the
+    target's own sentence while it owes more / fewer than n2 tokens."""
+    T, params = load_rule_trace(name)
+    r = oracle.generate_spec(tiny[0], tiny[1], T["prompt"], max_new_tokens=T["max_new"], force=T["force"], **params)
+    assert r.rc == 0
+    assert_matches_trace(r, T)
+    if "budget" in T:   # the same stream without an end-of-sequence id, cut by the token budget instead
+        params = dict(params, eos_id=-1)
+        r = oracle.generate_spec(tiny[0], tiny[1], T["prompt"], max_new_tokens=T["budget"], force=T["force"], **params)
+        assert r.rc == 0 and r.tokens.tolist() == T["budget_tokens"] and len(r.emission_tokens) == T["budget_steps"]
+        assert r.handoffs == T["handoffs"] and r.source.tolist() == T["source"][:T["budget"]]
 
 
 def test_three_takeovers_reduce_and_hold_invariants(oracle, tiny):
