@@ -129,13 +129,35 @@ class ClockSampler:
 
 
 def cpu_oracle_sample(w: W.Workload, stats: dict | None):
-    """Time the CPU oracle, as it stands, on a bounded sample of the workload: decode steps of the small
-    model (all layers) and decode steps of the large model cut to two layers plus its LM head, scaled
-    to the full depth; combined with the workload's pass mix into tokens/s."""
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload.
+
+    Small model: a teacher-forced window right after a short prompt (all layers, real per-token cost of the
+    projections and the LM head).  Large model: the same on a two-layer cut plus its LM head, scaled to the full
+    depth.  The oracle cannot afford to prefill the run's real contexts (its prefill costs seconds per token), so the
+    attention cost at the contexts of the run's start, middle and end is timed with the oracle's own attention
+    routine on vectors of those lengths and added per layer and head.  Combined with the workload's pass mix into
+    tokens/s."""
     import ctypes as C
     from oracle import oracle as O
     rng = np.random.default_rng(1)
     cores = os.cpu_count() or 1
+    contexts = [w.prompt_len, w.prompt_len + w.max_new_tokens // 2, w.prompt_len + w.max_new_tokens]
+
+    def attend_seconds(shape, n_keys):   # one query head over n_keys cached keys
+        d = shape.head_dim
+        q, k, v = rng.standard_normal(d), rng.standard_normal((n_keys, d)), rng.standard_normal((n_keys, d))
+        O.attend(q, k, v)
+        reps = 3
+        t0 = time.perf_counter()
+        for _ in range(reps):
+            O.attend(q, k, v)
+        return (time.perf_counter() - t0) / reps
+
+    def attention_extra(shape):   # mean over the window contexts of the attention time the short-context steps lack
+        per_head = np.mean([attend_seconds(shape, c) for c in contexts])
+        # the oracle spreads (row, head) pairs over its threads
+        return per_head * shape.n_q_heads * shape.n_layers / max(1, min(cores, shape.n_q_heads))
+
     om = O.Model(O.Config(**w.small.as_dict()), w.weight_seed, 0)
     kv = O.KV(om, 64)
     kv.forward(rng.integers(0, w.small.vocab, 4))
@@ -145,8 +167,9 @@ def cpu_oracle_sample(w: W.Workload, stats: dict | None):
         kv.forward(rng.integers(0, w.small.vocab, 1))
     t_small = (time.perf_counter() - t0) / n_s
     om.close()
-    t_large = None
-    sample = f"{n_s} decode steps of the {w.small.name} oracle"
+    att_small = attention_extra(w.small)
+    t_large = att_large = None
+    sample = f"{n_s} decode steps of the {w.small.name} oracle at a short context"
     if w.large is not None:
         sh = w.large.as_dict()
         sh["n_layers"] = 2
@@ -165,17 +188,21 @@ def cpu_oracle_sample(w: W.Workload, stats: dict | None):
         t_layers2 = (time.perf_counter() - t0) / n_l
         t_large = t_layers2 / 2 * w.large.n_layers + max(t_with_head - t_layers2, 0.0)
         ol.close()
+        att_large = attention_extra(w.large)
         sample += (f" + {2 * n_l} decode steps of the {w.large.name} oracle cut to 2 layers (with and without LM head), "
                    f"scaled to {w.large.n_layers} layers")
+    sample += f"; attention over the run's contexts {contexts} timed with the oracle's attention routine and added per layer and head"
+    ts, tl = t_small + att_small, (t_large or 0.0) + (att_large or 0.0)
     if stats:
-        total = stats["steps_small"] * t_small + stats["steps_large"] * (t_large or 0.0)
+        total = stats["steps_small"] * ts + stats["steps_large"] * tl
         value = stats["n_tokens"] / total
         sample += (f"; combined with the run's pass mix ({stats['steps_small']} small, {stats['steps_large']} large passes; "
                    "a catch-up pass counted as one decode pass)")
     else:
-        value = 1.0 / t_small
+        value = 1.0 / ts
     return {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
-            "s_per_small_step": t_small, "s_per_large_step": t_large}
+            "s_per_small_step": ts, "s_per_large_step": tl if w.large is not None else None,
+            "s_attention_small": att_small, "s_attention_large": att_large}
 
 
 def schedule_stats(w: W.Workload):
@@ -236,6 +263,155 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+def timed_decode_step(torch, model, shape, ctx, n_launches=20):
+    """Back-to-back single-kernel decode steps of one model at a context of `ctx` tokens, timed with CUDA events on
+    the launching stream (torch's current stream); every launch streams all weights (far larger than L2)."""
+    slot = model.st_seq_alloc()
+    for i in range(0, ctx, 256):
+        model.st_prefill(slot, W.prompt_ids(7 + i, min(256, ctx - i), shape.vocab))
+    tok_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    amax_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for _ in range(3):
+        model.st_decode_step([slot], tok_dev, None, amax_dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(n_launches):
+        model.st_decode_step([slot], tok_dev, None, amax_dev)
+    e1.record()
+    torch.cuda.synchronize()
+    sec = e0.elapsed_time(e1) * 1e-3 / n_launches
+    nbytes = model.st_weight_bytes() + model.st_kv_bytes_per_token() * (ctx + 3 + n_launches // 2)
+    model.st_seq_free(slot)
+    return sec, nbytes
+
+
+def timed_batched_step(torch, model, shape, batch, ctx, peak, n_launches=10):
+    slots = [model.st_seq_alloc() for _ in range(batch)]
+    for i, sl in enumerate(slots):
+        for j in range(0, ctx, 256):
+            model.st_prefill(sl, W.prompt_ids(50 + i, min(256, ctx - j), shape.vocab))
+    btok = torch.zeros(batch, dtype=torch.int32, device="cuda")
+    bamax = torch.zeros(batch, dtype=torch.int32, device="cuda")
+    for _ in range(3):
+        model.st_decode_step(slots, btok, None, bamax)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(n_launches):
+        model.st_decode_step(slots, btok, None, bamax)
+    e1.record()
+    torch.cuda.synchronize()
+    sec = e0.elapsed_time(e1) * 1e-3 / n_launches
+    nbytes = model.st_weight_bytes() + model.st_kv_bytes_per_token() * batch * (ctx + 3 + n_launches // 2)
+    for sl in slots:
+        model.st_seq_free(sl)
+    return {"model": shape.name, "batch": batch, "context": ctx, "ms_per_step": sec * 1e3, "tokens_per_s": batch / sec,
+            "hbm_gbs": nbytes / sec / 1e9, "frac_hbm": nbytes / sec / 1e9 / peak,
+            "note": "st_decode_step with 64 sequences: tcgen05 projections, per-sequence attention over paged K/V"}
+
+
+def timed_prompt_prefill(torch, model, shape, rows, peak):
+    """A long prompt ingested from an empty cache (passes of 256 rows): tokens/s and the tensor fraction."""
+    tensor_peak, tensor_kind = measured_tensor_peak()
+    toks = W.prompt_ids(123, rows, shape.vocab)
+    best = None
+    for rep in range(2):
+        slot = model.st_seq_alloc()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        model.st_prefill(slot, toks)
+        torch.cuda.synchronize()
+        t = time.perf_counter() - t0
+        model.st_seq_free(slot)
+        best = t if best is None else min(best, t)
+    lm_head_bytes = 2 * shape.vocab * shape.hidden
+    layer_params = (model.st_weight_bytes() - lm_head_bytes) / 2
+    flops = 2.0 * rows * layer_params + 4.0 * rows * (rows / 2) * shape.n_q_heads * shape.head_dim * shape.n_layers
+    passes = (rows + 255) // 256
+    return {"model": shape.name, "rows": rows, "passes": passes, "ms": best * 1e3, "tokens_per_s": rows / best,
+            "tflops_useful": flops / best / 1e12, "frac_tensor_useful": flops / best / 1e12 / tensor_peak,
+            "hbm_gbs": passes * model.st_weight_bytes() / best / 1e9, "tensor_peak": tensor_peak, "tensor_peak_source": tensor_kind,
+            "timing": "host clock around st_prefill + synchronize (the call syncs between passes)"}
+
+
+def generation_summary(r, peak):
+    """Figures of one timed generation (device time from the call's own CUDA events)."""
+    gbs = r.bytes_algorithmic / r.seconds / 1e9
+    return {"tokens": int(len(r.tokens)), "seconds": r.seconds, "tokens_per_s": len(r.tokens) / r.seconds, "handoffs": len(r.handoffs),
+            "passes": int(r.n_steps), "target_share": float(r.source.mean()) if len(r.source) else 0.0,
+            "achieved_gbs": gbs, "frac_of_measured_hbm": gbs / peak}
+
+
+def other_workloads(torch, B, small, large, peak, want_batch):
+    """One timed generation of each of the other workloads (after the main loop; single GPU only).  Returns a dict
+    keyed by workload name.  The 64-sequence workload needs most of the device memory for its KV pages, so the
+    models of the main loop are closed before it runs (the caller passes them in and must not use them after)."""
+    out = {}
+    # tiny pair (config 0): the case the oracle checks token by token
+    wl = W.CONFIGS["tiny_pair"]
+    prompt, force = W.workload_inputs(wl)
+    ts = B.Model(wl.small.as_dict(), seed=0, tag=0, max_tokens=512)
+    tl = B.Model(wl.large.as_dict(), seed=0, tag=1, max_tokens=512)
+    kw = dict(delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=W.N1, max_new_tokens=wl.max_new_tokens, force=force)
+    B.st_generate_spec(ts, tl, prompt, **kw)
+    out[wl.name] = generation_summary(B.st_generate_spec(ts, tl, prompt, **kw), peak)
+    ts.close()
+    tl.close()
+    # the small model alone (config 1)
+    wl = W.CONFIGS["qwen1p5b_alone"]
+    prompt, force = W.workload_inputs(wl)
+    kw = dict(delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=W.N1, max_new_tokens=wl.max_new_tokens, force=force)
+    B.st_generate_spec(small, None, prompt, **dict(kw, max_new_tokens=64))
+    out[wl.name] = generation_summary(B.st_generate_spec(small, None, prompt, **kw), peak)
+    # 7B + 32B with a 4096-token prompt (config 3): the target model is the one of the main loop
+    wl = W.CONFIGS["qwen7b_32b_long"]
+    if large is not None:
+        prompt, force = W.workload_inputs(wl)
+        cap = wl.prompt_len + wl.max_new_tokens + 64
+        mid = B.Model(wl.small.as_dict(), seed=wl.weight_seed, tag=0, max_tokens=cap)
+        kw = dict(delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=W.N1, max_new_tokens=wl.max_new_tokens, force=force)
+        out[wl.name] = generation_summary(B.st_generate_spec(mid, large, prompt, **kw), peak)
+        mid.close()
+    # 64 independent sequences on the 1.5B + 32B pair (config 4)
+    if want_batch and large is not None:
+        shape_s, shape_l = W.QWEN_1P5B, W.QWEN_32B
+        small.close()
+        large.close()
+        torch.cuda.empty_cache()
+        n = 64
+        prompts, budgets, forces = W.batch_inputs(5, n, min(shape_s.vocab, shape_l.vocab))
+        cap = sum(len(p) + b + 80 for p, b in zip(prompts, budgets))
+        bs = B.Model(shape_s.as_dict(), seed=0, tag=0, max_seqs=n, max_tokens=cap)
+        bl = B.Model(shape_l.as_dict(), seed=0, tag=1, max_seqs=n, max_tokens=cap)
+        t0 = time.perf_counter()
+        got = B.st_generate_spec_batch(bs, bl, prompts, delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=W.N1,
+                                       max_new_tokens=budgets, forces=forces)
+        wall = time.perf_counter() - t0
+        tok = sum(len(r.tokens) for r in got)
+        sec = got[0].seconds
+        # bytes the batch had to move: one pass over a model's weights per round and model is what batching saves, so the
+        # roofline compares against the per-sequence algorithmic bytes (what 64 separate generations would move)
+        alone = sum(r.bytes_algorithmic for r in got)
+        out["batch64_1p5b_32b"] = {"sequences": n, "tokens": int(tok), "seconds": sec, "wall_seconds": wall, "tokens_per_s": tok / sec,
+                                   "handoffs": int(sum(len(r.handoffs) for r in got)),
+                                   "target_share": float(sum(int((r.source == 1).sum()) for r in got) / max(tok, 1)),
+                                   "prompt_lens": [int(min(len(p) for p in prompts)), int(max(len(p) for p in prompts))],
+                                   "budgets": [int(min(budgets)), int(max(budgets))],
+                                   "bytes_if_run_one_by_one": int(alone), "speedup_bound_note":
+                                   "tokens/s of the whole batch; sequences share each round's pass over the weights"}
+        bs.close()
+        bl.close()
+    return out
+
+
+# DRAM bytes per launch of the dominant kernel, as a ratio to its algorithmic bytes: ncu dram__bytes_read.sum +
+# dram__bytes_write.sum of decode_mega_kernel<128, 5> (the 32B's instance) on a two-layer cut of the 32B's widths,
+# three launches.  None until a capture of the current kernel exists.
+DOMINANT_TRAFFIC_RATIO = None
+DOMINANT_TRAFFIC_SOURCE = None
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -244,6 +420,7 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--workload", default="qwen1p5b_32b", choices=sorted(W.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the per-kernel figures and the other workloads")
     ap.add_argument("--max-new", type=int, default=0, help="shorten the generation (profiling runs only)")
     ap.add_argument("--mean-interval", type=float, default=0.0, help="delimiter spacing override (profiling runs only)")
     ap.add_argument("--layers", type=int, default=0, help="cut both models to this many layers (profiling runs only)")
@@ -275,12 +452,17 @@ def main():
     # an independent replica of the workload (its own input seed); there is no data-path collective.
     wl = rank_workload(w, rank)
     prompt, force = W.workload_inputs(wl)
-    cap = wl.prompt_len + wl.max_new_tokens + 64
-    # room for the batched decode measurement at the end: BATCH more sequences of BATCH_CTX + 64 tokens on the large model
+    extras = not args.no_extras and args.layers == 0 and args.max_new == 0
+    main_is_headline = wl.name == "qwen1p5b_32b" or wl.name.startswith("qwen1p5b_32b")
+    # room for the other measurements on the same models: the 7B + 32B workload's 12k-token sequence and the batched
+    # decode step's BATCH sequences of BATCH_CTX + 64 tokens on the large model
     BATCH, BATCH_CTX = 64, 512
-    small = B.Model(wl.small.as_dict(), seed=wl.weight_seed, tag=0, max_tokens=cap)
+    cap = wl.prompt_len + wl.max_new_tokens + 64
+    cap_small = max(cap, 4096 + 64)
+    long_cap = W.CONFIGS["qwen7b_32b_long"].prompt_len + W.CONFIGS["qwen7b_32b_long"].max_new_tokens + 64
+    small = B.Model(wl.small.as_dict(), seed=wl.weight_seed, tag=0, max_tokens=cap_small)
     large = B.Model(wl.large.as_dict(), seed=wl.weight_seed, tag=1, max_seqs=BATCH + 1,
-                    max_tokens=cap + BATCH * (BATCH_CTX + 64)) if wl.large else None
+                    max_tokens=max(cap, long_cap) + BATCH * (BATCH_CTX + 64)) if wl.large else None
     kw = dict(delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=W.N1, max_new_tokens=wl.max_new_tokens, force=force)
 
     def barrier():
@@ -315,78 +497,40 @@ def main():
     e2e_value = n_tokens / e2e_s
 
     peak, peak_kind = measured_peaks()
-    # Dominant kernel: the single-kernel decode step of the large model (it moves ~3/4 of the run's bytes).
-    # Timed on its own after the run: back-to-back launches with CUDA events on the launching stream
-    # (torch's current stream), at a mid-run context length; every launch streams all weights (>> L2).
-    dom = large if large is not None else small
-    shp = wl.large if wl.large else wl.small
-    ctx = min(3000, cap - 64)
-    slot = dom.st_seq_alloc()
-    dom.st_prefill(slot, W.prompt_ids(7, ctx, shp.vocab))
-    tok_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
-    amax_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
-    for _ in range(3):
-        dom.st_decode_step([slot], tok_dev, None, amax_dev)
-    n_k = 20
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    e0.record()
-    for _ in range(n_k):
-        dom.st_decode_step([slot], tok_dev, None, amax_dev)
-    e1.record()
-    torch.cuda.synchronize()
-    kern_s = e0.elapsed_time(e1) * 1e-3 / n_k
-    kern_bytes = dom.st_weight_bytes() + dom.st_kv_bytes_per_token() * (ctx + 3 + n_k // 2)
-    achieved = kern_bytes / kern_s / 1e9
-    dom.st_seq_free(slot)
-    # multi-row passes (handoff catch-up and prompt prefill) of the same model, and the small model's decode step
-    mean_catchup = int(np.mean([h[2] for h in r.handoffs])) if len(r.handoffs) else 128
-    prefill = time_multi_row_passes(torch, dom, shp, max(0, min(1024, cap - 64 - 256)), [min(256, max(2, mean_catchup)), 256], peak)
-    small_step = None
-    if large is not None:
-        sslot = small.st_seq_alloc()
-        small.st_prefill(sslot, W.prompt_ids(7, ctx, wl.small.vocab))
-        for _ in range(3):
-            small.st_decode_step([sslot], tok_dev, None, amax_dev)
-        torch.cuda.synchronize()
-        e0.record()
-        for _ in range(n_k):
-            small.st_decode_step([sslot], tok_dev, None, amax_dev)
-        e1.record()
-        torch.cuda.synchronize()
-        s_s = e0.elapsed_time(e1) * 1e-3 / n_k
-        s_bytes = small.st_weight_bytes() + small.st_kv_bytes_per_token() * (ctx + 3 + n_k // 2)
-        small_step = {"kernel": f"decode_mega_kernel ({wl.small.name}, context {ctx})", "us_per_launch": s_s * 1e6,
-                      "achieved": s_bytes / s_s / 1e9, "frac": s_bytes / s_s / 1e9 / peak, "unit": "GB/s"}
-        small.st_seq_free(sslot)
-    # batched decode of the same model (the 64-sequence workload's step): one pass over the weights for all rows
-    batched = None
-    if large is not None:
-        bslots = [large.st_seq_alloc() for _ in range(BATCH)]
-        for i, sl in enumerate(bslots):
-            for j in range(0, BATCH_CTX, 256):
-                large.st_prefill(sl, W.prompt_ids(50 + i, min(256, BATCH_CTX - j), shp.vocab))
-        btok = torch.zeros(BATCH, dtype=torch.int32, device="cuda")
-        bamax = torch.zeros(BATCH, dtype=torch.int32, device="cuda")
-        for _ in range(3):
-            large.st_decode_step(bslots, btok, None, bamax)
-        torch.cuda.synchronize()
-        n_b = 10
-        e0.record()
-        for _ in range(n_b):
-            large.st_decode_step(bslots, btok, None, bamax)
-        e1.record()
-        torch.cuda.synchronize()
-        b_s = e0.elapsed_time(e1) * 1e-3 / n_b
-        b_bytes = large.st_weight_bytes() + large.st_kv_bytes_per_token() * BATCH * (BATCH_CTX + 3 + n_b // 2)
-        batched = {"model": shp.name, "batch": BATCH, "context": BATCH_CTX, "ms_per_step": b_s * 1e3, "tokens_per_s": BATCH / b_s,
-                   "hbm_gbs": b_bytes / b_s / 1e9, "frac_hbm": b_bytes / b_s / 1e9 / peak,
-                   "note": "st_decode_step with 64 sequences: tcgen05 projections, per-sequence attention over paged K/V"}
-        for sl in bslots:
-            large.st_seq_free(sl)
-    path_gbs = sum(x.bytes_algorithmic for x in results) / sum(x.seconds for x in results) / 1e9
+    # the metric's own fraction: algorithmic bytes of every pass of the timed generations / their device time
+    path_bytes = sum(x.bytes_algorithmic for x in results)
+    path_gbs = path_bytes / sum(x.seconds for x in results) / 1e9
     steps_small = int((r.emission_source == 0).sum())
     steps_large = int((r.emission_source == 1).sum())
+    dom = large if large is not None else small
+    shp = wl.large if wl.large else wl.small
+
+    dominant = small_step = prefill = prompt_prefill = batched = None
+    if extras:
+        # Dominant kernel by bytes: the single-kernel decode step of the large model, on its own, mid-run context
+        ctx = min(3000, cap - 64)
+        kern_s, kern_bytes = timed_decode_step(torch, dom, shp, ctx)
+        dominant = {"kernel": f"decode_mega_kernel ({shp.name}, one decode step per launch, context {ctx})", "bound": "hbm",
+                    "us_per_launch": kern_s * 1e6, "algorithmic_bytes_per_launch": int(kern_bytes), "achieved": kern_bytes / kern_s / 1e9,
+                    "peak": peak, "unit": "GB/s", "frac": kern_bytes / kern_s / 1e9 / peak,
+                    "traffic": int(DOMINANT_TRAFFIC_RATIO * kern_bytes) if DOMINANT_TRAFFIC_RATIO else None,
+                    "traffic_source": DOMINANT_TRAFFIC_SOURCE}
+        if large is not None:
+            s_s, s_bytes = timed_decode_step(torch, small, wl.small, ctx)
+            small_step = {"kernel": f"decode_mega_kernel ({wl.small.name}, context {ctx})", "us_per_launch": s_s * 1e6,
+                          "achieved": s_bytes / s_s / 1e9, "frac": s_bytes / s_s / 1e9 / peak, "unit": "GB/s"}
+        # multi-row passes (handoff catch-up and prompt prefill) of the large model
+        mean_catchup = int(np.mean([h[2] for h in r.handoffs])) if len(r.handoffs) else 128
+        prefill = time_multi_row_passes(torch, dom, shp, max(0, min(1024, cap - 64 - 256)), [min(256, max(2, mean_catchup)), 256], peak)
+        if world == 1:
+            prompt_prefill = timed_prompt_prefill(torch, dom, shp, 4096, peak)
+        if large is not None:
+            batched = timed_batched_step(torch, large, shp, BATCH, BATCH_CTX, peak)
+    accounting = paper_accounting(r, wl)
+    others = None
+    if extras and world == 1 and main_is_headline:
+        others = other_workloads(torch, B, small, large, peak, want_batch=True)
+        small = large = None   # closed by other_workloads
 
     if rank == 0:
         line = {
@@ -397,7 +541,7 @@ def main():
                        "prompt_len": wl.prompt_len, "max_new_tokens": wl.max_new_tokens, "n1": W.N1,
                        "handoffs": len(r.handoffs), "target_share": float(r.source.mean()),
                        "passes_small": steps_small, "passes_large": steps_large,
-                       "arithmetic": "bf16 weights and KV, fp32 activations and accumulation",
+                       "arithmetic": "bf16 weights, fp16 KV cache, fp32 activations and accumulation",
                        "l2": "inputs larger than L2: every pass streams 3.1 GB (small) or 64 GB (large) of weights",
                        "multi_gpu": "replicas only" if world > 1 else "single GPU"},
             "clocks": clocks,
@@ -405,29 +549,28 @@ def main():
                     "h2d_bytes_per_step": int(prompt.nbytes + (force.nbytes if force is not None else 0) + min(wl.small.vocab, shp.vocab)),
                     "d2h_bytes_per_step": int(5 * len(r.tokens) + 13 * r.n_steps + 12 * len(r.handoffs) + 80 * r.n_steps)},
             "gpu_launches": int(launches),
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         # DRAM bytes per launch: ncu measured read+write = 1.013 x the algorithmic bytes on a 4-layer
-                         # case of this kernel (profiles/decode_mega_kernel_4layer_pair.md); scaled to this launch
-                         "traffic": int(1.013 * kern_bytes),
-                         "traffic_source": "ncu dram__bytes_read+write on a 4-layer capture, scaled by streamed bytes",
-                         "kernel": f"decode_mega_kernel ({shp.name}, one decode step per launch, context {ctx})",
-                         "algorithmic_bytes_per_launch": int(kern_bytes),
-                         "peak_source": f"{peak_kind} copy bandwidth", "us_per_launch": kern_s * 1e6},
-            "path_roofline": {"achieved_gbs": path_gbs, "frac_of_measured_hbm": path_gbs / peak,
-                              "frac_of_nominal_8tbs": path_gbs / 8000.0,
-                              "note": "algorithmic bytes of every pass (weights + KV) / device time of the generation"},
-            "paper_accounting": paper_accounting(r, wl),
+            # the metric's fraction: the whole generation against the HBM roofline
+            "roofline": {"bound": "hbm", "achieved": path_gbs, "peak": peak, "unit": "GB/s", "frac": path_gbs / peak,
+                         "traffic": None, "kernel": "whole path: every pass of the timed generations",
+                         "algorithmic_bytes_per_step": int(path_bytes / len(results)),
+                         "frac_of_nominal_8tbs": path_gbs / 8000.0, "peak_source": f"{peak_kind} copy bandwidth",
+                         "note": "algorithmic bytes of every pass (weights + KV) / device time; per-kernel figures under dominant_kernel, decode_small, prefill, batched_decode"},
+            "dominant_kernel": dominant,
+            "decode_small": small_step,
             "prefill": prefill,
-            "small_model_decode": small_step,
+            "prompt_prefill": prompt_prefill,
             "batched_decode": batched,
+            "workloads": others,
+            "paper_accounting": accounting,
             "wall_s_timed_region": t_region,
         }
         if not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_oracle_sample(wl, {"steps_small": steps_small, "steps_large": steps_large,
                                                           "n_tokens": len(r.tokens)})
         print(json.dumps(line), flush=True)
-    small.close()
-    if large:
+    if small is not None:
+        small.close()
+    if large is not None:
         large.close()
     if world > 1:
         dist.destroy_process_group()

@@ -105,6 +105,11 @@ typedef struct {
                                          takeover the target's segment replaces the whole sentence (keep_probe 0: output
                                          and the speculative model's cached length go back to the sentence's start) or
                                          follows it (keep_probe 1).  Size emission logs for (1 + k) * max_new_tokens steps */
+    /* The delimiter as a family of ids (the paper's Table 1 and Appendix B: every token that ends in a blank line
+     * closes a paragraph).  n_delimiters == 0: the single delimiter_id above; otherwise delimiter_id is ignored and
+     * any of these ids (host array, ids below vocab_limit) counts as the delimiter wherever the rule tests for it. */
+    const int32_t *delimiter_ids;
+    int32_t n_delimiters;
 } st_spec_params;
 
 typedef struct {
@@ -134,6 +139,13 @@ typedef struct {
     int64_t bytes_algorithmic; /* weights + KV bytes the passes had to move (sum over steps) */
     uint8_t *handoff_kinds;   /* optional [cap_handoffs]: which takeover each handoff was (1 reflection / affirmation or
                                  every-delimiter, 2 verification, 3 excessive reflection) */
+    /* Device time of the generation by kind of pass (the split of the paper's Table "comparison of time": decode of one
+     * token against the "prefix" pass of a handoff), from device timestamps taken at the end of every pass:
+     * passes that ingest a model's first tokens (its prompt prefill, for the target inside its first catch-up), other
+     * passes of more than one token (catch-up after a handoff), and single-token decode passes.  Zero for
+     * st_generate_spec_batch (its passes serve many sequences at once). */
+    double t_prompt_prefill_s, t_catchup_s, t_decode_s;
+    int32_t n_prompt_prefill, n_catchup, n_decode;   /* passes of each kind (a catch-up cut into chunks counts once) */
 } st_spec_result;
 
 /* Create a model with seeded random-init weights: element idx of tensor tid of model `tag` is

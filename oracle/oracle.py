@@ -45,6 +45,7 @@ class _SpecParams(C.Structure):
         ("verification_ids", C.POINTER(C.c_int32)), ("n_verification", C.c_int32),
         ("n2", C.c_int32), ("neg_threshold", C.c_int32), ("n3", C.c_int32),
         ("aux_ids", C.POINTER(C.c_int32)), ("n_aux", C.c_int32), ("probe_len", C.c_int32),
+        ("delimiter_ids", C.POINTER(C.c_int32)), ("n_delimiters", C.c_int32),
     ]
 
 
@@ -280,18 +281,20 @@ def generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id: in
                   force=None, trace_first_step: int = 0, trace_n_steps: int = 0,
                   takeover_every_delimiter: bool = False, target_first_n: int = 0, affirmation_ids=(),
                   verification_ids=(), n2: int = 125, neg_threshold: int = -1, n3: int = 125, aux_ids=(),
-                  probe_len: int = 1) -> SpecResult:
+                  probe_len: int = 1, delimiter_ids=()) -> SpecResult:
     prompt = np.ascontiguousarray(prompt, dtype=np.int32)
     aff = np.ascontiguousarray(affirmation_ids, dtype=np.int32)
     ver = np.ascontiguousarray(verification_ids, dtype=np.int32)
     aux = np.ascontiguousarray(aux_ids, dtype=np.int32)
+    dl = np.ascontiguousarray(delimiter_ids, dtype=np.int32)
     ip = lambda a: a.ctypes.data_as(C.POINTER(C.c_int32))
     kw = np.ascontiguousarray(keyword_ids, dtype=np.int32)
     if vocab_limit <= 0:
         vocab_limit = small.cfg.vocab if large is None else min(small.cfg.vocab, large.cfg.vocab)
     P = _SpecParams(delimiter_id, kw.ctypes.data_as(C.POINTER(C.c_int32)), kw.size, n1, int(keep_probe), eos_id,
                     vocab_limit, max_new_tokens, int(takeover_every_delimiter), int(target_first_n),
-                    ip(aff), aff.size, ip(ver), ver.size, n2, neg_threshold, n3, ip(aux), aux.size, probe_len)
+                    ip(aff), aff.size, ip(ver), ver.size, n2, neg_threshold, n3, ip(aux), aux.size, probe_len,
+                    ip(dl), dl.size)
     cap_steps = (1 + max(1, probe_len)) * max_new_tokens + 8   # replaced probe sentences are steps without tokens
     tokens = np.zeros(max_new_tokens + 1, dtype=np.int32)
     source = np.zeros(max_new_tokens + 1, dtype=np.uint8)

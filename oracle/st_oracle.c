@@ -520,7 +520,20 @@ typedef struct {
     int32_t n_aux;
     int32_t probe_len;                /* tokens of the speculative model's sentence after a delimiter that are classified
                                          (paper: "one full sentence (i.e. n1 tokens)"); <= 1: only its first token */
+    /* The delimiter as a family of ids (the paper's Table 1 / Appendix B: any token ending in a blank line closes a
+     * paragraph).  n_delimiters == 0: delimiter_id alone; otherwise delimiter_id is ignored. */
+    const int32_t *delimiter_ids;
+    int32_t n_delimiters;
 } orc_spec_params;
+
+/* Does this token close a paragraph? */
+static int is_delimiter(const orc_spec_params *P, int32_t tok)
+{
+    if (P->n_delimiters <= 0) return tok == P->delimiter_id;
+    for (int i = 0; i < P->n_delimiters; ++i)
+        if (P->delimiter_ids[i] == tok) return 1;
+    return 0;
+}
 
 typedef struct { int32_t seg_start, step, catchup_len; } orc_handoff;
 
@@ -591,7 +604,7 @@ int orc_generate_spec(const orc_model *small, const orc_model *large, const orc_
         for (int i = 0; i < P->n_keywords; ++i) is_kw |= (P->keyword_ids[i] == tok);
         for (int i = 0; i < P->n_affirmation; ++i) is_aff |= (P->affirmation_ids[i] == tok);
         for (int i = 0; i < P->n_verification; ++i) is_ver |= (P->verification_ids[i] == tok);
-        const int after_delim = tokens[pos - 1] == P->delimiter_id;
+        const int after_delim = is_delimiter(P, tokens[pos - 1]);
         if (large && a == 0 && !P->takeover_every_delimiter && !probing && after_delim) {
             /* the speculative model opens a sentence: its next probe_len tokens are classified by cue counts */
             probing = 1;
@@ -671,7 +684,7 @@ int orc_generate_spec(const orc_model *small, const orc_model *large, const orc_
         R->n_tokens = generated;
         if (tok == P->eos_id) break;
         if (a == 1 && --remaining == 0) active = 0;
-        if (large && a == 0 && P->takeover_every_delimiter && tok == P->delimiter_id && generated < P->max_new_tokens) {
+        if (large && a == 0 && P->takeover_every_delimiter && is_delimiter(P, tok) && generated < P->max_new_tokens) {
             /* the speculative model closed a paragraph: the target writes the next n1 tokens */
             if (R->n_handoffs >= R->cap_handoffs) { rc = -3; break; }
             R->handoffs[R->n_handoffs].seg_start = pos;

@@ -42,6 +42,7 @@ class StSpecParams(C.Structure):
         ("verification_ids", C.POINTER(C.c_int32)), ("n_verification", C.c_int32),
         ("n2", C.c_int32), ("neg_threshold", C.c_int32), ("n3", C.c_int32),
         ("aux_ids", C.POINTER(C.c_int32)), ("n_aux", C.c_int32), ("probe_len", C.c_int32),
+        ("delimiter_ids", C.POINTER(C.c_int32)), ("n_delimiters", C.c_int32),
     ]
 
 
@@ -61,6 +62,8 @@ class StSpecResult(C.Structure):
         ("logits_trace", C.POINTER(C.c_float)), ("trace_first_step", C.c_int32), ("trace_n_steps", C.c_int32),
         ("seconds", C.c_double), ("bytes_algorithmic", C.c_int64),
         ("handoff_kinds", C.POINTER(C.c_uint8)),
+        ("t_prompt_prefill_s", C.c_double), ("t_catchup_s", C.c_double), ("t_decode_s", C.c_double),
+        ("n_prompt_prefill", C.c_int32), ("n_catchup", C.c_int32), ("n_decode", C.c_int32),
     ]
 
 
@@ -209,6 +212,7 @@ class SpecResult:
     bytes_algorithmic: int
     n_steps: int
     handoff_kinds: list = None   # 1 reflection / affirmation / every-delimiter, 2 verification, 3 excessive reflection
+    phase_times: dict = None     # kind of pass -> (device seconds, passes): prompt_prefill, catchup, decode
 
 
 class Model:
@@ -338,19 +342,21 @@ class _ResultBuffers:
                            for i in range(min(R.n_handoffs, self.cap_handoffs))],
                           self.e_tok[:s].copy(), self.e_src[:s].copy(), self.e_fed[:s].copy(), self.e_arg[:s].copy(),
                           R.kv_len_small, R.kv_len_large, self.trace, R.seconds, R.bytes_algorithmic, R.n_steps,
-                          self.kinds[:min(R.n_handoffs, self.cap_handoffs)].tolist())
+                          self.kinds[:min(R.n_handoffs, self.cap_handoffs)].tolist(),
+                          {"prompt_prefill": (R.t_prompt_prefill_s, R.n_prompt_prefill), "catchup": (R.t_catchup_s, R.n_catchup),
+                           "decode": (R.t_decode_s, R.n_decode)})
 
 
 def _spec_params(delimiter_id, keyword_ids, n1, keep_probe, eos_id, vocab_limit, max_new_tokens, takeover_every_delimiter,
                  target_first_n, affirmation_ids=(), verification_ids=(), n2=125, neg_threshold=-1, n3=125, aux_ids=(),
-                 probe_len=1):
+                 probe_len=1, delimiter_ids=()):
     """st_spec_params and the arrays it points at (keep both alive during the call)."""
-    arrs = [np.ascontiguousarray(a, dtype=np.int32) for a in (keyword_ids, affirmation_ids, verification_ids, aux_ids)]
+    arrs = [np.ascontiguousarray(a, dtype=np.int32) for a in (keyword_ids, affirmation_ids, verification_ids, aux_ids, delimiter_ids)]
     ip = lambda a: a.ctypes.data_as(C.POINTER(C.c_int32))
-    kw, aff, ver, aux = arrs
+    kw, aff, ver, aux, dl = arrs
     P = StSpecParams(delimiter_id, ip(kw), kw.size, n1, int(keep_probe), eos_id, vocab_limit, max_new_tokens,
                      int(takeover_every_delimiter), int(target_first_n), ip(aff), aff.size, ip(ver), ver.size, n2,
-                     neg_threshold, n3, ip(aux), aux.size, probe_len)
+                     neg_threshold, n3, ip(aux), aux.size, probe_len, ip(dl), dl.size)
     return P, arrs
 
 

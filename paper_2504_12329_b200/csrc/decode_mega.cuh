@@ -65,7 +65,7 @@ struct MegaParams {
     int32_t *tickets;         // [Hkv] attention tickets, zero between launches
     unsigned *sync;           // [1] exit tickets, [2] abort flag, [3] argmax tickets, [32 * (1 + i)] barrier counter i < 8
     int32_t *status;
-    int32_t n_layers, h, Hq, Hkv, f, vocab, n_splits, stages, xarea_bytes;
+    int32_t n_layers, h, Hq, Hkv, f, vocab, n_splits, unit_keys, stages, xarea_bytes;
     int32_t down_slab;        // K segments per slab of the down projection (0: the whole input vector is kept)
     int32_t kv_off, kv_cap;   // K/V staging area inside the activation area: byte offset, capacity in keys (multiple of 16)
     float eps, scale;
@@ -493,10 +493,10 @@ __device__ __forceinline__ uint32_t mega_kv_swz(const MegaUnit &u, int row, int 
     return (uint32_t)(d >> 6) * u.half_bytes + (uint32_t)row * 128 + (cb ^ ((uint32_t)(row & 7) << 4));
 }
 
-// Key splits of a decode step at position pos: 64 keys per unit while there are CTAs to spare.
-__host__ __device__ __forceinline__ int mega_key_splits(int pos, int n_splits_max, int n_cta, int Hkv)
+// Key splits of a decode step at position pos: unit_keys keys per unit while there are CTAs to spare.
+__host__ __device__ __forceinline__ int mega_key_splits(int pos, int n_splits_max, int n_cta, int Hkv, int unit_keys)
 {
-    int ns = (pos + 64) / 64;
+    int ns = (pos + unit_keys) / unit_keys;
     const int fit = n_cta / Hkv > 1 ? n_cta / Hkv : 1;
     const int cap = n_splits_max < fit ? n_splits_max : fit;
     return ns < cap ? ns : cap;
@@ -977,7 +977,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
         sh.cs[j] = make_float2((float)c, (float)s);
     }
     // every CTA derives the same split count
-    const int ns = mega_key_splits(pos, p.n_splits, (int)gridDim.x, p.Hkv);
+    const int ns = mega_key_splits(pos, p.n_splits, (int)gridDim.x, p.Hkv, p.unit_keys);
     const bool attn_active = (int)blockIdx.x < p.Hkv * ns;
     const MegaUnit unit = mega_unit<D>(p, base_ptr, base, pos, ns);
     if (attn_active && unit.n_cached > 0) {

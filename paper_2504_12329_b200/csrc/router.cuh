@@ -10,7 +10,8 @@
 
 namespace st {
 
-constexpr int kClsKeyword = 2;  // class-table bit of a reflection keyword
+constexpr int kClsDelim = 1;    // class-table bit of a delimiter
+constexpr int kClsKeyword = 2;  // ... of a reflection keyword
 constexpr int kClsAffirm = 4;   // ... of an affirmation cue
 constexpr int kClsVerify = 8;   // ... of a verification cue
 
@@ -44,7 +45,20 @@ struct GenState {
     int32_t every_delim;   // 1: no keyword test; the target takes over after every delimiter the speculative model writes
     int32_t prompt_len, cap_steps, cap_handoffs, max_chunk;
     int32_t trace_first, trace_n;
+    // --- device time by kind of pass: 0 prompt prefill, 1 catch-up, 2 decode ---
+    unsigned long long t_last;       // global timer at the end of the previous pass (or at the start)
+    unsigned long long t_pending;    // time of the ingest-only chunks of the catch-up in progress
+    unsigned long long t_kind[3];    // nanoseconds
+    int32_t n_kind[3];
+    int32_t pad_;
 };
+
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
 
 struct GenBuffers {
     int32_t *tokens;           // [prompt_len + max_new + 1] whole sequence
@@ -83,6 +97,14 @@ __device__ void router_step(GenState *g, const GenBuffers &b, int greedy, StepDe
     const int a = g->active;
     const int t = g->step;
     const int fed = g->pos - g->kv_len[a] + g->ingested;   // the whole catch-up, however it was chunked
+    {   // the pass that just ended, by kind: it began at position pos - fed of this model's cache
+        const unsigned long long now = global_timer_ns();
+        const int k = fed == 1 ? 2 : (g->pos - fed == 0 ? 0 : 1);
+        g->t_kind[k] += now - g->t_last + g->t_pending;
+        g->n_kind[k]++;
+        g->t_pending = 0;
+        g->t_last = now;
+    }
     g->ingested = 0;
     g->kv_len[a] = g->pos;
     g->bytes_algo += g->wbytes[a] + g->kvb[a] * (int64_t)g->pos;
@@ -100,7 +122,7 @@ __device__ void router_step(GenState *g, const GenBuffers &b, int greedy, StepDe
     if ((unsigned)tok >= (unsigned)g->vlimit) { atomicOr(status, DEV_BAD_TOKEN); tok = 0; }
     // Takeovers of Section 3 in token-id form: the token sampled right after a delimiter stands for the sentence.
     const int cls = b.cls[tok];
-    const bool after_delim = b.tokens[g->pos - 1] == g->delimiter;
+    const bool after_delim = (b.cls[b.tokens[g->pos - 1]] & kClsDelim) != 0;
     int kind = 0, len = 0;
     if (g->has_large && a == 0 && !g->every_delim && !g->probing && after_delim) {
         // the speculative model opens a sentence: its next probe_len tokens are classified by cue counts
@@ -173,7 +195,7 @@ __device__ void router_step(GenState *g, const GenBuffers &b, int greedy, StepDe
         g->generated++;
         if (tok == g->eos) g->done = 1;
         if (a == 1 && --g->remaining == 0) g->active = 0;
-        if (g->has_large && a == 0 && g->every_delim && tok == g->delimiter && !g->done && g->generated < g->max_new) {
+        if (g->has_large && a == 0 && g->every_delim && (cls & kClsDelim) && !g->done && g->generated < g->max_new) {
             // the speculative model closed a paragraph: the target writes the next n1 tokens
             log_handoff(g->pos, g->pos - g->kv_len[1], 1);
             g->active = 1;
@@ -199,6 +221,11 @@ __global__ void batch_router_kernel(GenState *gs, const GenBuffers *gb, const in
 __global__ void advance_ingest_kernel(GenState *g, StepDesc *desc_small, StepDesc *desc_large)
 {
     const int a = g->next_model;
+    {
+        const unsigned long long now = global_timer_ns();
+        g->t_pending += now - g->t_last;
+        g->t_last = now;
+    }
     g->kv_len[a] += g->next_m;
     g->ingested += g->next_m;
     g->bytes_algo += g->wbytes[a] + g->kvb[a] * (int64_t)g->kv_len[a];
@@ -207,6 +234,7 @@ __global__ void advance_ingest_kernel(GenState *g, StepDesc *desc_small, StepDes
 
 __global__ void plan_first_pass_kernel(GenState *g, StepDesc *desc_small, StepDesc *desc_large)
 {
+    g->t_last = global_timer_ns();
     plan_next_pass(g, desc_small, desc_large);
 }
 

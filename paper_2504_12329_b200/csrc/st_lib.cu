@@ -131,7 +131,7 @@ struct st_model {
     float *X0 = nullptr, *X1 = nullptr, *D1 = nullptr, *D2 = nullptr;   // [h] each
     unsigned *mega_sync = nullptr;      // [4]
     int32_t *mega_tickets = nullptr;    // [Hkv]
-    int mega_stages = 0, mega_xarea = 0, mega_splits = 0, mega_kv_off = 0, mega_kv_cap = 0, mega_down_slab = 0;
+    int mega_stages = 0, mega_xarea = 0, mega_splits = 0, mega_kv_off = 0, mega_kv_cap = 0, mega_down_slab = 0, mega_unit_keys = 64;
     size_t mega_smem = 0;
     bool multi_kernel_decode = false;   // debugging aid: one kernel per phase instead
 
@@ -798,6 +798,11 @@ static int model_build(st_model *m)
         int stages = (int)((budget - (long long)xarea) / kMegaTileBytes);
         if (stages < 2) return ST_ERR_UNSUPPORTED;
         m->mega_stages = stages > kMegaMaxStages ? kMegaMaxStages : stages;
+        // One or two KV heads mean many key splits per head, and merging the splits (every CTA of the O projection
+        // reads all partial results of its heads) then costs more than a ring stage buys: give one stage to the K/V
+        // staging so that a unit holds 128 keys (measured on the 1.5B shape: -4 % at 3000 cached tokens, -7 % at 6000).
+        const bool few_kv_heads = c.n_kv_heads <= 2;
+        if (few_kv_heads && m->mega_stages >= 5) m->mega_stages -= 1;
         if (const char *es = getenv("ST_MEGA_STAGES")) {   // tuning aid: fewer ring stages, more K/V staging
             const int want = atoi(es);
             if (want >= 2 && want < m->mega_stages) m->mega_stages = want;
@@ -816,6 +821,15 @@ static int model_build(st_model *m)
         m->mega_smem = 1024 + xarea + (size_t)m->mega_stages * kMegaTileBytes;
         m->mega_splits = m->sm_count / c.n_kv_heads > 0 ? m->sm_count / c.n_kv_heads : 1;
         if (m->mega_splits > kMaxAttnSplits) m->mega_splits = kMaxAttnSplits;
+        if (few_kv_heads) {   // as many keys per unit as one staging chunk holds (a unit's first key may sit 15 rows into its first box)
+            m->mega_unit_keys = (cap - 16) & ~15;
+            if (m->mega_unit_keys > 128) m->mega_unit_keys = 128;
+            if (m->mega_unit_keys < 64) m->mega_unit_keys = 64;
+        }
+        if (const char *eu = getenv("ST_MEGA_UNIT_KEYS")) {   // tuning aid: keys per attention unit while CTAs are to spare
+            const int want = atoi(eu) & ~15;
+            if (want >= 16 && want + 16 <= cap) m->mega_unit_keys = want;
+        }
         const char *e = getenv("ST_MULTI_KERNEL");
         m->multi_kernel_decode = e && e[0] == '1';
     }
@@ -957,7 +971,7 @@ static int pass_decode(st_model *m, const StepDesc *desc, const int32_t *tok, in
     p.logits = sc.logits_out ? sc.logits_out : m->logits;
     p.part_o = m->part_o; p.part_ml = m->part_ml; p.tickets = m->mega_tickets; p.sync = m->mega_sync; p.status = m->status;
     p.n_layers = c.n_layers; p.h = c.hidden; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.f = c.ffn; p.vocab = c.vocab;
-    p.n_splits = m->mega_splits; p.stages = m->mega_stages; p.xarea_bytes = m->mega_xarea;
+    p.n_splits = m->mega_splits; p.unit_keys = m->mega_unit_keys; p.stages = m->mega_stages; p.xarea_bytes = m->mega_xarea;
     p.kv_off = m->mega_kv_off; p.kv_cap = m->mega_kv_cap; p.down_slab = m->mega_down_slab;
     p.eps = c.rms_eps; p.scale = 1.f / sqrtf((float)c.head_dim);
     p.want_argmax = sc.want_argmax ? 1 : 0;
@@ -1247,7 +1261,7 @@ int64_t st_kernel_launches(void) { return g_launches; }
 int st_decode_geometry(const st_model *m, int32_t ctx, int32_t *n_splits, int32_t *kv_cap, int32_t *max_chunks, int32_t *own_chunk_empty)
 {
     if (!m || ctx < 0) return ST_ERR_ARG;
-    const int ns = mega_key_splits(ctx, m->mega_splits, m->sm_count, m->cfg.n_kv_heads);
+    const int ns = mega_key_splits(ctx, m->mega_splits, m->sm_count, m->cfg.n_kv_heads, m->mega_unit_keys);
     int most = 0, empty = 0;
     for (int sp = 0; sp < ns; ++sp) {
         const MegaUnitShape u = mega_unit_shape(ctx, ns, sp, m->mega_kv_cap);
@@ -1726,6 +1740,10 @@ static int check_rule_params(const st_spec_params *P, int vlimit)
     if ((P->n_affirmation > 0 && !P->affirmation_ids) || (P->n_verification > 0 && !P->verification_ids) || (P->n_aux > 0 && !P->aux_ids))
         return ST_ERR_ARG;
     if ((P->n_verification > 0 && P->n2 < 1) || (P->neg_threshold >= 0 && P->n3 < 1)) return ST_ERR_ARG;
+    if (P->n_delimiters < 0 || (P->n_delimiters > 0 && !P->delimiter_ids)) return ST_ERR_ARG;
+    for (int i = 0; i < P->n_delimiters; ++i)
+        if ((unsigned)P->delimiter_ids[i] >= (unsigned)vlimit) return ST_ERR_VOCAB;
+    if (P->n_delimiters == 0 && (unsigned)P->delimiter_id >= (unsigned)vlimit) return ST_ERR_VOCAB;
     if (P->n_aux > kMaxAuxTokens) return ST_ERR_CAPACITY;
     for (int i = 0; i < P->n_affirmation; ++i)
         if ((unsigned)P->affirmation_ids[i] >= (unsigned)vlimit) return ST_ERR_VOCAB;
@@ -1738,6 +1756,10 @@ static int check_rule_params(const st_spec_params *P, int vlimit)
 
 static void fill_class_table(const st_spec_params *P, std::vector<uint8_t> &cls)
 {
+    if (P->n_delimiters > 0)
+        for (int i = 0; i < P->n_delimiters; ++i) cls[P->delimiter_ids[i]] |= kClsDelim;
+    else
+        cls[P->delimiter_id] |= kClsDelim;
     for (int i = 0; i < P->n_keywords; ++i) cls[P->keyword_ids[i]] |= kClsKeyword;
     for (int i = 0; i < P->n_affirmation; ++i) cls[P->affirmation_ids[i]] |= kClsAffirm;
     for (int i = 0; i < P->n_verification; ++i) cls[P->verification_ids[i]] |= kClsVerify;
@@ -1759,7 +1781,6 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
         if (force[i] >= vlimit) return ST_ERR_VOCAB;
     for (int i = 0; i < P->n_keywords; ++i)
         if ((unsigned)P->keyword_ids[i] >= (unsigned)vlimit) return ST_ERR_VOCAB;
-    if ((unsigned)P->delimiter_id >= (unsigned)vlimit) return ST_ERR_VOCAB;
     TRY(check_rule_params(P, vlimit));
     const int max_new = P->max_new_tokens;
     if (out->cap_tokens < max_new || (max_new > 0 && (!out->tokens || !out->source))) return ST_ERR_CAPACITY;
@@ -1770,6 +1791,8 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     out->kv_len_small = out->kv_len_large = 0;
     out->seconds = 0.0;
     out->bytes_algorithmic = 0;
+    out->t_prompt_prefill_s = out->t_catchup_s = out->t_decode_s = 0.0;
+    out->n_prompt_prefill = out->n_catchup = out->n_decode = 0;
 
     cudaStream_t s = small->stream;
     CK(cudaMemsetAsync(small->status, 0, sizeof(int32_t), s));
@@ -1910,6 +1933,12 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     out->kv_len_large = gh.kv_len[1];
     out->seconds = ms * 1e-3;
     out->bytes_algorithmic = gh.bytes_algo;
+    out->t_prompt_prefill_s = (double)gh.t_kind[0] * 1e-9;
+    out->t_catchup_s = (double)gh.t_kind[1] * 1e-9;
+    out->t_decode_s = (double)gh.t_kind[2] * 1e-9;
+    out->n_prompt_prefill = gh.n_kind[0];
+    out->n_catchup = gh.n_kind[1];
+    out->n_decode = gh.n_kind[2];
     const int n_steps = gh.step < cap_steps ? gh.step : cap_steps;
     const int n_hand = gh.n_handoffs < cap_handoffs ? gh.n_handoffs : cap_handoffs;
     if (gh.generated > 0) {
@@ -1963,7 +1992,6 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
     if (vlimit > vshared) return ST_ERR_VOCAB;
     for (int i = 0; i < P->n_keywords; ++i)
         if ((unsigned)P->keyword_ids[i] >= (unsigned)vlimit) return ST_ERR_VOCAB;
-    if ((unsigned)P->delimiter_id >= (unsigned)vlimit) return ST_ERR_VOCAB;
     TRY(check_rule_params(P, vlimit));
     std::vector<int> plen(n), mnew(n), nforce(n), total(n);
     int longest = 0;
@@ -2213,6 +2241,10 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
             o.kv_len_large = g.kv_len[1];
             o.seconds = ms * 1e-3;   // of the whole batch
             o.bytes_algorithmic = g.bytes_algo;
+            o.t_prompt_prefill_s = o.t_catchup_s = o.t_decode_s = 0.0;
+            o.n_prompt_prefill = g.n_kind[0];
+            o.n_catchup = g.n_kind[1];
+            o.n_decode = g.n_kind[2];
             const int n_steps = g.step < o.cap_steps ? g.step : o.cap_steps;
             const int n_hand = g.n_handoffs < o.cap_handoffs ? g.n_handoffs : o.cap_handoffs;
             if (g.generated > 0) {

@@ -509,3 +509,27 @@ def test_hand_traced_rule_cases_on_device(B):
             assert cut.handoffs == T["handoffs"]
     gs.close()
     gl.close()
+
+
+def test_phase_times_and_pass_counts(B):
+    """The per-kind device times of st_spec_result (the split of the paper's Table "comparison of time"): the pass
+    counts must equal what the emission log says (one token ingested = decode, a model's first tokens = prompt
+    prefill, anything else = catch-up) and the three times must add up to the generation's device time."""
+    S, L = shape_dict(W.TINY_S), shape_dict(W.TINY_L)
+    gs = B.Model(S, seed=0, tag=0, max_tokens=1024)
+    gl = B.Model(L, seed=0, tag=1, max_tokens=1024)
+    prompt = W.prompt_ids(100, 300, 1024)          # longer than one 256-row pass: the prompt prefill is chunked
+    force = W.full_forcing(101, 1200, 1024, mean_interval=8, keyword_rate=0.5)
+    r = B.st_generate_spec(gs, gl, prompt, delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=5, max_new_tokens=400, force=force)
+    fed, src = r.emission_fed, r.emission_source
+    pt = r.phase_times
+    first = {int(m): int(np.argmax(src == m)) for m in (0, 1) if (src == m).any()}
+    n_prompt = sum(1 for m, t in first.items() if fed[t] > 1)
+    assert pt["decode"][1] == int((fed == 1).sum())
+    assert pt["prompt_prefill"][1] == n_prompt == 2
+    assert pt["catchup"][1] == int((fed > 1).sum()) - n_prompt and pt["catchup"][1] >= 5
+    total = sum(v[0] for v in pt.values())
+    assert all(v[0] > 0 for v in pt.values())
+    assert abs(total - r.seconds) <= 0.1 * r.seconds + 2e-4, (total, r.seconds)
+    gs.close()
+    gl.close()

@@ -28,9 +28,10 @@ def _trace(name):
     return out
 
 
-LIST_PARAMS = ("keyword_ids", "affirmation_ids", "verification_ids", "aux_ids")
+LIST_PARAMS = ("keyword_ids", "affirmation_ids", "verification_ids", "aux_ids", "delimiter_ids")
 RULE_TRACES = ["handoff_trace_verify_in_probe.txt", "handoff_trace_counter_reset.txt", "handoff_trace_probe_cut_replace.txt",
-               "handoff_trace_probe_cut_keep.txt", "handoff_trace_delimiter_in_probe.txt", "handoff_trace_target_verification.txt"]
+               "handoff_trace_probe_cut_keep.txt", "handoff_trace_delimiter_in_probe.txt", "handoff_trace_target_verification.txt",
+               "handoff_trace_delimiter_set.txt"]
 
 
 def load_rule_trace(name):
