@@ -203,6 +203,45 @@ int st_generate_spec_batch(st_model *small, st_model *large, const st_spec_param
                            const int32_t *prompts, const int32_t *prompt_offsets, const int32_t *max_new_per_seq,
                            const int32_t *force, const int32_t *force_offsets, st_spec_result *outs);
 
+/* Greedy speculative decoding on the same two models: the comparison system of the paper's section "Comparisons
+ * between Speculative Decoding and Speculative Thinking" (there with a 7B speculative and the 32B target model, the
+ * speculative model drafting 20 tokens per step).  Per round the speculative model drafts `gamma` tokens one by one,
+ * the target scores them in ONE multi-row pass, the longest prefix the target would have written itself is kept, and
+ * the target's own token follows (its next token when every draft was accepted; acceptance rule of Leviathan et al.
+ * 2023 for greedy decoding) -- so the output equals the target's own greedy continuation, and both KV caches are cut
+ * back to the accepted length after each round.  Both models must have the token ids below vocab_limit in common.
+ * force_draft[k] >= 0 (host, nullable) replaces the k-th draft, counted over all rounds; force_target[i] >= 0 replaces
+ * the target's choice for generated position i.  Rounds are host-driven: the host reads back only how far the text
+ * advanced, never a token.  All result arrays are caller-allocated host memory (optional ones may be NULL). */
+typedef struct {
+    int32_t gamma;          /* drafts per round (paper: 20); at most 254 */
+    int32_t eos_id;         /* -1: none */
+    int32_t vocab_limit;    /* 0 = min of the two vocabularies */
+    int32_t max_new_tokens;
+} st_specdec_params;
+
+typedef struct {
+    int32_t *tokens;         /* [cap_tokens] */
+    uint8_t *source;         /* [cap_tokens] 0 = accepted draft, 1 = written by the target */
+    int32_t cap_tokens, n_tokens;
+    int32_t *round_drafted;  /* [cap_rounds] drafts made in each round */
+    int32_t *round_accepted; /* [cap_rounds] drafts kept in each round */
+    int32_t cap_rounds, n_rounds;
+    int32_t kv_len_small, kv_len_large;
+    int32_t n_drafted, n_accepted;
+    int32_t *draft_tokens;   /* optional [cap_drafts] every draft, forcing applied */
+    int32_t *draft_argmax;   /* optional [cap_drafts] the speculative model's greedy choice behind each draft */
+    int32_t cap_drafts;
+    int32_t *choice_argmax;  /* optional [cap_tokens] the target's greedy choice (before forcing) for each generated position */
+    double seconds;          /* device time (CUDA events) */
+    int64_t bytes_algorithmic;
+} st_specdec_result;
+
+int st_generate_specdec(st_model *small, st_model *large, const st_specdec_params *params,
+                        const int32_t *prompt, int32_t prompt_len,
+                        const int32_t *force_draft, int32_t n_force_draft,
+                        const int32_t *force_target, int32_t n_force_target, st_specdec_result *out);
+
 /* Fill `out_dev` (bf16 bit patterns, device) with elements idx0.. of seeded tensor `tid`: the
  * generator behind st_model_create, exposed so that it can be compared bit for bit. */
 int st_fill_tensor_bf16(uint64_t seed, uint32_t model_tag, uint32_t tid, uint64_t idx0, uint64_t n,
@@ -219,6 +258,16 @@ int64_t st_kv_bytes_per_token(const st_model *m);
  * weight-streaming matrix-vector products of the decode pass).  Scratch activations are overwritten. */
 int64_t st_kernel_launches(void);
 int st_time_gemv(st_model *m, int32_t which, int32_t iters, double *seconds_out);
+
+/* Self-test of the bounded device-side waits (the paper has no counterpart; every spin of the kernels -- on an
+ * mbarrier, on the decode kernel's grid barrier -- gives up after a fixed number of polls, raises a status bit and
+ * lets the kernel run to its end instead of hanging the GPU).  Launches one CTA that waits, with a limit of 1000
+ * polls, for something that never happens: which = 0 an mbarrier nobody arms (the waits of the TMA / tensor-core
+ * pipelines), which = 1 the decode kernel's grid barrier with no other arrival.  Returns ST_ERR_TIMEOUT when the wait
+ * expired and the kernel returned normally (the expected outcome), ST_OK when it did not expire, ST_ERR_INTERNAL
+ * when the kernel never reached its end.  The model's status word and barrier state are clean afterwards.
+ * Synchronises the model's stream. */
+int st_selftest_bounded_wait(st_model *m, int32_t which);
 
 /* How the single-kernel decode step lays out its attention phase (Section 3 names no kernel; this describes the
  * split-KV decode attention of the hot path) when `ctx` tokens are cached: key splits per kv head, the capacity in
@@ -237,8 +286,9 @@ int st_decode_geometry(const st_model *m, int32_t ctx, int32_t *n_splits, int32_
  * maxima and a ticket word, 1 KB) is a fixed array inside the library image, present on every GPU
  * that loads the library until the process exits; n may be at most 4,194,304 (1 << 22), larger sizes
  * return ST_ERR_CAPACITY.  The first call on a device looks up the array's device address (no
- * allocation); make that first call outside any stream capture.  All calls share the one array:
- * calls that overlap on the GPU (different streams) race and must be serialised by the caller. */
+ * allocation); make that first call outside any stream capture.  `cuda_stream` must be a stream of the device that
+ * is current when the call is made (the array's address is looked up for the current device).  All calls share the
+ * one array: calls that overlap on the GPU (different streams) race and must be serialised by the caller. */
 int st_argmax_static(const float *logits_dev, int32_t n, int32_t *argmax_out_dev, void *cuda_stream);
 
 /* Sticky device status word (0 = clean) and message text. */

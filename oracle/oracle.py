@@ -68,6 +68,20 @@ class _SpecResult(C.Structure):
     ]
 
 
+class _SpecDecParams(C.Structure):
+    _fields_ = [("gamma", C.c_int32), ("eos_id", C.c_int32), ("vocab_limit", C.c_int32), ("max_new_tokens", C.c_int32)]
+
+
+class _SpecDecResult(C.Structure):
+    _fields_ = [
+        ("tokens", C.POINTER(C.c_int32)), ("source", C.POINTER(C.c_uint8)), ("cap_tokens", C.c_int32), ("n_tokens", C.c_int32),
+        ("round_drafted", C.POINTER(C.c_int32)), ("round_accepted", C.POINTER(C.c_int32)),
+        ("cap_rounds", C.c_int32), ("n_rounds", C.c_int32),
+        ("kv_len_small", C.c_int32), ("kv_len_large", C.c_int32), ("n_drafted", C.c_int32), ("n_accepted", C.c_int32),
+        ("choice_margin", C.POINTER(C.c_double)), ("draft_margin", C.POINTER(C.c_double)), ("cap_drafts", C.c_int32),
+    ]
+
+
 _lib = None
 
 
@@ -117,6 +131,9 @@ def lib():
         L.orc_forward_full.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
         L.orc_argmax.restype = C.c_int32
         L.orc_argmax.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_double)]
+        L.orc_generate_specdec.restype = C.c_int
+        L.orc_generate_specdec.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(_SpecDecParams), C.c_void_p, C.c_int32,
+                                           C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.POINTER(_SpecDecResult)]
         L.orc_generate_spec.restype = C.c_int
         L.orc_generate_spec.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(_SpecParams), C.c_void_p, C.c_int32,
                                         C.c_void_p, C.c_int32, C.POINTER(_SpecResult)]
@@ -330,3 +347,45 @@ def generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id: in
                       [(hand[i].seg_start, hand[i].step, hand[i].catchup_len) for i in range(R.n_handoffs)],
                       e_tok[:s].copy(), e_src[:s].copy(), e_fed[:s].copy(), e_arg[:s].copy(), e_mar[:s].copy(),
                       R.kv_len_small, R.kv_len_large, trace, rc, kinds[:R.n_handoffs].tolist())
+
+
+@dataclass
+class SpecDecResult:
+    tokens: np.ndarray
+    source: np.ndarray          # 0 = accepted draft, 1 = written by the target
+    rounds: list                # (drafted, accepted) per round
+    kv_len_small: int
+    kv_len_large: int
+    n_drafted: int
+    n_accepted: int
+    choice_margin: np.ndarray   # per generated position
+    draft_margin: np.ndarray    # per draft
+    rc: int
+
+
+def generate_specdec(small: Model, large: Model, prompt, *, gamma: int = 20, eos_id: int = -1, vocab_limit: int = 0,
+                     max_new_tokens: int, force_draft=None, force_target=None) -> SpecDecResult:
+    """Greedy speculative decoding (the paper's comparison system): see orc_generate_specdec."""
+    prompt = np.ascontiguousarray(prompt, dtype=np.int32)
+    if vocab_limit <= 0:
+        vocab_limit = min(small.cfg.vocab, large.cfg.vocab)
+    P = _SpecDecParams(gamma, eos_id, vocab_limit, max_new_tokens)
+    n = max_new_tokens + 1
+    tokens, source = np.zeros(n, dtype=np.int32), np.zeros(n, dtype=np.uint8)
+    rd, ra = np.zeros(n, dtype=np.int32), np.zeros(n, dtype=np.int32)
+    cap_drafts = gamma * n
+    cm, dm = np.zeros(n, dtype=np.float64), np.zeros(cap_drafts, dtype=np.float64)
+    R = _SpecDecResult()
+    ip = lambda a: a.ctypes.data_as(C.POINTER(C.c_int32))
+    R.tokens, R.source, R.cap_tokens = ip(tokens), source.ctypes.data_as(C.POINTER(C.c_uint8)), n
+    R.round_drafted, R.round_accepted, R.cap_rounds = ip(rd), ip(ra), n
+    R.choice_margin, R.draft_margin, R.cap_drafts = cm.ctypes.data_as(C.POINTER(C.c_double)), dm.ctypes.data_as(C.POINTER(C.c_double)), cap_drafts
+    fd = None if force_draft is None else np.ascontiguousarray(force_draft, dtype=np.int32)
+    ft = None if force_target is None else np.ascontiguousarray(force_target, dtype=np.int32)
+    rc = lib().orc_generate_specdec(small.h, large.h, C.byref(P), _p(prompt), prompt.size,
+                                    None if fd is None else _p(fd), 0 if fd is None else fd.size,
+                                    None if ft is None else _p(ft), 0 if ft is None else ft.size, C.byref(R))
+    k = R.n_rounds
+    return SpecDecResult(tokens[:R.n_tokens].copy(), source[:R.n_tokens].copy(), list(zip(rd[:k].tolist(), ra[:k].tolist())),
+                         R.kv_len_small, R.kv_len_large, R.n_drafted, R.n_accepted, cm[:R.n_tokens].copy(),
+                         dm[:R.n_drafted].copy(), rc)

@@ -704,3 +704,117 @@ int orc_generate_spec(const orc_model *small, const orc_model *large, const orc_
     free(z);
     return rc;
 }
+
+/* ------------------------------------------------------------------------- */
+/* Greedy speculative decoding: the comparison system of the paper's section  */
+/* "Comparisons between Speculative Decoding and Speculative Thinking"        */
+/* ------------------------------------------------------------------------- */
+
+/* The speculative model drafts gamma tokens one by one (the paper sets 20 "to match the number of intervention
+ * tokens"), the target model scores the drafts in one pass and keeps the longest prefix it would have written
+ * itself; the first draft it disagrees with is replaced by its own token, and when it agrees with all of them its
+ * next token comes for free (Leviathan et al., "Fast inference from transformers via speculative decoding", the
+ * greedy case).  Every round therefore writes (accepted drafts + 1) tokens, and the whole output equals the target
+ * model's own greedy continuation.  Both caches are cut back to the accepted length after a round.
+ *
+ * force_draft[k] >= 0 replaces the k-th drafted token (k counts drafts over all rounds); force_target[i] >= 0
+ * replaces the target's choice for the i-th generated position.  With both given the acceptance pattern is a pure
+ * function of the two arrays, which is how the hand-traced pins work. */
+typedef struct {
+    int32_t gamma;          /* drafts per round (paper: 20) */
+    int32_t eos_id;         /* -1: none */
+    int32_t vocab_limit;
+    int32_t max_new_tokens;
+} orc_specdec_params;
+
+typedef struct {
+    int32_t *tokens;        /* [cap_tokens] */
+    uint8_t *source;        /* [cap_tokens] 0 = accepted draft, 1 = written by the target */
+    int32_t cap_tokens, n_tokens;
+    int32_t *round_drafted, *round_accepted;   /* [cap_rounds] */
+    int32_t cap_rounds, n_rounds;
+    int32_t kv_len_small, kv_len_large;
+    int32_t n_drafted, n_accepted;             /* totals */
+    double *choice_margin;  /* optional [cap_tokens]: top-2 margin of the target's logits row that decided generated position i */
+    double *draft_margin;   /* optional [cap_drafts]: top-2 margin of the speculative model's logits behind draft k */
+    int32_t cap_drafts;
+} orc_specdec_result;
+
+int orc_generate_specdec(const orc_model *small, const orc_model *large, const orc_specdec_params *P,
+                         const int32_t *prompt, int32_t prompt_len, const int32_t *force_draft, int32_t n_force_draft,
+                         const int32_t *force_target, int32_t n_force_target, orc_specdec_result *R)
+{
+    if (prompt_len < 1 || P->max_new_tokens < 0 || P->gamma < 1) return -1;
+    int64_t cap = (int64_t)prompt_len + P->max_new_tokens + P->gamma + 2;
+    orc_kv *kvs = orc_kv_create(small, cap), *kvl = orc_kv_create(large, cap);
+    int32_t *tokens = (int32_t *)malloc((size_t)cap * sizeof(int32_t));
+    memcpy(tokens, prompt, (size_t)prompt_len * sizeof(int32_t));
+    int vmax = small->c.vocab > large->c.vocab ? small->c.vocab : large->c.vocab;
+    double *z = (double *)malloc((size_t)vmax * sizeof(double));
+    double *zrows = (double *)malloc((size_t)(P->gamma + 1) * (size_t)large->c.vocab * sizeof(double));
+    int32_t *draft = (int32_t *)malloc((size_t)P->gamma * sizeof(int32_t));
+    int32_t pos = prompt_len, generated = 0, k_draft = 0;
+    int rc = 0, stop = 0;
+    R->n_tokens = R->n_rounds = R->n_drafted = R->n_accepted = 0;
+    while (generated < P->max_new_tokens && !stop) {
+        /* drafts: as many as the round can still use (it always ends with one token of the target) */
+        int g = P->max_new_tokens - generated - 1;
+        if (g > P->gamma) g = P->gamma;
+        for (int i = 0; i < g; ++i) {
+            /* the speculative model ingests what it lacks (the prompt, the target's last token, its previous draft) */
+            int32_t fed = pos + i - (int32_t)kvs->len;
+            if (orc_forward(small, kvs, tokens + kvs->len, fed, 0, z) != 0) { rc = -2; break; }
+            double dm;
+            int32_t d = orc_argmax(z, P->vocab_limit, &dm);
+            if (force_draft && k_draft < n_force_draft && force_draft[k_draft] >= 0) d = force_draft[k_draft];
+            if (R->draft_margin && k_draft < R->cap_drafts) R->draft_margin[k_draft] = dm;
+            ++k_draft;
+            draft[i] = d;
+            tokens[pos + i] = d;   /* provisional: fed to both models, kept only if accepted */
+        }
+        if (rc) break;
+        /* the target scores the pending tokens and all drafts in one pass; the last g + 1 rows are its choices for
+         * positions pos .. pos + g */
+        int32_t fed_l = pos + g - (int32_t)kvl->len;
+        double *all = (double *)malloc((size_t)fed_l * (size_t)large->c.vocab * sizeof(double));
+        if (orc_forward(large, kvl, tokens + kvl->len, fed_l, 1, all) != 0) { free(all); rc = -2; break; }
+        memcpy(zrows, all + (size_t)(fed_l - (g + 1)) * large->c.vocab, (size_t)(g + 1) * large->c.vocab * sizeof(double));
+        free(all);
+        int n = 0;
+        int32_t choice = 0;
+        for (;;) {
+            double cm;
+            choice = orc_argmax(zrows + (size_t)n * large->c.vocab, P->vocab_limit, &cm);
+            if (R->choice_margin && generated + n < R->cap_tokens) R->choice_margin[generated + n] = cm;
+            if (force_target && generated + n < n_force_target && force_target[generated + n] >= 0) choice = force_target[generated + n];
+            if (n < g && draft[n] == choice) ++n; else break;
+        }
+        if (R->n_rounds >= R->cap_rounds) { rc = -3; break; }
+        R->round_drafted[R->n_rounds] = g;
+        R->round_accepted[R->n_rounds] = n;
+        R->n_rounds++;
+        R->n_drafted += g;
+        R->n_accepted += n;
+        /* write the accepted drafts and the target's token; an end-of-sequence id ends the output where it stands */
+        for (int i = 0; i <= n && !stop; ++i) {
+            int32_t tok = i < n ? draft[i] : choice;
+            if (generated >= R->cap_tokens) { rc = -3; stop = 1; break; }
+            tokens[pos] = tok;
+            R->tokens[generated] = tok;
+            R->source[generated] = (uint8_t)(i < n ? 0 : 1);
+            ++pos; ++generated;
+            if (tok == P->eos_id) stop = 1;
+        }
+        R->n_tokens = generated;
+        /* both caches keep the accepted prefix only (the target's own token has not been fed to anyone) */
+        int32_t keep = pos - 1;
+        if (kvl->len > keep) kvl->len = keep;
+        if (kvs->len > keep) kvs->len = keep;
+    }
+    R->kv_len_small = (int32_t)kvs->len;
+    R->kv_len_large = (int32_t)kvl->len;
+    orc_kv_destroy(kvs);
+    orc_kv_destroy(kvl);
+    free(tokens); free(z); free(zrows); free(draft);
+    return rc;
+}

@@ -67,11 +67,28 @@ class StSpecResult(C.Structure):
     ]
 
 
+class StSpecDecParams(C.Structure):
+    _fields_ = [("gamma", C.c_int32), ("eos_id", C.c_int32), ("vocab_limit", C.c_int32), ("max_new_tokens", C.c_int32)]
+
+
+class StSpecDecResult(C.Structure):
+    _fields_ = [
+        ("tokens", C.POINTER(C.c_int32)), ("source", C.POINTER(C.c_uint8)), ("cap_tokens", C.c_int32), ("n_tokens", C.c_int32),
+        ("round_drafted", C.POINTER(C.c_int32)), ("round_accepted", C.POINTER(C.c_int32)),
+        ("cap_rounds", C.c_int32), ("n_rounds", C.c_int32),
+        ("kv_len_small", C.c_int32), ("kv_len_large", C.c_int32), ("n_drafted", C.c_int32), ("n_accepted", C.c_int32),
+        ("draft_tokens", C.POINTER(C.c_int32)), ("draft_argmax", C.POINTER(C.c_int32)), ("cap_drafts", C.c_int32),
+        ("choice_argmax", C.POINTER(C.c_int32)),
+        ("seconds", C.c_double), ("bytes_algorithmic", C.c_int64),
+    ]
+
+
 EXPORTS = [
     "st_model_create", "st_model_destroy", "st_seq_alloc", "st_seq_free", "st_seq_reserve", "st_kv_len",
     "st_kv_truncate", "st_prefill", "st_decode_step", "st_generate_spec", "st_fill_tensor_bf16",
     "st_weight_bytes", "st_kv_bytes_per_token", "st_last_device_status", "st_strerror",
     "st_kernel_launches", "st_time_gemv", "st_argmax_static", "st_generate_spec_batch", "st_decode_geometry",
+    "st_generate_specdec", "st_selftest_bounded_wait",
 ]
 
 _lib = None
@@ -124,6 +141,11 @@ def lib():
         L.st_argmax_static.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.st_decode_geometry.restype = C.c_int
         L.st_decode_geometry.argtypes = [C.c_void_p, C.c_int32] + [C.POINTER(C.c_int32)] * 4
+        L.st_selftest_bounded_wait.restype = C.c_int
+        L.st_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_int32]
+        L.st_generate_specdec.restype = C.c_int
+        L.st_generate_specdec.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(StSpecDecParams), C.c_void_p, C.c_int32,
+                                          C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.POINTER(StSpecDecResult)]
         L.st_strerror.restype = C.c_char_p
         L.st_strerror.argtypes = [C.c_int]
         _lib = L
@@ -272,6 +294,10 @@ class Model:
     def st_kv_truncate(self, slot: int, new_len: int):
         _check(lib().st_kv_truncate(self.h, slot, new_len), "st_kv_truncate")
 
+    def st_selftest_bounded_wait(self, which: int) -> int:
+        """Status code of the bounded-wait self-test (ST_ERR_TIMEOUT is the expected outcome)."""
+        return int(lib().st_selftest_bounded_wait(self.h, which))
+
     def st_decode_geometry(self, ctx: int) -> dict:
         """Attention layout of the single-kernel decode step with ctx tokens cached (host arithmetic)."""
         v = [C.c_int32() for _ in range(4)]
@@ -413,3 +439,45 @@ def st_generate_spec_batch(small: Model, large: Model | None, prompts, *, delimi
                                       C.cast(Rs, C.c_void_p))
     _check(rc, "st_generate_spec_batch")
     return [b.result(Rs[i]) for i, b in enumerate(bufs)]
+
+
+@dataclass
+class SpecDecResult:
+    tokens: np.ndarray
+    source: np.ndarray          # 0 = accepted draft, 1 = written by the target
+    rounds: list                # (drafted, accepted) per round
+    kv_len_small: int
+    kv_len_large: int
+    n_drafted: int
+    n_accepted: int
+    draft_tokens: np.ndarray
+    draft_argmax: np.ndarray
+    choice_argmax: np.ndarray
+    seconds: float
+    bytes_algorithmic: int
+
+
+def st_generate_specdec(small: Model, large: Model, prompt, *, gamma: int = 20, eos_id: int = -1, vocab_limit: int = 0,
+                        max_new_tokens: int, force_draft=None, force_target=None) -> SpecDecResult:
+    """Greedy speculative decoding (the paper's comparison system): marshals the arguments of st_generate_specdec."""
+    prompt = np.ascontiguousarray(prompt, dtype=np.int32)
+    P = StSpecDecParams(gamma, eos_id, vocab_limit, max_new_tokens)
+    n = max_new_tokens + 1
+    ip = lambda a: a.ctypes.data_as(C.POINTER(C.c_int32))
+    tokens, source = np.zeros(n, dtype=np.int32), np.zeros(n, dtype=np.uint8)
+    rd, ra, ca = np.zeros(n, dtype=np.int32), np.zeros(n, dtype=np.int32), np.zeros(n, dtype=np.int32)
+    cap_drafts = gamma * n
+    dt, da = np.zeros(cap_drafts, dtype=np.int32), np.zeros(cap_drafts, dtype=np.int32)
+    R = StSpecDecResult()
+    R.tokens, R.source, R.cap_tokens = ip(tokens), source.ctypes.data_as(C.POINTER(C.c_uint8)), n
+    R.round_drafted, R.round_accepted, R.cap_rounds = ip(rd), ip(ra), n
+    R.draft_tokens, R.draft_argmax, R.cap_drafts, R.choice_argmax = ip(dt), ip(da), cap_drafts, ip(ca)
+    fd = None if force_draft is None else np.ascontiguousarray(force_draft, dtype=np.int32)
+    ft = None if force_target is None else np.ascontiguousarray(force_target, dtype=np.int32)
+    rc = lib().st_generate_specdec(small.h, large.h, C.byref(P), _np_ptr(prompt), prompt.size, _np_ptr(fd), 0 if fd is None else fd.size,
+                                   _np_ptr(ft), 0 if ft is None else ft.size, C.byref(R))
+    _check(rc, "st_generate_specdec")
+    k = R.n_rounds
+    return SpecDecResult(tokens[:R.n_tokens].copy(), source[:R.n_tokens].copy(), list(zip(rd[:k].tolist(), ra[:k].tolist())),
+                         R.kv_len_small, R.kv_len_large, R.n_drafted, R.n_accepted, dt[:R.n_drafted].copy(), da[:R.n_drafted].copy(),
+                         ca[:R.n_tokens].copy(), R.seconds, R.bytes_algorithmic)

@@ -68,6 +68,7 @@ struct MegaParams {
     int32_t n_layers, h, Hq, Hkv, f, vocab, n_splits, unit_keys, stages, xarea_bytes;
     int32_t down_slab;        // K segments per slab of the down projection (0: the whole input vector is kept)
     int32_t kv_off, kv_cap;   // K/V staging area inside the activation area: byte offset, capacity in keys (multiple of 16)
+    uint32_t spin_limit;      // polls of a grid barrier before it gives up (kMegaSpinLimit in normal use)
     float eps, scale;
     // sampling
     int32_t want_argmax, limit;
@@ -255,7 +256,7 @@ __device__ __forceinline__ bool mega_barrier_wait(const MegaParams &p, MegaShare
         const unsigned target = epoch * members;
         const unsigned *ctr = mega_bar_counter(p, i);
         bool ok = false;
-        for (uint32_t it = 0; it < kMegaSpinLimit; ++it) {
+        for (uint32_t it = 0; it < p.spin_limit; ++it) {
             const bool mine = ctid >= kMegaBarCounters || ld_acquire_u32(ctr) >= target;
             if (__all_sync(0xffffffffu, mine)) { ok = true; break; }
             if ((it & 63) == 63 && __any_sync(0xffffffffu, ld_acquire_u32(&p.sync[2]) != 0)) break;
@@ -895,6 +896,22 @@ __device__ __forceinline__ void mega_zero(float *buf, int n, int ctid)
         const int b = blockIdx.x * per, e = min(n, b + per);
         for (int i = b + ctid; i < e; i += kMegaCT) buf[i] = 0.f;
     }
+}
+
+// Exercises the grid barrier's bounded wait: one CTA waits for an arrival that never comes (it does not arrive
+// itself); the wait must give up after p.spin_limit polls, raise the abort flag and the status bit, and return.
+__global__ void __launch_bounds__(kMegaThreads, 1) mega_barrier_selftest_kernel(const MegaParams p, int32_t *returned)
+{
+    __shared__ MegaShared sh;
+    const int tid = threadIdx.x;
+    if (tid == 0) sh.abort = 0;
+    __syncthreads();
+    if (tid < 32) return;   // the producer warp has no part in barriers
+    const int ctid = tid - 32;
+    unsigned epoch = 0;
+    const bool ok = mega_barrier_wait(p, sh, epoch, ctid);
+    const bool ok2 = mega_barrier_wait(p, sh, epoch, ctid);   // returns at once: the abort flag is up
+    if (ctid == 0) *returned = (ok || ok2) ? 1 : 2;
 }
 
 template <int D, int G>

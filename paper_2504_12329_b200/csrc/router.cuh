@@ -353,6 +353,81 @@ __global__ void batch_plan_kernel(GenState *gs, const GenBuffers *gb, int n_seqs
     plan->all_done = live == 0;
 }
 
+// ---- greedy speculative decoding (the paper's comparison system): draft bookkeeping and the acceptance rule ----
+
+struct SpecDecState {
+    int32_t pos, generated;     // next position to write; tokens written after the prompt
+    int32_t k_draft;            // drafts made so far (index into the draft forcing array and logs)
+    int32_t g;                  // drafts of the round in progress
+    int32_t n_rounds, n_drafted, n_accepted;
+    int32_t last_accepted;      // accepted drafts of the round just closed (what the host reads back)
+    int32_t done;
+    int32_t eos, max_new, vlimit, n_force_draft, n_force_target, cap_rounds, cap_drafts, prompt_len;
+};
+
+struct SpecDecBuffers {
+    int32_t *tokens;            // [prompt_len + max_new + gamma + 2] whole sequence, drafts written provisionally
+    uint8_t *source;            // [max_new + 1] 0 = accepted draft, 1 = written by the target
+    int32_t *round_drafted, *round_accepted;   // [cap_rounds]
+    int32_t *draft_tok, *draft_arg;            // [cap_drafts] every draft (after forcing) and the greedy choice behind it
+    int32_t *choice_arg;                       // [max_new + 1] the target's greedy choice for each generated position it decided
+    const int32_t *force_draft, *force_target;
+};
+
+// The speculative model sampled draft i of the round: apply the forcing array, log, and place the draft at
+// position pos + i, where the next pass of either model reads it.
+__global__ void specdec_take_draft_kernel(SpecDecState *s, SpecDecBuffers b, const int32_t *greedy, int i, int32_t *status)
+{
+    const int k = s->k_draft;
+    int d = *greedy;
+    if (k < s->n_force_draft && b.force_draft[k] >= 0) d = b.force_draft[k];
+    if ((unsigned)d >= (unsigned)s->vlimit) { atomicOr(status, DEV_BAD_TOKEN); d = 0; }
+    if (k < s->cap_drafts) {
+        b.draft_tok[k] = d;
+        b.draft_arg[k] = *greedy;
+    }
+    b.tokens[s->pos + i] = d;
+    s->k_draft = k + 1;
+}
+
+// The target scored the round: choices[j] is its greedy token for position pos + j (j <= g).  Keep the longest
+// prefix of drafts it would have written itself, then its own token; an end-of-sequence id ends the output.
+__global__ void specdec_accept_kernel(SpecDecState *s, SpecDecBuffers b, const int32_t *choices, int32_t *status)
+{
+    const int g = s->g, pos = s->pos;
+    int n = 0, choice = 0;
+    for (;;) {
+        const int raw = choices[n];
+        choice = raw;
+        const int gi = s->generated + n;
+        if (gi < s->n_force_target && b.force_target[gi] >= 0) choice = b.force_target[gi];
+        if ((unsigned)choice >= (unsigned)s->vlimit) { atomicOr(status, DEV_BAD_TOKEN); choice = 0; }
+        if (gi <= s->max_new) b.choice_arg[gi] = raw;
+        if (n < g && b.tokens[pos + n] == choice) ++n; else break;
+    }
+    if (s->n_rounds < s->cap_rounds) {
+        b.round_drafted[s->n_rounds] = g;
+        b.round_accepted[s->n_rounds] = n;
+    } else {
+        atomicOr(status, DEV_LOG_FULL);
+    }
+    s->n_rounds++;
+    s->n_drafted += g;
+    s->n_accepted += n;
+    int written = 0;
+    for (int i = 0; i <= n && !s->done; ++i) {
+        const int tok = i < n ? b.tokens[pos + i] : choice;
+        b.tokens[pos + i] = tok;
+        b.source[s->generated] = (uint8_t)(i < n ? 0 : 1);
+        s->generated++;
+        ++written;
+        if (tok == s->eos) s->done = 1;
+    }
+    s->pos = pos + written;
+    s->last_accepted = n;
+    if (s->generated >= s->max_new) s->done = 1;
+}
+
 struct ArgmaxParams {
     const float *logits;   // [vocab]
     int32_t limit;         // ids < limit compete

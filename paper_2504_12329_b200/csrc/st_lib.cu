@@ -477,6 +477,10 @@ static int launch_tc_gemm(const CUtensorMap &tw, TcGemmParams p, int m_upper, in
             if (eff > best + 0.03) { best = eff; wt = cand; }
         }
     }
+    {   // tuning aid: force the weight tiles per CTA (when the forced count fits tensor and shared memory)
+        static const int forced = [] { const char *e = getenv("ST_TC_WT"); return e ? atoi(e) : 0; }();
+        if (forced >= 1 && forced <= 4 && forced * p.m_pad <= 512 && 2 * (forced * kTcWBytes + 2 * p.m_pad * kTcBlockK * 2) <= 220 * 1024) wt = forced;
+    }
     p.w_tiles = wt;
     int cols = wt * p.m_pad;
     p.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
@@ -973,6 +977,7 @@ static int pass_decode(st_model *m, const StepDesc *desc, const int32_t *tok, in
     p.n_layers = c.n_layers; p.h = c.hidden; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.f = c.ffn; p.vocab = c.vocab;
     p.n_splits = m->mega_splits; p.unit_keys = m->mega_unit_keys; p.stages = m->mega_stages; p.xarea_bytes = m->mega_xarea;
     p.kv_off = m->mega_kv_off; p.kv_cap = m->mega_kv_cap; p.down_slab = m->mega_down_slab;
+    p.spin_limit = kMegaSpinLimit;
     p.eps = c.rms_eps; p.scale = 1.f / sqrtf((float)c.head_dim);
     p.want_argmax = sc.want_argmax ? 1 : 0;
     p.limit = sc.vlimit > 0 ? sc.vlimit : c.vocab;
@@ -1257,6 +1262,37 @@ int64_t st_kv_bytes_per_token(const st_model *m)
 }
 
 int64_t st_kernel_launches(void) { return g_launches; }
+
+int st_selftest_bounded_wait(st_model *m, int32_t which)
+{
+    if (!m || which < 0 || which > 1) return ST_ERR_ARG;
+    cudaStream_t s = m->stream;
+    int32_t *d_ret = (int32_t *)m->tokbuf;   // a device word nobody uses between calls
+    CK(cudaMemsetAsync(m->status, 0, sizeof(int32_t), s));
+    CK(cudaMemsetAsync(d_ret, 0, sizeof(int32_t), s));
+    CK(cudaMemsetAsync(m->mega_sync, 0, kMegaSyncWords * sizeof(unsigned), s));
+    if (which == 0) {
+        wait_expiry_selftest_kernel<<<1, 64, 0, s>>>(m->status, 1000u, d_ret);
+    } else {
+        MegaParams p{};
+        p.sync = m->mega_sync;
+        p.status = m->status;
+        p.spin_limit = 1000u;
+        mega_barrier_selftest_kernel<<<1, kMegaThreads, 0, s>>>(p, d_ret);
+    }
+    ++g_launches;
+    CK(cudaGetLastError());
+    int32_t ret = 0, status = 0;
+    CK(cudaMemcpyAsync(&ret, d_ret, sizeof ret, cudaMemcpyDeviceToHost, s));
+    CK(cudaMemcpyAsync(&status, m->status, sizeof status, cudaMemcpyDeviceToHost, s));
+    CK(cudaStreamSynchronize(s));
+    // leave the model clean for the next ordinary call
+    CK(cudaMemsetAsync(m->status, 0, sizeof(int32_t), s));
+    CK(cudaMemsetAsync(m->mega_sync, 0, kMegaSyncWords * sizeof(unsigned), s));
+    if (ret == 0) return ST_ERR_INTERNAL;                          // the kernel did not reach its end
+    if (ret == 2 && (status & DEV_WAIT_EXPIRED)) return ST_ERR_TIMEOUT;   // the wait gave up as it should
+    return ST_OK;                                                  // the wait did not expire: the check failed
+}
 
 int st_decode_geometry(const st_model *m, int32_t ctx, int32_t *n_splits, int32_t *kv_cap, int32_t *max_chunks, int32_t *own_chunk_empty)
 {
@@ -1859,6 +1895,10 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     // every token costs a pass; a replaced probe sentence costs probe_len passes more per takeover
     const int64_t pass_cap = (1ll + g0.probe_len) * (max_new + 2) + 2ll * (total / g0.max_chunk + 2) * (max_new / P->n1 + 2);
     g0.pass_cap = pass_cap > 0x7fffffff ? 0x7fffffff : (int32_t)pass_cap;
+    if (const char *e = getenv("ST_TEST_PASS_CAP")) {   // test aid: makes the device loop's pass bound run out
+        const int cap = atoi(e);
+        if (cap > 0 && cap < g0.pass_cap) g0.pass_cap = cap;
+    }
     CK(cudaMemcpyAsync(gen, &g0, sizeof g0, cudaMemcpyHostToDevice, s));
     CK(cudaMemcpyAsync(b.tokens, prompt, (size_t)prompt_len * sizeof(int32_t), cudaMemcpyHostToDevice, s));
     if (n_force) CK(cudaMemcpyAsync(C.d_force, force, (size_t)n_force * sizeof(int32_t), cudaMemcpyHostToDevice, s));
@@ -2307,6 +2347,228 @@ extern "C" int st_generate_spec_batch(st_model *small, st_model *large, const st
         TRY(st_generate_spec(small, large, &pi, prompts + prompt_offsets[i], prompt_offsets[i + 1] - prompt_offsets[i],
                              nf > 0 ? f : nullptr, nf, &outs[i]));
     }
+    return ST_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// greedy speculative decoding (the paper's comparison system)
+// ------------------------------------------------------------------------------------------------
+
+namespace {
+struct DevArena {   // one cudaMalloc for the buffers of a call
+    uint8_t *base = nullptr;
+    size_t off = 0;
+    size_t take(size_t bytes) { off = (off + 255) & ~(size_t)255; const size_t o = off; off += bytes; return o; }
+    ~DevArena() { if (base) cudaFree(base); }
+};
+}  // namespace
+
+// Rounds are driven from the host: the speculative model drafts g tokens (single-kernel decode steps chained on the
+// device: each step reads the token the previous one placed), the target scores the pending tokens and the drafts in
+// one multi-row pass whose LM head covers every row (the ragged-batch pass with all rows on one sequence), a
+// one-thread kernel applies the acceptance rule, and the host reads back how far the text advanced (never a token)
+// to size the next round and to cut both caches back to the accepted length.
+extern "C" int st_generate_specdec(st_model *small, st_model *large, const st_specdec_params *P, const int32_t *prompt,
+                                   int32_t prompt_len, const int32_t *force_draft, int32_t n_force_draft,
+                                   const int32_t *force_target, int32_t n_force_target, st_specdec_result *out)
+{
+    if (!small || !large || !P || !prompt || !out || prompt_len < 1 || P->max_new_tokens < 0 || P->gamma < 1) return ST_ERR_ARG;
+    if (n_force_draft < 0 || n_force_target < 0 || (n_force_draft > 0 && !force_draft) || (n_force_target > 0 && !force_target)) return ST_ERR_ARG;
+    if (large->stream != small->stream || large->device != small->device) return ST_ERR_ARG;
+    const int gamma = P->gamma, max_new = P->max_new_tokens;
+    if (gamma + 1 > large->max_rows - 1) return ST_ERR_UNSUPPORTED;
+    const int vshared = small->cfg.vocab < large->cfg.vocab ? small->cfg.vocab : large->cfg.vocab;
+    const int vlimit = P->vocab_limit > 0 ? P->vocab_limit : vshared;
+    if (vlimit > vshared) return ST_ERR_VOCAB;
+    for (int i = 0; i < prompt_len; ++i)
+        if ((unsigned)prompt[i] >= (unsigned)vlimit) return ST_ERR_VOCAB;
+    for (int i = 0; i < n_force_draft; ++i)
+        if (force_draft[i] >= vlimit) return ST_ERR_VOCAB;
+    for (int i = 0; i < n_force_target; ++i)
+        if (force_target[i] >= vlimit) return ST_ERR_VOCAB;
+    if (out->cap_tokens < max_new || (max_new > 0 && (!out->tokens || !out->source))) return ST_ERR_CAPACITY;
+    if (out->cap_rounds > 0 && (!out->round_drafted || !out->round_accepted)) return ST_ERR_ARG;
+    out->n_tokens = out->n_rounds = out->n_drafted = out->n_accepted = 0;
+    out->kv_len_small = out->kv_len_large = 0;
+    out->seconds = 0.0;
+    out->bytes_algorithmic = 0;
+    if (max_new == 0) return ST_OK;
+
+    cudaStream_t s = small->stream;
+    st_model *models[2] = {small, large};
+    for (st_model *m : models) {
+        CK(cudaMemsetAsync(m->status, 0, sizeof(int32_t), s));
+        CK(cudaMemsetAsync(m->mega_sync, 0, kMegaSyncWords * sizeof(unsigned), s));
+    }
+    if (!large->batch_logits) {
+        large->batch_logits = (float *)large->dalloc((size_t)large->max_rows * large->cfg.vocab * sizeof(float));
+        if (!large->batch_logits) return ST_ERR_OOM;
+    }
+    const int total = prompt_len + max_new + gamma + 2;
+    SlotGuard gs{small}, gl{large};
+    TRY(st_seq_alloc(small, &gs.slot));
+    TRY(seq_reserve(small, gs.slot, total));
+    TRY(st_seq_alloc(large, &gl.slot));
+    TRY(seq_reserve(large, gl.slot, total));
+
+    const int cap_rounds = out->cap_rounds > 0 ? out->cap_rounds : 1;
+    const int cap_drafts = out->cap_drafts > 0 ? out->cap_drafts : 1;
+    DevArena A;
+    const size_t o_state = A.take(sizeof(SpecDecState)), o_tok = A.take((size_t)total * 4), o_src = A.take((size_t)max_new + 1);
+    const size_t o_rd = A.take((size_t)cap_rounds * 4), o_ra = A.take((size_t)cap_rounds * 4);
+    const size_t o_dt = A.take((size_t)cap_drafts * 4), o_da = A.take((size_t)cap_drafts * 4), o_ca = A.take(((size_t)max_new + 1) * 4);
+    const size_t o_fd = A.take((size_t)(n_force_draft > 0 ? n_force_draft : 1) * 4), o_ft = A.take((size_t)(n_force_target > 0 ? n_force_target : 1) * 4);
+    const size_t o_desc = A.take((size_t)(gamma + 8) * sizeof(StepDesc)), o_amax_s = A.take(4), o_amax_l = A.take((size_t)large->max_rows * 4);
+    if (cudaMalloc(&A.base, A.off + 256) != cudaSuccess) { cudaGetLastError(); return ST_ERR_OOM; }
+    SpecDecState *d_state = (SpecDecState *)(A.base + o_state);
+    SpecDecBuffers b{};
+    b.tokens = (int32_t *)(A.base + o_tok);
+    b.source = A.base + o_src;
+    b.round_drafted = (int32_t *)(A.base + o_rd);
+    b.round_accepted = (int32_t *)(A.base + o_ra);
+    b.draft_tok = (int32_t *)(A.base + o_dt);
+    b.draft_arg = (int32_t *)(A.base + o_da);
+    b.choice_arg = (int32_t *)(A.base + o_ca);
+    b.force_draft = (const int32_t *)(A.base + o_fd);
+    b.force_target = (const int32_t *)(A.base + o_ft);
+    StepDesc *d_desc = (StepDesc *)(A.base + o_desc);
+    int32_t *d_amax_s = (int32_t *)(A.base + o_amax_s), *d_amax_l = (int32_t *)(A.base + o_amax_l);
+
+    SpecDecState st{};
+    st.pos = prompt_len;
+    st.eos = P->eos_id;
+    st.max_new = max_new;
+    st.vlimit = vlimit;
+    st.n_force_draft = n_force_draft;
+    st.n_force_target = n_force_target;
+    st.cap_rounds = out->cap_rounds;
+    st.cap_drafts = out->cap_drafts;
+    st.prompt_len = prompt_len;
+    CK(cudaMemcpyAsync(d_state, &st, sizeof st, cudaMemcpyHostToDevice, s));
+    CK(cudaMemcpyAsync(b.tokens, prompt, (size_t)prompt_len * 4, cudaMemcpyHostToDevice, s));
+    if (n_force_draft) CK(cudaMemcpyAsync(A.base + o_fd, force_draft, (size_t)n_force_draft * 4, cudaMemcpyHostToDevice, s));
+    if (n_force_target) CK(cudaMemcpyAsync(A.base + o_ft, force_target, (size_t)n_force_target * 4, cudaMemcpyHostToDevice, s));
+
+    cudaEvent_t ev0, ev1;
+    CK(cudaEventCreate(&ev0));
+    CK(cudaEventCreate(&ev1));
+    CK(cudaEventRecord(ev0, s));
+    int kv_s = 0, kv_l = 0;   // cached lengths (host mirrors; the passes take their positions from descriptors)
+    int64_t bytes = 0;
+    int rc = ST_OK;
+    std::vector<StepDesc> descs;
+    std::vector<int32_t> rows;
+    // a model ingests `pending` tokens starting at position kv (chunks of a pass's rows); the last chunk samples into amax
+    auto ingest = [&](st_model *m, int slot, int &kv, int pending, int32_t *amax, bool sample_last) -> int {
+        while (pending > 0 && rc == ST_OK) {
+            const int rows_now = pending < m->max_rows ? pending : m->max_rows;
+            const bool last = rows_now == pending;
+            const bool emit = last && sample_last;
+            StepDesc d{kv, rows_now, kv, emit ? 1 : 0};
+            const int di = (int)descs.size();
+            if (di >= gamma + 8) { CK(cudaStreamSynchronize(s)); descs.clear(); }
+            descs.push_back(d);
+            StepDesc *dd = d_desc + (descs.size() - 1);
+            CK(cudaMemcpyAsync(dd, &descs.back(), sizeof d, cudaMemcpyHostToDevice, s));
+            SampleCtx sc{};
+            sc.argmax_out = amax;
+            sc.vlimit = vlimit;
+            sc.want_argmax = emit;
+            if (rows_now == 1 && emit) rc = pass_decode(m, dd, b.tokens, slot, kv + 1, sc);
+            else rc = pass_rows(m, dd, b.tokens, slot, rows_now, kv + rows_now, emit, sc);
+            bytes += m->weight_bytes + st_kv_bytes_per_token(m) * (int64_t)(kv + rows_now);
+            kv += rows_now;
+            pending -= rows_now;
+        }
+        return rc;
+    };
+    const int64_t round_cap = (int64_t)max_new + 4;
+    int generated = 0, pos = prompt_len;
+    for (int64_t round = 0; round < round_cap && rc == ST_OK; ++round) {
+        descs.clear();
+        descs.reserve(gamma + 8);
+        int g = max_new - generated - 1;
+        g = g > gamma ? gamma : g;
+        CK(cudaMemcpyAsync(&d_state->g, &g, sizeof g, cudaMemcpyHostToDevice, s));
+        // ---- drafts ----
+        for (int i = 0; i < g && rc == ST_OK; ++i) {
+            TRY(ingest(small, gs.slot, kv_s, pos + i - kv_s, d_amax_s, true));
+            specdec_take_draft_kernel<<<1, 1, 0, s>>>(d_state, b, d_amax_s, i, small->status);
+            ++g_launches;
+            CK(cudaGetLastError());
+        }
+        // ---- the target scores the pending tokens and the drafts: all rows of its last pass get logits ----
+        int pending = pos + g - kv_l;
+        if (pending > large->max_rows) TRY(ingest(large, gl.slot, kv_l, pending - (g + 1), nullptr, false));   // a long prompt first
+        pending = pos + g - kv_l;
+        {
+            rows.assign(2 * (size_t)pending, 0);
+            for (int j = 0; j < pending; ++j) { rows[j] = gl.slot; rows[pending + j] = kv_l + j; }
+            CK(cudaMemcpyAsync(large->row_slot, rows.data(), (size_t)pending * 4, cudaMemcpyHostToDevice, s));
+            CK(cudaMemcpyAsync(large->row_pos, rows.data() + pending, (size_t)pending * 4, cudaMemcpyHostToDevice, s));
+            StepDesc d{0, pending, kv_l, 1};
+            descs.push_back(d);
+            StepDesc *dd = d_desc + (descs.size() - 1);
+            CK(cudaMemcpyAsync(dd, &descs.back(), sizeof d, cudaMemcpyHostToDevice, s));
+            SampleCtx sc{};
+            sc.logits_out = large->batch_logits;
+            sc.argmax_out = d_amax_l;
+            sc.vlimit = vlimit;
+            sc.want_argmax = true;
+            int m_upper = (pending + 31) / 32 * 32;
+            if (m_upper > large->max_rows) m_upper = large->max_rows;
+            TRY(pass_rows(large, dd, b.tokens, -1, m_upper, kv_l + pending, true, sc, true));
+            bytes += large->weight_bytes + st_kv_bytes_per_token(large) * (int64_t)(kv_l + pending);
+        }
+        specdec_accept_kernel<<<1, 1, 0, s>>>(d_state, b, d_amax_l + (pending - (g + 1)), large->status);
+        ++g_launches;
+        CK(cudaGetLastError());
+        CK(cudaMemcpyAsync(&st, d_state, sizeof st, cudaMemcpyDeviceToHost, s));
+        CK(cudaStreamSynchronize(s));   // also makes the staging vectors reusable
+        kv_l += pending;
+        pos = st.pos;
+        generated = st.generated;
+        // both caches keep the accepted prefix only (the target's own token has not been fed to anyone)
+        if (kv_l > pos - 1) kv_l = pos - 1;
+        if (kv_s > pos - 1) kv_s = pos - 1;
+        if (st.done) break;
+    }
+    cudaEventRecord(ev1, s);
+    if (cudaStreamSynchronize(s) != cudaSuccess && rc == ST_OK) { set_error_text("speculative decoding", cudaGetLastError()); rc = ST_ERR_INTERNAL; }
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, ev0, ev1);
+    cudaEventDestroy(ev0);
+    cudaEventDestroy(ev1);
+    if (rc != ST_OK) return rc;
+    if (!st.done) return ST_ERR_TIMEOUT;
+    out->n_tokens = st.generated;
+    out->n_rounds = st.n_rounds;
+    out->n_drafted = st.n_drafted;
+    out->n_accepted = st.n_accepted;
+    out->kv_len_small = kv_s;
+    out->kv_len_large = kv_l;
+    out->seconds = ms * 1e-3;
+    out->bytes_algorithmic = bytes;
+    const int nr = st.n_rounds < out->cap_rounds ? st.n_rounds : out->cap_rounds;
+    const int nd = st.k_draft < out->cap_drafts ? st.k_draft : out->cap_drafts;
+    CK(cudaMemcpyAsync(out->tokens, b.tokens + prompt_len, (size_t)st.generated * 4, cudaMemcpyDeviceToHost, s));
+    CK(cudaMemcpyAsync(out->source, b.source, (size_t)st.generated, cudaMemcpyDeviceToHost, s));
+    if (nr > 0) {
+        CK(cudaMemcpyAsync(out->round_drafted, b.round_drafted, (size_t)nr * 4, cudaMemcpyDeviceToHost, s));
+        CK(cudaMemcpyAsync(out->round_accepted, b.round_accepted, (size_t)nr * 4, cudaMemcpyDeviceToHost, s));
+    }
+    if (nd > 0 && out->draft_tokens) CK(cudaMemcpyAsync(out->draft_tokens, b.draft_tok, (size_t)nd * 4, cudaMemcpyDeviceToHost, s));
+    if (nd > 0 && out->draft_argmax) CK(cudaMemcpyAsync(out->draft_argmax, b.draft_arg, (size_t)nd * 4, cudaMemcpyDeviceToHost, s));
+    if (out->choice_argmax) CK(cudaMemcpyAsync(out->choice_argmax, b.choice_arg, (size_t)st.generated * 4, cudaMemcpyDeviceToHost, s));
+    CK(cudaStreamSynchronize(s));
+    int32_t dev_status = 0, s2 = 0;
+    CK(cudaMemcpy(&dev_status, small->status, sizeof dev_status, cudaMemcpyDeviceToHost));
+    CK(cudaMemcpy(&s2, large->status, sizeof s2, cudaMemcpyDeviceToHost));
+    dev_status |= s2;
+    if (dev_status & DEV_LOG_FULL) return ST_ERR_CAPACITY;
+    if (dev_status & DEV_BAD_TOKEN) return ST_ERR_VOCAB;
+    if (dev_status & DEV_WAIT_EXPIRED) return ST_ERR_TIMEOUT;
+    if (dev_status) return ST_ERR_INTERNAL;
     return ST_OK;
 }
 

@@ -12,7 +12,7 @@
 // One CTA = w_tiles adjacent 128-row weight tiles x one K split.  Warp 0 issues TMA, warp 1 owns TMEM and issues
 // the MMAs, warps 2..5 drain the accumulator (tcgen05.ld) into the epilogue.  Stages hand over
 // through mbarriers; every wait is bounded and, when it runs out, raises a status bit, lets the CTA
-// drain what it armed, frees its TMEM and returns.  No multicast, no clusters.
+// drain what it armed, frees its TMEM and returns.  Every CTA stands alone: each loads its own tiles.
 #pragma once
 #include <cuda.h>
 
@@ -69,9 +69,10 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait: false (and a status bit) when the phase does not complete within the limit.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status,
+                                          uint32_t limit = kTcWaitLimit)
 {
-    for (uint32_t it = 0; it < kTcWaitLimit; ++it) {
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try(bar, parity)) return true;
         if (*abort_flag) return false;
         if (it > 64) __nanosleep(64);
@@ -130,6 +131,27 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v)
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Exercises the bounded wait without faulting anything: one CTA waits, with a short limit, on an mbarrier that
+// nobody arms; the wait must give up, raise the status bit and let the kernel return normally.
+__global__ void wait_expiry_selftest_kernel(int32_t *status, uint32_t limit, int32_t *returned)
+{
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    bool ok = true;
+    if (threadIdx.x == 0) ok = mbar_wait(smem_u32(&bar), 0, &abort_flag, status, limit);
+    __syncthreads();
+    // every later wait of the CTA returns at once after the first one gave up
+    if (threadIdx.x == 32) ok = mbar_wait(smem_u32(&bar), 0, &abort_flag, status, 1u << 30);
+    __syncthreads();
+    if (threadIdx.x == 0) *returned = ok ? 1 : 2;
 }
 
 // Sum the K-split partials of a projection in a fixed order: Y[i][n] (+)= sum_s Ws[s][i][n] (+ bias[n]).

@@ -133,3 +133,33 @@ def test_qwen7b_32b_long_context_routing(B, oracle):
     assert (got.kv_len_small, got.kv_len_large) == (want.kv_len_small, want.kv_len_large)
     small.close()
     large.close()
+
+
+def test_batch64_routing_at_full_size(B, oracle):
+    """The 64-sequence workload on the 1.5B + 32B shapes (ragged prompts of 64..512 tokens, one forcing schedule per
+    sequence, budgets shortened to 150..350 tokens), every step forced: the batched rounds must give every sequence
+    the routing the oracle's state machine gives it alone (tokens, sources, handoffs with catch-up lengths, per-step
+    ingested counts, KV lengths)."""
+    n = 64
+    rng = np.random.default_rng(17)
+    lens = rng.integers(64, 513, size=n)
+    budgets = [int(x) for x in rng.integers(150, 351, size=n)]
+    prompts = [W.prompt_ids(900 + i, int(lens[i]), 1024) for i in range(n)]
+    forces = [W.full_forcing(2000 + i, 2 * budgets[i], 1024, mean_interval=40.0, keyword_rate=0.3) for i in range(n)]
+    wants = [_routing_reference(oracle, prompts[i], forces[i], W.N1, budgets[i]) for i in range(n)]
+    assert sum(len(w.handoffs) for w in wants) >= 30
+    cap = sum(len(p) + b + 80 for p, b in zip(prompts, budgets))
+    small = B.Model(W.QWEN_1P5B.as_dict(), seed=0, tag=0, max_seqs=n, max_tokens=cap)
+    large = B.Model(W.QWEN_32B.as_dict(), seed=0, tag=1, max_seqs=n, max_tokens=cap)
+    gots = B.st_generate_spec_batch(small, large, prompts, delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=W.N1,
+                                    max_new_tokens=budgets, forces=forces)
+    for i, (want, got) in enumerate(zip(wants, gots)):
+        assert got.tokens.tolist() == want.tokens.tolist(), i
+        assert got.source.tolist() == want.source.tolist(), i
+        assert got.handoffs == want.handoffs, i
+        assert got.emission_fed.tolist() == want.emission_fed.tolist(), i
+        assert got.emission_source.tolist() == want.emission_source.tolist(), i
+        assert (got.kv_len_small, got.kv_len_large) == (want.kv_len_small, want.kv_len_large), i
+    assert small.st_last_device_status() == 0 and large.st_last_device_status() == 0
+    small.close()
+    large.close()

@@ -47,6 +47,20 @@ def test_static_argmax_matches_decode_step_twice():
     B.st_argmax_static(flat, 4096, got, stream)
     torch.cuda.synchronize()
     assert int(got.item()) == 77
+    # sizes that leave some of the 64 CTAs without an element, and sizes that are not a multiple of a CTA's 256 threads
+    rng = np.random.default_rng(2)
+    for n in (1, 255, 64 * 256 - 1, 64 * 256 + 3, 100_003):
+        v = torch.from_numpy(rng.standard_normal(n).astype(np.float32)).cuda()
+        B.st_argmax_static(v, n, got, stream)
+        torch.cuda.synchronize()
+        assert int(got.item()) == int(np.argmax(v.cpu().numpy())), n
+    # the property the entry point exists for: a call allocates no device memory and launches exactly one kernel
+    torch.cuda.synchronize()
+    free_before, launches_before = torch.cuda.mem_get_info()[0], B.st_kernel_launches()
+    B.st_argmax_static(flat, 4096, got, stream)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
+    assert B.st_kernel_launches() == launches_before + 1
     # sizes beyond the built-in scratch limit are refused
     with pytest.raises(B.StError) as e:
         B.st_argmax_static(flat, (1 << 22) + 1, got, stream)
