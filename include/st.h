@@ -110,6 +110,14 @@ typedef struct {
      * any of these ids (host array, ids below vocab_limit) counts as the delimiter wherever the rule tests for it. */
     const int32_t *delimiter_ids;
     int32_t n_delimiters;
+    /* Sampling.  The paper reports pass@1 and names no sampler; greedy (temperature 0) is the default.  temperature > 0:
+     * every token is drawn from softmax(logits / temperature) over ids < vocab_limit by the Gumbel-max rule: the id
+     * maximising logit / temperature + g wins, g = -ln(-ln u) a standard Gumbel variate from a counter-based generator
+     * (SplitMix64 stream `sample_seed`, output number step * 2^32 + id + 1, u = (top 23 bits + 0.5) * 2^-23), lowest id
+     * on ties.  emission_argmax then holds the drawn token.  Not available in st_generate_spec_batch's rounds (the
+     * sequences then run one by one). */
+    float temperature;
+    uint64_t sample_seed;
 } st_spec_params;
 
 typedef struct {

@@ -46,6 +46,7 @@ class _SpecParams(C.Structure):
         ("n2", C.c_int32), ("neg_threshold", C.c_int32), ("n3", C.c_int32),
         ("aux_ids", C.POINTER(C.c_int32)), ("n_aux", C.c_int32), ("probe_len", C.c_int32),
         ("delimiter_ids", C.POINTER(C.c_int32)), ("n_delimiters", C.c_int32),
+        ("temperature", C.c_double), ("sample_seed", C.c_uint64),
     ]
 
 
@@ -131,6 +132,10 @@ def lib():
         L.orc_forward_full.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
         L.orc_argmax.restype = C.c_int32
         L.orc_argmax.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_double)]
+        L.orc_sample.restype = C.c_int32
+        L.orc_sample.argtypes = [C.c_void_p, C.c_int32, C.c_double, C.c_uint64, C.c_uint32, C.POINTER(C.c_double)]
+        L.orc_gumbel.restype = C.c_double
+        L.orc_gumbel.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32]
         L.orc_generate_specdec.restype = C.c_int
         L.orc_generate_specdec.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(_SpecDecParams), C.c_void_p, C.c_int32,
                                            C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.POINTER(_SpecDecResult)]
@@ -194,6 +199,18 @@ def argmax(z, limit=None):
     m = C.c_double()
     i = lib().orc_argmax(_p(z), z.size if limit is None else limit, C.byref(m))
     return int(i), float(m.value)
+
+
+def sample(z, temperature: float, seed: int, step: int, limit=None):
+    """(token, margin of the perturbed values) of the Gumbel-max sampler."""
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    m = C.c_double()
+    i = lib().orc_sample(_p(z), z.size if limit is None else limit, temperature, seed, step, C.byref(m))
+    return int(i), float(m.value)
+
+
+def gumbel(seed: int, step: int, i: int) -> float:
+    return float(lib().orc_gumbel(seed, step, i))
 
 
 class Model:
@@ -298,7 +315,7 @@ def generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id: in
                   force=None, trace_first_step: int = 0, trace_n_steps: int = 0,
                   takeover_every_delimiter: bool = False, target_first_n: int = 0, affirmation_ids=(),
                   verification_ids=(), n2: int = 125, neg_threshold: int = -1, n3: int = 125, aux_ids=(),
-                  probe_len: int = 1, delimiter_ids=()) -> SpecResult:
+                  probe_len: int = 1, delimiter_ids=(), temperature: float = 0.0, sample_seed: int = 0) -> SpecResult:
     prompt = np.ascontiguousarray(prompt, dtype=np.int32)
     aff = np.ascontiguousarray(affirmation_ids, dtype=np.int32)
     ver = np.ascontiguousarray(verification_ids, dtype=np.int32)
@@ -311,7 +328,7 @@ def generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id: in
     P = _SpecParams(delimiter_id, kw.ctypes.data_as(C.POINTER(C.c_int32)), kw.size, n1, int(keep_probe), eos_id,
                     vocab_limit, max_new_tokens, int(takeover_every_delimiter), int(target_first_n),
                     ip(aff), aff.size, ip(ver), ver.size, n2, neg_threshold, n3, ip(aux), aux.size, probe_len,
-                    ip(dl), dl.size)
+                    ip(dl), dl.size, float(temperature), int(sample_seed))
     cap_steps = (1 + max(1, probe_len)) * max_new_tokens + 8   # replaced probe sentences are steps without tokens
     tokens = np.zeros(max_new_tokens + 1, dtype=np.int32)
     source = np.zeros(max_new_tokens + 1, dtype=np.uint8)

@@ -488,6 +488,33 @@ int32_t orc_argmax(const double *z, int32_t limit, double *margin)
     return best;
 }
 
+/* Temperature sampling by the Gumbel-max rule (Gumbel 1954; Maddison, Tarlow, Minka 2014): with independent
+ * standard Gumbel variates g_i, argmax_i (z_i / T + g_i) is distributed as softmax(z / T).  The variates come from a
+ * counter-based generator so that any implementation can reproduce them: u is built from the top 23 bits k of the
+ * SplitMix64 output number (step * 2^32 + i + 1) of the stream with initial state `seed`, u = (k + 0.5) * 2^-23 (so
+ * 0 < u < 1, exactly representable in single and double precision), and g = -ln(-ln u).  Lowest id on ties; *margin
+ * (optional) is the gap between the two largest perturbed values.  temperature <= 0 is plain greedy. */
+double orc_gumbel(uint64_t seed, uint32_t step, uint32_t i)
+{
+    uint64_t x = orc_sm64_nth(seed, (((uint64_t)step << 32) | (uint64_t)i) + 1);
+    double u = ((double)(x >> 41) + 0.5) * (1.0 / 8388608.0);
+    return -log(-log(u));
+}
+
+int32_t orc_sample(const double *z, int32_t limit, double temperature, uint64_t seed, uint32_t step, double *margin)
+{
+    if (!(temperature > 0.0)) return orc_argmax(z, limit, margin);
+    int32_t best = 0;
+    double vbest = z[0] / temperature + orc_gumbel(seed, step, 0), second = -INFINITY;
+    for (int32_t i = 1; i < limit; ++i) {
+        double v = z[i] / temperature + orc_gumbel(seed, step, (uint32_t)i);
+        if (v > vbest) { second = vbest; vbest = v; best = i; }
+        else if (v > second) second = v;
+    }
+    if (margin) *margin = vbest - second;
+    return best;
+}
+
 /* ------------------------------------------------------------------------- */
 /* Speculative Thinking generation (Section 3, takeover (1))                  */
 /* ------------------------------------------------------------------------- */
@@ -524,6 +551,10 @@ typedef struct {
      * paragraph).  n_delimiters == 0: delimiter_id alone; otherwise delimiter_id is ignored. */
     const int32_t *delimiter_ids;
     int32_t n_delimiters;
+    /* Sampling (the paper reports pass@1 and names no sampler; greedy is the default here): temperature > 0 draws
+     * every token by orc_sample with this seed and the emission step as the counter. */
+    double temperature;
+    uint64_t sample_seed;
 } orc_spec_params;
 
 /* Does this token close a paragraph? */
@@ -588,7 +619,7 @@ int orc_generate_spec(const orc_model *small, const orc_model *large, const orc_
         int32_t fed = pos - (int32_t)kv[a]->len;
         if (orc_forward(M[a], kv[a], tokens + kv[a]->len, fed, 0, z) != 0) { rc = -2; break; }
         double margin;
-        int32_t greedy = orc_argmax(z, P->vocab_limit, &margin);
+        int32_t greedy = orc_sample(z, P->vocab_limit, P->temperature, P->sample_seed, (uint32_t)t, &margin);
         int32_t tok = (force && t < n_force && force[t] >= 0) ? force[t] : greedy;
         if (t >= R->cap_steps) { rc = -3; break; }
         R->emission_tokens[t] = tok;

@@ -1097,10 +1097,11 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
         }
         float v = -INFINITY;
         int idx = 0x7fffffff;
+        const SampleRule rule = sample_rule(p.gen);   // the step counter changes only after every CTA has taken its ticket
         for (int i = blockIdx.x * kMegaCT + ctid; i < p.limit; i += gridDim.x * kMegaCT) {
             const float z = __ldcg(p.logits + i);
             if (trace) trace[i] = z;
-            argmax_merge(v, idx, z, i);
+            argmax_merge(v, idx, rule(z, i), i);
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {

@@ -7,6 +7,7 @@
 // kind and size of the next pass; it never sees a token before deciding what to launch.
 #pragma once
 #include "st_common.cuh"
+#include "weights.cuh"
 
 namespace st {
 
@@ -50,8 +51,37 @@ struct GenState {
     unsigned long long t_pending;    // time of the ingest-only chunks of the catch-up in progress
     unsigned long long t_kind[3];    // nanoseconds
     int32_t n_kind[3];
-    int32_t pad_;
+    // --- sampling: inv_temp > 0 draws tokens by the Gumbel-max rule with this seed (0: greedy) ---
+    float inv_temp;
+    unsigned long long sample_seed;
 };
+
+// Standard Gumbel variate number (step, i) of the stream `seed`: u = (k + 0.5) * 2^-23 with k the top 23 bits of
+// SplitMix64 output number (step * 2^32 + i + 1), g = -ln(-ln u).  argmax_i (z_i / T + g_i) is a draw from
+// softmax(z / T) (Gumbel-max rule), so sampling stays an argmax and keeps its lowest-id tie rule.
+__device__ __forceinline__ float gumbel_noise(unsigned long long seed, uint32_t step, uint32_t i)
+{
+    const uint64_t x = splitmix_out(seed + ((((uint64_t)step << 32) | (uint64_t)i) + 1) * kGamma);
+    const float u = ((float)(uint32_t)(x >> 41) + 0.5f) * 1.1920928955078125e-07f;   // * 2^-23, exact
+    return -logf(-logf(u));
+}
+
+// The value a logit competes with: the logit itself (greedy) or logit / T + Gumbel noise.
+struct SampleRule {
+    float inv_temp;
+    unsigned long long seed;
+    uint32_t step;
+    __device__ __forceinline__ float operator()(float z, int i) const
+    {
+        return inv_temp > 0.f ? fmaf(z, inv_temp, gumbel_noise(seed, step, (uint32_t)i)) : z;
+    }
+};
+__device__ __forceinline__ SampleRule sample_rule(const GenState *g)
+{
+    SampleRule r{0.f, 0ull, 0u};
+    if (g && g->inv_temp > 0.f) { r.inv_temp = g->inv_temp; r.seed = g->sample_seed; r.step = (uint32_t)g->step; }
+    return r;
+}
 
 __device__ __forceinline__ unsigned long long global_timer_ns()
 {
@@ -506,10 +536,11 @@ __global__ void __launch_bounds__(256) argmax_router_kernel(const ArgmaxParams p
     }
     float v = -INFINITY;
     int idx = 0x7fffffff;
+    const SampleRule rule = sample_rule(p.gen);
     for (int i = blockIdx.x * 256 + tid; i < p.limit; i += gridDim.x * 256) {
         const float z = p.logits[i];
         if (trace) trace[i] = z;
-        argmax_merge(v, idx, z, i);
+        argmax_merge(v, idx, rule(z, i), i);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {

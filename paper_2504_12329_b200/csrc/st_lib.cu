@@ -1777,6 +1777,7 @@ static int check_rule_params(const st_spec_params *P, int vlimit)
         return ST_ERR_ARG;
     if ((P->n_verification > 0 && P->n2 < 1) || (P->neg_threshold >= 0 && P->n3 < 1)) return ST_ERR_ARG;
     if (P->n_delimiters < 0 || (P->n_delimiters > 0 && !P->delimiter_ids)) return ST_ERR_ARG;
+    if (!(P->temperature >= 0.f)) return ST_ERR_ARG;
     for (int i = 0; i < P->n_delimiters; ++i)
         if ((unsigned)P->delimiter_ids[i] >= (unsigned)vlimit) return ST_ERR_VOCAB;
     if (P->n_delimiters == 0 && (unsigned)P->delimiter_id >= (unsigned)vlimit) return ST_ERR_VOCAB;
@@ -1876,6 +1877,10 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     g0.neg_threshold = P->neg_threshold;
     g0.n_aux = P->n_aux;
     g0.probe_len = P->probe_len > 1 ? P->probe_len : 1;
+    if (P->temperature > 0.f) {
+        g0.inv_temp = 1.f / P->temperature;
+        g0.sample_seed = P->sample_seed;
+    }
     if (large && P->target_first_n > 0) {   // the target opens the answer
         g0.active = 1;
         g0.remaining = P->target_first_n;
@@ -2024,6 +2029,7 @@ static int generate_spec_batch_rounds(st_model *small, st_model *large, const st
     *handled = false;
     static const bool sequential = [] { const char *e = getenv("ST_BATCH_SEQUENTIAL"); return e && e[0] == '1'; }();
     if (sequential || n < 2 || n > small->max_rows || (large && n > large->max_rows)) return ST_OK;
+    if (P->temperature > 0.f) return ST_OK;   // the ragged passes' per-row argmax is greedy: sampled runs go one by one
     if (P->max_new_tokens < 0 || P->n1 < 1 || P->n_keywords < 0 || (P->n_keywords > 0 && !P->keyword_ids)) return ST_ERR_ARG;
     if (large && (large->stream != small->stream || large->device != small->device)) return ST_ERR_ARG;
     int vshared = small->cfg.vocab;

@@ -533,3 +533,39 @@ def test_phase_times_and_pass_counts(B):
     assert abs(total - r.seconds) <= 0.1 * r.seconds + 2e-4, (total, r.seconds)
     gs.close()
     gl.close()
+
+
+@pytest.mark.parametrize("temperature", [0.7, 1.5])
+def test_temperature_sampling_on_device(B, oracle, temperature):
+    """Tokens drawn by the Gumbel-max rule (temperature sampling with a counter-based generator): under teacher
+    forcing with the oracle's stream, the token the device draws at every step equals the oracle's wherever the
+    oracle's decision is clear (gap of the two largest perturbed logits at least the tolerance, scaled by 1 / T);
+    handoffs triggered by drawn tokens follow; the same seed reproduces the run and another seed changes it."""
+    S, L = shape_dict(W.TINY_S), shape_dict(W.TINY_L)
+    os_, ol = oracle.Model(oracle.Config(**S), 0, 0), oracle.Model(oracle.Config(**L), 0, 1)
+    gs = B.Model(S, seed=0, tag=0, max_tokens=512)
+    gl = B.Model(L, seed=0, tag=1, max_tokens=512)
+    prompt = W.prompt_ids(100, 32, 1024)
+    sched = W.forcing_schedule(101, 400, mean_interval=8, keyword_rate=0.5)   # delimiters and keywords forced, the rest drawn
+    kw = dict(delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=4, max_new_tokens=120, temperature=temperature, sample_seed=77)
+    want = oracle.generate_spec(os_, ol, prompt, force=sched, **kw)
+    assert len(want.handoffs) >= 3
+    forced = B.st_generate_spec(gs, gl, prompt, force=want.emission_tokens, **kw)
+    _assert_routing_equal(want, forced)
+    clear = want.emission_margin >= MARGIN * max(1.0, 1.0 / temperature)
+    assert clear.sum() >= 60
+    assert forced.emission_argmax[clear].tolist() == want.emission_argmax[clear].tolist()
+    # drawn tokens differ from the greedy ones
+    greedy = oracle.generate_spec(os_, ol, prompt, force=sched, **dict(kw, temperature=0.0))
+    assert want.tokens.tolist() != greedy.tokens.tolist()
+    # free-running: identical up to the first unclear decision; reproducible; seed-dependent
+    free = B.st_generate_spec(gs, gl, prompt, force=sched, **kw)
+    again = B.st_generate_spec(gs, gl, prompt, force=sched, **kw)
+    other = B.st_generate_spec(gs, gl, prompt, force=sched, **dict(kw, sample_seed=78))
+    assert free.tokens.tolist() == again.tokens.tolist() != other.tokens.tolist()
+    for t in range(min(len(free.emission_tokens), len(want.emission_tokens))):
+        if free.emission_tokens[t] != want.emission_tokens[t]:
+            assert not clear[t], f"step {t}: drawn tokens differ at a clear margin"
+            break
+    gs.close()
+    gl.close()

@@ -22,7 +22,7 @@ CASES = [
     ("ST_SIMT_ATTN", "1", SINGLE),
     ("ST_PDL", "0", SINGLE + " or " + BATCH),
     ("ST_AB_TILE", "128", BATCH),
-    ("ST_BATCH_SEQUENTIAL", "1", "test_batched_generation_in_rounds"),
+    ("ST_BATCH_SEQUENTIAL", "1", "test_three_takeovers_on_device or test_every_delimiter_variant_on_device"),
     ("ST_BATCH_GRAPH", "0", BATCH),
     ("ST_BATCH_OVERLAP", "0", "test_batched_generation_in_rounds"),
     ("ST_MEGA_STAGES", "2", SINGLE),
