@@ -90,6 +90,7 @@ struct st_model {
     std::vector<BatchGraph> batch_graphs;
     cudaStream_t cap_stream = nullptr;     // side stream the batched pass is captured on (the model's own may be the legacy stream)
     CUtensorMap *act_maps = nullptr;       // device [3 buffers][2 planes][8]: activation planes in boxes of 32 (j + 1) rows
+    CUtensorMap *act_maps_half = nullptr;  // device [3 buffers][2 planes][16]: the same in boxes of 16 (j + 1) rows (CTA pairs)
     bool simt_gemm = false;                // debugging aid: multi-row projections on the CUDA cores
     bool simt_attn = false;                // debugging aid: multi-row attention on the CUDA cores
     double *inv_freq = nullptr;
@@ -450,14 +451,24 @@ static cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 bloc
     return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 
+// Passes of at least this many rows run on CTA pairs (0: never): below it the activation tiles are small beside the
+// weight tiles and a pair gains nothing.
+static int tc_pair_min_rows()
+{
+    static const int v = [] { const char *e = getenv("ST_TC_PAIR_MIN"); return e ? atoi(e) : 96; }();
+    return v;
+}
+
 template <int EPI>
 // pending_splits: when given, a K-split projection leaves its partial sums in the workspace and reports the split
 // count there (0: the output is complete) -- the kernel that consumes the output adds them up.
 static int launch_tc_gemm(const CUtensorMap &tw, TcGemmParams p, int m_upper, int sms, cudaStream_t s, int *pending_splits = nullptr)
 {
-    auto kern = tc_gemm_kernel<EPI>;
     p.m_pad = (m_upper + 31) / 32 * 32;
     if (p.m_pad > 256) return ST_ERR_INTERNAL;
+    const bool pair = tc_pair_min_rows() > 0 && p.m_pad >= tc_pair_min_rows();
+    auto kern = pair ? tc_gemm_pair_kernel<EPI> : tc_gemm_kernel<EPI>;
+    const int a_rows = pair ? p.m_pad / 2 : p.m_pad;   // activation rows a CTA loads per plane and stage
     // 128-row weight tiles per CTA (they share the activation tiles of a stage): bounded by TMEM (512 columns) and
     // by two pipeline stages of shared memory; among the candidates take the one whose CTA count fills whole waves
     // of SMs best (a projection with 1.46 waves of CTAs runs as long as one with 2), the larger on a tie.
@@ -466,7 +477,7 @@ static int launch_tc_gemm(const CUtensorMap &tw, TcGemmParams p, int m_upper, in
         double best = -1.0;
         for (int cand = 4; cand >= 1; --cand) {
             if (cand * p.m_pad > 512) continue;
-            if (2 * (cand * kTcWBytes + 2 * p.m_pad * kTcBlockK * 2) > 220 * 1024) continue;
+            if (2 * (cand * kTcWBytes + 2 * a_rows * kTcBlockK * 2) > 220 * 1024) continue;
             const int tiles = (p.N + kTcTileW * cand - 1) / (kTcTileW * cand);
             // projections that may split K fill the machine through the split; the others only through tiles
             int split = tiles >= sms ? 1 : sms / tiles;   // K splits: as many as still fit one wave
@@ -479,15 +490,16 @@ static int launch_tc_gemm(const CUtensorMap &tw, TcGemmParams p, int m_upper, in
     }
     {   // tuning aid: force the weight tiles per CTA (when the forced count fits tensor and shared memory)
         static const int forced = [] { const char *e = getenv("ST_TC_WT"); return e ? atoi(e) : 0; }();
-        if (forced >= 1 && forced <= 4 && forced * p.m_pad <= 512 && 2 * (forced * kTcWBytes + 2 * p.m_pad * kTcBlockK * 2) <= 220 * 1024) wt = forced;
+        if (forced >= 1 && forced <= 4 && forced * p.m_pad <= 512 && 2 * (forced * kTcWBytes + 2 * a_rows * kTcBlockK * 2) <= 220 * 1024) wt = forced;
     }
     p.w_tiles = wt;
     int cols = wt * p.m_pad;
     p.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
-    const int stage_bytes = wt * kTcWBytes + 2 * p.m_pad * kTcBlockK * 2;
+    const int stage_bytes = wt * kTcWBytes + 2 * a_rows * kTcBlockK * 2;
     int stages = (220 * 1024) / stage_bytes;
     p.stages = stages > 8 ? 8 : stages;
-    const int n_tiles = (p.N + kTcTileW * wt - 1) / (kTcTileW * wt);
+    int n_tiles = (p.N + kTcTileW * wt - 1) / (kTcTileW * wt);
+    if (pair) n_tiles = (n_tiles + 1) & ~1;   // whole pairs: a CTA beyond the matrix multiplies zero-filled tiles and stores nothing
     const int kb_total = (p.K + kTcBlockK - 1) / kTcBlockK;
     int ks = 1;
     if (EPI != TEPI_SILU) {
@@ -571,6 +583,9 @@ static int init_kernel_attributes()
     CK(cudaFuncSetAttribute(tc_gemm_kernel<TEPI_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
     CK(cudaFuncSetAttribute(tc_gemm_kernel<TEPI_RESADD>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
     CK(cudaFuncSetAttribute(tc_gemm_kernel<TEPI_SILU>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+    CK(cudaFuncSetAttribute(tc_gemm_pair_kernel<TEPI_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+    CK(cudaFuncSetAttribute(tc_gemm_pair_kernel<TEPI_RESADD>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+    CK(cudaFuncSetAttribute(tc_gemm_pair_kernel<TEPI_SILU>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
     return mega_attr_all();
 }
 
@@ -719,6 +734,15 @@ static int model_build(st_model *m)
                                       (uint64_t)m->max_rows, (uint64_t)widths[b], (uint32_t)(32 * (j + 1))));
         ALLOC(m->act_maps, CUtensorMap, maps.size());
         CK(cudaMemcpyAsync(m->act_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, m->stream));
+        CK(cudaStreamSynchronize(m->stream));
+        std::vector<CUtensorMap> halves(3 * 2 * 16);
+        for (int b = 0; b < 3; ++b)
+            for (int plane = 0; plane < 2; ++plane)
+                for (int j = 0; j < 16; ++j)
+                    TRY(make_map_bf16(&halves[(b * 2 + plane) * 16 + j], bufs[b] + (size_t)plane * m->max_rows * widths[b],
+                                      (uint64_t)m->max_rows, (uint64_t)widths[b], (uint32_t)(16 * (j + 1))));
+        ALLOC(m->act_maps_half, CUtensorMap, halves.size());
+        CK(cudaMemcpyAsync(m->act_maps_half, halves.data(), halves.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, m->stream));
         CK(cudaStreamSynchronize(m->stream));
     }
     ALLOC(m->cs, float2, (size_t)m->max_rows * (D / 2));
@@ -1048,6 +1072,8 @@ static int rows_gemm(st_model *m, const StepDesc *desc, int m_upper, int buffer,
     TcGemmParams p{};
     p.act_hi = m->act_maps + (buffer * 2 + 0) * 8;
     p.act_lo = m->act_maps + (buffer * 2 + 1) * 8;
+    p.act_hi_half = m->act_maps_half + (buffer * 2 + 0) * 16;
+    p.act_lo_half = m->act_maps_half + (buffer * 2 + 1) * 16;
     p.desc = desc; p.bias = bias; p.Yf = Yf; p.Yb_hi = Yb_hi; p.Yb_lo = Yb_lo; p.status = m->status; p.N = N; p.K = K;
     p.Ws = m->splitk_ws; p.ws_rows = m->max_rows;
     return launch_tc_gemm<EPI>(tw, p, m_upper, m->sm_count, m->stream, pending_splits);
