@@ -285,13 +285,17 @@ __device__ __forceinline__ void mega_load_x(MegaShared &sh, float4 *xa, float4 *
 {
     const int K8 = K >> 3;
     float ss = 0.f;
-    constexpr int XU = 4;   // loads in flight per thread
+    constexpr int XU = 4;   // items in flight per thread
+    // The gain is fetched together with x (one trip to L2 instead of two): shared memory first takes x * gain, the
+    // second pass only scales by 1 / rms.
+    const float4 *g4 = reinterpret_cast<const float4 *>(gain);
     for (int q0 = ctid; q0 < 2 * K8; q0 += XU * kMegaCT) {
-        float4 v[XU], a[XU];
+        float4 v[XU], a[XU], g[XU];
 #pragma unroll
         for (int u = 0; u < XU; ++u) {
             const int q = q0 + u * kMegaCT;
             v[u] = a[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            g[u] = make_float4(1.f, 1.f, 1.f, 1.f);
             if (q < 2 * K8) {
                 if (src_embed) {
                     const uint2 e = reinterpret_cast<const uint2 *>(src_embed)[q];
@@ -300,6 +304,7 @@ __device__ __forceinline__ void mega_load_x(MegaShared &sh, float4 *xa, float4 *
                     v[u] = __ldcg(reinterpret_cast<const float4 *>(x) + q);
                 }
                 if (add) a[u] = __ldcg(reinterpret_cast<const float4 *>(add) + q);
+                if (norm) g[u] = g4[q];
             }
         }
 #pragma unroll
@@ -310,7 +315,7 @@ __device__ __forceinline__ void mega_load_x(MegaShared &sh, float4 *xa, float4 *
                 t.x += a[u].x; t.y += a[u].y; t.z += a[u].z; t.w += a[u].w;
                 if (x_out && blockIdx.x == 0) reinterpret_cast<float4 *>(x_out)[q] = t;
                 ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
-                ((q & 1) ? xb : xa)[q >> 1] = t;
+                ((q & 1) ? xb : xa)[q >> 1] = make_float4(t.x * g[u].x, t.y * g[u].y, t.z * g[u].z, t.w * g[u].w);
             }
         }
     }
@@ -322,12 +327,10 @@ __device__ __forceinline__ void mega_load_x(MegaShared &sh, float4 *xa, float4 *
 #pragma unroll
         for (int w = 0; w < kMegaConsumers; ++w) tot += sh.red[w];
         const float inv = rsqrtf(tot / (float)K + eps);
-        const float4 *g4 = reinterpret_cast<const float4 *>(gain);
-        for (int q = ctid; q < 2 * K8; q += kMegaCT) {
+        for (int q = ctid; q < 2 * K8; q += kMegaCT) {   // each thread rescales what it wrote itself
             float4 *dst = ((q & 1) ? xb : xa) + (q >> 1);
             float4 v = *dst;
-            const float4 g = g4[q];
-            v.x *= inv * g.x; v.y *= inv * g.y; v.z *= inv * g.z; v.w *= inv * g.w;
+            v.x *= inv; v.y *= inv; v.z *= inv; v.w *= inv;
             *dst = v;
         }
     }
@@ -771,17 +774,24 @@ __device__ __forceinline__ void mega_attention_unit(const MegaParams &p, MegaSha
     const int hq0 = u.hk * G;
     for (int idx = gt; idx < G * D; idx += kMegaCT) {
         const int g = idx / D, c = idx - g * D;
+        // every load first (they do not depend on one another), then the arithmetic
+        float mw[kMegaAttnWarps], dw[kMegaAttnWarps], ow[kMegaAttnWarps];
+#pragma unroll
+        for (int w = 0; w < kMegaAttnWarps; ++w) {
+            mw[w] = sc.m[w][g];
+            dw[w] = sc.d[w][g];
+            ow[w] = sc.o[w][g][c];
+        }
         float mnew = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < kMegaAttnWarps; ++w) mnew = fmaxf(mnew, sc.m[w][g]);
+        for (int w = 0; w < kMegaAttnWarps; ++w) mnew = fmaxf(mnew, mw[w]);
         float dsum = 0.f, osum = 0.f;
 #pragma unroll
         for (int w = 0; w < kMegaAttnWarps; ++w) {
-            if (sc.m[w][g] != -INFINITY) {   // a warp without keys left its slots untouched
-                const float cw2 = __expf(sc.m[w][g] - mnew);
-                dsum += sc.d[w][g] * cw2;
-                osum += sc.o[w][g][c] * cw2;
-            }
+            const bool live = mw[w] != -INFINITY;   // a warp without keys left its sum and output slots untouched
+            const float cw2 = live ? __expf(mw[w] - mnew) : 0.f;
+            dsum += live ? dw[w] * cw2 : 0.f;
+            osum += live ? ow[w] * cw2 : 0.f;
         }
         const size_t pi = (size_t)(hq0 + g) * u.ns + u.split;
         p.part_o[pi * D + c] = osum;
