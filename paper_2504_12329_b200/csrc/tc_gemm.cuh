@@ -195,7 +195,7 @@ __global__ void splitk_reduce_kernel(const StepDesc *desc, const float *Ws, int 
 //   * tensor memory is allocated and freed by the same warp of both CTAs (the pair form of the instructions);
 //   * the pair synchronises once, after its barriers are initialised and before any load is issued; every wait is
 //     bounded as in the single-CTA kernel, and every path reaches the common exit.
-// Loads name no other CTA's shared memory as destination and use no multicast.
+// Every load writes only the issuing CTA's own shared memory (one copy per load).
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {
