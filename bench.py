@@ -335,10 +335,20 @@ def timed_prompt_prefill(torch, model, shape, rows, peak):
             "timing": "host clock around st_prefill + synchronize (the call syncs between passes)"}
 
 
+def pass_kind_times(r):
+    """Device time per kind of pass (stamped by the router on the device): the run's own version of the paper's table
+    of decode against prefix times."""
+    out = {}
+    for kind, (sec, n) in (r.phase_times or {}).items():
+        out[kind] = {"passes": int(n), "seconds": float(sec), "ms_per_pass": 1e3 * float(sec) / n if n else None}
+    return out
+
+
 def generation_summary(r, peak):
     """Figures of one timed generation (device time from the call's own CUDA events)."""
     gbs = r.bytes_algorithmic / r.seconds / 1e9
-    return {"tokens": int(len(r.tokens)), "seconds": r.seconds, "tokens_per_s": len(r.tokens) / r.seconds, "handoffs": len(r.handoffs),
+    phases = pass_kind_times(r)
+    return {"pass_kinds": phases, "tokens": int(len(r.tokens)), "seconds": r.seconds, "tokens_per_s": len(r.tokens) / r.seconds, "handoffs": len(r.handoffs),
             "passes": int(r.n_steps), "target_share": float(r.source.mean()) if len(r.source) else 0.0,
             "achieved_gbs": gbs, "frac_of_measured_hbm": gbs / peak}
 
@@ -556,6 +566,7 @@ def main():
                          "algorithmic_bytes_per_step": int(path_bytes / len(results)),
                          "frac_of_nominal_8tbs": path_gbs / 8000.0, "peak_source": f"{peak_kind} copy bandwidth",
                          "note": "algorithmic bytes of every pass (weights + KV) / device time; per-kernel figures under dominant_kernel, decode_small, prefill, batched_decode"},
+            "pass_kinds": pass_kind_times(r),
             "dominant_kernel": dominant,
             "decode_small": small_step,
             "prefill": prefill,
