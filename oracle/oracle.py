@@ -46,7 +46,7 @@ class _SpecParams(C.Structure):
         ("n2", C.c_int32), ("neg_threshold", C.c_int32), ("n3", C.c_int32),
         ("aux_ids", C.POINTER(C.c_int32)), ("n_aux", C.c_int32), ("probe_len", C.c_int32),
         ("delimiter_ids", C.POINTER(C.c_int32)), ("n_delimiters", C.c_int32),
-        ("temperature", C.c_double), ("sample_seed", C.c_uint64),
+        ("temperature", C.c_double), ("sample_seed", C.c_uint64), ("top_p", C.c_double),
     ]
 
 
@@ -134,6 +134,11 @@ def lib():
         L.orc_argmax.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_double)]
         L.orc_sample.restype = C.c_int32
         L.orc_sample.argtypes = [C.c_void_p, C.c_int32, C.c_double, C.c_uint64, C.c_uint32, C.POINTER(C.c_double)]
+        L.orc_nucleus_threshold.restype = C.c_double
+        L.orc_nucleus_threshold.argtypes = [C.c_void_p, C.c_int32, C.c_double, C.c_double, C.POINTER(C.c_double)]
+        L.orc_sample_top_p.restype = C.c_int32
+        L.orc_sample_top_p.argtypes = [C.c_void_p, C.c_int32, C.c_double, C.c_double, C.c_uint64, C.c_uint32,
+                                       C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.orc_gumbel.restype = C.c_double
         L.orc_gumbel.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32]
         L.orc_generate_specdec.restype = C.c_int
@@ -207,6 +212,22 @@ def sample(z, temperature: float, seed: int, step: int, limit=None):
     m = C.c_double()
     i = lib().orc_sample(_p(z), z.size if limit is None else limit, temperature, seed, step, C.byref(m))
     return int(i), float(m.value)
+
+
+def nucleus_threshold(z, temperature: float, top_p: float, limit=None):
+    """(threshold logit, gap): the nucleus of softmax(z / T) is {i: z[i] >= threshold}."""
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    g = C.c_double()
+    t = lib().orc_nucleus_threshold(_p(z), z.size if limit is None else limit, temperature, top_p, C.byref(g))
+    return float(t), float(g.value)
+
+
+def sample_top_p(z, temperature: float, top_p: float, seed: int, step: int, limit=None):
+    """(token, margin of the perturbed values, gap of the nucleus cut) of the Gumbel-max sampler restricted to the nucleus."""
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    m, g = C.c_double(), C.c_double()
+    i = lib().orc_sample_top_p(_p(z), z.size if limit is None else limit, temperature, top_p, seed, step, C.byref(m), C.byref(g))
+    return int(i), float(m.value), float(g.value)
 
 
 def gumbel(seed: int, step: int, i: int) -> float:
@@ -315,7 +336,8 @@ def generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id: in
                   force=None, trace_first_step: int = 0, trace_n_steps: int = 0,
                   takeover_every_delimiter: bool = False, target_first_n: int = 0, affirmation_ids=(),
                   verification_ids=(), n2: int = 125, neg_threshold: int = -1, n3: int = 125, aux_ids=(),
-                  probe_len: int = 1, delimiter_ids=(), temperature: float = 0.0, sample_seed: int = 0) -> SpecResult:
+                  probe_len: int = 1, delimiter_ids=(), temperature: float = 0.0, sample_seed: int = 0,
+                  top_p: float = 0.0) -> SpecResult:
     prompt = np.ascontiguousarray(prompt, dtype=np.int32)
     aff = np.ascontiguousarray(affirmation_ids, dtype=np.int32)
     ver = np.ascontiguousarray(verification_ids, dtype=np.int32)
@@ -328,7 +350,7 @@ def generate_spec(small: Model, large: Model | None, prompt, *, delimiter_id: in
     P = _SpecParams(delimiter_id, kw.ctypes.data_as(C.POINTER(C.c_int32)), kw.size, n1, int(keep_probe), eos_id,
                     vocab_limit, max_new_tokens, int(takeover_every_delimiter), int(target_first_n),
                     ip(aff), aff.size, ip(ver), ver.size, n2, neg_threshold, n3, ip(aux), aux.size, probe_len,
-                    ip(dl), dl.size, float(temperature), int(sample_seed))
+                    ip(dl), dl.size, float(temperature), int(sample_seed), float(top_p))
     cap_steps = (1 + max(1, probe_len)) * max_new_tokens + 8   # replaced probe sentences are steps without tokens
     tokens = np.zeros(max_new_tokens + 1, dtype=np.int32)
     source = np.zeros(max_new_tokens + 1, dtype=np.uint8)

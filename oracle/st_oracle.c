@@ -515,6 +515,58 @@ int32_t orc_sample(const double *z, int32_t limit, double temperature, uint64_t 
     return best;
 }
 
+/* Nucleus (top-p) of softmax(z / T) (Holtzman et al. 2020): order the ids by probability, largest first; the nucleus
+ * is the shortest prefix whose probabilities sum to at least top_p, and -- so that the set does not depend on how
+ * equal probabilities are ordered -- every id that ties with the prefix's last member.  Returns the logit of that last
+ * member: the nucleus is { i : z[i] >= threshold }.  *gap (optional) is the distance between top_p and the nearest of
+ * the two cumulative sums around the cut (the sum that reaches top_p and the one before it): a cut with a small gap
+ * may fall differently in lower precision.  The paper names no sampler; this is the standard definition written out
+ * (selection sort over what is needed, sums in double precision). */
+double orc_nucleus_threshold(const double *z, int32_t limit, double temperature, double top_p, double *gap)
+{
+    double zmax = z[0], Z = 0.0;
+    for (int32_t i = 1; i < limit; ++i) if (z[i] > zmax) zmax = z[i];
+    for (int32_t i = 0; i < limit; ++i) Z += exp((z[i] - zmax) / temperature);
+    unsigned char *taken = (unsigned char *)calloc((size_t)limit, 1);
+    double cum = 0.0, thr = zmax, before = 0.0;
+    for (int32_t k = 0; k < limit; ++k) {
+        int32_t best = -1;
+        for (int32_t i = 0; i < limit; ++i)
+            if (!taken[i] && (best < 0 || z[i] > z[best])) best = i;   /* largest remaining, lowest id first */
+        taken[best] = 1;
+        before = cum;
+        cum += exp((z[best] - zmax) / temperature) / Z;
+        thr = z[best];
+        if (cum >= top_p) break;
+    }
+    free(taken);
+    if (gap) {
+        double a = fabs(cum - top_p), b = fabs(top_p - before);
+        *gap = a < b ? a : b;
+    }
+    return thr;
+}
+
+/* Top-p sampling: the Gumbel-max draw of orc_sample restricted to the nucleus (ids outside it cannot win), which is
+ * a draw from softmax(z / T) renormalised over the nucleus.  top_p <= 0 or >= 1: no restriction. */
+int32_t orc_sample_top_p(const double *z, int32_t limit, double temperature, double top_p, uint64_t seed, uint32_t step,
+                         double *margin, double *gap)
+{
+    if (gap) *gap = 1.0;
+    if (!(temperature > 0.0) || !(top_p > 0.0) || top_p >= 1.0) return orc_sample(z, limit, temperature, seed, step, margin);
+    const double thr = orc_nucleus_threshold(z, limit, temperature, top_p, gap);
+    int32_t best = -1;
+    double vbest = -INFINITY, second = -INFINITY;
+    for (int32_t i = 0; i < limit; ++i) {
+        if (z[i] < thr) continue;
+        double v = z[i] / temperature + orc_gumbel(seed, step, (uint32_t)i);
+        if (best < 0 || v > vbest) { second = vbest; vbest = v; best = i; }
+        else if (v > second) second = v;
+    }
+    if (margin) *margin = vbest - second;
+    return best;
+}
+
 /* ------------------------------------------------------------------------- */
 /* Speculative Thinking generation (Section 3, takeover (1))                  */
 /* ------------------------------------------------------------------------- */
@@ -555,6 +607,7 @@ typedef struct {
      * every token by orc_sample with this seed and the emission step as the counter. */
     double temperature;
     uint64_t sample_seed;
+    double top_p;        /* 0 < top_p < 1: every draw is restricted to the nucleus (orc_sample_top_p) */
 } orc_spec_params;
 
 /* Does this token close a paragraph? */
@@ -619,7 +672,7 @@ int orc_generate_spec(const orc_model *small, const orc_model *large, const orc_
         int32_t fed = pos - (int32_t)kv[a]->len;
         if (orc_forward(M[a], kv[a], tokens + kv[a]->len, fed, 0, z) != 0) { rc = -2; break; }
         double margin;
-        int32_t greedy = orc_sample(z, P->vocab_limit, P->temperature, P->sample_seed, (uint32_t)t, &margin);
+        int32_t greedy = orc_sample_top_p(z, P->vocab_limit, P->temperature, P->top_p, P->sample_seed, (uint32_t)t, &margin, NULL);
         int32_t tok = (force && t < n_force && force[t] >= 0) ? force[t] : greedy;
         if (t >= R->cap_steps) { rc = -3; break; }
         R->emission_tokens[t] = tok;

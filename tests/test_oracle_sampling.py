@@ -68,3 +68,72 @@ def test_generation_with_sampling(oracle):
     # temperature -> 0 is the greedy stream
     cold = oracle.generate_spec(ms, None, prompt, temperature=1e-5, sample_seed=5, **kw)
     assert cold.tokens.tolist() == greedy.tokens.tolist()
+
+
+def test_nucleus_closed_form_on_four_tokens(oracle):
+    """Top-p on a distribution small enough to do by hand.  With z = ln p the softmax at T = 1 is p itself:
+    p = (0.5, 0.25, 0.15, 0.1), cumulative 0.5, 0.75, 0.9, 1.0 in order of probability."""
+    p = np.array([0.15, 0.5, 0.1, 0.25])           # ids in no particular order
+    z = np.log(p)
+    members = lambda top_p, T=1.0: [i for i in range(4) if z[i] >= oracle.nucleus_threshold(z, T, top_p)[0]]
+    assert members(0.3) == [1]                      # the most probable id alone already holds 0.5 >= 0.3
+    assert members(0.5) == [1]                      # "at least top_p": 0.5 reaches 0.5
+    assert members(0.6) == [1, 3]                   # 0.5 < 0.6 <= 0.75
+    assert members(0.76) == [0, 1, 3]
+    assert members(0.95) == [0, 1, 2, 3]
+    # the reported gap is the distance of top_p to the nearer cumulative sum around the cut
+    assert abs(oracle.nucleus_threshold(z, 1.0, 0.6)[1] - 0.1) < 1e-12
+    assert abs(oracle.nucleus_threshold(z, 1.0, 0.74)[1] - 0.01) < 1e-12
+    # the temperature acts before the cut: at T = 0.5 the probabilities are p^2 / sum = (.0625, .25, .0225, .01) / .345
+    assert members(0.7, T=0.5) == [1]               # 0.7246 >= 0.7
+    assert members(0.8, T=0.5) == [1, 3]            # 0.7246 < 0.8 <= 0.9058
+    # ids that tie with the last member come along, whatever their order
+    zt = np.log(np.array([0.2, 0.4, 0.2, 0.2]))
+    assert [i for i in range(4) if zt[i] >= oracle.nucleus_threshold(zt, 1.0, 0.5)[0]] == [0, 1, 2, 3]
+    # only ids below the limit count
+    z5 = np.append(z, 10.0)
+    assert oracle.nucleus_threshold(z5, 1.0, 0.6, limit=4)[0] == oracle.nucleus_threshold(z, 1.0, 0.6)[0]
+
+
+def test_top_p_sampling_is_the_renormalised_distribution(oracle):
+    p = np.array([0.15, 0.5, 0.1, 0.25])
+    z = np.log(p)
+    # nucleus {1, 3} renormalised: (2/3, 1/3); nothing else is ever drawn
+    n = 30_000
+    draws = [oracle.sample_top_p(z, 1.0, 0.6, 77, step)[0] for step in range(n)]
+    counts = np.bincount(draws, minlength=4)
+    assert counts[0] == 0 and counts[2] == 0
+    want = n * np.array([2 / 3, 1 / 3])
+    chi2 = float(((counts[[1, 3]] - want) ** 2 / want).sum())
+    assert chi2 < 15.1, counts                       # 1 degree of freedom: p < 1e-4
+    # top_p outside (0, 1) is no restriction: the same draws as plain temperature sampling
+    for step in range(200):
+        assert oracle.sample_top_p(z, 1.0, 1.0, 9, step)[0] == oracle.sample(z, 1.0, 9, step)[0]
+        assert oracle.sample_top_p(z, 1.0, 0.0, 9, step)[0] == oracle.sample(z, 1.0, 9, step)[0]
+    # a nucleus of one id is greedy
+    rng = np.random.default_rng(1)
+    big = rng.standard_normal(3000)
+    for step in range(50):
+        assert oracle.sample_top_p(big, 1.0, 1e-6, 3, step)[0] == int(np.argmax(big))
+    # inside the nucleus the draw is the unrestricted Gumbel-max draw whenever that one falls inside
+    thr, _ = oracle.nucleus_threshold(big, 1.0, 0.9)
+    same = 0
+    for step in range(300):
+        free = oracle.sample(big, 1.0, 4, step)[0]
+        if big[free] >= thr:
+            assert oracle.sample_top_p(big, 1.0, 0.9, 4, step)[0] == free
+            same += 1
+    assert same > 200
+
+
+def test_generation_with_top_p(oracle):
+    cfg_s = oracle.Config(**W.TINY_S.as_dict())
+    ms = oracle.Model(cfg_s, 0, 0)
+    prompt = W.prompt_ids(3, 8, 1024)
+    kw = dict(delimiter_id=10, keyword_ids=[], n1=3, max_new_tokens=24, temperature=1.0, sample_seed=5)
+    free = oracle.generate_spec(ms, None, prompt, **kw)
+    cut = oracle.generate_spec(ms, None, prompt, top_p=0.5, **kw)
+    assert cut.tokens.tolist() != free.tokens.tolist()
+    z = oracle.KV(ms, 16).forward(prompt)
+    assert cut.tokens[0] == oracle.sample_top_p(z, 1.0, 0.5, 5, 0)[0]
+    assert oracle.generate_spec(ms, None, prompt, top_p=1.0, **kw).tokens.tolist() == free.tokens.tolist()
