@@ -118,6 +118,12 @@ typedef struct {
      * sequences then run one by one). */
     float temperature;
     uint64_t sample_seed;
+    /* Top-p (nucleus) sampling, with temperature > 0 only: 0 < top_p < 1 restricts every draw to the nucleus of
+     * softmax(logits / temperature) -- the shortest prefix of the ids ordered by probability whose probabilities sum to
+     * at least top_p, plus every id tying with its last member -- i.e. draws from the distribution renormalised over
+     * it.  0 (or >= 1): no restriction.  The cut is found on the device without a sort (three histogram passes over the
+     * logits' bit patterns, probability mass summed as 64-bit integers). */
+    float top_p;
 } st_spec_params;
 
 typedef struct {

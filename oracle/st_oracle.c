@@ -521,25 +521,30 @@ int32_t orc_sample(const double *z, int32_t limit, double temperature, uint64_t 
  * member: the nucleus is { i : z[i] >= threshold }.  *gap (optional) is the distance between top_p and the nearest of
  * the two cumulative sums around the cut (the sum that reaches top_p and the one before it): a cut with a small gap
  * may fall differently in lower precision.  The paper names no sampler; this is the standard definition written out
- * (selection sort over what is needed, sums in double precision). */
+ * (the ids sorted with the C library's qsort, sums in double precision). */
+typedef struct { double z; int32_t id; } orc_zid;
+static int orc_zid_desc(const void *a, const void *b)   /* larger logit first, lower id first among equals */
+{
+    const orc_zid *x = (const orc_zid *)a, *y = (const orc_zid *)b;
+    if (x->z != y->z) return x->z > y->z ? -1 : 1;
+    return x->id < y->id ? -1 : x->id > y->id;
+}
 double orc_nucleus_threshold(const double *z, int32_t limit, double temperature, double top_p, double *gap)
 {
     double zmax = z[0], Z = 0.0;
     for (int32_t i = 1; i < limit; ++i) if (z[i] > zmax) zmax = z[i];
     for (int32_t i = 0; i < limit; ++i) Z += exp((z[i] - zmax) / temperature);
-    unsigned char *taken = (unsigned char *)calloc((size_t)limit, 1);
+    orc_zid *order = (orc_zid *)malloc((size_t)limit * sizeof(orc_zid));
+    for (int32_t i = 0; i < limit; ++i) { order[i].z = z[i]; order[i].id = i; }
+    qsort(order, (size_t)limit, sizeof(orc_zid), orc_zid_desc);
     double cum = 0.0, thr = zmax, before = 0.0;
     for (int32_t k = 0; k < limit; ++k) {
-        int32_t best = -1;
-        for (int32_t i = 0; i < limit; ++i)
-            if (!taken[i] && (best < 0 || z[i] > z[best])) best = i;   /* largest remaining, lowest id first */
-        taken[best] = 1;
         before = cum;
-        cum += exp((z[best] - zmax) / temperature) / Z;
-        thr = z[best];
+        cum += exp((order[k].z - zmax) / temperature) / Z;
+        thr = order[k].z;
         if (cum >= top_p) break;
     }
-    free(taken);
+    free(order);
     if (gap) {
         double a = fabs(cum - top_p), b = fabs(top_p - before);
         *gap = a < b ? a : b;

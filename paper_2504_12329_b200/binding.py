@@ -43,7 +43,7 @@ class StSpecParams(C.Structure):
         ("n2", C.c_int32), ("neg_threshold", C.c_int32), ("n3", C.c_int32),
         ("aux_ids", C.POINTER(C.c_int32)), ("n_aux", C.c_int32), ("probe_len", C.c_int32),
         ("delimiter_ids", C.POINTER(C.c_int32)), ("n_delimiters", C.c_int32),
-        ("temperature", C.c_float), ("sample_seed", C.c_uint64),
+        ("temperature", C.c_float), ("sample_seed", C.c_uint64), ("top_p", C.c_float),
     ]
 
 
@@ -376,14 +376,14 @@ class _ResultBuffers:
 
 def _spec_params(delimiter_id, keyword_ids, n1, keep_probe, eos_id, vocab_limit, max_new_tokens, takeover_every_delimiter,
                  target_first_n, affirmation_ids=(), verification_ids=(), n2=125, neg_threshold=-1, n3=125, aux_ids=(),
-                 probe_len=1, delimiter_ids=(), temperature=0.0, sample_seed=0):
+                 probe_len=1, delimiter_ids=(), temperature=0.0, sample_seed=0, top_p=0.0):
     """st_spec_params and the arrays it points at (keep both alive during the call)."""
     arrs = [np.ascontiguousarray(a, dtype=np.int32) for a in (keyword_ids, affirmation_ids, verification_ids, aux_ids, delimiter_ids)]
     ip = lambda a: a.ctypes.data_as(C.POINTER(C.c_int32))
     kw, aff, ver, aux, dl = arrs
     P = StSpecParams(delimiter_id, ip(kw), kw.size, n1, int(keep_probe), eos_id, vocab_limit, max_new_tokens,
                      int(takeover_every_delimiter), int(target_first_n), ip(aff), aff.size, ip(ver), ver.size, n2,
-                     neg_threshold, n3, ip(aux), aux.size, probe_len, ip(dl), dl.size, float(temperature), int(sample_seed))
+                     neg_threshold, n3, ip(aux), aux.size, probe_len, ip(dl), dl.size, float(temperature), int(sample_seed), float(top_p))
     return P, arrs
 
 

@@ -1099,6 +1099,16 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
     MEGA_MARK();
 
     // ---- sampling + router ----
+    if (p.want_argmax && top_p_active(p.gen)) {   // the same decision in every CTA
+        // top-p: CTA 0 finds the nucleus' threshold (the ring is free by now), the others learn it after one more barrier
+        if (blockIdx.x == 0) {
+            unsigned long long *hist = reinterpret_cast<unsigned long long *>(base_ptr + p.xarea_bytes);
+            const float tau = nucleus_threshold_cta(p.logits, p.limit, p.gen->inv_temp, p.gen->top_p, hist, hist + kNucleusBins,
+                                                    hist + kNucleusBins + 256, ctid, [] { consumer_sync(); });
+            if (ctid == 0) p.gen->tau = tau;
+        }
+        mega_grid_barrier(p, sh, epoch, ctid);
+    }
     if (p.want_argmax) {
         float *trace = nullptr;
         if (p.gen && p.buf.trace && p.gen->trace_n > 0) {

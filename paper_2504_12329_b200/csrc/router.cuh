@@ -54,6 +54,8 @@ struct GenState {
     // --- sampling: inv_temp > 0 draws tokens by the Gumbel-max rule with this seed (0: greedy) ---
     float inv_temp;
     unsigned long long sample_seed;
+    // --- top-p: 0 < top_p < 1 restricts every draw to the nucleus; tau is the nucleus' lowest logit of the pass at hand ---
+    float top_p, tau;
 };
 
 // Standard Gumbel variate number (step, i) of the stream `seed`: u = (k + 0.5) * 2^-23 with k the top 23 bits of
@@ -66,21 +68,123 @@ __device__ __forceinline__ float gumbel_noise(unsigned long long seed, uint32_t 
     return -logf(-logf(u));
 }
 
-// The value a logit competes with: the logit itself (greedy) or logit / T + Gumbel noise.
+// The value a logit competes with: the logit itself (greedy) or logit / T + Gumbel noise; a logit below the nucleus'
+// threshold cannot win.
 struct SampleRule {
     float inv_temp;
     unsigned long long seed;
     uint32_t step;
+    float tau;
     __device__ __forceinline__ float operator()(float z, int i) const
     {
+        if (z < tau) return -INFINITY;
         return inv_temp > 0.f ? fmaf(z, inv_temp, gumbel_noise(seed, step, (uint32_t)i)) : z;
     }
 };
+__device__ __forceinline__ bool top_p_active(const GenState *g) { return g && g->inv_temp > 0.f && g->top_p > 0.f && g->top_p < 1.f; }
 __device__ __forceinline__ SampleRule sample_rule(const GenState *g)
 {
-    SampleRule r{0.f, 0ull, 0u};
+    SampleRule r{0.f, 0ull, 0u, -INFINITY};
     if (g && g->inv_temp > 0.f) { r.inv_temp = g->inv_temp; r.seed = g->sample_seed; r.step = (uint32_t)g->step; }
+    if (top_p_active(g)) r.tau = __ldcg(&g->tau);
     return r;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Nucleus (top-p) threshold of softmax(logits / T) over ids < limit, by one CTA of 256 threads.
+//
+// The nucleus is the shortest prefix of the ids ordered by probability whose probabilities sum to at least top_p,
+// plus every id that ties with its last member; the function returns that member's logit.  No sort: the logits'
+// bit patterns, mapped to unsigned keys that keep their order, are narrowed down in three histogram passes (11, 11
+// and 10 key bits); a bin holds the probability mass of its ids as a 64-bit integer (exp(y - max y) in units of
+// 2^-32), so the sums do not depend on the order of the additions and every CTA that runs this gets the same cut.
+// hist: 2048 64-bit words of shared memory; part: 256 more; sel: 2.
+// ---------------------------------------------------------------------------------------------
+constexpr int kNucleusBins = 2048;
+__device__ __forceinline__ uint32_t nucleus_key(float z)
+{
+    const uint32_t b = __float_as_uint(z);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float nucleus_unkey(uint32_t k)
+{
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+// sync: the barrier of the 256 calling threads.
+template <class Sync>
+__device__ __noinline__ float nucleus_threshold_cta(const float *logits, int limit, float inv_temp, float top_p, unsigned long long *hist,
+                                                    unsigned long long *part, unsigned long long *sel, int tid, Sync sync)
+{
+    constexpr int NT = 256;
+    // ---- max of the scaled logits ----
+    float ymax = -INFINITY;
+    for (int i = tid; i < limit; i += NT) ymax = fmaxf(ymax, __ldcg(logits + i) * inv_temp);
+    float *fred = reinterpret_cast<float *>(part);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ymax = fmaxf(ymax, __shfl_xor_sync(0xffffffffu, ymax, o));
+    if ((tid & 31) == 0) fred[tid >> 5] = ymax;
+    sync();
+    ymax = fred[0];
+    for (int w = 1; w < NT / 32; ++w) ymax = fmaxf(ymax, fred[w]);
+    sync();
+    unsigned long long above = 0, target = 0;   // mass of the keys above the prefix found so far; top_p of the total mass
+    uint32_t prefix = 0;
+    const int shifts[3] = {21, 10, 0}, bits[3] = {11, 11, 10};
+    for (int level = 0; level < 3; ++level) {
+        const int sh = shifts[level], nb = 1 << bits[level];
+        for (int b = tid; b < kNucleusBins; b += NT) hist[b] = 0ull;
+        sync();
+        for (int i = tid; i < limit; i += NT) {
+            const float z = __ldcg(logits + i);
+            const uint32_t k = nucleus_key(z);
+            if (level > 0 && (k >> (sh + bits[level])) != (prefix >> (sh + bits[level]))) continue;
+            const float m = expf(z * inv_temp - ymax);   // in (0, 1]
+            atomicAdd(&hist[(k >> sh) & (uint32_t)(nb - 1)], (unsigned long long)(m * 4294967296.f));
+        }
+        sync();
+        // chunk sums: thread t owns bins [8 t, 8 t + 8)
+        unsigned long long mine = 0;
+        for (int j = 0; j < kNucleusBins / NT; ++j) mine += hist[tid * (kNucleusBins / NT) + j];
+        part[tid] = mine;
+        sync();
+        if (level == 0) {   // the total mass, identical in every thread
+            unsigned long long tot = 0;
+            for (int t = 0; t < NT; ++t) tot += part[t];
+            target = (unsigned long long)__double2ull_ru((double)top_p * (double)tot);
+            if (target > tot) target = tot;
+            if (target == 0) target = 1;
+        }
+        // the bin where the mass counted from the top reaches the target: thread t checks its chunk
+        unsigned long long suffix = above;
+        for (int t = NT - 1; t > tid; --t) suffix += part[t];   // mass above this thread's chunk
+        if (suffix < target && target <= suffix + mine) {
+            unsigned long long run = suffix;
+            for (int j = kNucleusBins / NT - 1; j >= 0; --j) {
+                const unsigned long long h = hist[tid * (kNucleusBins / NT) + j];
+                if (run + h >= target) {
+                    sel[0] = (unsigned long long)(tid * (kNucleusBins / NT) + j);
+                    sel[1] = run;
+                    break;
+                }
+                run += h;
+            }
+        }
+        sync();
+        prefix |= (uint32_t)sel[0] << sh;
+        above = sel[1];
+        sync();
+    }
+    return nucleus_unkey(prefix);
+}
+
+// The threshold for a pass whose sampling runs in a kernel of its own (multi-row passes): one CTA of 256 threads
+// writes gen->tau when top-p sampling is on, and does nothing otherwise.
+__global__ void __launch_bounds__(256) nucleus_kernel(const float *logits, int limit, GenState *gen)
+{
+    __shared__ unsigned long long hist[kNucleusBins], part[256], sel[2];
+    if (!top_p_active(gen)) return;
+    const float tau = nucleus_threshold_cta(logits, limit, gen->inv_temp, gen->top_p, hist, part, sel, (int)threadIdx.x, [] { __syncthreads(); });
+    if (threadIdx.x == 0) gen->tau = tau;
 }
 
 __device__ __forceinline__ unsigned long long global_timer_ns()

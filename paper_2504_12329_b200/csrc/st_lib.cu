@@ -932,6 +932,11 @@ static int sample_tail(st_model *m, const StepDesc *desc, const SampleCtx &sc)
         a.argmax_out = sc.argmax_out;
         a.gen = sc.gen; a.buf = sc.buf; a.desc_small = sc.desc_small; a.desc_large = sc.desc_large;
         a.status = m->status;
+        if (sc.gen) {   // top-p sampling: the nucleus' threshold first (the kernel returns at once when it is off)
+            nucleus_kernel<<<1, 256, 0, m->stream>>>(a.logits, a.limit, sc.gen);
+            ++g_launches;
+            CK(cudaGetLastError());
+        }
         argmax_router_kernel<<<kArgmaxBlocks, 256, 0, m->stream>>>(a);
         ++g_launches;
         CK(cudaGetLastError());
@@ -1803,7 +1808,7 @@ static int check_rule_params(const st_spec_params *P, int vlimit)
         return ST_ERR_ARG;
     if ((P->n_verification > 0 && P->n2 < 1) || (P->neg_threshold >= 0 && P->n3 < 1)) return ST_ERR_ARG;
     if (P->n_delimiters < 0 || (P->n_delimiters > 0 && !P->delimiter_ids)) return ST_ERR_ARG;
-    if (!(P->temperature >= 0.f)) return ST_ERR_ARG;
+    if (!(P->temperature >= 0.f) || !(P->top_p >= 0.f)) return ST_ERR_ARG;
     for (int i = 0; i < P->n_delimiters; ++i)
         if ((unsigned)P->delimiter_ids[i] >= (unsigned)vlimit) return ST_ERR_VOCAB;
     if (P->n_delimiters == 0 && (unsigned)P->delimiter_id >= (unsigned)vlimit) return ST_ERR_VOCAB;
@@ -1906,6 +1911,7 @@ extern "C" int st_generate_spec(st_model *small, st_model *large, const st_spec_
     if (P->temperature > 0.f) {
         g0.inv_temp = 1.f / P->temperature;
         g0.sample_seed = P->sample_seed;
+        g0.top_p = P->top_p;
     }
     if (large && P->target_first_n > 0) {   // the target opens the answer
         g0.active = 1;

@@ -28,7 +28,7 @@ def test_struct_layouts_match_header():
     # sizes implied by the header on LP64: st_config = 14 int32/float + 3 pointers; st_handoff = 3 int32
     assert C.sizeof(binding.StConfig) == 14 * 4 + 3 * 8
     assert C.sizeof(binding.StHandoff) == 12
-    assert C.sizeof(binding.StSpecParams) == 4 + 4 + 8 + 8 * 4 + (8 + 4 + 4) + (8 + 4) + 3 * 4 + 8 + 4 + 4 + (8 + 4 + 4) + 8
+    assert C.sizeof(binding.StSpecParams) == 4 + 4 + 8 + 8 * 4 + (8 + 4 + 4) + (8 + 4) + 3 * 4 + 8 + 4 + 4 + (8 + 4 + 4) + 8 + (4 + 4)   # ... sample_seed, top_p + tail padding
     # st_spec_result ends with three doubles and three int32 (8-byte aligned tail)
     assert binding.StSpecResult.t_prompt_prefill_s.offset % 8 == 0
     assert C.sizeof(binding.StSpecResult) == binding.StSpecResult.n_decode.offset + 8

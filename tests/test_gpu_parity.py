@@ -569,3 +569,66 @@ def test_temperature_sampling_on_device(B, oracle, temperature):
             break
     gs.close()
     gl.close()
+
+
+@pytest.mark.parametrize("top_p", [0.5, 0.9])
+def test_top_p_sampling_on_device(B, oracle, top_p):
+    """Top-p (nucleus) sampling: under teacher forcing with the oracle's stream, the token the device draws equals the
+    oracle's at every step where the oracle's decision is clear -- the gap of the two largest perturbed logits at least
+    the tolerance, and the same token wins for every nucleus between those of top_p - 0.03 and top_p + 0.03 (the sets
+    are nested, so one winner at both ends is the winner of every set in between; the device sums the probability mass
+    in single precision from its own logits, which moves the cut by a few boundary ids at most).  Covers the decode kernel's in-kernel cut and the cut that precedes
+    the sampling kernel of multi-row passes (the first token after the prompt, every token after a catch-up)."""
+    S, L = shape_dict(W.TINY_S), shape_dict(W.TINY_L)
+    os_, ol = oracle.Model(oracle.Config(**S), 0, 0), oracle.Model(oracle.Config(**L), 0, 1)
+    gs = B.Model(S, seed=0, tag=0, max_tokens=512)
+    gl = B.Model(L, seed=0, tag=1, max_tokens=512)
+    prompt = W.prompt_ids(100, 32, 1024)
+    sched = W.forcing_schedule(101, 400, mean_interval=8, keyword_rate=0.5)
+    T = 1.0
+    kw = dict(delimiter_id=W.DELIMITER_ID, keyword_ids=W.KEYWORD_IDS, n1=4, max_new_tokens=120, temperature=T, sample_seed=77,
+              top_p=top_p)
+    want = oracle.generate_spec(os_, ol, prompt, force=sched, trace_n_steps=400, **kw)
+    n = len(want.emission_tokens)
+    ends = [[oracle.sample_top_p(want.logits_trace[t], T, q, 77, t)[:2] for q in (top_p - 0.03, top_p + 0.03)] for t in range(n)]
+    robust = np.array([lo[0] == hi[0] and min(lo[1], hi[1]) >= MARGIN for lo, hi in ends])
+    forced = B.st_generate_spec(gs, gl, prompt, force=want.emission_tokens, **kw)
+    _assert_routing_equal(want, forced)
+    clear = (want.emission_margin >= MARGIN) & robust
+    assert clear.sum() >= 50
+    assert forced.emission_argmax[clear].tolist() == want.emission_argmax[clear].tolist()
+    # the restriction matters: the unrestricted draws differ somewhere, and every drawn token lies in the oracle's nucleus
+    free = oracle.generate_spec(os_, ol, prompt, force=sched, **dict(kw, top_p=0.0))
+    assert free.emission_argmax.tolist() != want.emission_argmax.tolist()
+    for t in np.flatnonzero(clear):
+        thr = oracle.nucleus_threshold(want.logits_trace[t], T, top_p)[0]
+        assert want.logits_trace[t][forced.emission_argmax[t]] >= thr
+    # top_p = 1 is plain temperature sampling
+    a = B.st_generate_spec(gs, gl, prompt, force=sched, **dict(kw, top_p=1.0))
+    b = B.st_generate_spec(gs, gl, prompt, force=sched, **dict(kw, top_p=0.0))
+    assert a.tokens.tolist() == b.tokens.tolist()
+    gs.close()
+    gl.close()
+
+
+def test_top_p_large_vocabulary(B, oracle):
+    """The nucleus cut over a vocabulary of 151 936 ids (two layers at the 1.5B's widths): all three histogram levels
+    of the device's threshold search are exercised with ~10^5 ids inside the nucleus."""
+    import dataclasses
+    shape = shape_dict(dataclasses.replace(W.QWEN_1P5B, n_layers=2))
+    om = oracle.Model(oracle.Config(**shape), 0, 0)
+    gm = B.Model(shape, seed=0, tag=0, max_tokens=256)
+    prompt = W.prompt_ids(5, 12, shape["vocab"])
+    T, top_p = 0.8, 0.7
+    kw = dict(delimiter_id=W.DELIMITER_ID, keyword_ids=[], n1=4, max_new_tokens=10, temperature=T, sample_seed=11, top_p=top_p)
+    want = oracle.generate_spec(om, None, prompt, trace_n_steps=16, **kw)
+    n = len(want.emission_tokens)
+    forced = B.st_generate_spec(gm, None, prompt, force=want.emission_tokens, **kw)
+    ends = [[oracle.sample_top_p(want.logits_trace[t], T, q, 11, t)[:2] for q in (top_p - 0.03, top_p + 0.03)] for t in range(n)]
+    clear = np.array([lo[0] == hi[0] and min(lo[1], hi[1]) >= MARGIN for lo, hi in ends]) & (want.emission_margin >= MARGIN)
+    assert clear.sum() >= 5
+    assert forced.emission_argmax[clear].tolist() == want.emission_argmax[clear].tolist()
+    # the cut removes a real share of the vocabulary and the unrestricted draw differs somewhere
+    inside = [(want.logits_trace[t] >= oracle.nucleus_threshold(want.logits_trace[t], T, top_p)[0]).sum() for t in range(n)]
+    assert 1000 < min(inside) and max(inside) < shape["vocab"] - 1000
+    gm.close()
