@@ -459,6 +459,17 @@ static int tc_pair_min_rows()
     return v;
 }
 
+// Shared memory a projection CTA spends on its pipeline stages.  With at most half of an SM's shared memory (and of its
+// tensor memory) per CTA two CTAs share an SM: while one drains its accumulators the other -- of the same kernel or,
+// launched as a programmatic dependent, of the next -- already streams weights.
+// Measured on the 32B: passes of up to 64 rows gain 3 % that way (20 rows 16.3 -> 15.7 ms, 64 rows 19.0 -> 18.4 ms), wider
+// ones lose 2 % (their activation tiles leave too few stages in half an SM), so the default halves the budget up to 64 rows.
+static int tc_stage_smem(int m_pad)
+{
+    static const int forced = [] { const char *e = getenv("ST_TC_SMEM_KB"); const int kb = e ? atoi(e) : 0; return kb <= 0 ? 0 : (kb < 64 ? 64 : kb > 220 ? 220 : kb) * 1024; }();
+    return forced ? forced : (m_pad <= 64 ? 108 : 220) * 1024;
+}
+
 template <int EPI>
 // pending_splits: when given, a K-split projection leaves its partial sums in the workspace and reports the split
 // count there (0: the output is complete) -- the kernel that consumes the output adds them up.
@@ -469,6 +480,11 @@ static int launch_tc_gemm(const CUtensorMap &tw, TcGemmParams p, int m_upper, in
     const bool pair = tc_pair_min_rows() > 0 && p.m_pad >= tc_pair_min_rows();
     auto kern = pair ? tc_gemm_pair_kernel<EPI> : tc_gemm_kernel<EPI>;
     const int a_rows = pair ? p.m_pad / 2 : p.m_pad;   // activation rows a CTA loads per plane and stage
+    // two CTAs per SM when two stages of one weight tile fit the halved budget; the whole SM otherwise
+    const int smem_want = tc_stage_smem(p.m_pad);
+    const bool shared_sm = smem_want <= 110 * 1024 && 2 * (kTcWBytes + 2 * a_rows * kTcBlockK * 2) <= smem_want && p.m_pad <= 256;
+    const int smem_budget = shared_sm ? smem_want : 220 * 1024, tmem_budget = shared_sm ? 256 : 512;
+    const int slots = shared_sm ? 2 * sms : sms;   // CTAs resident at a time
     // 128-row weight tiles per CTA (they share the activation tiles of a stage): bounded by TMEM (512 columns) and
     // by two pipeline stages of shared memory; among the candidates take the one whose CTA count fills whole waves
     // of SMs best (a projection with 1.46 waves of CTAs runs as long as one with 2), the larger on a tie.
@@ -476,34 +492,34 @@ static int launch_tc_gemm(const CUtensorMap &tw, TcGemmParams p, int m_upper, in
     {
         double best = -1.0;
         for (int cand = 4; cand >= 1; --cand) {
-            if (cand * p.m_pad > 512) continue;
-            if (2 * (cand * kTcWBytes + 2 * a_rows * kTcBlockK * 2) > 220 * 1024) continue;
+            if (cand * p.m_pad > tmem_budget) continue;
+            if (2 * (cand * kTcWBytes + 2 * a_rows * kTcBlockK * 2) > smem_budget) continue;
             const int tiles = (p.N + kTcTileW * cand - 1) / (kTcTileW * cand);
             // projections that may split K fill the machine through the split; the others only through tiles
-            int split = tiles >= sms ? 1 : sms / tiles;   // K splits: as many as still fit one wave
+            int split = tiles >= slots ? 1 : slots / tiles;   // K splits: as many as still fit one wave
             split = split > kMaxKSplits ? kMaxKSplits : split;
             const int ctas = EPI == TEPI_SILU ? tiles : tiles * split;
-            const int waves = (ctas + sms - 1) / sms;
-            const double eff = (double)ctas / ((double)waves * sms);
+            const int waves = (ctas + slots - 1) / slots;
+            const double eff = (double)ctas / ((double)waves * slots);
             if (eff > best + 0.03) { best = eff; wt = cand; }
         }
     }
     {   // tuning aid: force the weight tiles per CTA (when the forced count fits tensor and shared memory)
         static const int forced = [] { const char *e = getenv("ST_TC_WT"); return e ? atoi(e) : 0; }();
-        if (forced >= 1 && forced <= 4 && forced * p.m_pad <= 512 && 2 * (forced * kTcWBytes + 2 * a_rows * kTcBlockK * 2) <= 220 * 1024) wt = forced;
+        if (forced >= 1 && forced <= 4 && forced * p.m_pad <= tmem_budget && 2 * (forced * kTcWBytes + 2 * a_rows * kTcBlockK * 2) <= smem_budget) wt = forced;
     }
     p.w_tiles = wt;
     int cols = wt * p.m_pad;
     p.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
     const int stage_bytes = wt * kTcWBytes + 2 * a_rows * kTcBlockK * 2;
-    int stages = (220 * 1024) / stage_bytes;
+    int stages = smem_budget / stage_bytes;
     p.stages = stages > 8 ? 8 : stages;
     int n_tiles = (p.N + kTcTileW * wt - 1) / (kTcTileW * wt);
     if (pair) n_tiles = (n_tiles + 1) & ~1;   // whole pairs: a CTA beyond the matrix multiplies zero-filled tiles and stores nothing
     const int kb_total = (p.K + kTcBlockK - 1) / kTcBlockK;
     int ks = 1;
     if (EPI != TEPI_SILU) {
-        ks = n_tiles >= sms ? 1 : sms / n_tiles;
+        ks = n_tiles >= slots ? 1 : slots / n_tiles;
         const int ks_max = kb_total / 8 > 1 ? kb_total / 8 : 1;
         ks = ks > ks_max ? ks_max : ks;
         ks = ks > kMaxKSplits ? kMaxKSplits : ks;
